@@ -1,0 +1,394 @@
+/*
+ * seq_oracle.c -- TEST INFRASTRUCTURE, NOT PRODUCT CODE.
+ *
+ * A plain, slow, fp64 CPU statement of what Sequoia's token-tree verification
+ * step computes (Chen et al., "Sequoia: Scalable, Robust, and Hardware-aware
+ * Speculative Decoding"):
+ *   - the ancestor relation of a token tree given as a parent array
+ *     (Section 2.2: verification proceeds from the root along parent links);
+ *   - the target model's attention over that tree, where a tree token sees
+ *     the committed prefix and its own root-to-node path (Section 1: the
+ *     whole tree is verified by one forward pass of the target model);
+ *   - Algorithm 2 ("Sequoia Sampling and Verification") applied recursively
+ *     from the root (Section 2.2), ending with the draw x ~ R.
+ *
+ * Nothing here is blocked, fused or reordered: every function is the
+ * definition, or the algorithm's steps in the paper's order and notation, so
+ * it can be checked against the paper by eye.  It shares no code, headers,
+ * tables or constants with the CUDA library.  Only tests, the smoke check and
+ * the benchmark's cpu_baseline leg may call it.
+ *
+ * Parity pins (tests marked "not gpu"): exact enumeration of Algorithm 2's
+ * output distribution (must equal P, Appendix "Proof of correctness"), the
+ * printed P=[1,0], Q=[.5,.5] example of Theorem 3.7's proof, the optimal-
+ * transport closed form 1-|P-Q|_1/2 at k=1, the cover property, the lemma
+ * P(reject at i) = sum max(0, t_i - d_i), reduction of a chain to Algorithm 3,
+ * Monte-Carlo; attention against library causal attention (chain tree),
+ * single-query decode (star tree) and explicit-sequence brute force.
+ *
+ * Build: gcc -O2 -fopenmp -shared -fPIC seq_oracle.c -o liboracle.so -lm
+ */
+#include <math.h>
+#include <stdint.h>
+#include <stdlib.h>
+#include <string.h>
+#ifdef _OPENMP
+#include <omp.h>
+#endif
+
+/* data-problem flags reported by the oracle (its own numbering) */
+#define ORC_BAD_PARENT 1
+#define ORC_BAD_TOKEN 2
+#define ORC_NONFINITE 4
+#define ORC_DEGENERATE 8
+
+#define ORC_VARIANT_SEQUOIA 0   /* Algorithm 2 as printed */
+#define ORC_VARIANT_SPECINFER 1 /* Algorithm 2 without its blue lines 10-16 */
+
+int orc_num_threads(void) {
+#ifdef _OPENMP
+  return omp_get_max_threads();
+#else
+  return 1;
+#endif
+}
+
+/* A parent entry is usable iff it is -1 (no parent) or an earlier node.
+ * Anything else is flagged and read as -1, so every walk below terminates. */
+static int32_t clean_parent(const int32_t* parent, int32_t i, int* flags) {
+  int32_t p = parent[i];
+  if (p == -1) return -1;
+  if (p < -1 || p >= i) {
+    if (flags) *flags |= ORC_BAD_PARENT;
+    return -1;
+  }
+  return p;
+}
+
+/*
+ * Ancestor relation (Section 2.2, "starting at the root of the tree"):
+ * bit j of row i is set iff j lies on the walk i, parent[i], parent[parent[i]], ...
+ * depth[i] = number of parent links on that walk.
+ */
+int orc_mask_from_parents(const int32_t* parent, int32_t n, uint32_t* mask_bits,
+                          int32_t words_per_row, int32_t* depth) {
+  int flags = 0;
+  for (int32_t i = 0; i < n; ++i) {
+    uint32_t* row = mask_bits + (size_t)i * words_per_row;
+    memset(row, 0, sizeof(uint32_t) * (size_t)words_per_row);
+    int32_t j = i, links = 0;
+    for (;;) {
+      row[j >> 5] |= (uint32_t)1 << (j & 31);
+      int32_t p = clean_parent(parent, j, &flags);
+      if (p < 0) break;
+      j = p;
+      ++links;
+    }
+    if (depth) depth[i] = links;
+  }
+  return flags;
+}
+
+/*
+ * Tree attention by its definition (Section 1: one target forward pass over
+ * all tree tokens; each tree token conditions on the prefix x_{<n} followed by
+ * the tokens on its own path, which is the context Algorithm 2's input
+ * P(. | x_{<n}) refers to at that node).
+ *
+ * For query head h (kv head g = h / (Hq/Hkv)) and node i the key set is
+ *   J = {0..L-1}  union  {L + a : a on the walk i -> root},
+ * and out[i,h,:] = sum_j softmax_j(scale * q.k_j) v_j over j in J.
+ * q,out: [n][Hq][d]; k,v: [Hkv][kv_rows][d]; lse: [Hq][n] (natural log), nullable.
+ * No mask array is used: the path is gathered by walking parent[].
+ */
+int orc_tree_attention(const double* q, const double* k, const double* v,
+                       const int32_t* parent, int32_t n, int32_t L, int32_t Hq,
+                       int32_t Hkv, int32_t d, int32_t kv_rows, double scale,
+                       double* out, double* lse) {
+  int flags = 0;
+  int32_t G = Hq / Hkv;
+#pragma omp parallel for collapse(2) schedule(dynamic, 4) reduction(| : flags)
+  for (int32_t h = 0; h < Hq; ++h) {
+    for (int32_t i = 0; i < n; ++i) {
+      int32_t g = h / G;
+      int32_t nkeys = 0;
+      int32_t* J = (int32_t*)malloc(sizeof(int32_t) * (size_t)(L + n));
+      double* s = (double*)malloc(sizeof(double) * (size_t)(L + n));
+      for (int32_t j = 0; j < L; ++j) J[nkeys++] = j;
+      for (int32_t a = i; a >= 0; a = clean_parent(parent, a, &flags)) J[nkeys++] = L + a;
+      const double* qi = q + ((size_t)i * Hq + h) * d;
+      double m = -INFINITY;
+      for (int32_t t = 0; t < nkeys; ++t) {
+        const double* kj = k + ((size_t)g * kv_rows + J[t]) * d;
+        double acc = 0.0;
+        for (int32_t c = 0; c < d; ++c) acc += qi[c] * kj[c];
+        s[t] = scale * acc;
+        if (s[t] > m) m = s[t];
+      }
+      double denom = 0.0;
+      for (int32_t t = 0; t < nkeys; ++t) {
+        s[t] = exp(s[t] - m);
+        denom += s[t];
+      }
+      double* o = out + ((size_t)i * Hq + h) * d;
+      for (int32_t c = 0; c < d; ++c) o[c] = 0.0;
+      for (int32_t t = 0; t < nkeys; ++t) {
+        const double* vj = v + ((size_t)g * kv_rows + J[t]) * d;
+        double w = s[t] / denom;
+        for (int32_t c = 0; c < d; ++c) o[c] += w * vj[c];
+      }
+      if (lse) lse[(size_t)h * n + i] = m + log(denom);
+      free(J);
+      free(s);
+    }
+  }
+  return flags;
+}
+
+/* softmax(logits / T) in fp64, max-subtracted (Algorithm 2's inputs P and Q
+ * are the models' distributions at temperature T, Table 1 column "T"). */
+void orc_softmax_T(const float* logits, int32_t V, double T, double* out) {
+  double m = -INFINITY;
+  for (int32_t t = 0; t < V; ++t) {
+    double x = (double)logits[t] / T;
+    if (x > m) m = x;
+  }
+  double z = 0.0;
+  for (int32_t t = 0; t < V; ++t) {
+    out[t] = exp((double)logits[t] / T - m);
+    z += out[t];
+  }
+  for (int32_t t = 0; t < V; ++t) out[t] /= z;
+}
+
+/*
+ * Algorithm 2, lines 3-17, for ONE node whose k children were already drawn
+ * (the draws s_i ~ D of line 5 are the caller's: child_tok[i] in draw order)
+ * and whose uniforms r_i are supplied.
+ *
+ *   R, D       in: P and Q (length V); out: the residual and draft after the
+ *              last executed line, i.e. R is what line 18 (x ~ R) samples if
+ *              no child was accepted.
+ *   accepted   index i (0-based) of the accepted child, or -1.
+ *   ratio/rnum/dden (nullable, length k): R[s_i]/D[s_i], R[s_i], D[s_i] as
+ *              seen by the test of line 6 (NaN where the test never ran).
+ *   min_gap    (nullable) min over executed tests of |r_i - ratio_i|.
+ * Returns flags.
+ */
+int orc_alg2_node(double* R, double* D, int32_t V, const int32_t* child_tok,
+                  const double* child_u, int32_t k, int32_t variant,
+                  int32_t* accepted, double* ratio_out, double* rnum_out,
+                  double* dden_out, double* min_gap) {
+  int flags = 0;
+  *accepted = -1;
+  unsigned char* S = (unsigned char*)calloc((size_t)V, 1); /* line 3: S = {} */
+  double* Rn = (double*)malloc(sizeof(double) * (size_t)V);
+  if (min_gap) *min_gap = INFINITY;
+  for (int32_t i = 0; i < k; ++i) {
+    if (ratio_out) ratio_out[i] = NAN;
+    if (rnum_out) rnum_out[i] = NAN;
+    if (dden_out) dden_out[i] = NAN;
+  }
+  int32_t n_rejected = 0;
+  for (int32_t i = 0; i < k; ++i) { /* line 4 */
+    int32_t s = child_tok[i];
+    if (s < 0 || s >= V) { /* not a token: cannot be accepted, touches nothing */
+      flags |= ORC_BAD_TOKEN;
+      continue;
+    }
+    double ratio; /* line 6: R[s]/D[s] */
+    if (D[s] > 0.0)
+      ratio = R[s] / D[s];
+    else
+      ratio = (R[s] > 0.0) ? INFINITY : 0.0;
+    if (ratio_out) ratio_out[i] = ratio;
+    if (rnum_out) rnum_out[i] = R[s];
+    if (dden_out) dden_out[i] = D[s];
+    if (min_gap) {
+      double gap = fabs(child_u[i] - ratio);
+      if (gap < *min_gap) *min_gap = gap;
+    }
+    if (child_u[i] < ratio) { /* line 6, strict */
+      *accepted = i;          /* line 7 */
+      break;
+    }
+    /* line 9: R <- norm(max(R - D, 0)), with D as it stands (s not yet removed) */
+    double Z = 0.0;
+    for (int32_t t = 0; t < V; ++t) {
+      double x = R[t] - D[t];
+      Rn[t] = x > 0.0 ? x : 0.0;
+      Z += Rn[t];
+    }
+    if (Z > 0.0) {
+      for (int32_t t = 0; t < V; ++t) R[t] = Rn[t] / Z;
+    } else {
+      flags |= ORC_DEGENERATE; /* impossible in exact arithmetic; keep R */
+    }
+    if (variant == ORC_VARIANT_SEQUOIA) {
+      D[s] = 0.0; /* line 10 */
+      if (!S[s]) { /* line 11 */
+        S[s] = 1;
+        ++n_rejected;
+      }
+      double sumD = 0.0; /* line 12 */
+      for (int32_t t = 0; t < V; ++t) sumD += D[t];
+      if (sumD == 0.0) { /* lines 13-15: uniform over the non-rejected set */
+        for (int32_t t = 0; t < V; ++t) D[t] = S[t] ? 0.0 : 1.0;
+        sumD = (double)(V - n_rejected);
+      }
+      if (sumD > 0.0) /* line 16 (nothing left to normalise once S is everything) */
+        for (int32_t t = 0; t < V; ++t) D[t] /= sumD;
+    }
+  }
+  free(S);
+  free(Rn);
+  return flags;
+}
+
+/* Line 18, x ~ R, realised by inverse CDF in index order with one uniform:
+ * the first t whose inclusive cumulative sum exceeds u; if rounding leaves the
+ * total at or below u, the last t with R[t] > 0. */
+int32_t orc_sample_inverse_cdf(const double* R, int32_t V, double u) {
+  double c = 0.0;
+  int32_t last_pos = -1;
+  for (int32_t t = 0; t < V; ++t) {
+    c += R[t];
+    if (R[t] > 0.0) last_pos = t;
+    if (c > u) return t;
+  }
+  return last_pos;
+}
+
+/*
+ * The whole verification of one tree (Section 2.2: start at the root, apply
+ * the per-node algorithm, recurse into the accepted child), Algorithm 2 at
+ * every visited node, then line 18 at the node where the walk stops.
+ *
+ *   parent, tokens        [n]; node 0 is the root (parent[0] = -1), tokens[0] unused.
+ *   target_logits         row v = next-token logits after node v.
+ *   draft_logits          row v = logits v's children were drawn from
+ *                         (rows of leaves are never read).
+ *   T                     temperature of both distributions; 0 = greedy.
+ *   uniforms              [n+1]: entry c tests child node c, entry n draws the bonus.
+ *   path/path_len/bonus   visited nodes (root first), their count, the token from line 18.
+ *   residual_out          nullable [V]: R at line 18.
+ *   next_child            nullable [n]: accepted child of each visited node,
+ *                         -1 if none, -2 for nodes the walk never reached.
+ *   ratio_out             nullable [n]: ratio tested for child node c (NaN if untested).
+ *   min_gap               nullable: min |u - ratio| over executed tests.
+ * Children of a node are taken in ascending node index (= draw order).
+ */
+int orc_tree_verify(int32_t n, int32_t V, const int32_t* parent, const int32_t* tokens,
+                    const float* target_logits, int64_t target_row_stride,
+                    const float* draft_logits, int64_t draft_row_stride, double T,
+                    const float* uniforms, int32_t variant, int32_t* path,
+                    int32_t* path_len, int32_t* bonus, double* residual_out,
+                    int32_t* next_child, double* ratio_out, double* min_gap) {
+  int flags = 0;
+  double* R = (double*)malloc(sizeof(double) * (size_t)V);
+  double* D = (double*)malloc(sizeof(double) * (size_t)V);
+  int32_t* kids = (int32_t*)malloc(sizeof(int32_t) * (size_t)n);
+  int32_t* ktok = (int32_t*)malloc(sizeof(int32_t) * (size_t)n);
+  double* ku = (double*)malloc(sizeof(double) * (size_t)n);
+  double* kr = (double*)malloc(sizeof(double) * (size_t)n);
+  if (next_child)
+    for (int32_t i = 0; i < n; ++i) next_child[i] = -2;
+  if (ratio_out)
+    for (int32_t i = 0; i < n; ++i) ratio_out[i] = NAN;
+  if (min_gap) *min_gap = INFINITY;
+  for (int32_t i = 1; i < n; ++i) (void)clean_parent(parent, i, &flags);
+
+  int32_t cur = 0, plen = 0;
+  path[plen++] = 0;
+  for (;;) {
+    const float* trow = target_logits + (size_t)cur * (size_t)target_row_stride;
+    int32_t k = 0;
+    for (int32_t c = cur + 1; c < n; ++c)
+      if (parent[c] == cur) kids[k++] = c;
+    for (int32_t t = 0; t < V; ++t)
+      if (!isfinite(trow[t]) && !(trow[t] < 0 && isinf(trow[t]))) flags |= ORC_NONFINITE;
+    int32_t acc = -1;
+    if (T == 0.0) {
+      /* greedy: P is the one-hot at the target arg-max (lowest index on ties);
+       * a child is accepted iff its token is that arg-max. */
+      int32_t a = 0;
+      for (int32_t t = 1; t < V; ++t)
+        if (trow[t] > trow[a]) a = t;
+      for (int32_t t = 0; t < V; ++t) R[t] = 0.0;
+      R[a] = 1.0;
+      for (int32_t i = 0; i < k && acc < 0; ++i) {
+        int32_t s = tokens[kids[i]];
+        if (s < 0 || s >= V) {
+          flags |= ORC_BAD_TOKEN;
+          continue;
+        }
+        if (s == a) acc = i;
+      }
+    } else {
+      orc_softmax_T(trow, V, T, R); /* line 3: R <- P */
+      if (k > 0) {
+        const float* drow = draft_logits + (size_t)cur * (size_t)draft_row_stride;
+        orc_softmax_T(drow, V, T, D); /* line 3: D <- Q */
+        for (int32_t i = 0; i < k; ++i) {
+          ktok[i] = tokens[kids[i]];
+          ku[i] = (double)uniforms[kids[i]];
+        }
+        double gap;
+        flags |= orc_alg2_node(R, D, V, ktok, ku, k, variant, &acc, kr, NULL, NULL, &gap);
+        if (min_gap && gap < *min_gap) *min_gap = gap;
+        if (ratio_out)
+          for (int32_t i = 0; i < k; ++i) ratio_out[kids[i]] = kr[i];
+      }
+    }
+    if (next_child) next_child[cur] = acc >= 0 ? kids[acc] : -1;
+    if (acc < 0) break;
+    cur = kids[acc]; /* recurse into the accepted child with fresh R, D */
+    path[plen++] = cur;
+  }
+  *path_len = plen;
+  *bonus = orc_sample_inverse_cdf(R, V, (double)uniforms[n]); /* line 18 */
+  if (residual_out) memcpy(residual_out, R, sizeof(double) * (size_t)V);
+  free(R);
+  free(D);
+  free(kids);
+  free(ktok);
+  free(ku);
+  free(kr);
+  return flags;
+}
+
+/*
+ * Algorithm 3 (sequence-based speculative decoding) for one chain, with the
+ * two misprints of the listing read as: the target distributions come from the
+ * target model, and the final residual is taken iff fewer than gamma tokens
+ * were accepted.  p,q: [gamma+1][V] and [gamma][V] distributions; x: the gamma
+ * drafted tokens; r: gamma uniforms; u_final: uniform for the last draw.
+ * Returns the number of accepted tokens; *t_out is the final token.
+ */
+int32_t orc_alg3_chain(const double* p, const double* q, int32_t V, int32_t gamma,
+                       const int32_t* x, const double* r, double u_final,
+                       int32_t* t_out) {
+  int32_t s = 0;
+  for (int32_t i = 0; i < gamma; ++i) {
+    double pi = p[(size_t)i * V + x[i]], qi = q[(size_t)i * V + x[i]];
+    double ratio = qi > 0.0 ? pi / qi : (pi > 0.0 ? INFINITY : 0.0);
+    if (r[i] < ratio)
+      ++s;
+    else
+      break;
+  }
+  double* pp = (double*)malloc(sizeof(double) * (size_t)V);
+  memcpy(pp, p + (size_t)s * V, sizeof(double) * (size_t)V);
+  if (s < gamma) {
+    double Z = 0.0;
+    for (int32_t t = 0; t < V; ++t) {
+      double dlt = p[(size_t)s * V + t] - q[(size_t)s * V + t];
+      pp[t] = dlt > 0.0 ? dlt : 0.0;
+      Z += pp[t];
+    }
+    for (int32_t t = 0; t < V; ++t) pp[t] /= Z;
+  }
+  *t_out = orc_sample_inverse_cdf(pp, V, u_final);
+  free(pp);
+  return s;
+}
