@@ -1,0 +1,201 @@
+/*
+ * seq_tree.h -- C ABI of the B200 (sm_100a) token-tree verification library.
+ *
+ * The library computes the per-step numerics of Sequoia's tree-based
+ * speculative decoding (Chen et al., arXiv 2402.12374):
+ *   (a) the target model's attention over a speculated token tree, and
+ *   (b) Algorithm 2 ("Sequoia Sampling and Verification") applied from the
+ *       root down the tree, ending in the bonus token drawn from the residual.
+ *
+ * Conventions shared by every entry point
+ *   - All data pointers are DEVICE pointers owned by the caller, valid on the
+ *     device that is current when the call is made.  The library allocates
+ *     nothing, keeps no state between calls and never synchronises the host.
+ *   - `stream` is a cudaStream_t passed as void* (NULL = the legacy default
+ *     stream).  Work is enqueued on it and the call returns at once.
+ *   - Problems the host can see (null pointers, sizes out of range, bad
+ *     alignment, workspace too small) return a negative seq_status and
+ *     enqueue nothing.
+ *   - Problems only the device can see (a parent that is not an earlier node,
+ *     a token id outside the vocabulary, NaN/+inf logits) OR a bit into
+ *     *dev_status (nullable), clamp the offending index, and still produce
+ *     defined outputs.  Kernels never trap and never wait without a bound;
+ *     a bounded wait that runs out sets SEQ_DEV_TIMEOUT.
+ *     *dev_status is only ever OR-ed into: the caller zeroes it.
+ *   - Trees: n nodes, node 0 is the root (the last committed token, Section
+ *     2.1: "the tree root corresponds to the current prefix"); parent[0] = -1
+ *     and 0 <= parent[i] < i.  Siblings are ordered by node index, which is
+ *     the order they were drawn in.  1 <= n <= SEQ_MAX_TREE.
+ */
+#ifndef SEQ_TREE_H_
+#define SEQ_TREE_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define SEQ_MAX_TREE 1024
+
+typedef enum {
+  SEQ_OK = 0,
+  SEQ_ERR_INVALID_ARG = -1, /* null pointer, size/stride/alignment out of range */
+  SEQ_ERR_UNSUPPORTED = -2, /* valid request this build has no kernel for */
+  SEQ_ERR_WORKSPACE = -3,   /* workspace_bytes below seq_*_workspace_bytes() */
+  SEQ_ERR_CUDA = -4         /* a CUDA runtime/driver call failed */
+} seq_status;
+
+typedef enum { SEQ_F16 = 0, SEQ_BF16 = 1, SEQ_F32 = 2 } seq_dtype;
+
+/* bits OR-ed into *dev_status by kernels; 0 = clean */
+enum {
+  SEQ_DEV_BAD_PARENT = 1,  /* parent[i] not in {-1} u [0,i): read as -1 */
+  SEQ_DEV_BAD_TOKEN = 2,   /* token id outside [0,vocab): the child is rejected, R and D untouched */
+  SEQ_DEV_NONFINITE = 4,   /* NaN or +inf logit on a visited row */
+  SEQ_DEV_DEGENERATE = 8,  /* sum max(R-D,0) == 0 after a rejection (impossible in exact arithmetic): R kept */
+  SEQ_DEV_TIMEOUT = 16     /* a bounded on-chip wait ran out; outputs of that call are undefined */
+};
+
+/*
+ * seq_tree_mask_from_parents -- ancestor bitmasks of a token tree.
+ *
+ * Defines which tree tokens a tree token may attend to: itself and the nodes
+ * on its path to the root (Section 2.2: verification walks "starting at the
+ * root of the tree"; Algorithm 2's input P(.|x_<n) at a node is conditioned on
+ * exactly that path).  Bit j of row i is set iff j is i or an ancestor of i.
+ *
+ *   parent        [n] int32, device.  parent[i] = -1 also allowed for i > 0
+ *                 (a node with no ancestors).
+ *   mask_bits     [n][words_per_row] uint32, device, written in full (unused
+ *                 high bits cleared).  words_per_row >= ceil(n/32).
+ *   depth         [n] int32, device, nullable: number of parent links from i
+ *                 to its root (callers use prefix_len + depth as position id).
+ *   dev_status    nullable.
+ * Returns SEQ_OK or SEQ_ERR_INVALID_ARG.  Run once per tree: the tree is fixed
+ * across decoding steps (Section 4.1, "we determine the optimal tree structure
+ * in advance").
+ */
+int seq_tree_mask_from_parents(const int32_t* parent, int32_t n, uint32_t* mask_bits,
+                               int32_t words_per_row, int32_t* depth, int32_t* dev_status,
+                               void* stream);
+
+/*
+ * seq_tree_attention -- attention of the n tree tokens in one target forward
+ * pass (Section 1: "the speculated tokens are then verified in parallel
+ * through a single forward pass of the target model").
+ *
+ * For query head h (kv head h / (num_q_heads/num_kv_heads)) and node i:
+ *     out[i,h,:] = sum_j softmax_j(softmax_scale * q[i,h,:].k[g,j,:]) * v[g,j,:]
+ * over j in [0, prefix_len)  and  j = prefix_len + a for every a whose bit is
+ * set in row i of mask_bits.  Scores, softmax and accumulation are fp32; with
+ * 16-bit inputs the probabilities are rounded to the input type before the
+ * P.V product on the tensor-core path.
+ *
+ * Layouts (strides in ELEMENTS, innermost head_dim contiguous):
+ *   q, out        element (i,h,c) at i*stride_tok + h*stride_head + c
+ *   k_cache,      element (g,j,c) at g*kv_stride_head + j*kv_stride_tok + c;
+ *   v_cache       rows [0,prefix_len) hold the prefix, rows [prefix_len,
+ *                 prefix_len+n_tree) the tree tokens in node order; rows
+ *                 beyond that (up to kv_capacity) are never read into the
+ *                 result and may hold anything, NaN included.
+ *   lse           nullable, [num_q_heads][n_tree] fp32: natural-log
+ *                 sum-exp of the scaled scores of each row.
+ * head_dim must be 128.  Base pointers and strides must keep every row
+ * 16-byte aligned.  dtype selects f16/bf16/f32 for q, k, v and out alike.
+ * workspace: at least seq_tree_attention_workspace_bytes(p) bytes, 256-byte
+ * aligned, device; contents undefined before and after.
+ */
+typedef struct {
+  int32_t n_tree, prefix_len, num_q_heads, num_kv_heads, head_dim;
+  int32_t dtype;       /* seq_dtype */
+  float softmax_scale; /* <= 0 selects 1/sqrt(head_dim) */
+  const void* q;
+  int64_t q_stride_tok, q_stride_head;
+  const void* k_cache;
+  const void* v_cache;
+  int64_t kv_stride_tok, kv_stride_head;
+  int32_t kv_capacity; /* rows per kv head; >= prefix_len + n_tree */
+  const uint32_t* mask_bits;
+  int32_t mask_words_per_row;
+  void* out;
+  int64_t o_stride_tok, o_stride_head;
+  float* lse;
+  void* workspace;
+  size_t workspace_bytes;
+  int32_t* dev_status;
+  int32_t kernel; /* 0 = choose; 1 = force the CUDA-core kernel; 2 = force the tensor-core kernel */
+} seq_tree_attention_params;
+
+size_t seq_tree_attention_workspace_bytes(const seq_tree_attention_params* p);
+int seq_tree_attention(const seq_tree_attention_params* p, void* stream);
+
+/*
+ * seq_tree_verify -- Algorithm 2 applied recursively from the root (Section
+ * 2.2), then its last line x ~ R at the node where the walk stops.
+ *
+ * At the current node v with children c_1 < c_2 < ... (node order):
+ *   R <- softmax(target_logits[v]/T), D <- softmax(draft_logits[v]/T), S <- {}
+ *   for each child c, s = tokens[c]:
+ *     accept c  iff  uniforms[c] < R[s]/D[s]          (strict; D[s]=0: +inf if R[s]>0 else 0)
+ *     otherwise R <- norm(max(R-D,0)); D[s] <- 0; S <- S u {s};
+ *               if sum(D) = 0: D <- uniform over tokens not in S;  D <- norm(D)
+ *   an accepted child becomes the current node with fresh R, D, S; when no
+ *   child is accepted (or v is a leaf) the bonus token is the first t with
+ *   R[0]+..+R[t] > uniforms[n] (the last t with R[t] > 0 if rounding leaves
+ *   none).
+ * T = 0 is greedy: R is the one-hot at the target arg-max (lowest index on
+ * ties), a child is accepted iff its token is that arg-max, draft logits and
+ * uniforms are not read.
+ *
+ *   parent, tokens      [n] int32; tokens[0] is ignored.  A single root.
+ *   target_logits       fp32, row v at v*target_row_stride: next-token logits after node v.
+ *   draft_logits        fp32, row v at v*draft_row_stride: the logits whose softmax at T
+ *                       v's children were drawn from without replacement; rows of leaves
+ *                       are never read.  -inf entries are legal (probability 0).
+ *   temperature         >= 0, finite; one value for both models.
+ *   uniforms            [n+1] fp32 in [0,1): entry c decides child node c, entry n the bonus.
+ *   path                [n] int32 out: visited nodes, root first; path_len out: their count
+ *                       (accepted tokens are tokens[path[1..path_len-1]]; the step emits
+ *                       path_len tokens counting the bonus).
+ *   bonus_token         out.
+ *   residual_out        nullable [vocab] fp32: the R the bonus token was drawn from.
+ *   next_child_out      nullable [n] int32: accepted child of each visited node, -1 if none,
+ *                       -2 for nodes the walk did not visit.  With SEQ_VERIFY_ALL_NODES
+ *                       every node is processed and gets its own decision.
+ * workspace may be NULL when seq_tree_verify_workspace_bytes() returns 0.
+ */
+enum { SEQ_VERIFY_ALL_NODES = 1 };
+
+typedef struct {
+  int32_t n_tree, vocab;
+  const int32_t* parent;
+  const int32_t* tokens;
+  const float* target_logits;
+  int64_t target_row_stride;
+  const float* draft_logits;
+  int64_t draft_row_stride;
+  float temperature;
+  const float* uniforms;
+  int32_t* path;
+  int32_t* path_len;
+  int32_t* bonus_token;
+  float* residual_out;
+  int32_t* next_child_out;
+  void* workspace;
+  size_t workspace_bytes;
+  int32_t* dev_status;
+  int32_t flags; /* 0 or SEQ_VERIFY_ALL_NODES */
+} seq_tree_verify_params;
+
+size_t seq_tree_verify_workspace_bytes(const seq_tree_verify_params* p);
+int seq_tree_verify(const seq_tree_verify_params* p, void* stream);
+
+/* Library build string ("seqtree <version> sm_100a"); static storage. */
+const char* seq_tree_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* SEQ_TREE_H_ */

@@ -1,0 +1,272 @@
+"""Thin ctypes binding of ``libseqtree.so`` (see ``include/seq_tree.h``).
+
+Argument marshalling only: every step of the token-tree verification path runs in the
+library's CUDA kernels.  torch supplies device memory and streams.  There is no CPU fallback:
+if the library is missing or a tensor is not on a CUDA device the call raises.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libseqtree.so")
+
+SEQ_OK, SEQ_ERR_INVALID_ARG, SEQ_ERR_UNSUPPORTED, SEQ_ERR_WORKSPACE, SEQ_ERR_CUDA = 0, -1, -2, -3, -4
+SEQ_F16, SEQ_BF16, SEQ_F32 = 0, 1, 2
+SEQ_DEV_BAD_PARENT, SEQ_DEV_BAD_TOKEN, SEQ_DEV_NONFINITE, SEQ_DEV_DEGENERATE, SEQ_DEV_TIMEOUT = 1, 2, 4, 8, 16
+SEQ_VERIFY_ALL_NODES = 1
+SEQ_MAX_TREE = 1024
+KERNEL_AUTO, KERNEL_CUDA_CORE, KERNEL_TENSOR_CORE = 0, 1, 2
+
+_STATUS_NAMES = {0: "SEQ_OK", -1: "SEQ_ERR_INVALID_ARG", -2: "SEQ_ERR_UNSUPPORTED", -3: "SEQ_ERR_WORKSPACE",
+                 -4: "SEQ_ERR_CUDA"}
+_DTYPES = {torch.float16: SEQ_F16, torch.bfloat16: SEQ_BF16, torch.float32: SEQ_F32}
+
+EXPORTED_SYMBOLS = (
+    "seq_tree_mask_from_parents",
+    "seq_tree_attention_workspace_bytes",
+    "seq_tree_attention",
+    "seq_tree_verify_workspace_bytes",
+    "seq_tree_verify",
+    "seq_tree_version",
+)
+
+
+class SeqTreeError(RuntimeError):
+    def __init__(self, fn: str, code: int):
+        super().__init__(f"{fn} returned {_STATUS_NAMES.get(code, code)}")
+        self.code = code
+
+
+class AttentionParams(C.Structure):
+    _fields_ = [
+        ("n_tree", C.c_int32), ("prefix_len", C.c_int32), ("num_q_heads", C.c_int32),
+        ("num_kv_heads", C.c_int32), ("head_dim", C.c_int32), ("dtype", C.c_int32),
+        ("softmax_scale", C.c_float),
+        ("q", C.c_void_p), ("q_stride_tok", C.c_int64), ("q_stride_head", C.c_int64),
+        ("k_cache", C.c_void_p), ("v_cache", C.c_void_p),
+        ("kv_stride_tok", C.c_int64), ("kv_stride_head", C.c_int64), ("kv_capacity", C.c_int32),
+        ("mask_bits", C.c_void_p), ("mask_words_per_row", C.c_int32),
+        ("out", C.c_void_p), ("o_stride_tok", C.c_int64), ("o_stride_head", C.c_int64),
+        ("lse", C.c_void_p), ("workspace", C.c_void_p), ("workspace_bytes", C.c_size_t),
+        ("dev_status", C.c_void_p), ("kernel", C.c_int32),
+    ]
+
+
+class VerifyParams(C.Structure):
+    _fields_ = [
+        ("n_tree", C.c_int32), ("vocab", C.c_int32),
+        ("parent", C.c_void_p), ("tokens", C.c_void_p),
+        ("target_logits", C.c_void_p), ("target_row_stride", C.c_int64),
+        ("draft_logits", C.c_void_p), ("draft_row_stride", C.c_int64),
+        ("temperature", C.c_float), ("uniforms", C.c_void_p),
+        ("path", C.c_void_p), ("path_len", C.c_void_p), ("bonus_token", C.c_void_p),
+        ("residual_out", C.c_void_p), ("next_child_out", C.c_void_p),
+        ("workspace", C.c_void_p), ("workspace_bytes", C.c_size_t),
+        ("dev_status", C.c_void_p), ("flags", C.c_int32),
+    ]
+
+
+_lib = None
+
+
+def load() -> C.CDLL:
+    """Load the CUDA library; raises if it has not been built (``python -m paper_2402_12374_b200.build``)."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise RuntimeError(f"{LIB_PATH} is missing: build it with `python -m paper_2402_12374_b200.build`; "
+                               "there is no fallback path")
+        lib = C.CDLL(LIB_PATH)
+        lib.seq_tree_mask_from_parents.argtypes = [C.c_void_p, C.c_int32, C.c_void_p, C.c_int32, C.c_void_p,
+                                                   C.c_void_p, C.c_void_p]
+        lib.seq_tree_mask_from_parents.restype = C.c_int
+        lib.seq_tree_attention_workspace_bytes.argtypes = [C.POINTER(AttentionParams)]
+        lib.seq_tree_attention_workspace_bytes.restype = C.c_size_t
+        lib.seq_tree_attention.argtypes = [C.POINTER(AttentionParams), C.c_void_p]
+        lib.seq_tree_attention.restype = C.c_int
+        lib.seq_tree_verify_workspace_bytes.argtypes = [C.POINTER(VerifyParams)]
+        lib.seq_tree_verify_workspace_bytes.restype = C.c_size_t
+        lib.seq_tree_verify.argtypes = [C.POINTER(VerifyParams), C.c_void_p]
+        lib.seq_tree_verify.restype = C.c_int
+        lib.seq_tree_version.restype = C.c_char_p
+        _lib = lib
+    return _lib
+
+
+def _dev(t: torch.Tensor | None, name: str, dtype=None) -> int | None:
+    if t is None:
+        return None
+    if not t.is_cuda:
+        raise ValueError(f"{name} must live on a CUDA device (there is no CPU path)")
+    if dtype is not None and t.dtype != dtype:
+        raise ValueError(f"{name} must be {dtype}, got {t.dtype}")
+    return t.data_ptr()
+
+
+def _stream(stream) -> int:
+    s = stream if stream is not None else torch.cuda.current_stream()
+    return s.cuda_stream if hasattr(s, "cuda_stream") else int(s)
+
+
+def _check(fn: str, code: int) -> None:
+    if code != SEQ_OK:
+        raise SeqTreeError(fn, code)
+
+
+def seq_tree_version() -> str:
+    return load().seq_tree_version().decode()
+
+
+def seq_tree_mask_from_parents(parent: torch.Tensor, *, words_per_row: int | None = None,
+                               mask_bits: torch.Tensor | None = None, depth: torch.Tensor | None = None,
+                               dev_status: torch.Tensor | None = None, stream=None):
+    """parent int32 [n] (device) -> (mask_bits int32-typed uint32 words [n, words_per_row], depth int32 [n])."""
+    n = parent.shape[0]
+    wpr = words_per_row or (n + 31) // 32
+    if mask_bits is None:
+        mask_bits = torch.empty((n, wpr), dtype=torch.int32, device=parent.device)
+    if depth is None:
+        depth = torch.empty(n, dtype=torch.int32, device=parent.device)
+    rc = load().seq_tree_mask_from_parents(_dev(parent, "parent", torch.int32), n, _dev(mask_bits, "mask_bits", torch.int32),
+                                           wpr, _dev(depth, "depth", torch.int32), _dev(dev_status, "dev_status", torch.int32),
+                                           _stream(stream))
+    _check("seq_tree_mask_from_parents", rc)
+    return mask_bits, depth
+
+
+class AttentionCall:
+    """A prepared seq_tree_attention call: the parameter struct is filled once and can be launched many times."""
+
+    def __init__(self, q, k_cache, v_cache, mask_bits, prefix_len: int, *, out=None, lse=None,
+                 softmax_scale: float = 0.0, workspace=None, dev_status=None, kernel: int = KERNEL_AUTO):
+        if q.dtype not in _DTYPES or k_cache.dtype != q.dtype or v_cache.dtype != q.dtype:
+            raise ValueError("q, k_cache, v_cache must share one of float16/bfloat16/float32")
+        n, Hq, d = q.shape
+        Hkv, cap, dk = k_cache.shape
+        if v_cache.shape != k_cache.shape or dk != d:
+            raise ValueError("k_cache and v_cache must be [Hkv, capacity, head_dim]")
+        for t, nm in ((q, "q"), (k_cache, "k_cache"), (v_cache, "v_cache")):
+            if t.stride(-1) != 1:
+                raise ValueError(f"{nm}: head_dim must be contiguous")
+        if k_cache.stride() != v_cache.stride():
+            raise ValueError("k_cache and v_cache must share strides")
+        if out is None:
+            out = torch.empty_like(q)
+        p = AttentionParams()
+        p.n_tree, p.prefix_len, p.num_q_heads, p.num_kv_heads, p.head_dim = n, prefix_len, Hq, Hkv, d
+        p.dtype, p.softmax_scale = _DTYPES[q.dtype], softmax_scale
+        p.q, p.q_stride_tok, p.q_stride_head = _dev(q, "q"), q.stride(0), q.stride(1)
+        p.k_cache, p.v_cache = _dev(k_cache, "k_cache"), _dev(v_cache, "v_cache")
+        p.kv_stride_tok, p.kv_stride_head, p.kv_capacity = k_cache.stride(1), k_cache.stride(0), cap
+        p.mask_bits, p.mask_words_per_row = _dev(mask_bits, "mask_bits", torch.int32), mask_bits.shape[1]
+        p.out, p.o_stride_tok, p.o_stride_head = _dev(out, "out", q.dtype), out.stride(0), out.stride(1)
+        p.lse = _dev(lse, "lse", torch.float32)
+        p.dev_status = _dev(dev_status, "dev_status", torch.int32)
+        p.kernel = kernel
+        need = load().seq_tree_attention_workspace_bytes(C.byref(p))
+        if workspace is None and need:
+            workspace = torch.empty(need, dtype=torch.uint8, device=q.device)
+        p.workspace = _dev(workspace, "workspace") if workspace is not None else None
+        p.workspace_bytes = workspace.numel() * workspace.element_size() if workspace is not None else 0
+        self.params, self.out, self.lse, self.workspace_bytes_needed = p, out, lse, need
+        self._keep = (q, k_cache, v_cache, mask_bits, out, lse, workspace, dev_status)
+
+    def run(self, stream=None):
+        _check("seq_tree_attention", load().seq_tree_attention(C.byref(self.params), _stream(stream)))
+        return self.out
+
+
+def seq_tree_attention(q, k_cache, v_cache, mask_bits, prefix_len: int, **kw):
+    """Tree-masked attention of the n tree tokens; returns out [n, Hq, d] (same dtype as q)."""
+    stream = kw.pop("stream", None)
+    return AttentionCall(q, k_cache, v_cache, mask_bits, prefix_len, **kw).run(stream)
+
+
+class VerifyCall:
+    """A prepared seq_tree_verify call."""
+
+    def __init__(self, parent, tokens, target_logits, draft_logits, temperature: float, uniforms, *,
+                 path=None, path_len=None, bonus_token=None, residual_out=None, next_child_out=None,
+                 all_nodes: bool = False, dev_status=None):
+        n, V = target_logits.shape
+        dev = target_logits.device
+        if path is None:
+            path = torch.empty(n, dtype=torch.int32, device=dev)
+        if path_len is None:
+            path_len = torch.zeros(1, dtype=torch.int32, device=dev)
+        if bonus_token is None:
+            bonus_token = torch.full((1,), -1, dtype=torch.int32, device=dev)
+        if all_nodes and next_child_out is None:
+            next_child_out = torch.empty(n, dtype=torch.int32, device=dev)
+        for t, nm in ((target_logits, "target_logits"), (draft_logits, "draft_logits")):
+            if t is not None and t.stride(-1) != 1:
+                raise ValueError(f"{nm}: vocabulary dimension must be contiguous")
+        p = VerifyParams()
+        p.n_tree, p.vocab = n, V
+        p.parent, p.tokens = _dev(parent, "parent", torch.int32), _dev(tokens, "tokens", torch.int32)
+        p.target_logits, p.target_row_stride = _dev(target_logits, "target_logits", torch.float32), target_logits.stride(0)
+        p.draft_logits = _dev(draft_logits, "draft_logits", torch.float32)
+        p.draft_row_stride = draft_logits.stride(0) if draft_logits is not None else 0
+        p.temperature = temperature
+        p.uniforms = _dev(uniforms, "uniforms", torch.float32)
+        p.path, p.path_len = _dev(path, "path", torch.int32), _dev(path_len, "path_len", torch.int32)
+        p.bonus_token = _dev(bonus_token, "bonus_token", torch.int32)
+        p.residual_out = _dev(residual_out, "residual_out", torch.float32)
+        p.next_child_out = _dev(next_child_out, "next_child_out", torch.int32)
+        p.workspace, p.workspace_bytes = None, 0
+        p.dev_status = _dev(dev_status, "dev_status", torch.int32)
+        p.flags = SEQ_VERIFY_ALL_NODES if all_nodes else 0
+        self.params = p
+        self.path, self.path_len, self.bonus_token = path, path_len, bonus_token
+        self.residual_out, self.next_child_out = residual_out, next_child_out
+        self._keep = (parent, tokens, target_logits, draft_logits, uniforms, dev_status)
+
+    def run(self, stream=None):
+        _check("seq_tree_verify", load().seq_tree_verify(C.byref(self.params), _stream(stream)))
+        return self.path, self.path_len, self.bonus_token
+
+
+def seq_tree_verify(parent, tokens, target_logits, draft_logits, temperature: float, uniforms, **kw):
+    """Algorithm 2 walked from the root; returns device tensors (path [n], path_len [1], bonus_token [1])."""
+    stream = kw.pop("stream", None)
+    return VerifyCall(parent, tokens, target_logits, draft_logits, temperature, uniforms, **kw).run(stream)
+
+
+class HostStep:
+    """One whole verify step fed from pinned HOST buffers: per call it copies the step's inputs to
+    the device, builds the ancestor mask, runs attention and verification, and copies the results
+    (attention output, path, bonus token) back.  Device staging buffers are allocated once here."""
+
+    def __init__(self, q, k_cache, v_cache, parent, prefix_len, tokens, target_logits, draft_logits, temperature,
+                 uniforms, device="cuda"):
+        self.host_in = [t if t.is_pinned() else t.pin_memory()
+                        for t in (q, k_cache, v_cache, parent, tokens, target_logits, draft_logits, uniforms)]
+        self.dev_in = [torch.empty_like(t, device=device) for t in self.host_in]
+        dq, dk, dv, dparent, dtok, dtl, ddl, du = self.dev_in
+        n = parent.shape[0]
+        self.mask = torch.empty((n, (n + 31) // 32), dtype=torch.int32, device=device)
+        self.depth = torch.empty(n, dtype=torch.int32, device=device)
+        self.status = torch.zeros(1, dtype=torch.int32, device=device)
+        self.attn = AttentionCall(dq, dk, dv, self.mask, prefix_len, dev_status=self.status)
+        self.verify = VerifyCall(dparent, dtok, dtl, ddl, temperature, du, dev_status=self.status)
+        self.host_out = [torch.empty_like(self.attn.out, device="cpu").pin_memory(),
+                         torch.empty(n, dtype=torch.int32).pin_memory(),
+                         torch.empty(1, dtype=torch.int32).pin_memory(),
+                         torch.empty(1, dtype=torch.int32).pin_memory()]
+        self.h2d_bytes = sum(t.numel() * t.element_size() for t in self.host_in)
+        self.d2h_bytes = sum(t.numel() * t.element_size() for t in self.host_out)
+
+    def run(self, stream=None):
+        for h, d in zip(self.host_in, self.dev_in):
+            d.copy_(h, non_blocking=True)
+        seq_tree_mask_from_parents(self.dev_in[3], mask_bits=self.mask, depth=self.depth, dev_status=self.status,
+                                   stream=stream)
+        self.attn.run(stream)
+        self.verify.run(stream)
+        for h, d in zip(self.host_out, (self.attn.out, self.verify.path, self.verify.path_len, self.verify.bonus_token)):
+            h.copy_(d, non_blocking=True)
+        return self.host_out

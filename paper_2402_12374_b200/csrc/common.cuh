@@ -1,0 +1,86 @@
+// Shared host/device helpers of the token-tree verification library (sm_100a only).
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_fp16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "seq_tree.h"
+
+namespace seqtree {
+
+constexpr int kHeadDim = 128;
+constexpr float kLog2e = 1.4426950408889634f;
+constexpr float kLn2 = 0.6931471805599453f;
+
+#define SEQ_CUDA_OK(expr)                     \
+  do {                                        \
+    cudaError_t _e = (expr);                  \
+    if (_e != cudaSuccess) return SEQ_ERR_CUDA; \
+  } while (0)
+
+__device__ __forceinline__ void dev_flag(int32_t* dev_status, int bit) {
+  if (dev_status != nullptr) atomicOr(dev_status, bit);
+}
+
+__device__ __forceinline__ float warp_max(float v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, o));
+  return v;
+}
+__device__ __forceinline__ float warp_sum(float v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+  return v;
+}
+__device__ __forceinline__ double warp_sum(double v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+  return v;
+}
+
+template <typename T>
+__device__ __forceinline__ float to_float(T x);
+template <>
+__device__ __forceinline__ float to_float<float>(float x) { return x; }
+template <>
+__device__ __forceinline__ float to_float<__half>(__half x) { return __half2float(x); }
+template <>
+__device__ __forceinline__ float to_float<__nv_bfloat16>(__nv_bfloat16 x) { return __bfloat162float(x); }
+
+template <typename T>
+__device__ __forceinline__ T from_float(float x);
+template <>
+__device__ __forceinline__ float from_float<float>(float x) { return x; }
+template <>
+__device__ __forceinline__ __half from_float<__half>(float x) { return __float2half_rn(x); }
+template <>
+__device__ __forceinline__ __nv_bfloat16 from_float<__nv_bfloat16>(float x) { return __float2bfloat16_rn(x); }
+
+// Split-KV partial results: every attention kernel writes, per (split, query head, node),
+// an unnormalised fp32 accumulator row plus (m, l): the running maximum of the scores in the
+// log2 domain and the sum of 2^(score - m).  combine_splits() merges them.
+struct SplitLayout {
+  float* o_part;  // [splits][Hq][n][128]
+  float2* ml;     // [splits][Hq][n]
+};
+
+inline size_t split_workspace_bytes(int splits, int Hq, int n) {
+  size_t rows = (size_t)splits * Hq * n;
+  return rows * kHeadDim * sizeof(float) + rows * sizeof(float2);
+}
+inline SplitLayout split_layout(void* workspace, int splits, int Hq, int n) {
+  SplitLayout s;
+  size_t rows = (size_t)splits * Hq * n;
+  s.o_part = reinterpret_cast<float*>(workspace);
+  s.ml = reinterpret_cast<float2*>(s.o_part + rows * kHeadDim);
+  return s;
+}
+
+// attention kernels (host launchers; defined in their own .cu files)
+int launch_attention_simt(const seq_tree_attention_params& p, int splits, cudaStream_t stream);
+int simt_default_splits(const seq_tree_attention_params& p);
+int launch_combine_splits(const seq_tree_attention_params& p, int splits, cudaStream_t stream);
+
+}  // namespace seqtree

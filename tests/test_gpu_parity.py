@@ -1,0 +1,203 @@
+"""GPU parity: the CUDA path, called through the C ABI, against the fp64 oracle on the same seeded
+inputs.  Integer results bit-exact; attention within 2e-2 abs (16-bit inputs) / 1e-5 (fp32 mode);
+residual probabilities within 1e-5 abs; accepted path and bonus identical outside the band
+|u - ratio| < 1e-5."""
+import dataclasses
+
+import numpy as np
+import pytest
+import torch
+
+from oracle import oracle as O
+from paper_2402_12374_b200 import binding as B
+from paper_2402_12374_b200 import workloads as W
+from tests import gpu_util as G
+
+pytestmark = pytest.mark.gpu
+
+
+# ---------------------------------------------------------------- mask ------------------------------
+@pytest.mark.parametrize("n,seed", [(1, 0), (2, 0), (16, 1), (17, 2), (64, 3), (100, 4), (130, 5), (768, 6), (1024, 7)])
+def test_mask_bit_exact(n, seed):
+    parent = W.random_tree(n, 20, 16, np.random.default_rng(seed))
+    for p in (parent, W.chain_tree(n), W.star_tree(n)):
+        mask, depth, st = G.gpu_mask(p)
+        omask, odepth, _ = O.mask_from_parents(p)
+        assert np.array_equal(mask.cpu().numpy().view(np.uint32), omask)
+        assert np.array_equal(depth.cpu().numpy(), odepth) and int(st.item()) == 0
+
+
+def test_mask_wide_rows_forest_and_bad_parent():
+    d = G.dev()
+    parent = np.array([-1, 0, -1, 2, 9, 1, -5], np.int32)
+    st = torch.zeros(1, dtype=torch.int32, device=d)
+    mask = torch.full((7, 3), -1, dtype=torch.int32, device=d)
+    B.seq_tree_mask_from_parents(torch.from_numpy(parent).to(d), words_per_row=3, mask_bits=mask, dev_status=st)
+    omask, odepth, oflags = O.mask_from_parents(parent, words_per_row=3)
+    assert np.array_equal(mask.cpu().numpy().view(np.uint32), omask)
+    assert int(st.item()) == B.SEQ_DEV_BAD_PARENT and oflags == O.BAD_PARENT
+
+
+# ---------------------------------------------------------------- attention -------------------------
+def _cfg(name, **kw):
+    return dataclasses.replace(W.CONFIGS[name], **kw)
+
+
+@pytest.mark.parametrize("seed", range(4))
+def test_attention_tiny_config(seed):
+    G.check_attention(W.make_attention_inputs(W.CONFIGS["tiny"], seed))
+
+
+@pytest.mark.parametrize("dtype", ["fp16", "bf16", "fp32"])
+@pytest.mark.parametrize("kernel", [B.KERNEL_AUTO, B.KERNEL_CUDA_CORE])
+def test_attention_dtypes_small(dtype, kernel):
+    cfg = _cfg("tiny", num_q_heads=8, num_kv_heads=8, prefix_len=300, n_tree=40)
+    G.check_attention(W.make_attention_inputs(cfg, 1, dtype=dtype), kernel=kernel)
+
+
+def test_attention_fp32_mode_config_shapes():
+    G.check_attention(W.make_attention_inputs(W.CONFIGS["tiny"], 0, dtype="fp32"))
+    cfg = _cfg("llama2-7b", num_q_heads=8, num_kv_heads=8)  # config-2 shape, fewer heads for the oracle's sake
+    G.check_attention(W.make_attention_inputs(cfg, 0, dtype="fp32"))
+
+
+@pytest.mark.parametrize("n,L", [(1, 0), (1, 77), (5, 0), (17, 33), (100, 129), (130, 1000)])
+def test_attention_edge_sizes(n, L):
+    cfg = _cfg("tiny", num_q_heads=4, num_kv_heads=2, prefix_len=L, n_tree=n, max_depth=12)
+    for dtype in ("bf16", "fp32"):
+        G.check_attention(W.make_attention_inputs(cfg, 2, dtype=dtype))
+
+
+@pytest.mark.parametrize("tree", ["chain", "star"])
+def test_attention_chain_and_star(tree):
+    cfg = _cfg("tiny", num_q_heads=4, num_kv_heads=4, prefix_len=200, n_tree=64)
+    parent = W.chain_tree(64) if tree == "chain" else W.star_tree(64)
+    G.check_attention(W.make_attention_inputs(cfg, 3, parent=parent))
+
+
+def test_attention_gqa_and_custom_scale():
+    cfg = _cfg("tiny", num_q_heads=16, num_kv_heads=2, prefix_len=150, n_tree=48)
+    G.check_attention(W.make_attention_inputs(cfg, 4, dtype="bf16"), scale=0.05)
+
+
+def test_attention_masked_keys_contribute_exactly_zero_and_nan_tail_is_never_read():
+    cfg = _cfg("tiny", num_q_heads=4, num_kv_heads=4, prefix_len=96, n_tree=40)
+    ai = W.make_attention_inputs(cfg, 5, dtype="bf16", extra_capacity=24)  # NaN rows past L+n
+    base, lse, st = G.run_attention(ai)
+    assert st == 0 and torch.isfinite(base).all() and torch.isfinite(lse).all()
+    G.check_attention(ai)
+    # junk in every tree row that node i cannot see leaves row i bitwise unchanged
+    M, _, _ = O.mask_from_parents(ai.parent)
+    n, L = 40, 96
+    for i in (0, 7, 23, 39):
+        k2, v2 = ai.k_cache.clone(), ai.v_cache.clone()
+        for a in range(n):
+            if not (M[i, a >> 5] >> (a & 31)) & 1:
+                k2[:, L + a] = 1e4 * (-1) ** a
+                v2[:, L + a] = -1e4
+        out2, lse2, _ = G.run_attention(dataclasses.replace(ai, k_cache=k2, v_cache=v2))
+        assert torch.equal(out2[i], base[i]) and torch.equal(lse2[:, i], lse[:, i])
+
+
+def test_attention_strided_views():
+    """q/out as slices of a fused [n, Hq+2Hkv, d] projection; K/V cache with spare capacity."""
+    cfg = _cfg("tiny", num_q_heads=8, num_kv_heads=4, prefix_len=64, n_tree=20)
+    ai = W.make_attention_inputs(cfg, 6, dtype="bf16", extra_capacity=16, tail_fill=0.0)
+    d = G.dev()
+    fused = torch.zeros((20, 16, 128), dtype=torch.bfloat16, device=d)
+    fused[:, :8] = ai.q.to(d)
+    out_buf = torch.zeros((20, 12, 128), dtype=torch.bfloat16, device=d)
+    mask, _, _ = G.gpu_mask(ai.parent.numpy())
+    B.seq_tree_attention(fused[:, :8], ai.k_cache.to(d), ai.v_cache.to(d), mask, 64, out=out_buf[:, 2:10])
+    torch.cuda.synchronize()
+    ref, _, _ = O.tree_attention(ai.q, ai.k_cache, ai.v_cache, ai.parent, 64)
+    assert np.abs(out_buf[:, 2:10].double().cpu().numpy() - ref).max() < 2e-2
+    assert out_buf[:, :2].abs().sum() == 0 and out_buf[:, 10:].abs().sum() == 0
+
+
+# ---------------------------------------------------------------- verification ----------------------
+def _verify_cases(name, T, seeds, vocab=None, parent=None):
+    cfg = W.CONFIGS[name]
+    outcomes = []
+    for seed in seeds:
+        vi = W.make_verify_inputs(cfg, T, seed, vocab=vocab, parent=parent)
+        outcomes.append(G.check_verify(vi))
+    assert outcomes.count("ok") >= max(1, len(outcomes) - 1), outcomes
+    return outcomes
+
+
+def test_verify_tiny_config():
+    _verify_cases("tiny", 0.6, range(8))
+
+
+@pytest.mark.parametrize("T", [0.0, 0.6, 1.0])
+def test_verify_llama2_7b_config(T):
+    _verify_cases("llama2-7b", T, range(4))
+
+
+def test_verify_llama2_13b_config():
+    _verify_cases("llama2-13b", 1.0, range(2))
+
+
+def test_verify_vicuna_33b_config():
+    _verify_cases("vicuna-33b", 0.6, range(2))
+
+
+@pytest.mark.parametrize("V", [1, 2, 7, 8, 33, 1000, 4099, 50257])
+def test_verify_ragged_vocab_sizes(V):
+    cfg = _cfg("tiny", n_tree=min(12, V + 1), max_fanout=max(1, min(3, V)))
+    for seed in range(3):
+        G.check_verify(W.make_verify_inputs(cfg, 0.8, seed, vocab=V))
+
+
+@pytest.mark.parametrize("T", [0.0, 0.6])
+def test_verify_every_node_hook(T):
+    vi = W.make_verify_inputs(W.CONFIGS["llama2-13b"], T, 0, vocab=8192)
+    checked, excluded = G.check_verify_all_nodes(vi)
+    assert checked >= 20 and excluded <= 2
+
+
+def test_verify_chain_star_single_node():
+    cfg = W.CONFIGS["tiny"]
+    for parent in (W.chain_tree(24), W.star_tree(24), np.array([-1], np.int32)):
+        for seed in range(3):
+            G.check_verify(W.make_verify_inputs(cfg, 0.7, seed, parent=parent, vocab=3000))
+
+
+def test_verify_uniform_fallback_duplicates_and_bad_tokens():
+    """A node with more children than the draft's support (-inf draft logits) drives the uniform
+    fallback; a duplicated sibling token and an out-of-range token take their documented paths."""
+    rng = np.random.default_rng(0)
+    V, n = 64, 12
+    parent = W.star_tree(n)
+    for trial in range(20):
+        tl = (2 * rng.standard_normal((n, V))).astype(np.float32)
+        dl = np.full((n, V), -np.inf, np.float32)
+        supp = rng.choice(V, 4, replace=False)
+        dl[:, supp] = tl[:, supp] + rng.standard_normal((n, 4)).astype(np.float32)
+        tokens = W.draw_children_tokens(parent, dl, 0.9, rng)
+        u = (0.9 + 0.1 * rng.random(n + 1)).astype(np.float32)  # large uniforms: many rejections
+        u[-1] = rng.random()
+        vi = W.VerifyInputs(torch.from_numpy(parent), torch.from_numpy(tokens), torch.from_numpy(tl),
+                            torch.from_numpy(dl), torch.from_numpy(u), 0.9)
+        G.check_verify(vi)
+    # duplicate sibling + bad token
+    tokens = W.draw_children_tokens(parent, tl, 0.9, rng)
+    tokens[3] = tokens[1]
+    tokens[5] = V + 3
+    tokens[6] = -1
+    u = np.full(n + 1, 0.999, np.float32)
+    vi = W.VerifyInputs(torch.from_numpy(parent), torch.from_numpy(tokens), torch.from_numpy(tl),
+                        torch.from_numpy((tl + 1).astype(np.float32)), torch.from_numpy(u), 0.9)
+    got = G.run_verify(vi)
+    ref = O.tree_verify(parent, tokens, tl, (tl + 1).astype(np.float32), 0.9, u)
+    assert got["status"] == B.SEQ_DEV_BAD_TOKEN and ref["flags"] == O.BAD_TOKEN
+    assert got["path"].tolist() == ref["path"].tolist() and got["bonus"] == ref["bonus"]
+    assert np.abs(got["residual"] - ref["residual"]).max() < 1e-5
+
+
+def test_verify_nonfinite_logits_are_flagged_not_trapped():
+    vi = W.make_verify_inputs(W.CONFIGS["tiny"], 0.6, 0, vocab=512)
+    vi.target_logits[0, 5] = float("nan")
+    got = G.run_verify(vi)
+    assert got["status"] & B.SEQ_DEV_NONFINITE and 0 <= got["bonus"] < 512 and got["path_len"] >= 1
