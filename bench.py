@@ -1,0 +1,361 @@
+#!/usr/bin/env python
+"""Benchmark of the token-tree verify step (ancestor mask -> tree attention -> Algorithm 2 walk).
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload NAME] [--temperature T]
+    python bench.py --impl reference ...      # the fp64 CPU oracle on the host cores, same metric
+
+One "step" is one pass of the whole hot path over one synthetic request.  The K timed steps are
+captured in one CUDA graph and replayed between two CUDA events; inputs rotate over enough
+independent copies that every step reads memory that is not in L2.  One JSON line is printed by
+rank 0.  With N > 1 (torchrun) every rank verifies its own requests (weak scaling, no data-path
+collective) and the time is the maximum over ranks.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import math
+import os
+import statistics
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import numpy as np
+import torch
+
+from paper_2402_12374_b200 import workloads as W
+
+METRIC = "us_per_tree_verify_step"
+UNIT = "us/step"
+L2_BYTES = 126 * 1024 * 1024
+
+# DRAM traffic per launch (dram__bytes_read.sum + dram__bytes_write.sum) of the attention kernel, from
+# the ncu captures summarised under profiles/; None where no capture exists for that workload.
+NCU_TRAFFIC_BYTES = {}
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        d = json.load(open(path))
+        return dict(hbm_gbs=d["hbm_gbs"], bf16_tflops=d["bf16_tflops"], source="measured")
+    return dict(hbm_gbs=6650.0, bf16_tflops=1590.0, source="fallback")
+
+
+class ClockSampler:
+    """Samples SM clock and throttle reasons through NVML (read-only) while the timed region runs."""
+
+    def __init__(self, index: int, period_s: float = 0.002):
+        self.samples, self.reasons, self.max_mhz = [], set(), None
+        self._stop = threading.Event()
+        self._thread = None
+        try:
+            import pynvml
+
+            pynvml.nvmlInit()
+            self.nv = pynvml
+            self.h = pynvml.nvmlDeviceGetHandleByIndex(index)
+            self.max_mhz = pynvml.nvmlDeviceGetMaxClockInfo(self.h, pynvml.NVML_CLOCK_SM)
+        except Exception:  # NVML missing: report nulls rather than fail the run
+            self.nv = None
+        self.period = period_s
+
+    def _loop(self):
+        nv = self.nv
+        names = {
+            "hw_slowdown": nv.nvmlClocksEventReasonHwSlowdown if hasattr(nv, "nvmlClocksEventReasonHwSlowdown") else 0x8,
+            "hw_thermal_slowdown": 0x40, "sw_thermal_slowdown": 0x20, "sw_power_cap": 0x4, "hw_power_brake": 0x80,
+        }
+        while not self._stop.is_set():
+            try:
+                self.samples.append(nv.nvmlDeviceGetClockInfo(self.h, nv.NVML_CLOCK_SM))
+                try:
+                    r = nv.nvmlDeviceGetCurrentClocksEventReasons(self.h)
+                except Exception:
+                    r = nv.nvmlDeviceGetCurrentClocksThrottleReasons(self.h)
+                for k, bit in names.items():
+                    if r & bit:
+                        self.reasons.add(k)
+            except Exception:
+                pass
+            time.sleep(self.period)
+
+    def __enter__(self):
+        if self.nv is not None:
+            self._thread = threading.Thread(target=self._loop, daemon=True)
+            self._thread.start()
+        return self
+
+    def __exit__(self, *exc):
+        self._stop.set()
+        if self._thread is not None:
+            self._thread.join()
+
+    def summary(self):
+        return {"sm_mhz": statistics.median(self.samples) if self.samples else None, "sm_max_mhz": self.max_mhz,
+                "reasons": sorted(self.reasons), "samples": len(self.samples)}
+
+
+def n_sets(bytes_per_set: int, lo: int = 2, hi: int = 48) -> int:
+    return max(lo, min(hi, math.ceil(3 * L2_BYTES / max(1, bytes_per_set))))
+
+
+def build_requests(cfg, T, rank, n_attn, n_verify):
+    """Host-side inputs for this rank: n_attn attention sets and n_verify logit sets (seeds differ by rank)."""
+    base = 1000 * rank
+    parent = W.make_tree(cfg, base)
+    attn = [W.make_attention_inputs(cfg, base + s, parent=parent) for s in range(n_attn)]
+    ver = [W.make_verify_inputs(cfg, T, base + s, parent=parent) for s in range(n_verify)]
+    return parent, attn, ver
+
+
+def oracle_step_sample(cfg, parent, ai, vi, T, budget_flops=1.5e9):
+    """Times the oracle on one step, attention restricted to a leading block of nodes (closed under
+    'parent') when the whole tree would take too long; returns (seconds scaled to a full step, note)."""
+    from oracle import oracle as O
+
+    n = len(parent)
+    L = cfg.prefix_len
+    per_node = 4.0 * cfg.head_dim * cfg.num_q_heads * (L + 8)
+    m = int(max(1, min(n, budget_flops // per_node)))
+    t0 = time.perf_counter()
+    O.tree_attention(ai.q[:m], ai.k_cache[:, : L + m], ai.v_cache[:, : L + m], parent[:m], L)
+    t_attn = (time.perf_counter() - t0) * (n / m)
+    t0 = time.perf_counter()
+    O.mask_from_parents(parent)
+    O.tree_verify(vi.parent, vi.tokens, vi.target_logits, vi.draft_logits, T, vi.uniforms)
+    t_ver = time.perf_counter() - t0
+    note = (f"1 step: mask + Algorithm 2 walk in full, attention on the first {m} of {n} nodes "
+            f"(time scaled by {n}/{m}), fp64, gcc -O2 -fopenmp")
+    return t_attn + t_ver, note
+
+
+def run_reference(args, cfg, T):
+    """--impl reference: the oracle, as it stands, on the host cores."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    from oracle import oracle as O
+
+    parent, attn, ver = build_requests(cfg, T, 0, 1, 1)
+    for _ in range(min(args.warmup, 2)):
+        oracle_step_sample(cfg, parent, attn[0], ver[0], T)
+    steps = min(args.steps, 20)
+    times, note = [], ""
+    for _ in range(steps):
+        t, note = oracle_step_sample(cfg, parent, attn[0], ver[0], T)
+        times.append(t)
+    us = 1e6 * sum(times) / len(times)
+    cores = O.num_threads()
+    line = {
+        "impl": "reference", "metric": METRIC, "value": us, "unit": UNIT, "n_gpus": args.gpus, "steps": steps,
+        "warmup": min(args.warmup, 2), "ms_per_step": us / 1e3, "higher_is_better": False, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": cfg.name, "temperature": T},
+        "cpu_baseline": {"value": us, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": note},
+        "e2e": {"value": us, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line), flush=True)
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=500)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="llama2-7b", choices=sorted(W.CONFIGS))
+    ap.add_argument("--temperature", type=float, default=0.6)
+    ap.add_argument("--kernel", type=int, default=0, help="0 auto, 1 CUDA-core, 2 tensor-core attention")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    cfg = W.CONFIGS[args.workload]
+    T = args.temperature
+    if args.impl == "reference":
+        run_reference(args, cfg, T)
+        return
+
+    from paper_2402_12374_b200 import binding as B
+
+    B.load()  # fails loudly if the CUDA library is missing: there is no fallback
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    if not torch.cuda.is_available():
+        raise RuntimeError("bench.py needs a CUDA device")
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    if world > 1:
+        import torch.distributed as dist
+
+        dist.init_process_group("nccl", device_id=dev)
+    K, Wm = args.steps, max(3, args.warmup)
+
+    attn_bytes = W.attention_algorithmic_bytes(cfg)
+    n = cfg.n_tree
+    logits_bytes_touched = 4 * 2 * cfg.vocab * 4  # a walk reads a few rows of each matrix
+    na = n_sets(attn_bytes)
+    nv = min(n_sets(logits_bytes_touched), 8 if cfg.vocab * n * 8 < (1 << 28) else 3)
+    parent, attn_h, ver_h = build_requests(cfg, T, rank, na, nv)
+
+    status = torch.zeros(1, dtype=torch.int32, device=dev)
+    parent_d = torch.from_numpy(parent).to(dev)
+    mask = torch.empty((n, (n + 31) // 32), dtype=torch.int32, device=dev)
+    depth = torch.empty(n, dtype=torch.int32, device=dev)
+    attn_calls, ver_calls = [], []
+    workspace = None
+    for ai in attn_h:
+        call = B.AttentionCall(ai.q.to(dev), ai.k_cache.to(dev), ai.v_cache.to(dev), mask, cfg.prefix_len,
+                               workspace=workspace, dev_status=status, kernel=args.kernel)
+        workspace = call._keep[6]
+        attn_calls.append(call)
+    for vi in ver_h:
+        ver_calls.append(B.VerifyCall(parent_d, vi.tokens.to(dev), vi.target_logits.to(dev), vi.draft_logits.to(dev),
+                                      T, vi.uniforms.to(dev), dev_status=status))
+    launches_per_step = 1 + (2 if attn_calls[0].workspace_bytes_needed else 1) + 1
+
+    stream = torch.cuda.Stream(device=dev)
+
+    def step(i, s, ev=None):
+        B.seq_tree_mask_from_parents(parent_d, mask_bits=mask, depth=depth, dev_status=status, stream=s)
+        if ev:
+            ev[0].record(s)
+        attn_calls[i % na].run(s)
+        if ev:
+            ev[1].record(s)
+        ver_calls[i % nv].run(s)
+        if ev:
+            ev[2].record(s)
+
+    with torch.cuda.stream(stream):
+        for i in range(Wm):
+            step(i, stream)
+        stream.synchronize()
+        # graph A: the K timed steps, nothing else
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph, stream=stream):
+            for i in range(K):
+                step(Wm + i, stream)
+        # graph B: the same K steps with event nodes around the kernels (per-kernel durations)
+        Kb = min(K, 200)
+        evs = [[torch.cuda.Event(enable_timing=True, external=True) for _ in range(3)] for _ in range(Kb)]
+        graph_b = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph_b, stream=stream):
+            for i in range(Kb):
+                step(Wm + i, stream, evs[i])
+        graph.replay()  # untimed replay: uploads the graph
+        graph_b.replay()
+        stream.synchronize()
+
+        def barrier():
+            torch.cuda.synchronize()
+            if world > 1:
+                dist.barrier()
+            torch.cuda.synchronize()
+
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        barrier()
+        with ClockSampler(local_rank) as clocks:
+            e0.record(stream)
+            graph.replay()
+            e1.record(stream)
+            stream.synchronize()
+            # keep sampling over a few more replays so that short regions still see clocks under load
+            t_end = time.time() + 0.25
+            while time.time() < t_end:
+                graph.replay()
+                stream.synchronize()
+        barrier()
+        ms_total = e0.elapsed_time(e1)
+        graph_b.replay()
+        stream.synchronize()
+        t_attn = [evs[i][0].elapsed_time(evs[i][1]) * 1e3 for i in range(Kb)]
+        t_ver = [evs[i][1].elapsed_time(evs[i][2]) * 1e3 for i in range(Kb)]
+
+    if int(status.item()) != 0:
+        raise RuntimeError(f"dev_status = {int(status.item())} after the timed region")
+    if world > 1:
+        t = torch.tensor([ms_total], dtype=torch.float64, device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms_total = float(t.item())
+    ms_per_step = ms_total / K
+    value_us = 1e3 * ms_per_step / world  # whole job: N requests verified per step time
+
+    # end to end from pinned host buffers through the public API, copies inside the timed region
+    host = B.HostStep(attn_h[0].q, attn_h[0].k_cache, attn_h[0].v_cache, torch.from_numpy(parent), cfg.prefix_len,
+                      ver_h[0].tokens, ver_h[0].target_logits, ver_h[0].draft_logits, T, ver_h[0].uniforms, device=dev)
+    Ke = min(K, 20)
+    with torch.cuda.stream(stream):
+        for _ in range(3):
+            host.run(stream)
+            stream.synchronize()
+        torch.cuda.synchronize()
+        t0 = time.perf_counter()
+        for _ in range(Ke):
+            host.run(stream)
+            stream.synchronize()
+        e2e_us = 1e6 * (time.perf_counter() - t0) / Ke
+    if world > 1:
+        t = torch.tensor([e2e_us], dtype=torch.float64, device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        e2e_us = float(t.item()) / world
+
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return
+
+    peaks = measured_peaks()
+    attn_us = statistics.mean(t_attn)
+    ver_us = statistics.mean(t_ver)
+    flops = W.attention_algorithmic_flops(cfg, parent)
+    hbm_time = attn_bytes / (peaks["hbm_gbs"] * 1e9)
+    tensor_time = flops / (peaks["bf16_tflops"] * 1e12)
+    if hbm_time >= tensor_time:
+        achieved = attn_bytes / (attn_us * 1e-6) / 1e9
+        roofline = {"bound": "hbm", "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                    "frac": achieved / peaks["hbm_gbs"]}
+    else:
+        achieved = flops / (attn_us * 1e-6) / 1e12
+        roofline = {"bound": "tensor", "achieved": achieved, "peak": peaks["bf16_tflops"], "unit": "TFLOP/s",
+                    "frac": achieved / peaks["bf16_tflops"]}
+    roofline.update({
+        "traffic": NCU_TRAFFIC_BYTES.get(cfg.name), "kernel": "seq_tree_attention", "us_per_launch": attn_us,
+        "algorithmic_bytes": attn_bytes, "algorithmic_flops": flops, "peak_source": f"of {peaks['source']}",
+        "timing": f"CUDA events around each call in a replay of the same steps ({Kb} of them), mean",
+    })
+
+    line = {
+        "metric": METRIC, "value": value_us, "unit": UNIT, "n_gpus": world, "steps": K, "warmup": Wm,
+        "ms_per_step": ms_per_step, "higher_is_better": False, "scaling": "weak", "vs_baseline": None,
+        "dtype": cfg.dtype, "data": "synthetic",
+        "config": {"workload": cfg.name, "temperature": T, "n_tree": n, "prefix_len": cfg.prefix_len,
+                   "heads": f"{cfg.num_q_heads}/{cfg.num_kv_heads}", "vocab": cfg.vocab, "requests_per_gpu": 1,
+                   "l2": f"inputs rotate over {na} attention sets ({na * attn_bytes >> 20} MiB) and {nv} logit sets, "
+                         f"larger than the 126 MiB L2", "launch": "CUDA graph of the K steps"},
+        "clocks": clocks.summary(),
+        "e2e": {"value": e2e_us, "unit": UNIT, "h2d_bytes_per_step": host.h2d_bytes, "d2h_bytes_per_step": host.d2h_bytes,
+                "steps": Ke},
+        "gpu_launches": K * launches_per_step,
+        "roofline": roofline,
+        "breakdown_us": {"attention": attn_us, "verify": ver_us,
+                         "verify_bytes_visited_rows_x2": None},
+    }
+    if not args.no_cpu_baseline:
+        from oracle import oracle as O
+
+        t, note = oracle_step_sample(cfg, parent, attn_h[0], ver_h[0], T)
+        line["cpu_baseline"] = {"value": 1e6 * t, "unit": UNIT, "cores": O.num_threads(), "kind": "oracle", "sample": note}
+    print(json.dumps(line), flush=True)
+    if world > 1:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

@@ -181,17 +181,19 @@ def test_verify_uniform_fallback_duplicates_and_bad_tokens():
         vi = W.VerifyInputs(torch.from_numpy(parent), torch.from_numpy(tokens), torch.from_numpy(tl),
                             torch.from_numpy(dl), torch.from_numpy(u), 0.9)
         G.check_verify(vi)
-    # duplicate sibling + bad token
-    tokens = W.draw_children_tokens(parent, tl, 0.9, rng)
-    tokens[3] = tokens[1]
-    tokens[5] = V + 3
-    tokens[6] = -1
+    # bad tokens first (always reached), then a duplicated sibling
+    dl = (tl + 2 * rng.standard_normal((n, V))).astype(np.float32)
+    tokens = W.draw_children_tokens(parent, dl, 0.9, rng)
+    tokens[1] = V + 3
+    tokens[2] = -1
+    tokens[4] = tokens[3]
     u = np.full(n + 1, 0.999, np.float32)
     vi = W.VerifyInputs(torch.from_numpy(parent), torch.from_numpy(tokens), torch.from_numpy(tl),
-                        torch.from_numpy((tl + 1).astype(np.float32)), torch.from_numpy(u), 0.9)
+                        torch.from_numpy(dl), torch.from_numpy(u), 0.9)
     got = G.run_verify(vi)
-    ref = O.tree_verify(parent, tokens, tl, (tl + 1).astype(np.float32), 0.9, u)
+    ref = O.tree_verify(parent, tokens, tl, dl, 0.9, u)
     assert got["status"] == B.SEQ_DEV_BAD_TOKEN and ref["flags"] == O.BAD_TOKEN
+    assert ref["min_gap"] > 1e-5 and ref["ratio"][4] == 0.0  # the duplicate was tested and had ratio 0
     assert got["path"].tolist() == ref["path"].tolist() and got["bonus"] == ref["bonus"]
     assert np.abs(got["residual"] - ref["residual"]).max() < 1e-5
 
