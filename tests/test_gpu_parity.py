@@ -203,3 +203,71 @@ def test_verify_nonfinite_logits_are_flagged_not_trapped():
     vi.target_logits[0, 5] = float("nan")
     got = G.run_verify(vi)
     assert got["status"] & B.SEQ_DEV_NONFINITE and 0 <= got["bonus"] < 512 and got["path_len"] >= 1
+
+
+# ---------------------------------------------------------------- tensor-core attention kernel ------
+@pytest.mark.parametrize("dtype", ["fp16", "bf16"])
+@pytest.mark.parametrize("n,L,Hq,Hkv", [(1, 0, 2, 2), (1, 77, 2, 1), (5, 0, 4, 2), (17, 33, 4, 4), (64, 128, 2, 2),
+                                        (100, 129, 8, 2), (130, 1000, 4, 4), (257, 5, 16, 1), (40, 300, 128, 1)])
+def test_tensor_core_attention_edge_sizes(dtype, n, L, Hq, Hkv):
+    cfg = _cfg("tiny", num_q_heads=Hq, num_kv_heads=Hkv, prefix_len=L, n_tree=n, max_depth=12)
+    G.check_attention(W.make_attention_inputs(cfg, 7, dtype=dtype), kernel=B.KERNEL_TENSOR_CORE)
+
+
+@pytest.mark.parametrize("tree", ["chain", "star"])
+def test_tensor_core_attention_chain_and_star(tree):
+    cfg = _cfg("tiny", num_q_heads=4, num_kv_heads=2, prefix_len=200, n_tree=160)
+    parent = W.chain_tree(160) if tree == "chain" else W.star_tree(160)
+    G.check_attention(W.make_attention_inputs(cfg, 3, parent=parent, dtype="bf16"), kernel=B.KERNEL_TENSOR_CORE)
+
+
+def test_tensor_core_attention_masked_keys_are_exactly_zero_and_nan_tail_is_never_read():
+    cfg = _cfg("tiny", num_q_heads=4, num_kv_heads=2, prefix_len=96, n_tree=150, max_depth=12)
+    ai = W.make_attention_inputs(cfg, 5, dtype="bf16", extra_capacity=200)  # NaN rows past L+n
+    base, lse, st = G.run_attention(ai, kernel=B.KERNEL_TENSOR_CORE)
+    assert st == 0 and torch.isfinite(base).all() and torch.isfinite(lse).all()
+    G.check_attention(ai, kernel=B.KERNEL_TENSOR_CORE)
+    M, _, _ = O.mask_from_parents(ai.parent)
+    n, L = 150, 96
+    for i in (0, 31, 77, 149):
+        k2, v2 = ai.k_cache.clone(), ai.v_cache.clone()
+        for a in range(n):
+            if not (M[i, a >> 5] >> (a & 31)) & 1:
+                k2[:, L + a] = 1e4 * (-1) ** a
+                v2[:, L + a] = -1e4
+        out2, lse2, _ = G.run_attention(dataclasses.replace(ai, k_cache=k2, v_cache=v2), kernel=B.KERNEL_TENSOR_CORE)
+        assert torch.equal(out2[i], base[i]) and torch.equal(lse2[:, i], lse[:, i])
+
+
+def test_tensor_core_attention_garbage_in_unused_mask_words_is_ignored():
+    cfg = _cfg("tiny", num_q_heads=2, num_kv_heads=2, prefix_len=50, n_tree=70)
+    ai = W.make_attention_inputs(cfg, 8, dtype="bf16", extra_capacity=64, tail_fill=1.0)
+    d = G.dev()
+    mask, _, _ = G.gpu_mask(ai.parent.numpy())
+    wide = torch.full((70, 6), -1, dtype=torch.int32, device=d)  # all-ones beyond the 3 live words
+    wide[:, :3] = mask
+    wide[:, 2] |= torch.tensor(-(1 << 6), dtype=torch.int32, device=d)  # bits 70..95 set too
+    for kernel in (B.KERNEL_TENSOR_CORE, B.KERNEL_CUDA_CORE):
+        out = B.seq_tree_attention(ai.q.to(d), ai.k_cache.to(d), ai.v_cache.to(d), wide, 50, kernel=kernel)
+        torch.cuda.synchronize()
+        ref, _, _ = O.tree_attention(ai.q, ai.k_cache, ai.v_cache, ai.parent, 50)
+        assert np.abs(out.double().cpu().numpy() - ref).max() < 2e-2
+
+
+def test_tensor_core_attention_large_magnitude_scores_rescale_path():
+    """Scores that grow block after block force the accumulator rescale in tensor memory."""
+    cfg = _cfg("tiny", num_q_heads=2, num_kv_heads=2, prefix_len=700, n_tree=64)
+    ai = W.make_attention_inputs(cfg, 9, dtype="bf16")
+    ramp = torch.linspace(0.2, 6.0, 764).view(1, -1, 1)
+    k = (ai.k_cache.float() * ramp).to(torch.bfloat16)
+    G.check_attention(dataclasses.replace(ai, k_cache=k), kernel=B.KERNEL_TENSOR_CORE)
+
+
+@pytest.mark.parametrize("name,rows", [("llama2-7b", [0, 1, 13, 40, 63]), ("llama2-13b", [0, 5, 64, 127]),
+                                       ("vicuna-33b", [0, 100, 128, 255]), ("llama3-70b", [0, 31, 32, 400, 767])])
+def test_attention_full_size_configs_sampled_rows(name, rows):
+    """BASELINE sizes in the launch configuration the benchmark times; the oracle recomputes the
+    sampled nodes (and their ancestors) one by one."""
+    cfg = W.CONFIGS[name]
+    ai = W.make_attention_inputs(cfg, 0)
+    G.check_attention(ai, rows=rows)
