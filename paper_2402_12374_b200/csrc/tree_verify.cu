@@ -2,11 +2,13 @@
 // cluster, plus the final draw x ~ R.
 //
 // Schedule.  One cluster of 8 CTAs follows the walk.  At each visited node the two logit rows
-// are cut into 8 contiguous vocabulary slices, one per CTA, read from HBM once and kept in shared
-// memory as unnormalised exponentials; everything that is vocabulary-wide (max, sums, the
-// residual's normaliser, the inverse CDF) is a block reduction followed by one exchange over
-// distributed shared memory.  The walk's scalar state is replicated: every CTA derives it from
-// the same exchanged numbers with the same instructions, so all CTAs take the same branches.
+// are cut into 8 contiguous vocabulary slices, one per CTA, brought from HBM once by bulk
+// asynchronous copies and kept in shared memory as unnormalised exponentials.  Everything that is
+// vocabulary-wide (max, sums, the residual's normaliser, the inverse CDF) is a block reduction
+// followed by one exchange over distributed shared memory.  The walk's scalar state is replicated:
+// every CTA derives it from the same exchanged numbers with the same instructions, so all CTAs take
+// the same branches.  While a node is processed, the rows of its children are prefetched into L2.
+// Per visited node there is one cluster barrier (softmax statistics), per rejection one more.
 //
 // Arithmetic.  R and D of Algorithm 2 are never materialised.  With p, q the two softmaxes and S
 // the rejected set (their entries zeroed in shared memory when rejected), the state after any
@@ -16,6 +18,10 @@
 // for scalars C, U, Z, ZD: line 9's  R <- norm(max(R - D, 0))  becomes  C += Z/ZD  (or
 // U += Z/(V-|S|) after the fallback) followed by one vocabulary-wide sum for the new Z, and
 // line 12's sum(D) is the direct sum ZD of the surviving q, never a subtraction.
+//
+// Each warp owns a contiguous segment of its CTA's slice and keeps its exponentials relative to
+// the segment's own maximum (no block-wide maximum is needed); the per-warp sums of the last pass
+// are exactly the coarse levels of the final inverse CDF.
 #include <cooperative_groups.h>
 #include <float.h>
 #include <math.h>
@@ -26,10 +32,29 @@ namespace cg = cooperative_groups;
 
 namespace seqtree {
 
-constexpr int kVThreads = 512;
+#ifdef SEQ_TRACE
+__device__ unsigned long long g_trace[512];
+__device__ int g_trace_n;
+__shared__ int s_trace_i;
+#define TRACE(tag)                                                        \
+  do {                                                                    \
+    if (blockIdx.x == 0 && threadIdx.x == 0) {                            \
+      if ((tag) == 0) s_trace_i = 0;                                      \
+      int _i = s_trace_i++;                                               \
+      if (_i < 256) { g_trace[2 * _i] = (tag); g_trace[2 * _i + 1] = clock64(); g_trace_n = _i + 1; } \
+    }                                                                     \
+  } while (0)
+#else
+#define TRACE(tag) do { } while (0)
+#endif
+
+constexpr int kVThreads = 256;
 constexpr int kVWarps = kVThreads / 32;
 constexpr int kVCluster = 8;
-constexpr int kVStaticSmem = 24 * 1024;  // upper bound of the kernel's static shared memory
+constexpr int kVParts = kVCluster * kVWarps;  // 64 (rank, warp) segments cover the vocabulary
+constexpr uint32_t kVSpinLimit = 1u << 22;
+constexpr int kPrefetchChildren = 4;          // rows of the first few children are prefetched into L2
+static_assert(kVParts == 64, "the exchange reads two entries per lane");
 
 struct VerifyArgs {
   int32_t n, V, slice_cap, flags;
@@ -47,94 +72,94 @@ struct VShared {
   int32_t tokens[SEQ_MAX_TREE];
   float uniforms[SEQ_MAX_TREE + 1];
   int32_t kids[SEQ_MAX_TREE];
-  double xbuf[2][kVCluster][4];   // cluster exchange slots, double-buffered
-  double wbuf[2][kVWarps][4];     // block reduction slots, double-buffered
+  // (target exp, draft exp, target segment max, draft segment max) of each child's token, written by
+  // the warp that owns the token into every CTA; double-buffered by node so that a CTA that runs
+  // ahead never overwrites what a sibling still reads
+  float4 kid_pq[2][SEQ_MAX_TREE];
+  uint8_t dup[SEQ_MAX_TREE];            // child i carries the token of an earlier sibling
+  uint32_t has_child[SEQ_MAX_TREE / 32];
+  float4 xbuf[2][kVParts];              // cluster exchange: one entry per (rank, warp), double-buffered
   int32_t wcnt[kVWarps];
-  int32_t misc[4];
+  uint64_t bar[2];                      // completion of the target / draft slice copies
 };
 
 // Per-thread copy of the replicated walk state at the current node.
 struct NodeState {
-  float ip, iq;       // this CTA's factors turning stored exponentials into probabilities
-  float mlp[kVCluster], ipr[kVCluster], mlq[kVCluster], iqr[kVCluster];
+  float c2;             // log2(e)/T
+  float Mp, Mq;         // global maxima of the two rows
+  float invSp, invSq;   // 1 / sum of exponentials relative to the global maxima
+  float ipw, iqw;       // this warp's factors turning its stored exponentials into probabilities
   double C, U, Z, ZD;
-  int mode;           // 0: D proportional to q; 1: uniform over the non-rejected set
-  int nS;             // |S|
+  double part_sum[2];   // residual mass of segments `lane` and `lane + 32` (probability units)
+  int mode;             // 0: D proportional to q; 1: uniform over the non-rejected set
+  int nS;               // |S|
+  int has_q;            // qs holds this node's draft slice
   int greedy_token;
 };
 
 struct Ctx {
   VShared* sh;
   float* ps; float* qs;
-  int rank, lo, cnt;
-  int wpar, xpar;
+  int rank, lo, cnt, seg, s_lo, s_hi;  // slice, and this warp's segment of it
+  int xpar, npar;
+  uint32_t ph[2];
   int tid, warp, lane;
 };
 
+__device__ __forceinline__ uint32_t vsmem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
 __device__ __forceinline__ float sanitize_logit(float x, int32_t* dev_status) {
-  if (x != x) { dev_flag(dev_status, SEQ_DEV_NONFINITE); return -INFINITY; }
-  if (x == INFINITY) { dev_flag(dev_status, SEQ_DEV_NONFINITE); return FLT_MAX; }
-  return x;
+  if (x < INFINITY) return x;  // finite or -inf
+  dev_flag(dev_status, SEQ_DEV_NONFINITE);
+  return x != x ? -INFINITY : FLT_MAX;
 }
-// exponential of one logit relative to its slice maximum (c2 = log2(e)/T)
-__device__ __forceinline__ float slice_exp(float x, float mloc, float c2) {
-  return mloc == -INFINITY ? 0.f : exp2f((x - mloc) * c2);
+// 2^((m - M) c2), and 0 for an empty (all -inf) part
+__device__ __forceinline__ float rel_exp(float m, float M, float c2) {
+  return m == -INFINITY ? 0.f : exp2f((m - M) * c2);
 }
 // unnormalised residual max(p - C q - U, 0) of one token
 __device__ __forceinline__ float resid(float pn, float qn, float Cf, float Uf) {
   return fmaxf(fmaf(-Cf, qn, pn) - Uf, 0.f);
 }
 
-template <int K, bool kMax>
-__device__ __forceinline__ void block_allreduce(Ctx& c, double (&v)[K]) {
-#pragma unroll
-  for (int k = 0; k < K; ++k) {
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) {
-      const double other = __shfl_xor_sync(0xffffffffu, v[k], o);
-      v[k] = kMax ? fmax(v[k], other) : v[k] + other;
-    }
-  }
-  double (*w)[4] = c.sh->wbuf[c.wpar];
-  if (c.lane == 0) {
-#pragma unroll
-    for (int k = 0; k < K; ++k) w[c.warp][k] = v[k];
-  }
-  __syncthreads();
-#pragma unroll
-  for (int k = 0; k < K; ++k) {
-    double acc = w[0][k];
-#pragma unroll
-    for (int ww = 1; ww < kVWarps; ++ww) acc = kMax ? fmax(acc, w[ww][k]) : acc + w[ww][k];
-    v[k] = acc;
-  }
-  c.wpar ^= 1;
+// Visit this warp's segment four elements per lane at a time (conflict-free 16-byte accesses);
+// f4(t) handles elements t..t+3, f1(t) a single element of the ragged end.
+template <typename F4, typename F1>
+__device__ __forceinline__ void sweep(const Ctx& c, F4 f4, F1 f1) {
+  int t = c.s_lo + 4 * c.lane;
+  for (; t + 131 < c.s_hi; t += 256) { f4(t); f4(t + 128); }  // two independent steps per trip
+  for (; t + 3 < c.s_hi; t += 128) f4(t);
+  for (int e = t; e < c.s_hi && e < t + 4; ++e) f1(e);
+}
+__device__ __forceinline__ float fast_ex2(float x) {  // 2^x, relative error 2^-22; 2^-inf = 0
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
 }
 
-// Every CTA publishes K doubles to every CTA of the cluster; on return out[r][k] holds rank r's.
-template <int K>
-__device__ __forceinline__ void cluster_exchange(cg::cluster_group& cluster, Ctx& c, const double (&v)[K],
-                                                 double (&out)[kVCluster][K]) {
-  if (c.tid < kVCluster) {
-    double* remote = cluster.map_shared_rank(&c.sh->xbuf[c.xpar][c.rank][0], c.tid);
-#pragma unroll
-    for (int k = 0; k < K; ++k) remote[k] = v[k];
-  }
+__device__ __forceinline__ double sum_lanes(double v, int width) {  // butterfly over `width` lanes
+  for (int o = width >> 1; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+  return v;
+}
+
+// Every warp of every CTA publishes one float4 to every CTA of the cluster.  On return e0/e1 hold the
+// entries of segments `lane` and `lane + 32` (segment index = rank * 8 + warp).  One cluster barrier.
+__device__ __forceinline__ void cluster_exchange(cg::cluster_group& cluster, Ctx& c, float4 mine, float4& e0, float4& e1) {
+  if (c.lane < kVCluster) *cluster.map_shared_rank(&c.sh->xbuf[c.xpar][c.rank * kVWarps + c.warp], c.lane) = mine;
   cluster.sync();
-#pragma unroll
-  for (int r = 0; r < kVCluster; ++r)
-#pragma unroll
-    for (int k = 0; k < K; ++k) out[r][k] = c.sh->xbuf[c.xpar][r][k];
+  e0 = c.sh->xbuf[c.xpar][c.lane];
+  e1 = c.sh->xbuf[c.xpar][c.lane + 32];
   c.xpar ^= 1;
 }
 
-// Children of v in ascending node order -> sh->kids; returns their count.
+// Children of v in ascending node order -> sh->kids; returns their count.  Two barriers.
 __device__ int build_kids(Ctx& c, int v, int n) {
-  // each thread owns two consecutive candidates so that warps and lanes are in node order
-  const int c0 = v + 1 + 2 * c.tid;
-  const bool f0 = c0 < n && c.sh->parent[c0] == v;
-  const bool f1 = c0 + 1 < n && c.sh->parent[c0 + 1] == v;
-  const int mine = (int)f0 + (int)f1;
+  // each thread owns four consecutive candidates so that warps and lanes are in node order
+  const int c0 = v + 1 + 4 * c.tid;
+  int f = 0;
+#pragma unroll
+  for (int e = 0; e < 4; ++e) f |= (int)(c0 + e < n && c.sh->parent[c0 + e] == v) << e;
+  const int mine = __popc(f);
   int incl = mine;
 #pragma unroll
   for (int o = 1; o < 32; o <<= 1) {
@@ -151,64 +176,112 @@ __device__ int build_kids(Ctx& c, int v, int n) {
     total += x;
   }
   int pos = base + incl - mine;
-  if (f0) c.sh->kids[pos++] = c0;
-  if (f1) c.sh->kids[pos] = c0 + 1;
+#pragma unroll
+  for (int e = 0; e < 4; ++e)
+    if ((f >> e) & 1) c.sh->kids[pos++] = c0 + e;
   __syncthreads();
   return total;
 }
 
-// Read this CTA's slice of one logit row into shared memory (sanitised); returns the slice max.
-__device__ float load_slice(const Ctx& c, const float* __restrict__ row, float* dst, int32_t* dev_status) {
-  float m = -INFINITY;
-  const float* src = row + c.lo;
-  const int n4 = c.cnt >> 2;
-  for (int i = c.tid; i < n4; i += kVThreads) {
-    float4 x = __ldg(reinterpret_cast<const float4*>(src) + i);
-    x.x = sanitize_logit(x.x, dev_status); x.y = sanitize_logit(x.y, dev_status);
-    x.z = sanitize_logit(x.z, dev_status); x.w = sanitize_logit(x.w, dev_status);
-    reinterpret_cast<float4*>(dst)[i] = x;
-    m = fmaxf(fmaxf(m, fmaxf(x.x, x.y)), fmaxf(x.z, x.w));
-  }
-  for (int i = (n4 << 2) + c.tid; i < c.cnt; i += kVThreads) {
-    const float x = sanitize_logit(__ldg(src + i), dev_status);
-    dst[i] = x;
-    m = fmaxf(m, x);
-  }
-  return m;
+// Start the asynchronous copy of this CTA's slice of one row into shared memory (16-byte body only).
+__device__ __forceinline__ void start_slice_copy(const Ctx& c, const float* row, float* dst, int which) {
+  const uint32_t bytes = (uint32_t)(c.cnt & ~3) * 4u;
+  if (bytes == 0) return;
+  const uint32_t bar = vsmem_u32(&c.sh->bar[which]);
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+               ::"r"(vsmem_u32(dst)), "l"(row + c.lo), "r"(bytes), "r"(bar) : "memory");
 }
+// Bounded wait for a slice copy; the ragged tail (at most 3 elements) is fetched by the warp that owns it.
+__device__ __forceinline__ void finish_slice_copy(Ctx& c, const float* row, float* dst, int which, int32_t* dev_status) {
+  if ((c.cnt & ~3) != 0) {
+    const uint32_t bar = vsmem_u32(&c.sh->bar[which]);
+    uint32_t ok = 0;
+    for (uint32_t it = 0; it < kVSpinLimit && !ok; ++it) {
+      asm volatile(
+          "{\n\t.reg .pred p;\n\t"
+          "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+          "selp.u32 %0, 1, 0, p;\n\t}"
+          : "=r"(ok) : "r"(bar), "r"(c.ph[which]) : "memory");
+    }
+    if (!ok) dev_flag(dev_status, SEQ_DEV_TIMEOUT);
+    c.ph[which] ^= 1u;
+  }
+  const int t = (c.cnt & ~3) + c.lane;
+  if (t < c.cnt && t >= c.s_lo && t < c.s_hi) dst[t] = __ldg(row + c.lo + t);
+  __syncwarp();
+}
+__device__ __forceinline__ void prefetch_slice_l2(const Ctx& c, const float* row) {
+  const uint32_t bytes = (uint32_t)(c.cnt & ~3) * 4u;
+  if (bytes) asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(row + c.lo), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool node_has_child(const Ctx& c, int v) { return (c.sh->has_child[v >> 5] >> (v & 31)) & 1u; }
 
 // Runs Algorithm 2's loop at node v.  Returns the accepted child's node id or -1 and leaves in
-// `st` (and in ps/qs) the state the final draw needs.
+// `st` (and in ps/qs/wseg) the state the final draw needs.
 __device__ int process_node(cg::cluster_group& cluster, Ctx& c, const VerifyArgs& a, int v, NodeState& st,
-                            bool skip_leaves) {
-  const int k = build_kids(c, v, a.n);
-  if (k == 0 && skip_leaves) return -1;
+                            bool skip_leaves, bool copies_started) {
   const bool greedy = a.temperature == 0.f;
+  const bool has_kids = node_has_child(c, v);
+  if (skip_leaves && !has_kids) return -1;
+  const bool need_draft = !greedy && (has_kids || (copies_started && a.n > 1));
   const float* trow = a.target + (int64_t)v * a.target_stride;
   const float* drow = a.draft + (int64_t)v * a.draft_stride;
+  c.npar ^= 1;
+  float4* kid_pq = c.sh->kid_pq[c.npar];
+  if (c.tid == 0 && !copies_started) {
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");  // earlier plain writes to the slices come first
+    start_slice_copy(c, trow, c.ps, 0);
+    if (need_draft) start_slice_copy(c, drow, c.qs, 1);
+  }
+  TRACE(1);
+  const int k = build_kids(c, v, a.n);  // overlaps the copies
+  // duplicates among siblings, and L2 prefetch of the first children's rows
+  for (int i = c.tid; i < k; i += kVThreads) {
+    const int s = c.sh->tokens[c.sh->kids[i]];
+    int d = 0;
+    for (int j = 0; j < i; ++j) d |= c.sh->tokens[c.sh->kids[j]] == s;
+    c.sh->dup[i] = (uint8_t)d;
+    if (i < kPrefetchChildren) {
+      const int ch = c.sh->kids[i];
+      prefetch_slice_l2(c, a.target + (int64_t)ch * a.target_stride);
+      if (!greedy && node_has_child(c, ch)) prefetch_slice_l2(c, a.draft + (int64_t)ch * a.draft_stride);
+    }
+  }
+  TRACE(2);
+  finish_slice_copy(c, trow, c.ps, 0, a.dev_status);
+  if (need_draft) finish_slice_copy(c, drow, c.qs, 1, a.dev_status);
+  TRACE(3);
 
   if (greedy) {
-    // arg-max of the target row, lowest index on ties
+    // arg-max of the target row, lowest index on ties (each lane meets its elements in ascending order)
     float best = -INFINITY;
     int best_idx = 0x7fffffff;
-    for (int i = c.tid; i < c.cnt; i += kVThreads) {
-      const float x = sanitize_logit(__ldg(trow + c.lo + i), a.dev_status);
-      if (x > best || (x == best && c.lo + i < best_idx)) { best = x; best_idx = c.lo + i; }
-    }
-    double mv[1] = {(double)best};
-    block_allreduce<1, true>(c, mv);
-    double iv[1] = {(best == (float)mv[0] && best_idx != 0x7fffffff) ? -(double)best_idx : -2147483647.0};
-    block_allreduce<1, true>(c, iv);  // max of negated indices = lowest index
-    double mine[2] = {mv[0], iv[0]};
-    double all[kVCluster][2];
-    cluster_exchange<2>(cluster, c, mine, all);
-    double gbest = -INFINITY, gidx = -2147483647.0;
+    auto upd = [&](int t) {
+      const float x = sanitize_logit(c.ps[t], a.dev_status);
+      if (x > best || best_idx == 0x7fffffff) { best = x; best_idx = c.lo + t; }
+    };
+    sweep(c, [&](int t) { upd(t); upd(t + 1); upd(t + 2); upd(t + 3); }, upd);
 #pragma unroll
-    for (int r = 0; r < kVCluster; ++r) {
-      if (all[r][1] == -2147483647.0) continue;  // empty slice or nothing comparable
-      if (all[r][0] > gbest || (all[r][0] == gbest && all[r][1] > gidx)) { gbest = all[r][0]; gidx = all[r][1]; }
+    for (int o = 16; o > 0; o >>= 1) {
+      const float ob = __shfl_xor_sync(0xffffffffu, best, o);
+      const int oi = __shfl_xor_sync(0xffffffffu, best_idx, o);
+      if (oi != 0x7fffffff && (best_idx == 0x7fffffff || ob > best || (ob == best && oi < best_idx))) { best = ob; best_idx = oi; }
     }
-    st.greedy_token = gidx == -2147483647.0 ? 0 : (int)(-gidx);
+    float4 e0, e1;
+    cluster_exchange(cluster, c, make_float4(best, __int_as_float(best_idx), 0.f, 0.f), e0, e1);
+    float gb = e0.x; int gi = __float_as_int(e0.y);
+    {
+      const float ob = e1.x; const int oi = __float_as_int(e1.y);
+      if (oi != 0x7fffffff && (gi == 0x7fffffff || ob > gb || (ob == gb && oi < gi))) { gb = ob; gi = oi; }
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+      const float ob = __shfl_xor_sync(0xffffffffu, gb, o);
+      const int oi = __shfl_xor_sync(0xffffffffu, gi, o);
+      if (oi != 0x7fffffff && (gi == 0x7fffffff || ob > gb || (ob == gb && oi < gi))) { gb = ob; gi = oi; }
+    }
+    st.greedy_token = gi == 0x7fffffff ? 0 : gi;
     for (int i = 0; i < k; ++i) {
       const int ch = c.sh->kids[i];
       const int s = c.sh->tokens[ch];
@@ -218,111 +291,156 @@ __device__ int process_node(cg::cluster_group& cluster, Ctx& c, const VerifyArgs
     return -1;
   }
 
-  const float c2 = kLog2e / a.temperature;
-  const bool need_draft = k > 0;
-
-  // slices -> shared memory as exponentials relative to the slice maxima, with their sums
-  double mx[2];
-  mx[0] = (double)load_slice(c, trow, c.ps, a.dev_status);
-  mx[1] = need_draft ? (double)load_slice(c, drow, c.qs, a.dev_status) : -INFINITY;
-  block_allreduce<2, true>(c, mx);  // its barrier also publishes the raw logits to the block
-  const float mlp = (float)mx[0], mlq = (float)mx[1];
-  float sp = 0.f, sq = 0.f;
-  for (int i = c.tid; i < c.cnt; i += kVThreads) {
-    const float e = slice_exp(c.ps[i], mlp, c2);
-    c.ps[i] = e;
-    sp += e;
-    if (need_draft) {
-      const float f = slice_exp(c.qs[i], mlq, c2);
-      c.qs[i] = f;
-      sq += f;
-    }
-  }
-  double sums[2] = {(double)sp, (double)sq};
-  block_allreduce<2, false>(c, sums);
-  double mine[4] = {mx[0], sums[0], mx[1], sums[1]};
-  double all[kVCluster][4];
-  cluster_exchange<4>(cluster, c, mine, all);
+  const float c2 = st.c2;
+  // segment maxima; a NaN or +inf logit is flagged and replaced in place (rare path)
+  float mp = -INFINITY, mq = -INFINITY;
   {
-    double Mp = -INFINITY, Mq = -INFINITY;
-#pragma unroll
-    for (int r = 0; r < kVCluster; ++r) { Mp = fmax(Mp, all[r][0]); Mq = fmax(Mq, all[r][2]); }
-    double fp[kVCluster], fq[kVCluster], Sp = 0.0, Sq = 0.0;
-#pragma unroll
-    for (int r = 0; r < kVCluster; ++r) {
-      fp[r] = all[r][0] == -INFINITY ? 0.0 : (double)exp2f(((float)all[r][0] - (float)Mp) * c2);
-      fq[r] = all[r][2] == -INFINITY ? 0.0 : (double)exp2f(((float)all[r][2] - (float)Mq) * c2);
-      Sp += all[r][1] * fp[r];
-      Sq += all[r][3] * fq[r];
+    auto fix = [&](float* p) { *p = sanitize_logit(*p, a.dev_status); return *p; };
+    auto f1 = [&](int t) {
+      float x = c.ps[t];
+      if (!(x < INFINITY)) x = fix(c.ps + t);
+      mp = fmaxf(mp, x);
+      if (need_draft) {
+        float y = c.qs[t];
+        if (!(y < INFINITY)) y = fix(c.qs + t);
+        mq = fmaxf(mq, y);
+      }
+    };
+    auto f4 = [&](int t) {
+      const float4 x = *reinterpret_cast<const float4*>(c.ps + t);
+      const float m4 = fmaxf(fmaxf(x.x, x.y), fmaxf(x.z, x.w));
+      if (m4 < INFINITY && x.x == x.x && x.y == x.y && x.z == x.z && x.w == x.w) mp = fmaxf(mp, m4);
+      else { f1(t); f1(t + 1); f1(t + 2); f1(t + 3); return; }
+      if (need_draft) {
+        const float4 y = *reinterpret_cast<const float4*>(c.qs + t);
+        const float n4 = fmaxf(fmaxf(y.x, y.y), fmaxf(y.z, y.w));
+        if (n4 < INFINITY && y.x == y.x && y.y == y.y && y.z == y.z && y.w == y.w) mq = fmaxf(mq, n4);
+        else { f1(t); f1(t + 1); f1(t + 2); f1(t + 3); }
+      }
+    };
+    sweep(c, f4, f1);
+  }
+  mp = warp_max(mp);
+  mq = warp_max(mq);
+  TRACE(4);
+  // exponentials relative to the segment maxima, with their sums
+  float sp = 0.f, sq = 0.f;
+  {
+    const float mpe = mp == -INFINITY ? 0.f : mp, mqe = mq == -INFINITY ? 0.f : mq;  // an all -inf segment stays 0
+    auto f1 = [&](int t) {
+      const float e = fast_ex2((c.ps[t] - mpe) * c2);
+      c.ps[t] = e; sp += e;
+      if (need_draft) { const float f = fast_ex2((c.qs[t] - mqe) * c2); c.qs[t] = f; sq += f; }
+    };
+    auto f4 = [&](int t) {
+      float4 x = *reinterpret_cast<const float4*>(c.ps + t);
+      x.x = fast_ex2((x.x - mpe) * c2); x.y = fast_ex2((x.y - mpe) * c2);
+      x.z = fast_ex2((x.z - mpe) * c2); x.w = fast_ex2((x.w - mpe) * c2);
+      *reinterpret_cast<float4*>(c.ps + t) = x;
+      sp += (x.x + x.y) + (x.z + x.w);
+      if (need_draft) {
+        float4 y = *reinterpret_cast<const float4*>(c.qs + t);
+        y.x = fast_ex2((y.x - mqe) * c2); y.y = fast_ex2((y.y - mqe) * c2);
+        y.z = fast_ex2((y.z - mqe) * c2); y.w = fast_ex2((y.w - mqe) * c2);
+        *reinterpret_cast<float4*>(c.qs + t) = y;
+        sq += (y.x + y.y) + (y.z + y.w);
+      }
+    };
+    sweep(c, f4, f1);
+  }
+  sp = warp_sum(sp);
+  sq = warp_sum(sq);
+  __syncwarp();
+  // every child's stored exponentials go from the warp that owns its token to all CTAs
+  for (int i = c.lane; i < k; i += 32) {
+    const int s = c.sh->tokens[c.sh->kids[i]] - c.lo;
+    if (s >= c.s_lo && s < c.s_hi) {
+      const float4 pq = make_float4(c.ps[s], need_draft ? c.qs[s] : 0.f, mp, mq);
+      for (int r = 0; r < kVCluster; ++r) *cluster.map_shared_rank(&kid_pq[i], r) = pq;
     }
+  }
+  TRACE(5);
+  float4 e0, e1;
+  cluster_exchange(cluster, c, make_float4(mp, sp, mq, sq), e0, e1);
+  TRACE(6);
+  {
+    float Mp = warp_max(fmaxf(e0.x, e1.x)), Mq = warp_max(fmaxf(e0.z, e1.z));
+    const double a0 = (double)e0.y * (double)rel_exp(e0.x, Mp, c2), a1 = (double)e1.y * (double)rel_exp(e1.x, Mp, c2);
+    const double b0 = (double)e0.w * (double)rel_exp(e0.z, Mq, c2), b1 = (double)e1.w * (double)rel_exp(e1.z, Mq, c2);
+    const double Sp = sum_lanes(a0 + a1, 32), Sq = sum_lanes(b0 + b1, 32);
     if (!(Sp > 0.0)) dev_flag(a.dev_status, SEQ_DEV_DEGENERATE);
-#pragma unroll
-    for (int r = 0; r < kVCluster; ++r) {
-      st.mlp[r] = (float)all[r][0];
-      st.mlq[r] = (float)all[r][2];
-      st.ipr[r] = Sp > 0.0 ? (float)(fp[r] / Sp) : 0.f;
-      st.iqr[r] = (need_draft && Sq > 0.0) ? (float)(fq[r] / Sq) : 0.f;
-    }
-    st.ip = st.ipr[c.rank];
-    st.iq = st.iqr[c.rank];
+    st.Mp = Mp; st.Mq = Mq;
+    st.invSp = Sp > 0.0 ? (float)(1.0 / Sp) : 0.f;
+    st.invSq = (need_draft && Sq > 0.0) ? (float)(1.0 / Sq) : 0.f;
+    st.part_sum[0] = a0 * (double)st.invSp;
+    st.part_sum[1] = a1 * (double)st.invSp;
+    st.mode = (need_draft && !(Sq > 0.0)) ? 1 : 0;  // a draft row without mass: the fallback from the start
   }
-  st.C = 0.0; st.U = 0.0; st.Z = 1.0; st.ZD = 1.0; st.mode = 0; st.nS = 0;
-  if (need_draft && st.iqr[0] == 0.f) {
-    // the draft row has no mass at all (every logit -inf): Algorithm 2's fallback from the start
-    bool any = false;
-#pragma unroll
-    for (int r = 0; r < kVCluster; ++r) any |= st.iqr[r] != 0.f;
-    if (!any) st.mode = 1;
-  }
+  st.ipw = rel_exp(mp, st.Mp, c2) * st.invSp;
+  st.iqw = rel_exp(mq, st.Mq, c2) * st.invSq;
+  st.C = 0.0; st.U = 0.0; st.Z = 1.0; st.ZD = 1.0; st.nS = 0; st.has_q = need_draft;
+  TRACE(7);
 
   for (int i = 0; i < k; ++i) {
     const int ch = c.sh->kids[i];
     const int s = c.sh->tokens[ch];
     if (s < 0 || s >= a.V) { dev_flag(a.dev_status, SEQ_DEV_BAD_TOKEN); continue; }
-    // s is in S iff an earlier (hence rejected) sibling carried the same token
-    int dup = 0;
-    for (int j = c.tid; j < i; j += kVThreads) dup |= c.sh->tokens[c.sh->kids[j]] == s;
-    const bool in_S = __syncthreads_or(dup) != 0;
-    const int owner = s / a.slice_cap;
+    const bool in_S = c.sh->dup[i] != 0;  // an earlier (hence rejected) sibling carried the same token
     float pn = 0.f, qn = 0.f;
     if (!in_S) {
-      const float xp = sanitize_logit(__ldg(trow + s), nullptr);
-      const float xq = sanitize_logit(__ldg(drow + s), nullptr);
-      pn = slice_exp(xp, st.mlp[owner], c2) * st.ipr[owner];
-      qn = slice_exp(xq, st.mlq[owner], c2) * st.iqr[owner];
+      const float4 pq = kid_pq[i];
+      pn = pq.x * (rel_exp(pq.z, st.Mp, c2) * st.invSp);
+      qn = pq.y * (rel_exp(pq.w, st.Mq, c2) * st.invSq);
     }
-    const float Cf = (float)st.C, Uf = (float)st.U;
-    const double Rs = in_S ? 0.0 : (double)resid(pn, qn, Cf, Uf) / st.Z;
-    const double Ds = in_S ? 0.0 : (st.mode == 0 ? (double)qn / st.ZD : 1.0 / (double)(a.V - st.nS));
-    const double ratio = Ds > 0.0 ? Rs / Ds : (Rs > 0.0 ? (double)INFINITY : 0.0);
-    if ((double)c.sh->uniforms[ch] < ratio) return ch;  // line 6-7: accept
+    // line 6: accept iff u < R[s]/D[s], with R[s] = rs/Z and D[s] = qn/ZD (or 1/(V-|S|)); cross-multiplied,
+    // which also covers D[s] = 0 (accept iff R[s] > 0)
+    const double rs = in_S ? 0.0 : (double)resid(pn, qn, (float)st.C, (float)st.U);
+    const double u = (double)c.sh->uniforms[ch];
+    const bool accept = st.mode == 0 ? (u * st.Z * (double)qn < rs * st.ZD) : (u * st.Z < rs * (double)(a.V - st.nS));
+    TRACE(8);
+    if (accept) return ch;
 
     // line 9: R <- norm(max(R - D, 0)) with D as it stands
     double Cn = st.C, Un = st.U;
     if (st.mode == 0) Cn += st.Z / st.ZD;
     else if (a.V - st.nS > 0) Un += st.Z / (double)(a.V - st.nS);
-    // lines 10-11: D[s] <- 0, S.add(s)
+    // lines 10-11: D[s] <- 0, S.add(s); done by the warp that owns s
     if (!in_S) {
-      if (owner == c.rank && c.tid == 0) { c.ps[s - c.lo] = 0.f; c.qs[s - c.lo] = 0.f; }
+      const int sl = s - c.lo;
+      if (sl >= c.s_lo && sl < c.s_hi && c.lane == 0) { c.ps[sl] = 0.f; c.qs[sl] = 0.f; }
       st.nS += 1;
     }
-    __syncthreads();
-    const float Cnf = (float)Cn, Unf = (float)Un;
+    __syncwarp();
+    const float Cnf = (float)Cn, Unf = (float)Un, ipw = st.ipw, iqw = st.iqw;
     float zr = 0.f, zd = 0.f;
-    for (int t = c.tid; t < c.cnt; t += kVThreads) {
-      const float qt = c.qs[t] * st.iq;
-      zr += resid(c.ps[t] * st.ip, qt, Cnf, Unf);
-      zd += qt;
+    {
+      auto f1 = [&](int t) {
+        const float qt = c.qs[t] * iqw;
+        zr += resid(c.ps[t] * ipw, qt, Cnf, Unf);
+        zd += qt;
+      };
+      auto f4 = [&](int t) {
+        const float4 x = *reinterpret_cast<const float4*>(c.ps + t);
+        const float4 y = *reinterpret_cast<const float4*>(c.qs + t);
+        const float q0 = y.x * iqw, q1 = y.y * iqw, q2 = y.z * iqw, q3 = y.w * iqw;
+        zr += (resid(x.x * ipw, q0, Cnf, Unf) + resid(x.y * ipw, q1, Cnf, Unf)) +
+              (resid(x.z * ipw, q2, Cnf, Unf) + resid(x.w * ipw, q3, Cnf, Unf));
+        zd += (q0 + q1) + (q2 + q3);
+      };
+      sweep(c, f4, f1);
     }
-    double z2[2] = {(double)zr, (double)zd};
-    block_allreduce<2, false>(c, z2);
-    double zall[kVCluster][2];
-    cluster_exchange<2>(cluster, c, z2, zall);
-    double Zn = 0.0, ZDn = 0.0;
-#pragma unroll
-    for (int r = 0; r < kVCluster; ++r) { Zn += zall[r][0]; ZDn += zall[r][1]; }
-    if (Zn > 0.0) { st.C = Cn; st.U = Un; st.Z = Zn; }
-    else dev_flag(a.dev_status, SEQ_DEV_DEGENERATE);  // keep R
+    zr = warp_sum(zr);
+    zd = warp_sum(zd);
+    TRACE(9);
+    cluster_exchange(cluster, c, make_float4(zr, zd, 0.f, 0.f), e0, e1);
+    TRACE(10);
+    const double Zn = sum_lanes((double)e0.x + (double)e1.x, 32), ZDn = sum_lanes((double)e0.y + (double)e1.y, 32);
+    if (Zn > 0.0) {
+      st.C = Cn; st.U = Un; st.Z = Zn;
+      st.part_sum[0] = (double)e0.x; st.part_sum[1] = (double)e1.x;
+    } else {
+      dev_flag(a.dev_status, SEQ_DEV_DEGENERATE);  // keep R
+    }
     st.ZD = ZDn;
     if (st.mode == 0 && !(ZDn > 0.0)) st.mode = 1;  // lines 12-15: uniform over the non-rejected set
   }
@@ -330,79 +448,68 @@ __device__ int process_node(cg::cluster_group& cluster, Ctx& c, const VerifyArgs
 }
 
 // Line 18, x ~ R by inverse CDF in index order with uniforms[n]; optionally writes R.
-__device__ void draw_bonus(cg::cluster_group& cluster, Ctx& c, const VerifyArgs& a, const NodeState& st) {
-  const bool greedy = a.temperature == 0.f;
-  if (greedy) {
+__device__ void draw_bonus(Ctx& c, const VerifyArgs& a, const NodeState& st) {
+  if (a.temperature == 0.f) {
     if (a.residual_out != nullptr)
       for (int t = c.tid; t < c.cnt; t += kVThreads) a.residual_out[c.lo + t] = (c.lo + t == st.greedy_token) ? 1.f : 0.f;
     if (c.rank == 0 && c.tid == 0) *a.bonus = st.greedy_token;
     return;
   }
   const float Cf = (float)st.C, Uf = (float)st.U;
-  const bool has_q = st.C != 0.0;  // qs holds this node's draft only if a rejection happened
-  // contiguous segment of the slice per warp, a multiple of 32 long
-  const int seg = (((c.cnt + kVWarps - 1) / kVWarps) + 31) & ~31;
-  const int s_lo = min(c.warp * seg, c.cnt), s_hi = min(s_lo + seg, c.cnt);
-  float part = 0.f;
-  for (int t = s_lo + c.lane; t < s_hi; t += 32)
-    part += resid(c.ps[t] * st.ip, has_q ? c.qs[t] * st.iq : 0.f, Cf, Uf);
-  double wsum = warp_sum((double)part);
-  double (*w)[4] = c.sh->wbuf[c.wpar];
-  if (c.lane == 0) w[c.warp][0] = wsum;
-  __syncthreads();
-  double cta_sum[1] = {0.0};
-#pragma unroll
-  for (int ww = 0; ww < kVWarps; ++ww) cta_sum[0] += w[ww][0];
-  double ranks[kVCluster][1];
-  cluster_exchange<1>(cluster, c, cta_sum, ranks);
-  double total = 0.0;
-#pragma unroll
-  for (int r = 0; r < kVCluster; ++r) total += ranks[r][0];
-  const double inv_total = total > 0.0 ? 1.0 / total : 0.0;
+  const bool has_q = st.has_q && (st.C != 0.0);
+  const float ipw = st.ipw, iqw = has_q ? st.iqw : 0.f;
+  const float* qsrc = has_q ? c.qs : c.ps;  // never dereference a slice that was not loaded
+  const double total = sum_lanes(st.part_sum[0] + st.part_sum[1], 32);
 
   if (a.residual_out != nullptr) {
-    const float it = (float)inv_total;
-    for (int t = c.tid; t < c.cnt; t += kVThreads)
-      a.residual_out[c.lo + t] = resid(c.ps[t] * st.ip, has_q ? c.qs[t] * st.iq : 0.f, Cf, Uf) * it;
+    const float it = total > 0.0 ? (float)(1.0 / total) : 0.f;
+    for (int t = c.s_lo + c.lane; t < c.s_hi; t += 32)
+      a.residual_out[c.lo + t] = resid(c.ps[t] * ipw, qsrc[t] * iqw, Cf, Uf) * it;
   }
 
+  // inverse CDF over the 64 (rank, warp) segments: inclusive scan across lanes, segments `lane` first
   const double tgt = (double)c.sh->uniforms[a.n] * total;
-  // rank holding the crossing: first rank whose inclusive sum exceeds tgt, else the last with mass
-  int rstar = -1, rlast = -1;
-  double excl = 0.0, run = 0.0;
+  double inc0 = st.part_sum[0];
 #pragma unroll
-  for (int r = 0; r < kVCluster; ++r) {
-    if (ranks[r][0] > 0.0) rlast = r;
-    if (rstar < 0 && run + ranks[r][0] > tgt) { rstar = r; excl = run; }
-    run += ranks[r][0];
+  for (int o = 1; o < 32; o <<= 1) {
+    const double up = __shfl_up_sync(0xffffffffu, inc0, o);
+    if (c.lane >= o) inc0 += up;
   }
+  const double half = __shfl_sync(0xffffffffu, inc0, 31);
+  double inc1 = st.part_sum[1];
+#pragma unroll
+  for (int o = 1; o < 32; o <<= 1) {
+    const double up = __shfl_up_sync(0xffffffffu, inc1, o);
+    if (c.lane >= o) inc1 += up;
+  }
+  inc1 += half;
+  const uint32_t hit0 = __ballot_sync(0xffffffffu, st.part_sum[0] > 0.0 && inc0 > tgt);
+  const uint32_t hit1 = __ballot_sync(0xffffffffu, st.part_sum[1] > 0.0 && inc1 > tgt);
+  const uint32_t pos0 = __ballot_sync(0xffffffffu, st.part_sum[0] > 0.0);
+  const uint32_t pos1 = __ballot_sync(0xffffffffu, st.part_sum[1] > 0.0);
+  int part;          // segment holding the crossing
   bool take_last = false;
-  if (rstar < 0) { rstar = rlast; take_last = true; }
-  if (rstar < 0) {  // no mass anywhere: degenerate input, defined output
-    if (c.rank == 0 && c.tid == 0) { *a.bonus = 0; dev_flag(a.dev_status, SEQ_DEV_DEGENERATE); }
-    return;
+  if (hit0) part = __ffs(hit0) - 1;
+  else if (hit1) part = 32 + __ffs(hit1) - 1;
+  else {             // rounding left the total at or below the target: the last segment with mass
+    take_last = true;
+    if (pos1) part = 63 - __clz(pos1);
+    else if (pos0) part = 31 - __clz(pos0);
+    else {           // no mass anywhere: degenerate input, defined output
+      if (c.rank == 0 && c.tid == 0) { *a.bonus = 0; dev_flag(a.dev_status, SEQ_DEV_DEGENERATE); }
+      return;
+    }
   }
-  if (c.rank != rstar) return;
-  // warp holding the crossing
-  double tl = tgt - excl;
-  int wstar = -1, wlast = -1;
-  double wexcl = 0.0;
-  run = 0.0;
-#pragma unroll
-  for (int ww = 0; ww < kVWarps; ++ww) {
-    const double x = w[ww][0];
-    if (x > 0.0) wlast = ww;
-    if (!take_last && wstar < 0 && run + x > tl) { wstar = ww; wexcl = run; }
-    run += x;
-  }
-  if (wstar < 0) { wstar = wlast; take_last = true; }
-  if (c.warp != wstar) return;
-  tl -= wexcl;
+  if (part != c.rank * kVWarps + c.warp) return;
+  const double incl_part = part < 32 ? __shfl_sync(0xffffffffu, inc0, part & 31) : __shfl_sync(0xffffffffu, inc1, part & 31);
+  const double mass_part = part < 32 ? __shfl_sync(0xffffffffu, st.part_sum[0], part & 31)
+                                     : __shfl_sync(0xffffffffu, st.part_sum[1], part & 31);
+  const double tl = tgt - (incl_part - mass_part);  // target within this warp's segment
   double carry = 0.0;
   int found = -1, last_pos = -1;
-  for (int base = s_lo; base < s_hi && found < 0; base += 32) {
+  for (int base = c.s_lo; base < c.s_hi && found < 0; base += 32) {
     const int t = base + c.lane;
-    const float val = t < s_hi ? resid(c.ps[t] * st.ip, has_q ? c.qs[t] * st.iq : 0.f, Cf, Uf) : 0.f;
+    const float val = t < c.s_hi ? resid(c.ps[t] * ipw, qsrc[t] * iqw, Cf, Uf) : 0.f;
     double incl = (double)val;
 #pragma unroll
     for (int o = 1; o < 32; o <<= 1) {
@@ -418,47 +525,67 @@ __device__ void draw_bonus(cg::cluster_group& cluster, Ctx& c, const VerifyArgs&
     carry += __shfl_sync(0xffffffffu, incl, 31);
   }
   if (found < 0) found = last_pos;
-  if (c.lane == 0) *a.bonus = c.lo + (found < 0 ? 0 : found);
+  if (c.lane == 0) *a.bonus = c.lo + (found < 0 ? c.s_lo : found);
 }
 
 __global__ void __launch_bounds__(kVThreads, 1) tree_verify_kernel(const VerifyArgs a) {
   cg::cluster_group cluster = cg::this_cluster();
-  extern __shared__ __align__(16) float dyn_smem[];
-  __shared__ VShared sh;
+  extern __shared__ __align__(16) uint8_t dyn_smem[];  // VShared, then the two slices
+  VShared& sh = *reinterpret_cast<VShared*>(dyn_smem);
+  TRACE(0);
   Ctx c;
   c.sh = &sh;
-  c.ps = dyn_smem;
-  c.qs = dyn_smem + a.slice_cap;
+  c.ps = reinterpret_cast<float*>(dyn_smem + sizeof(VShared));
+  c.qs = c.ps + a.slice_cap;
   c.rank = (int)cluster.block_rank();
   c.lo = min(c.rank * a.slice_cap, a.V);
   c.cnt = min(a.V - c.lo, a.slice_cap);
-  c.wpar = 0; c.xpar = 0;
+  c.xpar = 0; c.npar = 0; c.ph[0] = 0; c.ph[1] = 0;
   c.tid = threadIdx.x; c.warp = threadIdx.x >> 5; c.lane = threadIdx.x & 31;
+  c.seg = (((a.slice_cap + kVWarps - 1) / kVWarps) + 31) & ~31;  // contiguous, a multiple of 32 long
+  c.s_lo = min(c.warp * c.seg, c.cnt);
+  c.s_hi = min(c.s_lo + c.seg, c.cnt);
+  const bool all_nodes = a.flags & SEQ_VERIFY_ALL_NODES;
+  const bool greedy = a.temperature == 0.f;
 
+  if (c.tid == 0) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(vsmem_u32(&sh.bar[0])) : "memory");
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(vsmem_u32(&sh.bar[1])) : "memory");
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    if (!all_nodes) {  // the walk always starts at the root: fetch its rows while the tree is being read
+      start_slice_copy(c, a.target, c.ps, 0);
+      if (!greedy && a.n > 1) start_slice_copy(c, a.draft, c.qs, 1);  // draft row 0 is read whenever the tree has children
+    }
+  }
+  if (c.tid < SEQ_MAX_TREE / 32) sh.has_child[c.tid] = 0u;
+  __syncthreads();
   for (int i = c.tid; i < a.n; i += kVThreads) {
     int p = a.parent[i];
     if (i == 0) p = -1;
     else if (p < -1 || p >= i) { dev_flag(a.dev_status, SEQ_DEV_BAD_PARENT); p = -1; }
     sh.parent[i] = p;
     sh.tokens[i] = a.tokens[i];
+    if (p >= 0) atomicOr(&sh.has_child[p >> 5], 1u << (p & 31));
   }
-  if (a.temperature != 0.f)
+  if (!greedy)
     for (int i = c.tid; i <= a.n; i += kVThreads) sh.uniforms[i] = a.uniforms[i];
+  TRACE(20);
   __syncthreads();
   cluster.sync();  // every CTA of the cluster is resident before any remote shared-memory write
+  TRACE(21);
 
   NodeState st;
   st.greedy_token = 0;
+  st.c2 = greedy ? 0.f : kLog2e / a.temperature;
   const int cluster_id = blockIdx.x / kVCluster, n_clusters = gridDim.x / kVCluster;
 
-  if (a.flags & SEQ_VERIFY_ALL_NODES) {
+  if (all_nodes) {
     // test hook: every node gets its own run of Algorithm 2's loop; no walk, no final draw
     for (int v = cluster_id; v < a.n; v += n_clusters) {
-      const int acc = process_node(cluster, c, a, v, st, true);
+      const int acc = process_node(cluster, c, a, v, st, true, false);
       if (c.rank == 0 && c.tid == 0) a.next_child_out[v] = acc;
       __syncthreads();
     }
-    cluster.sync();
     return;
   }
 
@@ -469,15 +596,18 @@ __global__ void __launch_bounds__(kVThreads, 1) tree_verify_kernel(const VerifyA
   for (int hop = 0; hop < a.n; ++hop) {  // a walk visits at most n nodes
     if (c.rank == 0 && c.tid == 0) a.path[plen] = cur;
     ++plen;
-    const int acc = process_node(cluster, c, a, cur, st, false);
+    const int acc = process_node(cluster, c, a, cur, st, false, hop == 0);
     if (c.rank == 0 && c.tid == 0 && a.next_child_out != nullptr) a.next_child_out[cur] = acc;
     if (acc < 0) break;
     cur = acc;
-    __syncthreads();
+    __syncthreads();  // all reads of this node's slices are done before the next copies land
   }
   if (c.rank == 0 && c.tid == 0) *a.path_len = plen;
-  draw_bonus(cluster, c, a, st);
-  cluster.sync();  // no CTA leaves while a sibling may still address its shared memory
+  TRACE(11);
+  draw_bonus(c, a, st);
+  TRACE(12);
+  // No closing cluster barrier: remote shared memory is only written before a cluster barrier that
+  // every CTA joins, so nothing can still address a CTA that has left.
 }
 
 }  // namespace seqtree
@@ -526,8 +656,9 @@ extern "C" int seq_tree_verify(const seq_tree_verify_params* p, void* stream) {
   a.path = p->path; a.path_len = p->path_len; a.bonus = p->bonus_token;
   a.residual_out = p->residual_out; a.next_child_out = p->next_child_out; a.dev_status = p->dev_status;
 
-  const size_t dyn = (size_t)2 * a.slice_cap * sizeof(float);
-  if (dyn + kVStaticSmem > 227 * 1024) return SEQ_ERR_UNSUPPORTED;  // vocabulary too large for 8 slices
+  static_assert(sizeof(VShared) % 16 == 0, "the slices behind VShared must stay 16-byte aligned");
+  const size_t dyn = sizeof(VShared) + (size_t)2 * a.slice_cap * sizeof(float);
+  if (dyn > 227 * 1024) return SEQ_ERR_UNSUPPORTED;  // vocabulary too large for 8 slices
   SEQ_CUDA_OK(cudaFuncSetAttribute(tree_verify_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)dyn));
 
   int n_clusters = 1;
@@ -547,3 +678,17 @@ extern "C" int seq_tree_verify(const seq_tree_verify_params* p, void* stream) {
   SEQ_CUDA_OK(cudaLaunchKernelEx(&cfg, tree_verify_kernel, a));
   return SEQ_OK;
 }
+
+#ifdef SEQ_TRACE
+// debug builds only: copy out and reset the phase timeline recorded by TRACE()
+extern "C" int seq_debug_trace_dump(unsigned long long* host_out) {
+  int n = 0;
+  cudaDeviceSynchronize();
+  cudaMemcpyFromSymbol(&n, seqtree::g_trace_n, sizeof(int));
+  if (n > 256) n = 256;
+  cudaMemcpyFromSymbol(host_out, seqtree::g_trace, sizeof(unsigned long long) * 2 * n);
+  int zero = 0;
+  cudaMemcpyToSymbol(seqtree::g_trace_n, &zero, sizeof(int));
+  return n;
+}
+#endif
