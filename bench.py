@@ -101,13 +101,34 @@ class ClockSampler:
                 "reasons": sorted(self.reasons), "samples": len(self.samples)}
 
 
+def max_over_ranks(value: float, device=None) -> float:
+    """Maximum of a per-rank number over all ranks of the default process group (1 rank: itself)."""
+    import torch.distributed as dist
+
+    if not (dist.is_available() and dist.is_initialized()) or dist.get_world_size() == 1:
+        return float(value)
+    t = torch.tensor([value], dtype=torch.float64, device=device or "cpu")
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def whole_job_us_per_step(ms_total_max: float, steps: int, world: int) -> float:
+    """Every rank verifies its own request per step (weak scaling): the job completes `world` steps in
+    the time of one, so the whole-job figure is the max-over-ranks step time divided by `world`."""
+    return 1e3 * ms_total_max / steps / world
+
+
+def rank_seed_base(rank: int) -> int:
+    return 1000 * rank
+
+
 def n_sets(bytes_per_set: int, lo: int = 2, hi: int = 48) -> int:
     return max(lo, min(hi, math.ceil(3 * L2_BYTES / max(1, bytes_per_set))))
 
 
 def build_requests(cfg, T, rank, n_attn, n_verify):
     """Host-side inputs for this rank: n_attn attention sets and n_verify logit sets (seeds differ by rank)."""
-    base = 1000 * rank
+    base = rank_seed_base(rank)
     parent = W.make_tree(cfg, base)
     attn = [W.make_attention_inputs(cfg, base + s, parent=parent) for s in range(n_attn)]
     ver = [W.make_verify_inputs(cfg, T, base + s, parent=parent) for s in range(n_verify)]
@@ -280,12 +301,9 @@ def main():
 
     if int(status.item()) != 0:
         raise RuntimeError(f"dev_status = {int(status.item())} after the timed region")
-    if world > 1:
-        t = torch.tensor([ms_total], dtype=torch.float64, device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms_total = float(t.item())
+    ms_total = max_over_ranks(ms_total, dev)
     ms_per_step = ms_total / K
-    value_us = 1e3 * ms_per_step / world  # whole job: N requests verified per step time
+    value_us = whole_job_us_per_step(ms_total, K, world)
 
     # end to end from pinned host buffers through the public API, copies inside the timed region
     host = B.HostStep(attn_h[0].q, attn_h[0].k_cache, attn_h[0].v_cache, torch.from_numpy(parent), cfg.prefix_len,
@@ -301,10 +319,7 @@ def main():
             host.run(stream)
             stream.synchronize()
         e2e_us = 1e6 * (time.perf_counter() - t0) / Ke
-    if world > 1:
-        t = torch.tensor([e2e_us], dtype=torch.float64, device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        e2e_us = float(t.item()) / world
+    e2e_us = max_over_ranks(e2e_us, dev) / world
 
     if rank != 0:
         if world > 1:
