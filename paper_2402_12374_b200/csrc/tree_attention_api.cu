@@ -58,7 +58,8 @@ extern "C" size_t seq_tree_attention_workspace_bytes(const seq_tree_attention_pa
   if (validate(p) != SEQ_OK) return 0;
   const int which = choose_kernel(*p);
   if (which == 0) return 0;
-  const int splits = which == 2 ? umma_default_splits(*p) : simt_default_splits(*p);
+  if (which == 2) return 0;  // the tensor-core kernel merges its key-range shares on chip
+  const int splits = simt_default_splits(*p);
   size_t bytes = splits > 1 ? split_workspace_bytes(splits, p->num_q_heads, p->n_tree) : 0;
   return (bytes + 255) & ~(size_t)255;
 }
@@ -68,12 +69,12 @@ extern "C" int seq_tree_attention(const seq_tree_attention_params* p, void* stre
   if (rc != SEQ_OK) return rc;
   const int which = choose_kernel(*p);
   if (which == 0) return SEQ_ERR_UNSUPPORTED;
-  const int splits = which == 2 ? umma_default_splits(*p) : simt_default_splits(*p);
+  if (which == 2) return launch_attention_umma(*p, umma_default_splits(*p), (cudaStream_t)stream);
+  const int splits = simt_default_splits(*p);
   if (splits > 1) {
     if (p->workspace == nullptr || p->workspace_bytes < split_workspace_bytes(splits, p->num_q_heads, p->n_tree))
       return SEQ_ERR_WORKSPACE;
     if (reinterpret_cast<uintptr_t>(p->workspace) % 256 != 0) return SEQ_ERR_INVALID_ARG;
   }
-  if (which == 2) return launch_attention_umma(*p, splits, (cudaStream_t)stream);
   return launch_attention_simt(*p, splits, (cudaStream_t)stream);
 }

@@ -1,16 +1,28 @@
 // Tree-masked attention on the 5th-generation tensor cores (tcgen05.mma, accumulators in tensor
 // memory, K/V/Q tiles staged by TMA), for 16-bit inputs.
 //
-// Work unit: one CTA = (kv head g, tile of 128 query rows, split of the key range).  A query row is
+// Work unit: one CTA = (kv head g, tile of 128 query rows, share of the key range).  A query row is
 // a (node, head-in-group) pair, r = i_local * G + hg, so under GQA the G heads that share a kv head
 // share every K/V tile.  Keys are taken in blocks of 128:
 //     S = Q K^T      128x128x128  tcgen05.mma, Q and K K-major in 128-byte-swizzled shared memory
-//     P = 2^(scale*S - m) masked  one thread per row, S read from tensor memory
-//     O += P V       128x128x128  tcgen05.mma, P (16-bit) in shared memory, V MN-major
-// Warp 0 issues TMA loads, warp 1 issues MMAs, warps 2..5 own the 128 rows.  S is double-buffered
-// in tensor memory so that S(j+1) is computed while the row threads work on block j.  The running
-// maximum is only moved when a row's block maximum exceeds it by more than 2^8 (the accumulator is
-// then rescaled in tensor memory), so in steady state O is never touched by the row threads.
+//     P = 2^(scale*S - m) masked  one thread per row: S read from tensor memory, P written back over
+//                                 it as packed 16-bit values
+//     O += P V       128x128x128  tcgen05.mma, A = P from tensor memory, V MN-major in shared memory
+//
+// Two chains per CTA.  Even blocks of the CTA's key range belong to chain A, odd blocks to chain B.
+// Each chain has its own S/P buffer and its own accumulator O in tensor memory (4 x 128 columns),
+// its own K/V stage in shared memory, its own 128 row threads (one warp group) and its own running
+// (m, l); the chains only share Q, the TMA warp and the MMA warp.  While the row threads of one chain
+// exponentiate, the tensor pipe works for the other.  The running maximum of a row is only moved
+// when a block maximum exceeds it by more than 2^8 (the accumulator row is then rescaled in tensor
+// memory).  Registers are rebalanced with setmaxnreg: 40 for the TMA/MMA warp group, 232 for the rows.
+//
+// Merge.  The CTAs that share (tile, kv head) form a thread-block cluster along the key
+// range (cs = 1, 2, 4 or 8); its 2*cs chains share the 16 slices of 8 output columns round-robin.  Every chain pushes,
+// for every row, each 8-column piece of its unnormalised fp32 accumulator into the shared memory of
+// the chain that owns that slice (the K/V stages, dead by then) and its (m, l) into every CTA, with
+// plain remote stores over distributed shared memory; after one cluster barrier each owner reduces
+// its slices from local shared memory and writes the final output.  No workspace, no second kernel.
 //
 // Masking: key j < prefix_len is visible; key prefix_len + t is visible iff bit t of the row's
 // ancestor mask; masked scores become -inf before the maximum, so their probability is exactly 0.
@@ -18,29 +30,47 @@
 // the rest of a tile with zeros.
 //
 // Every mbarrier wait is bounded; a wait that runs out raises SEQ_DEV_TIMEOUT and the CTA drains.
+#include <cooperative_groups.h>
 #include <cuda.h>
+#include <stdlib.h>
 
 #include "common.cuh"
 
+namespace cg = cooperative_groups;
+
 namespace seqtree {
 
-constexpr int kTileM = 128;      // query rows per CTA
-constexpr int kBlockN = 128;     // keys per block
-constexpr int kStages = 2;       // K and V stages each
-constexpr int kUmmaThreads = 192;
-constexpr uint32_t kTileBytes = 128 * 128 * 2;  // one 128x128 16-bit tile
-constexpr uint32_t kHalfBytes = kTileBytes / 2; // one 128-row x 64-element sub-tile (128 B rows)
-constexpr float kRescaleThreshold = 8.f;        // log2 units
+#ifdef SEQ_TRACE
+__device__ unsigned long long g_utrace[4][512];
+#define UTRACE(role, tag)                                                       \
+  do {                                                                          \
+    if (blockIdx.x == 0 && blockIdx.y == 0 && blockIdx.z == 0) {                \
+      int _i = utrace_i++;                                                      \
+      if (_i < 255) { g_utrace[role][2 * _i + 2] = (tag); g_utrace[role][2 * _i + 3] = clock64(); g_utrace[role][0] = _i + 1; } \
+    }                                                                           \
+  } while (0)
+#else
+#define UTRACE(role, tag) do { } while (0)
+#endif
+
+constexpr int kTileM = 128;         // query rows per CTA
+constexpr int kBlockN = 128;        // keys per block
+constexpr int kUmmaThreads = 384;   // warp group 0: TMA warp, MMA warp, two spare; warp groups 1, 2: rows of chains A, B
+constexpr int kRegsLight = 40, kRegsRows = 232;  // after setmaxnreg: 128*40 + 256*232 = 384*168
+constexpr int kMaxClusterSplit = 8;
+constexpr int kNumSMs = 148;
+constexpr uint32_t kTileBytes = 128 * 128 * 2;   // one 128x128 16-bit tile
+constexpr uint32_t kHalfBytes = kTileBytes / 2;  // one 128-row x 64-element sub-tile (128 B rows)
+constexpr float kRescaleThreshold = 8.f;         // log2 units
 constexpr uint32_t kSpinLimit = 1u << 22;
 
 struct UmmaSmem {
   // all tiles 1024-byte aligned (128-byte swizzle atoms are 8 rows x 128 B)
   uint8_t q[kTileBytes];
-  uint8_t k[kStages][kTileBytes];
-  uint8_t v[kStages][kTileBytes];
-  uint8_t p[kTileBytes];
-  uint64_t q_full, k_full[kStages], k_empty[kStages], v_full[kStages], v_empty[kStages];
-  uint64_t s_full[2], s_empty[2], p_full, pv_done;
+  uint8_t k[2][kTileBytes];  // K stage of chain A, of chain B; after the last block: chain A's 128x128 fp32 accumulator
+  uint8_t v[2][kTileBytes];  // V stage of chain A, of chain B; after the last block: chain B's accumulator
+  float2 ml[2 * kMaxClusterSplit][kTileM];  // (m, l) of every row of every chain of the cluster, for the merge
+  uint64_t q_full, k_full[2], k_empty[2], v_full[2], v_empty[2], s_full[2], p_full[2], pv_done[2];
   uint32_t tmem_base;
   volatile int abort_flag;
 };
@@ -51,7 +81,7 @@ struct UmmaArgs {
   uint32_t idesc_qk, idesc_pv;
   const uint32_t* mask_bits;
   void* out; int64_t o_stride_tok, o_stride_head;
-  float* lse; float* o_part; float2* ml;
+  float* lse;
   int32_t* dev_status;
 };
 
@@ -115,6 +145,14 @@ __device__ __forceinline__ void tc_mma(uint32_t d_tmem, uint64_t adesc, uint64_t
       ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate) : "memory");
 }
 
+__device__ __forceinline__ void tc_mma_tmem_a(uint32_t d_tmem, uint32_t a_tmem, uint64_t bdesc, uint32_t idesc, uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t}"
+      ::"r"(d_tmem), "r"(a_tmem), "l"(bdesc), "r"(idesc), "r"(accumulate) : "memory");
+}
+
 #define SEQ_R32(a, o) \
   "=r"(a[o + 0]), "=r"(a[o + 1]), "=r"(a[o + 2]), "=r"(a[o + 3]), "=r"(a[o + 4]), "=r"(a[o + 5]), "=r"(a[o + 6]),   \
   "=r"(a[o + 7]), "=r"(a[o + 8]), "=r"(a[o + 9]), "=r"(a[o + 10]), "=r"(a[o + 11]), "=r"(a[o + 12]),               \
@@ -143,6 +181,14 @@ __device__ __forceinline__ void tmem_st32(uint32_t taddr, const uint32_t* r, int
       "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16, %17, %18, %19, %20, %21, %22, "
       "%23, %24, %25, %26, %27, %28, %29, %30, %31};"
       ::SEQ_W32(r, o), "r"(taddr) : "memory");
+}
+
+__device__ __forceinline__ void tmem_st16(uint32_t taddr, const uint32_t* r) {
+  asm volatile(
+      "tcgen05.st.sync.aligned.32x32b.x16.b32 [%16], "
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15};"
+      ::"r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]), "r"(r[8]), "r"(r[9]),
+        "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15]), "r"(taddr) : "memory");
 }
 
 __device__ __forceinline__ float ex2(float x) {
@@ -188,12 +234,16 @@ tree_attention_umma_kernel(const __grid_constant__ CUtensorMap q_map, const __gr
                            const __grid_constant__ CUtensorMap v_map, const UmmaArgs a) {
   extern __shared__ uint8_t smem_raw[];
   UmmaSmem* sm = reinterpret_cast<UmmaSmem*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+  cg::cluster_group cluster = cg::this_cluster();
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int tile = blockIdx.x, g = blockIdx.y, split = blockIdx.z;
+#ifdef SEQ_TRACE
+  int utrace_i = 0;
+#endif
+  const int tile = blockIdx.x, g = blockIdx.y, split = blockIdx.z;  // the cluster spans blockIdx.z
 
   const int i0 = tile * a.nodes_per_tile;
   const int i1 = min(i0 + a.nodes_per_tile, a.n);
-  // keys this tile can see end at L + i1 (a node sees no later node); blocks of this split
+  // keys this tile can see end at L + i1 (a node sees no later node); blocks of this CTA
   const int nblk_tile = (a.L + i1 + kBlockN - 1) / kBlockN;
   const int blk_lo = (int)(((long)split * nblk_tile) / a.splits);
   const int blk_hi = (int)(((long)(split + 1) * nblk_tile) / a.splits);
@@ -201,17 +251,15 @@ tree_attention_umma_kernel(const __grid_constant__ CUtensorMap q_map, const __gr
 
   if (threadIdx.x == 0) {
     mbar_init(&sm->q_full, 1);
-    for (int s = 0; s < kStages; ++s) {
-      mbar_init(&sm->k_full[s], 1); mbar_init(&sm->k_empty[s], 1);
-      mbar_init(&sm->v_full[s], 1); mbar_init(&sm->v_empty[s], 1);
+    for (int c = 0; c < 2; ++c) {
+      mbar_init(&sm->k_full[c], 1); mbar_init(&sm->k_empty[c], 1);
+      mbar_init(&sm->v_full[c], 1); mbar_init(&sm->v_empty[c], 1);
+      mbar_init(&sm->s_full[c], 1); mbar_init(&sm->p_full[c], 128); mbar_init(&sm->pv_done[c], 1);
     }
-    for (int b = 0; b < 2; ++b) { mbar_init(&sm->s_full[b], 1); mbar_init(&sm->s_empty[b], 128); }
-    mbar_init(&sm->p_full, 128);
-    mbar_init(&sm->pv_done, 1);
     sm->abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
-  if (warp == 1) {  // 512 tensor-memory columns: S0, S1, O (128 each) + spare
+  if (warp == 1) {  // all 512 tensor-memory columns: S_A, S_B (P over them), O_A, O_B
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], 512;" ::"r"(smem_u32(&sm->tmem_base)) : "memory");
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
   }
@@ -219,209 +267,255 @@ tree_attention_umma_kernel(const __grid_constant__ CUtensorMap q_map, const __gr
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem = sm->tmem_base;
-  const uint32_t tmem_s[2] = {tmem, tmem + 128u};
-  const uint32_t tmem_o = tmem + 256u;
+  if (threadIdx.x == 128) UTRACE(2, 0);
 
-  if (warp == 0) {
-    // ------------------------------------------------------------ TMA producer ------------------
-    if (lane == 0 && nblk > 0) {
-      mbar_expect_tx(&sm->q_full, kTileBytes);
-      tma_load_4d(sm->q, &q_map, &sm->q_full, 0, 0, i0, g);
-      tma_load_4d(sm->q + kHalfBytes, &q_map, &sm->q_full, 64, 0, i0, g);
-      for (int jj = 0; jj < nblk; ++jj) {
-        const int s = jj % kStages;
-        const int row = (blk_lo + jj) * kBlockN;
-        if (jj >= kStages && !mbar_wait(sm, &sm->k_empty[s], ((jj / kStages) - 1) & 1, a.dev_status)) break;
-        mbar_expect_tx(&sm->k_full[s], kTileBytes);
-        tma_load_3d(sm->k[s], &k_map, &sm->k_full[s], 0, row, g);
-        tma_load_3d(sm->k[s] + kHalfBytes, &k_map, &sm->k_full[s], 64, row, g);
-        if (jj >= kStages && !mbar_wait(sm, &sm->v_empty[s], ((jj / kStages) - 1) & 1, a.dev_status)) break;
-        mbar_expect_tx(&sm->v_full[s], kTileBytes);
-        tma_load_3d(sm->v[s], &v_map, &sm->v_full[s], 0, row, g);
-        tma_load_3d(sm->v[s] + kHalfBytes, &v_map, &sm->v_full[s], 64, row, g);
-      }
-    }
-    __syncwarp();
-  } else if (warp == 1) {
-    // ------------------------------------------------------------ MMA issuer --------------------
-    if (lane == 0 && nblk > 0) {
-      bool ok = mbar_wait(sm, &sm->q_full, 0, a.dev_status);
-      auto issue_qk = [&](int j) -> bool {
-        const int s = j % kStages, b = j & 1;
-        if (!mbar_wait(sm, &sm->k_full[s], (j / kStages) & 1, a.dev_status)) return false;
-        if (j >= 2 && !mbar_wait(sm, &sm->s_empty[b], ((j >> 1) - 1) & 1, a.dev_status)) return false;
-        tc_fence_after();
-        const uint32_t qa = smem_u32(sm->q), ka = smem_u32(sm->k[s]);
-#pragma unroll
-        for (int ks = 0; ks < 8; ++ks) {  // 8 steps of 16 along head_dim; 4 per 64-element sub-tile
-          const uint32_t off = (ks >> 2) * kHalfBytes + (ks & 3) * 32;
-          tc_mma(tmem_s[b], make_desc(qa + off, 16, 1024), make_desc(ka + off, 16, 1024), a.idesc_qk, ks > 0);
+  if (warp < 4) {
+    // ============================ warp group 0: data movement and MMA issue, few registers =========
+    asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(kRegsLight));
+    if (warp == 0) {
+      // ---------------------------------------------------------- TMA producer ------------------
+      if (lane == 0 && nblk > 0) {
+        mbar_expect_tx(&sm->q_full, kTileBytes);
+        tma_load_4d(sm->q, &q_map, &sm->q_full, 0, 0, i0, g);
+        tma_load_4d(sm->q + kHalfBytes, &q_map, &sm->q_full, 64, 0, i0, g);
+        for (int jj = 0; jj < nblk; ++jj) {
+          const int c = jj & 1, u = jj >> 1;  // chain (= stage) and its use count
+          const int row = (blk_lo + jj) * kBlockN;
+          if (u > 0 && !mbar_wait(sm, &sm->k_empty[c], (u - 1) & 1, a.dev_status)) break;
+          UTRACE(0, 1);
+          mbar_expect_tx(&sm->k_full[c], kTileBytes);
+          tma_load_3d(sm->k[c], &k_map, &sm->k_full[c], 0, row, g);
+          tma_load_3d(sm->k[c] + kHalfBytes, &k_map, &sm->k_full[c], 64, row, g);
+          if (u > 0 && !mbar_wait(sm, &sm->v_empty[c], (u - 1) & 1, a.dev_status)) break;
+          UTRACE(0, 2);
+          mbar_expect_tx(&sm->v_full[c], kTileBytes);
+          tma_load_3d(sm->v[c], &v_map, &sm->v_full[c], 0, row, g);
+          tma_load_3d(sm->v[c] + kHalfBytes, &v_map, &sm->v_full[c], 64, row, g);
         }
-        tc_commit(&sm->k_empty[s]);
-        tc_commit(&sm->s_full[b]);
-        return true;
-      };
-      if (ok) ok = issue_qk(0);
-      for (int jj = 0; jj < nblk && ok; ++jj) {
-        if (jj + 1 < nblk && !issue_qk(jj + 1)) break;
-        const int s = jj % kStages;
-        if (!mbar_wait(sm, &sm->p_full, jj & 1, a.dev_status)) break;
-        if (!mbar_wait(sm, &sm->v_full[s], (jj / kStages) & 1, a.dev_status)) break;
-        tc_fence_after();
-        const uint32_t pa = smem_u32(sm->p), va = smem_u32(sm->v[s]);
-#pragma unroll
-        for (int ks = 0; ks < 8; ++ks) {  // 8 steps of 16 keys
-          const uint64_t adesc = make_desc(pa + (ks >> 2) * kHalfBytes + (ks & 3) * 32, 16, 1024);
-          const uint64_t bdesc = make_desc(va + ks * 2048, kHalfBytes, 1024);
-          tc_mma(tmem_o, adesc, bdesc, a.idesc_pv, (jj > 0 || ks > 0) ? 1u : 0u);
-        }
-        tc_commit(&sm->v_empty[s]);
-        tc_commit(&sm->pv_done);
       }
+      __syncwarp();
+    } else if (warp == 1) {
+      // ---------------------------------------------------------- MMA issuer --------------------
+      if (lane == 0 && nblk > 0) {
+        bool go = mbar_wait(sm, &sm->q_full, 0, a.dev_status);
+        // A step along the contraction only moves a descriptor's 14-bit start-address field (16-byte units).
+        const uint64_t qd0 = make_desc(smem_u32(sm->q), 16, 1024);
+        auto issue_qk = [&](int jj) -> bool {
+          const int c = jj & 1, u = jj >> 1;
+          if (!mbar_wait(sm, &sm->k_full[c], u & 1, a.dev_status)) return false;
+          tc_fence_after();
+          const uint64_t kd0 = make_desc(smem_u32(sm->k[c]), 16, 1024);
+#pragma unroll
+          for (int ks = 0; ks < 8; ++ks) {  // 16 elements of head_dim per step: 32 bytes inside a 64-element sub-tile
+            const uint64_t off = (uint64_t)(((ks >> 2) * kHalfBytes + (ks & 3) * 32) >> 4);
+            tc_mma(tmem + 128u * c, qd0 + off, kd0 + off, a.idesc_qk, ks > 0);
+          }
+          tc_commit(&sm->k_empty[c]);
+          tc_commit(&sm->s_full[c]);
+          UTRACE(1, 2);
+          return true;
+        };
+        if (go) go = issue_qk(0);
+        if (go && nblk > 1) go = issue_qk(1);
+        for (int jj = 0; jj < nblk && go; ++jj) {
+          const int c = jj & 1, u = jj >> 1;
+          if (!mbar_wait(sm, &sm->p_full[c], u & 1, a.dev_status)) break;
+          UTRACE(1, 3);
+          if (!mbar_wait(sm, &sm->v_full[c], u & 1, a.dev_status)) break;
+          tc_fence_after();
+          const uint64_t vd0 = make_desc(smem_u32(sm->v[c]), kHalfBytes, 1024);
+#pragma unroll
+          for (int ks = 0; ks < 8; ++ks)  // A = 8 packed columns of P, B = 16 key rows of V per step
+            tc_mma_tmem_a(tmem + 256u + 128u * c, tmem + 128u * c + 8u * ks, vd0 + (uint64_t)(ks * (2048 >> 4)), a.idesc_pv,
+                          (u > 0 || ks > 0) ? 1u : 0u);
+          tc_commit(&sm->v_empty[c]);
+          tc_commit(&sm->pv_done[c]);
+          UTRACE(1, 5);
+          // The chain's next S goes where its P lives.  tcgen05.mma operations issued by one thread
+          // execute in issue order, so this QK^T cannot overtake the P.V just issued.
+          if (jj + 2 < nblk && !issue_qk(jj + 2)) break;
+        }
+      }
+      __syncwarp();
     }
-    __syncwarp();
-  } else {
-    // ------------------------------------------------------------ row threads -------------------
-    const int quad = warp & 3;                  // tensor-memory lane quarter this warp may access
-    const int r = quad * 32 + lane;             // row of the tile = tensor-memory lane
-    const uint32_t lane_sel = (uint32_t)(quad * 32) << 16;
-    const int i = i0 + r / a.group;             // node of this row
-    const int hg = r % a.group;
-    const bool row_valid = i < a.n;
-    const uint32_t* mrow = a.mask_bits + (size_t)min(i, a.n - 1) * a.mask_wpr;
-
-    float m_used = -INFINITY, l = 0.f;
-    bool ok = true;
-    uint32_t sreg[128];
-    for (int jj = 0; jj < nblk && ok; ++jj) {
-      const int b = jj & 1;
-      if (!mbar_wait(sm, &sm->s_full[b], (jj >> 1) & 1, a.dev_status)) { ok = false; break; }
+    cluster.sync();  // the two cluster barriers of the merge (see the row threads)
+    cluster.sync();
+    UTRACE(1, 9);
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1) {
       tc_fence_after();
-#pragma unroll
-      for (int c = 0; c < 4; ++c) tmem_ld32(tmem_s[b] + lane_sel + 32u * c, sreg, 32 * c);
-      tc_wait_ld();
-      tc_fence_before();
-      mbar_arrive(&sm->s_empty[b]);
-
-      // scale, mask, block maximum
-      const int kb = (blk_lo + jj) * kBlockN;
-      const bool needs_mask = kb + kBlockN > a.L;
-      float m_blk = -INFINITY;
-#pragma unroll
-      for (int c = 0; c < 4; ++c) {
-        uint32_t vis = 0xFFFFFFFFu;
-        if (needs_mask) vis = mask_window(mrow, a.mask_wpr, a.n, kb - a.L + 32 * c);
-#pragma unroll
-        for (int e = 0; e < 32; ++e) {
-          float s = __uint_as_float(sreg[32 * c + e]) * a.scale_log2;
-          s = (vis >> e) & 1u ? s : -INFINITY;
-          sreg[32 * c + e] = __float_as_uint(s);
-          m_blk = fmaxf(m_blk, s);
-        }
-      }
-      // move the reference maximum only when it is first set or exceeded by more than the threshold
-      float alpha = 1.f;
-      if (m_blk > m_used + kRescaleThreshold || (m_used == -INFINITY && m_blk != -INFINITY)) {
-        alpha = m_used == -INFINITY ? 0.f : ex2(m_used - m_blk);
-        m_used = m_blk;
-      }
-      const float m_eff = m_used == -INFINITY ? 0.f : m_used;
-      float sum = 0.f;
-      uint32_t packed[64];
-#pragma unroll
-      for (int e = 0; e < 128; e += 2) {
-        const float p0 = ex2(__uint_as_float(sreg[e]) - m_eff);
-        const float p1 = ex2(__uint_as_float(sreg[e + 1]) - m_eff);
-        sum += p0 + p1;
-        packed[e >> 1] = pack2<kBf16>(p0, p1);
-      }
-      l = l * alpha + sum;
-
-      if (jj > 0) {
-        if (!mbar_wait(sm, &sm->pv_done, (jj - 1) & 1, a.dev_status)) { ok = false; break; }
-        tc_fence_after();
-        if (__any_sync(0xffffffffu, alpha != 1.f)) {  // rescale the accumulator rows of this warp
-#pragma unroll
-          for (int c = 0; c < 4; ++c) {
-            uint32_t o[32];
-            tmem_ld32(tmem_o + lane_sel + 32u * c, o, 0);
-            tc_wait_ld();
-#pragma unroll
-            for (int e = 0; e < 32; ++e) o[e] = __float_as_uint(__uint_as_float(o[e]) * alpha);
-            tmem_st32(tmem_o + lane_sel + 32u * c, o, 0);
-          }
-          tc_wait_st();
-        }
-        tc_fence_before();
-      }
-      // P tile -> shared memory, K-major with 128-byte swizzle: 16-byte chunk c of row r sits at chunk c ^ (r & 7)
-      uint8_t* prow = sm->p + r * 128;
-#pragma unroll
-      for (int half = 0; half < 2; ++half) {
-#pragma unroll
-        for (int c = 0; c < 8; ++c) {
-          const int src = half * 32 + c * 4;
-          uint4 val = make_uint4(packed[src], packed[src + 1], packed[src + 2], packed[src + 3]);
-          *reinterpret_cast<uint4*>(prow + half * kHalfBytes + ((c ^ (r & 7)) << 4)) = val;
-        }
-      }
-      fence_async_smem();
-      mbar_arrive(&sm->p_full);
+      asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, 512;" ::"r"(tmem) : "memory");
     }
+    return;
+  }
 
-    // ------------------------------------------------------------ epilogue ----------------------
-    if (nblk > 0 && ok) ok = mbar_wait(sm, &sm->pv_done, (nblk - 1) & 1, a.dev_status);
+  // ============================== warp groups 1, 2: one thread per query row of chain A, B ============
+  asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(kRegsRows));
+  const int chain = (warp >> 2) - 1;
+  const int quad = warp & 3;                  // tensor-memory lane quarter this warp may access
+  const int r = quad * 32 + lane;             // row of the tile = tensor-memory lane
+  const uint32_t lane_sel = (uint32_t)(quad * 32) << 16;
+  const uint32_t tmem_s = tmem + 128u * chain + lane_sel, tmem_o = tmem + 256u + 128u * chain + lane_sel;
+  const int i = i0 + r / a.group;             // node of this row
+  const int h = g * a.group + r % a.group;
+  const bool row_valid = i < a.n;
+  const uint32_t* mrow = a.mask_bits + (size_t)min(i, a.n - 1) * a.mask_wpr;
+  const float sc = a.scale_log2;
+
+  float m_used = -INFINITY, l = 0.f;
+  bool ok = true;
+  const int n_mine = nblk > chain ? (nblk - chain + 1) >> 1 : 0;  // blocks of this chain
+  for (int u = 0; u < n_mine && ok; ++u) {
+    const int jj = 2 * u + chain;
+    if (!mbar_wait(sm, &sm->s_full[chain], u & 1, a.dev_status)) { ok = false; break; }
+    if (threadIdx.x == 128) UTRACE(2, 1);
     tc_fence_after();
-    const int h = g * a.group + hg;
-    if (a.splits == 1) {
-      if (ok && nblk > 0) {
-        const float inv = 1.f / l;
+    uint32_t sreg[128];
 #pragma unroll
-        for (int c = 0; c < 4; ++c) {
-          uint32_t o[32];
-          tmem_ld32(tmem_o + lane_sel + 32u * c, o, 0);
-          tc_wait_ld();
-          if (row_valid) {
-            uint8_t* dst = reinterpret_cast<uint8_t*>(a.out) + 2 * ((int64_t)i * a.o_stride_tok + (int64_t)h * a.o_stride_head + 32 * c);
+    for (int c = 0; c < 4; ++c) tmem_ld32(tmem_s + 32u * c, sreg, 32 * c);
+    const int kb = (blk_lo + jj) * kBlockN;
+    const bool masked = kb + kBlockN > a.L;  // the block reaches into the tree keys (or past the end)
+    uint32_t vis[4] = {0xFFFFFFFFu, 0xFFFFFFFFu, 0xFFFFFFFFu, 0xFFFFFFFFu};
+    if (masked) {
 #pragma unroll
-            for (int e = 0; e < 32; e += 8) {
-              uint4 val;
-              val.x = pack2<kBf16>(__uint_as_float(o[e]) * inv, __uint_as_float(o[e + 1]) * inv);
-              val.y = pack2<kBf16>(__uint_as_float(o[e + 2]) * inv, __uint_as_float(o[e + 3]) * inv);
-              val.z = pack2<kBf16>(__uint_as_float(o[e + 4]) * inv, __uint_as_float(o[e + 5]) * inv);
-              val.w = pack2<kBf16>(__uint_as_float(o[e + 6]) * inv, __uint_as_float(o[e + 7]) * inv);
-              *reinterpret_cast<uint4*>(dst + 2 * e) = val;
-            }
-          }
-        }
-        if (row_valid && a.lse != nullptr) a.lse[(size_t)h * a.n + i] = (m_used + log2f(l)) * kLn2;
+      for (int c = 0; c < 4; ++c) vis[c] = mask_window(mrow, a.mask_wpr, a.n, kb - a.L + 32 * c);
+    }
+    tc_wait_ld();
+    if (threadIdx.x == 128) UTRACE(2, 2);
+    // block maximum of the raw scores (four independent chains); masked scores become -inf first
+    float mx[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
+    if (masked) {
+#pragma unroll
+      for (int e = 0; e < 128; ++e) {
+        const float sv = (vis[e >> 5] & (1u << (e & 31))) ? __uint_as_float(sreg[e]) : -INFINITY;
+        sreg[e] = __float_as_uint(sv);
+        mx[e & 3] = fmaxf(mx[e & 3], sv);
       }
     } else {
-      const size_t prow_idx = ((size_t)split * a.Hq + h) * a.n + i;
-      if (ok && nblk > 0) {
 #pragma unroll
-        for (int c = 0; c < 4; ++c) {
-          uint32_t o[32];
-          tmem_ld32(tmem_o + lane_sel + 32u * c, o, 0);
-          tc_wait_ld();
-          if (row_valid) {
-            float* dst = a.o_part + prow_idx * kHeadDim + 32 * c;
+      for (int e = 0; e < 128; ++e) mx[e & 3] = fmaxf(mx[e & 3], __uint_as_float(sreg[e]));
+    }
+    const float m_blk = fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3])) * sc;  // scale > 0
+    // move the reference maximum only when it is first set or exceeded by more than the threshold
+    float alpha = 1.f;
+    if (m_blk > m_used + kRescaleThreshold || (m_used == -INFINITY && m_blk != -INFINITY)) {
+      alpha = m_used == -INFINITY ? 0.f : ex2(m_used - m_blk);
+      m_used = m_blk;
+    }
+    // this S was issued after O took the chain's previous block, so O is quiescent here
+    if (u > 0 && __any_sync(0xffffffffu, alpha != 1.f)) {  // rescale the accumulator rows of this warp
 #pragma unroll
-            for (int e = 0; e < 32; e += 4)
-              *reinterpret_cast<uint4*>(dst + e) = make_uint4(o[e], o[e + 1], o[e + 2], o[e + 3]);
-          }
+      for (int c = 0; c < 4; ++c) {
+        uint32_t o[32];
+        tmem_ld32(tmem_o + 32u * c, o, 0);
+        tc_wait_ld();
+#pragma unroll
+        for (int e = 0; e < 32; ++e) o[e] = __float_as_uint(__uint_as_float(o[e]) * alpha);
+        tmem_st32(tmem_o + 32u * c, o, 0);
+      }
+    }
+    if (threadIdx.x == 128) UTRACE(2, 3);
+    const float neg_m = m_used == -INFINITY ? 0.f : -m_used;
+    float sm4[4] = {0.f, 0.f, 0.f, 0.f};
+    // P = 2^(scale*s - m) written over S as packed 16-bit values: 64 columns, four stores of 16
+#pragma unroll
+    for (int c = 0; c < 4; ++c) {
+      uint32_t packed[16];
+#pragma unroll
+      for (int e = 0; e < 16; ++e) {
+        const float p0 = ex2(fmaf(__uint_as_float(sreg[32 * c + 2 * e]), sc, neg_m));
+        const float p1 = ex2(fmaf(__uint_as_float(sreg[32 * c + 2 * e + 1]), sc, neg_m));
+        sm4[e & 1] += p0;
+        sm4[2 + (e & 1)] += p1;
+        packed[e] = pack2<kBf16>(p0, p1);
+      }
+      tmem_st16(tmem_s + 16u * c, packed);
+    }
+    l = l * alpha + ((sm4[0] + sm4[1]) + (sm4[2] + sm4[3]));
+    if (threadIdx.x == 128) UTRACE(2, 4);
+    tc_wait_st();
+    tc_fence_before();
+    mbar_arrive(&sm->p_full[chain]);
+  }
+  // both chains must be done with the tensor pipe before the K/V stages are reused as staging
+  for (int c = 0; c < 2; ++c) {
+    const int n_c = nblk > c ? (nblk - c + 1) >> 1 : 0;
+    if (n_c > 0 && ok) ok = mbar_wait(sm, &sm->pv_done[c], (n_c - 1) & 1, a.dev_status);
+  }
+  tc_fence_after();
+
+  // ---------------------------------------------------------------- merge ------------------------
+  // Slice s (output columns [8s, 8s+8)) is owned by chain w = s % workers, workers = 2*splits, chain
+  // index = 2*cta + chain.  An owner's receive buffer is its chain's 64 KB staging area, laid out as
+  // float4 planes [contributor][owned slice][half][row], so that a warp's 32 rows are contiguous.
+  const int workers = 2 * a.splits, me = 2 * split + chain;
+  const int per_owner = (16 + workers - 1) / workers;  // slices an owner can hold
+  if (threadIdx.x == 128) UTRACE(2, 6);
+  tc_fence_before();
+  cluster.sync();  // every CTA of the cluster is done with its K/V stages before anyone writes into them
+  if (threadIdx.x == 128) UTRACE(2, 7);
+  {
+    const bool have = ok && n_mine > 0;
+    const float2 mine_ml = have ? make_float2(m_used, l) : make_float2(-INFINITY, 0.f);
+    for (int q = 0; q < a.splits; ++q) *cluster.map_shared_rank(&sm->ml[me][r], q) = mine_ml;
+    if (have) {
+#pragma unroll
+      for (int c = 0; c < 4; ++c) {
+        uint32_t o[32];
+        tmem_ld32(tmem_o + 32u * c, o, 0);
+        tc_wait_ld();
+#pragma unroll
+        for (int e = 0; e < 32; e += 8) {
+          const int slice = 4 * c + (e >> 3);
+          const int w = slice % workers;
+          uint4* base = reinterpret_cast<uint4*>((w & 1) == 0 ? sm->k[0] : sm->v[0]);
+          uint4* dst = cluster.map_shared_rank(base, w >> 1) + ((size_t)(me * per_owner + slice / workers) * 2) * kTileM + r;
+          dst[0] = make_uint4(o[e], o[e + 1], o[e + 2], o[e + 3]);
+          dst[kTileM] = make_uint4(o[e + 4], o[e + 5], o[e + 6], o[e + 7]);
         }
       }
-      if (row_valid) a.ml[prow_idx] = (ok && nblk > 0) ? make_float2(m_used, l) : make_float2(-INFINITY, 0.f);
     }
-    tc_fence_before();
   }
-
-  __syncthreads();
-  if (warp == 1) {
-    tc_fence_after();
-    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, 512;" ::"r"(tmem) : "memory");
+  cluster.sync();
+  if (threadIdx.x == 128) UTRACE(2, 8);
+  {
+    float M = -INFINITY;
+    for (int p = 0; p < workers; ++p) M = fmaxf(M, sm->ml[p][r].x);
+    float Ls = 0.f;
+    for (int p = 0; p < workers; ++p) {
+      const float2 mlp = sm->ml[p][r];
+      if (mlp.x != -INFINITY) Ls += mlp.y * ex2(mlp.x - M);
+    }
+    const float inv = 1.f / Ls;  // some chain saw the row's own key, so Ls > 0
+    const float4* mine = reinterpret_cast<const float4*>(chain == 0 ? sm->k[0] : sm->v[0]);
+    for (int slot = 0, slice = me; slice < 16; ++slot, slice += workers) {
+      float acc[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+      for (int p = 0; p < workers; ++p) {
+        const float mp = sm->ml[p][r].x;
+        if (mp == -INFINITY) continue;
+        const float f = ex2(mp - M);
+        const float4* src = mine + ((size_t)(p * per_owner + slot) * 2) * kTileM + r;
+        const float4 x = src[0], y = src[kTileM];
+        acc[0] = fmaf(x.x, f, acc[0]); acc[1] = fmaf(x.y, f, acc[1]); acc[2] = fmaf(x.z, f, acc[2]); acc[3] = fmaf(x.w, f, acc[3]);
+        acc[4] = fmaf(y.x, f, acc[4]); acc[5] = fmaf(y.y, f, acc[5]); acc[6] = fmaf(y.z, f, acc[6]); acc[7] = fmaf(y.w, f, acc[7]);
+      }
+      if (row_valid) {
+        uint4 val;
+        val.x = pack2<kBf16>(acc[0] * inv, acc[1] * inv);
+        val.y = pack2<kBf16>(acc[2] * inv, acc[3] * inv);
+        val.z = pack2<kBf16>(acc[4] * inv, acc[5] * inv);
+        val.w = pack2<kBf16>(acc[6] * inv, acc[7] * inv);
+        *reinterpret_cast<uint4*>(reinterpret_cast<uint8_t*>(a.out) +
+                                  2 * ((int64_t)i * a.o_stride_tok + (int64_t)h * a.o_stride_head + 8 * slice)) = val;
+      }
+    }
+    if (me == 0 && row_valid && a.lse != nullptr) a.lse[(size_t)h * a.n + i] = (M + log2f(Ls)) * kLn2;
   }
+  if (threadIdx.x == 128) UTRACE(2, 9);
+  // no remote access happens after the second cluster barrier, so CTAs may leave independently
+  tc_fence_before();
+  __syncthreads();  // pairs with warp group 0, whose MMA warp then frees the tensor memory
 }
 
 // ---------------------------------------------------------------- host side ---------------------
@@ -449,17 +543,27 @@ bool umma_supported(const seq_tree_attention_params& p) {
   return true;
 }
 
+// Size of the cluster that shares one (tile, kv head): 1, 2, 4 or 8 CTAs along the key range, chosen for the
+// shortest estimated makespan with one CTA per SM (about 0.9 us per key block with both chains busy,
+// about 4 us of fixed cost per CTA).
 int umma_default_splits(const seq_tree_attention_params& p) {
   const int G = p.num_q_heads / p.num_kv_heads;
   const int nodes_per_tile = kTileM / G;
   const int tiles = (p.n_tree + nodes_per_tile - 1) / nodes_per_tile;
-  const int ctas = tiles * p.num_kv_heads;
+  const long units = (long)tiles * p.num_kv_heads;
   const int nblk = (p.prefix_len + p.n_tree + kBlockN - 1) / kBlockN;
-  int splits = 148 / ctas;  // one CTA per SM: fill the machine in one wave when the tiles alone cannot
-  if (splits < 1) splits = 1;
-  if (splits > nblk) splits = nblk;
-  if (splits > 32) splits = 32;
-  return splits;
+#ifdef SEQ_TRACE
+  if (const char* e = getenv("SEQ_DEBUG_SPLITS")) return atoi(e);  // debug builds only
+#endif
+  int best = 1;
+  double best_cost = -1.0;
+  for (int cs = 1; cs <= kMaxClusterSplit; cs *= 2) {  // powers of two: 16 slices divide evenly among 2*cs chains
+    if (cs > 1 && cs > nblk) break;
+    const long waves = (units * cs + kNumSMs - 1) / kNumSMs;
+    const double cost = (double)waves * (0.9 * ((nblk + cs - 1) / cs) + 4.0);
+    if (best_cost < 0 || cost < best_cost - 1e-9) { best = cs; best_cost = cost; }
+  }
+  return best;
 }
 
 int launch_attention_umma(const seq_tree_attention_params& p, int splits, cudaStream_t stream) {
@@ -508,22 +612,39 @@ int launch_attention_umma(const seq_tree_attention_params& p, int splits, cudaSt
   a.mask_bits = p.mask_bits;
   a.out = p.out; a.o_stride_tok = p.o_stride_tok; a.o_stride_head = p.o_stride_head;
   a.lse = p.lse;
-  SplitLayout sl = split_layout(p.workspace, splits, p.num_q_heads, p.n_tree);
-  a.o_part = sl.o_part; a.ml = sl.ml;
   a.dev_status = p.dev_status;
 
   const size_t smem = sizeof(UmmaSmem) + 1024;
-  dim3 grid(tiles, p.num_kv_heads, splits);
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(tiles, p.num_kv_heads, splits);
+  cfg.blockDim = dim3(kUmmaThreads);
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = stream;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeClusterDimension;
+  attr[0].val.clusterDim.x = 1;
+  attr[0].val.clusterDim.y = 1;
+  attr[0].val.clusterDim.z = splits;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
   if (p.dtype == SEQ_BF16) {
     SEQ_CUDA_OK(cudaFuncSetAttribute(tree_attention_umma_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-    tree_attention_umma_kernel<true><<<grid, kUmmaThreads, smem, stream>>>(q_map, k_map, v_map, a);
+    SEQ_CUDA_OK(cudaLaunchKernelEx(&cfg, tree_attention_umma_kernel<true>, q_map, k_map, v_map, a));
   } else {
     SEQ_CUDA_OK(cudaFuncSetAttribute(tree_attention_umma_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-    tree_attention_umma_kernel<false><<<grid, kUmmaThreads, smem, stream>>>(q_map, k_map, v_map, a);
+    SEQ_CUDA_OK(cudaLaunchKernelEx(&cfg, tree_attention_umma_kernel<false>, q_map, k_map, v_map, a));
   }
-  SEQ_CUDA_OK(cudaGetLastError());
-  if (splits > 1) return launch_combine_splits(p, splits, stream);
   return SEQ_OK;
 }
 
 }  // namespace seqtree
+
+#ifdef SEQ_TRACE
+extern "C" int seq_debug_utrace_dump(unsigned long long* host_out) {
+  cudaDeviceSynchronize();
+  cudaMemcpyFromSymbol(host_out, seqtree::g_utrace, sizeof(unsigned long long) * 4 * 512);
+  static unsigned long long zeros[4 * 512];
+  cudaMemcpyToSymbol(seqtree::g_utrace, zeros, sizeof(zeros));
+  return 0;
+}
+#endif
