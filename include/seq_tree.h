@@ -132,6 +132,33 @@ size_t seq_tree_attention_workspace_bytes(const seq_tree_attention_params* p);
 int seq_tree_attention(const seq_tree_attention_params* p, void* stream);
 
 /*
+ * seq_tree_attention_noalloc -- the CUDA-core variant of seq_tree_attention for callers that
+ * cannot provide scratch memory.  (The paper has no counterpart: this is a deployment convenience.)
+ *
+ * Who needs it: a serving process whose device memory is handed out once at start-up and frozen
+ * afterwards (no allocator is reachable from the decoding loop, or an allocation there would
+ * synchronise the device and stall every other stream), and small embedders that link this library
+ * without any tensor framework and so have nothing to size or own a workspace with.
+ *
+ * Same arguments, semantics and results as seq_tree_attention run with kernel = 1 (the CUDA-core
+ * kernel, any dtype); p->workspace, p->workspace_bytes and p->kernel are ignored.  The split-KV
+ * partial results go to a fixed array of SEQ_NOALLOC_SCRATCH_BYTES that lives inside the library
+ * image on every device that loads it, until the process exits.  The call allocates nothing: no
+ * cudaMalloc/cudaFree and no allocating library routine.
+ *
+ *   - A request whose partials need more than SEQ_NOALLOC_SCRATCH_BYTES returns SEQ_ERR_WORKSPACE
+ *     and launches nothing (use seq_tree_attention with your own workspace instead).
+ *   - The first call on a device looks up the array's device address (one cheap runtime query with
+ *     that device current) and remembers it; make that first call during start-up, before any
+ *     stream capture is begun on that device.
+ *   - All calls share the one array, and it keeps whatever the previous call left there.  Nothing
+ *     in it has to start at zero: every partial a call reads was written by that same call.  Two
+ *     calls that overlap on the GPU (different streams) race on it; serialise them.
+ */
+#define SEQ_NOALLOC_SCRATCH_BYTES (384u << 10)
+int seq_tree_attention_noalloc(const seq_tree_attention_params* p, void* stream);
+
+/*
  * seq_tree_verify -- Algorithm 2 applied recursively from the root (Section
  * 2.2), then its last line x ~ R at the node where the walk stops.
  *

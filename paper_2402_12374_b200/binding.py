@@ -19,6 +19,7 @@ SEQ_F16, SEQ_BF16, SEQ_F32 = 0, 1, 2
 SEQ_DEV_BAD_PARENT, SEQ_DEV_BAD_TOKEN, SEQ_DEV_NONFINITE, SEQ_DEV_DEGENERATE, SEQ_DEV_TIMEOUT = 1, 2, 4, 8, 16
 SEQ_VERIFY_ALL_NODES = 1
 SEQ_MAX_TREE = 1024
+SEQ_NOALLOC_SCRATCH_BYTES = 384 << 10
 KERNEL_AUTO, KERNEL_CUDA_CORE, KERNEL_TENSOR_CORE = 0, 1, 2
 
 _STATUS_NAMES = {0: "SEQ_OK", -1: "SEQ_ERR_INVALID_ARG", -2: "SEQ_ERR_UNSUPPORTED", -3: "SEQ_ERR_WORKSPACE",
@@ -29,6 +30,7 @@ EXPORTED_SYMBOLS = (
     "seq_tree_mask_from_parents",
     "seq_tree_attention_workspace_bytes",
     "seq_tree_attention",
+    "seq_tree_attention_noalloc",
     "seq_tree_verify_workspace_bytes",
     "seq_tree_verify",
     "seq_tree_version",
@@ -88,6 +90,8 @@ def load() -> C.CDLL:
         lib.seq_tree_attention_workspace_bytes.restype = C.c_size_t
         lib.seq_tree_attention.argtypes = [C.POINTER(AttentionParams), C.c_void_p]
         lib.seq_tree_attention.restype = C.c_int
+        lib.seq_tree_attention_noalloc.argtypes = [C.POINTER(AttentionParams), C.c_void_p]
+        lib.seq_tree_attention_noalloc.restype = C.c_int
         lib.seq_tree_verify_workspace_bytes.argtypes = [C.POINTER(VerifyParams)]
         lib.seq_tree_verify_workspace_bytes.restype = C.c_size_t
         lib.seq_tree_verify.argtypes = [C.POINTER(VerifyParams), C.c_void_p]
@@ -142,7 +146,10 @@ class AttentionCall:
     """A prepared seq_tree_attention call: the parameter struct is filled once and can be launched many times."""
 
     def __init__(self, q, k_cache, v_cache, mask_bits, prefix_len: int, *, out=None, lse=None,
-                 softmax_scale: float = 0.0, workspace=None, dev_status=None, kernel: int = KERNEL_AUTO):
+                 softmax_scale: float = 0.0, workspace=None, dev_status=None, kernel: int = KERNEL_AUTO,
+                 noalloc: bool = False):
+        """``noalloc=True`` prepares a call of ``seq_tree_attention_noalloc``: no workspace tensor is
+        created or passed; the library's built-in scratch array is used (CUDA-core kernel)."""
         if q.dtype not in _DTYPES or k_cache.dtype != q.dtype or v_cache.dtype != q.dtype:
             raise ValueError("q, k_cache, v_cache must share one of float16/bfloat16/float32")
         n, Hq, d = q.shape
@@ -167,7 +174,8 @@ class AttentionCall:
         p.lse = _dev(lse, "lse", torch.float32)
         p.dev_status = _dev(dev_status, "dev_status", torch.int32)
         p.kernel = kernel
-        need = load().seq_tree_attention_workspace_bytes(C.byref(p))
+        self.noalloc = noalloc
+        need = 0 if noalloc else load().seq_tree_attention_workspace_bytes(C.byref(p))
         if workspace is None and need:
             workspace = torch.empty(need, dtype=torch.uint8, device=q.device)
         p.workspace = _dev(workspace, "workspace") if workspace is not None else None
@@ -176,7 +184,10 @@ class AttentionCall:
         self._keep = (q, k_cache, v_cache, mask_bits, out, lse, workspace, dev_status)
 
     def run(self, stream=None):
-        _check("seq_tree_attention", load().seq_tree_attention(C.byref(self.params), _stream(stream)))
+        if self.noalloc:
+            _check("seq_tree_attention_noalloc", load().seq_tree_attention_noalloc(C.byref(self.params), _stream(stream)))
+        else:
+            _check("seq_tree_attention", load().seq_tree_attention(C.byref(self.params), _stream(stream)))
         return self.out
 
 
@@ -184,6 +195,13 @@ def seq_tree_attention(q, k_cache, v_cache, mask_bits, prefix_len: int, **kw):
     """Tree-masked attention of the n tree tokens; returns out [n, Hq, d] (same dtype as q)."""
     stream = kw.pop("stream", None)
     return AttentionCall(q, k_cache, v_cache, mask_bits, prefix_len, **kw).run(stream)
+
+
+def seq_tree_attention_noalloc(q, k_cache, v_cache, mask_bits, prefix_len: int, **kw):
+    """seq_tree_attention for callers that cannot provide scratch memory: same result as the CUDA-core
+    kernel, split-KV partials in the library's built-in array (see ``include/seq_tree.h``)."""
+    stream = kw.pop("stream", None)
+    return AttentionCall(q, k_cache, v_cache, mask_bits, prefix_len, noalloc=True, **kw).run(stream)
 
 
 class VerifyCall:

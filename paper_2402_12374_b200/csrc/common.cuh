@@ -78,7 +78,8 @@ inline SplitLayout split_layout(void* workspace, int splits, int Hq, int n) {
   return s;
 }
 
-// attention kernels (host launchers; defined in their own .cu files)
+// attention: argument checks shared by the entry points, and the kernels' host launchers
+int validate_attention_params(const seq_tree_attention_params* p);
 int launch_attention_simt(const seq_tree_attention_params& p, int splits, cudaStream_t stream);
 int simt_default_splits(const seq_tree_attention_params& p);
 int launch_combine_splits(const seq_tree_attention_params& p, int splits, cudaStream_t stream);

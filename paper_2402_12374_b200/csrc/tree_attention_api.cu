@@ -12,7 +12,7 @@ int launch_attention_umma(const seq_tree_attention_params& p, int splits, cudaSt
 
 static size_t elem_size(int dtype) { return dtype == SEQ_F32 ? 4 : 2; }
 
-static int validate(const seq_tree_attention_params* p) {
+int validate_attention_params(const seq_tree_attention_params* p) {
   if (p == nullptr) return SEQ_ERR_INVALID_ARG;
   if (p->q == nullptr || p->k_cache == nullptr || p->v_cache == nullptr || p->out == nullptr ||
       p->mask_bits == nullptr)
@@ -55,7 +55,7 @@ static int choose_kernel(const seq_tree_attention_params& p) {
 using namespace seqtree;
 
 extern "C" size_t seq_tree_attention_workspace_bytes(const seq_tree_attention_params* p) {
-  if (validate(p) != SEQ_OK) return 0;
+  if (validate_attention_params(p) != SEQ_OK) return 0;
   const int which = choose_kernel(*p);
   if (which == 0) return 0;
   if (which == 2) return 0;  // the tensor-core kernel merges its key-range shares on chip
@@ -65,7 +65,7 @@ extern "C" size_t seq_tree_attention_workspace_bytes(const seq_tree_attention_pa
 }
 
 extern "C" int seq_tree_attention(const seq_tree_attention_params* p, void* stream) {
-  int rc = validate(p);
+  int rc = validate_attention_params(p);
   if (rc != SEQ_OK) return rc;
   const int which = choose_kernel(*p);
   if (which == 0) return SEQ_ERR_UNSUPPORTED;

@@ -297,3 +297,42 @@ int launch_combine_splits(const seq_tree_attention_params& p, int splits, cudaSt
 }
 
 }  // namespace seqtree
+
+// ---------------------------------------------------------------------------------------------------
+// seq_tree_attention_noalloc: the same CUDA-core kernels, with the split-KV partials in a fixed array
+// that is part of the library image instead of a caller-provided workspace.
+//
+// `g_noalloc_scratch` names the array in device code.  In host code the same identifier is only a
+// handle for the runtime: its device address has to be asked for with cudaGetSymbolAddress, once per
+// device, with that device current; passing the identifier itself to a kernel would hand it a host
+// address.
+static __device__ __align__(256) unsigned char g_noalloc_scratch[SEQ_NOALLOC_SCRATCH_BYTES];
+
+namespace {
+constexpr int kMaxDevices = 64;
+void* g_noalloc_ptr[kMaxDevices];  // device address of g_noalloc_scratch on each device, 0 = not looked up yet
+}  // namespace
+
+extern "C" int seq_tree_attention_noalloc(const seq_tree_attention_params* p, void* stream) {
+  using namespace seqtree;
+  int rc = validate_attention_params(p);
+  if (rc != SEQ_OK) return rc;
+  const int splits = simt_default_splits(*p);
+  const size_t need = splits > 1 ? split_workspace_bytes(splits, p->num_q_heads, p->n_tree) : 0;
+  if (need > SEQ_NOALLOC_SCRATCH_BYTES) return SEQ_ERR_WORKSPACE;  // too large for the built-in array
+
+  int dev = -1;
+  SEQ_CUDA_OK(cudaGetDevice(&dev));
+  if (dev < 0 || dev >= kMaxDevices) return SEQ_ERR_UNSUPPORTED;
+  if (g_noalloc_ptr[dev] == nullptr) {  // set-up: first call on this device
+    void* ptr = nullptr;
+    SEQ_CUDA_OK(cudaGetSymbolAddress(&ptr, g_noalloc_scratch));
+    if (ptr == nullptr) return SEQ_ERR_CUDA;
+    g_noalloc_ptr[dev] = ptr;
+  }
+  seq_tree_attention_params q = *p;
+  q.workspace = g_noalloc_ptr[dev];
+  q.workspace_bytes = SEQ_NOALLOC_SCRATCH_BYTES;
+  q.kernel = 1;
+  return launch_attention_simt(q, splits, (cudaStream_t)stream);
+}
