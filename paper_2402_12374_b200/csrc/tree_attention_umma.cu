@@ -69,7 +69,8 @@ struct UmmaSmem {
   uint8_t q[kTileBytes];
   uint8_t k[2][kTileBytes];  // K stage of chain A, of chain B; after the last block: chain A's 128x128 fp32 accumulator
   uint8_t v[2][kTileBytes];  // V stage of chain A, of chain B; after the last block: chain B's accumulator
-  float2 ml[2 * kMaxClusterSplit][kTileM];  // (m, l) of every row of every chain of the cluster, for the merge
+  float2 ml_chain[2][kTileM];                // (m, l) of every row of the two chains of this CTA
+  float2 ml_cta[kMaxClusterSplit][kTileM];   // (m, l) of every row of every CTA of the cluster, after its chains are merged
   uint64_t q_full, k_full[2], k_empty[2], v_full[2], v_empty[2], s_full[2], p_full[2], pv_done[2];
   uint32_t tmem_base;
   volatile int abort_flag;
@@ -240,6 +241,7 @@ tree_attention_umma_kernel(const __grid_constant__ CUtensorMap q_map, const __gr
   int utrace_i = 0;
 #endif
   const int tile = blockIdx.x, g = blockIdx.y, split = blockIdx.z;  // the cluster spans blockIdx.z
+  if (threadIdx.x == 128) UTRACE(2, 10);
 
   const int i0 = tile * a.nodes_per_tile;
   const int i1 = min(i0 + a.nodes_per_tile, a.n);
@@ -259,6 +261,7 @@ tree_attention_umma_kernel(const __grid_constant__ CUtensorMap q_map, const __gr
     sm->abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
+  if (threadIdx.x == 128) UTRACE(2, 11);
   if (warp == 1) {  // all 512 tensor-memory columns: S_A, S_B (P over them), O_A, O_B
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], 512;" ::"r"(smem_u32(&sm->tmem_base)) : "memory");
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
@@ -338,9 +341,11 @@ tree_attention_umma_kernel(const __grid_constant__ CUtensorMap q_map, const __gr
       }
       __syncwarp();
     }
-    cluster.sync();  // the two cluster barriers of the merge (see the row threads)
-    cluster.sync();
-    UTRACE(1, 9);
+    if (a.splits > 1) {  // the two cluster barriers of the merge (see the row threads)
+      cluster.sync();
+      cluster.sync();
+    }
+    if (threadIdx.x == 32) UTRACE(1, 9);
     tc_fence_before();
     __syncthreads();
     if (warp == 1) {
@@ -383,56 +388,65 @@ tree_attention_umma_kernel(const __grid_constant__ CUtensorMap q_map, const __gr
     }
     tc_wait_ld();
     if (threadIdx.x == 128) UTRACE(2, 2);
-    // block maximum of the raw scores (four independent chains); masked scores become -inf first
-    float mx[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
-    if (masked) {
+    if (masked) {  // masked scores become -inf: probability exactly 0, and they cannot raise the maximum
 #pragma unroll
-      for (int e = 0; e < 128; ++e) {
-        const float sv = (vis[e >> 5] & (1u << (e & 31))) ? __uint_as_float(sreg[e]) : -INFINITY;
-        sreg[e] = __float_as_uint(sv);
-        mx[e & 3] = fmaxf(mx[e & 3], sv);
-      }
-    } else {
-#pragma unroll
-      for (int e = 0; e < 128; ++e) mx[e & 3] = fmaxf(mx[e & 3], __uint_as_float(sreg[e]));
+      for (int e = 0; e < 128; ++e)
+        if (!(vis[e >> 5] & (1u << (e & 31)))) sreg[e] = __float_as_uint(-INFINITY);
     }
-    const float m_blk = fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3])) * sc;  // scale > 0
-    // move the reference maximum only when it is first set or exceeded by more than the threshold
-    float alpha = 1.f;
-    if (m_blk > m_used + kRescaleThreshold || (m_used == -INFINITY && m_blk != -INFINITY)) {
-      alpha = m_used == -INFINITY ? 0.f : ex2(m_used - m_blk);
-      m_used = m_blk;
-    }
-    // this S was issued after O took the chain's previous block, so O is quiescent here
-    if (u > 0 && __any_sync(0xffffffffu, alpha != 1.f)) {  // rescale the accumulator rows of this warp
+    // P = 2^(scale*s - m) written over S as packed 16-bit values (64 columns, four stores of 16), with the
+    // block maximum taken in the same sweep: the exponentials are MUFU-bound, so the comparisons ride
+    // along.  The sweep first assumes the reference maximum does not have to move; if the block maximum
+    // turns out to exceed it by more than the threshold (or there is no reference yet) it is redone once.
+    // (A row without a reference that sees nothing in this block has all scores -inf: its P are 0.)
+    auto sweep = [&](float neg_m, float& m_raw) -> float {
+      float sm4[4] = {0.f, 0.f, 0.f, 0.f};
+      float mx[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
 #pragma unroll
       for (int c = 0; c < 4; ++c) {
-        uint32_t o[32];
-        tmem_ld32(tmem_o + 32u * c, o, 0);
-        tc_wait_ld();
+        uint32_t packed[16];
 #pragma unroll
-        for (int e = 0; e < 32; ++e) o[e] = __float_as_uint(__uint_as_float(o[e]) * alpha);
-        tmem_st32(tmem_o + 32u * c, o, 0);
+        for (int e = 0; e < 16; ++e) {
+          const float s0 = __uint_as_float(sreg[32 * c + 2 * e]), s1 = __uint_as_float(sreg[32 * c + 2 * e + 1]);
+          mx[e & 1] = fmaxf(mx[e & 1], s0);
+          mx[2 + (e & 1)] = fmaxf(mx[2 + (e & 1)], s1);
+          const float p0 = ex2(fmaf(s0, sc, neg_m));
+          const float p1 = ex2(fmaf(s1, sc, neg_m));
+          sm4[e & 1] += p0;
+          sm4[2 + (e & 1)] += p1;
+          packed[e] = pack2<kBf16>(p0, p1);
+        }
+        tmem_st16(tmem_s + 16u * c, packed);
+      }
+      m_raw = fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3]));
+      return (sm4[0] + sm4[1]) + (sm4[2] + sm4[3]);
+    };
+    float alpha = 1.f, m_raw;
+    float sum = sweep(m_used == -INFINITY ? 0.f : -m_used, m_raw);
+    {
+      const float m_blk = m_raw * sc;  // scale > 0
+      const bool move = m_blk > m_used + kRescaleThreshold || (m_used == -INFINITY && m_blk != -INFINITY);
+      if (__any_sync(0xffffffffu, move)) {  // rare: the whole warp redoes the block (rows that do not move get the same P again)
+        if (move) {
+          alpha = m_used == -INFINITY ? 0.f : ex2(m_used - m_blk);
+          m_used = m_blk;
+        }
+        // this S was issued after O took the chain's previous block, so O is quiescent here
+        if (u > 0) {
+#pragma unroll
+          for (int c = 0; c < 4; ++c) {
+            uint32_t o[32];
+            tmem_ld32(tmem_o + 32u * c, o, 0);
+            tc_wait_ld();
+#pragma unroll
+            for (int e = 0; e < 32; ++e) o[e] = __float_as_uint(__uint_as_float(o[e]) * alpha);
+            tmem_st32(tmem_o + 32u * c, o, 0);
+          }
+        }
+        sum = sweep(m_used == -INFINITY ? 0.f : -m_used, m_raw);
       }
     }
     if (threadIdx.x == 128) UTRACE(2, 3);
-    const float neg_m = m_used == -INFINITY ? 0.f : -m_used;
-    float sm4[4] = {0.f, 0.f, 0.f, 0.f};
-    // P = 2^(scale*s - m) written over S as packed 16-bit values: 64 columns, four stores of 16
-#pragma unroll
-    for (int c = 0; c < 4; ++c) {
-      uint32_t packed[16];
-#pragma unroll
-      for (int e = 0; e < 16; ++e) {
-        const float p0 = ex2(fmaf(__uint_as_float(sreg[32 * c + 2 * e]), sc, neg_m));
-        const float p1 = ex2(fmaf(__uint_as_float(sreg[32 * c + 2 * e + 1]), sc, neg_m));
-        sm4[e & 1] += p0;
-        sm4[2 + (e & 1)] += p1;
-        packed[e] = pack2<kBf16>(p0, p1);
-      }
-      tmem_st16(tmem_s + 16u * c, packed);
-    }
-    l = l * alpha + ((sm4[0] + sm4[1]) + (sm4[2] + sm4[3]));
+    l = l * alpha + sum;
     if (threadIdx.x == 128) UTRACE(2, 4);
     tc_wait_st();
     tc_fence_before();
@@ -446,56 +460,95 @@ tree_attention_umma_kernel(const __grid_constant__ CUtensorMap q_map, const __gr
   tc_fence_after();
 
   // ---------------------------------------------------------------- merge ------------------------
-  // Slice s (output columns [8s, 8s+8)) is owned by chain w = s % workers, workers = 2*splits, chain
-  // index = 2*cta + chain.  An owner's receive buffer is its chain's 64 KB staging area, laid out as
-  // float4 planes [contributor][owned slice][half][row], so that a warp's 32 rows are contiguous.
-  const int workers = 2 * a.splits, me = 2 * split + chain;
-  const int per_owner = (16 + workers - 1) / workers;  // slices an owner can hold
+  // Step 1, inside the CTA: both accumulators live in this CTA's tensor memory and a warp may read
+  // any column of its 32 lanes, so the thread of chain c and row r merges columns [64c, 64c+64) of
+  // O_A and O_B itself; only (m, l) goes through shared memory.
   if (threadIdx.x == 128) UTRACE(2, 6);
-  tc_fence_before();
-  cluster.sync();  // every CTA of the cluster is done with its K/V stages before anyone writes into them
-  if (threadIdx.x == 128) UTRACE(2, 7);
+  sm->ml_chain[chain][r] = (ok && n_mine > 0) ? make_float2(m_used, l) : make_float2(-INFINITY, 0.f);
+  asm volatile("bar.sync 1, 256;" ::: "memory");  // the 256 row threads only
+  float M, Lc;           // reference maximum and denominator of the CTA's merged partial
+  float merged[64];      // its columns [64*chain, 64*chain + 64), unnormalised
   {
-    const bool have = ok && n_mine > 0;
-    const float2 mine_ml = have ? make_float2(m_used, l) : make_float2(-INFINITY, 0.f);
-    for (int q = 0; q < a.splits; ++q) *cluster.map_shared_rank(&sm->ml[me][r], q) = mine_ml;
-    if (have) {
+    const float2 mlA = sm->ml_chain[0][r], mlB = sm->ml_chain[1][r];
+    M = fmaxf(mlA.x, mlB.x);
+    const float fA = mlA.x == -INFINITY ? 0.f : ex2(mlA.x - M), fB = mlB.x == -INFINITY ? 0.f : ex2(mlB.x - M);
+    Lc = mlA.y * fA + mlB.y * fB;
+    const int nA = nblk > 0 ? (nblk + 1) >> 1 : 0, nB = nblk >> 1;  // CTA-uniform: which accumulators were written
+    const uint32_t oA = tmem + 256u + lane_sel + 64u * chain, oB = oA + 128u;
 #pragma unroll
-      for (int c = 0; c < 4; ++c) {
-        uint32_t o[32];
-        tmem_ld32(tmem_o + 32u * c, o, 0);
-        tc_wait_ld();
+    for (int e = 0; e < 64; ++e) merged[e] = 0.f;
+    if (nA > 0 && ok) {
+      uint32_t o[64];
+      tmem_ld32(oA, o, 0);
+      tmem_ld32(oA + 32u, o, 32);
+      tc_wait_ld();
 #pragma unroll
-        for (int e = 0; e < 32; e += 8) {
-          const int slice = 4 * c + (e >> 3);
-          const int w = slice % workers;
-          uint4* base = reinterpret_cast<uint4*>((w & 1) == 0 ? sm->k[0] : sm->v[0]);
-          uint4* dst = cluster.map_shared_rank(base, w >> 1) + ((size_t)(me * per_owner + slice / workers) * 2) * kTileM + r;
-          dst[0] = make_uint4(o[e], o[e + 1], o[e + 2], o[e + 3]);
-          dst[kTileM] = make_uint4(o[e + 4], o[e + 5], o[e + 6], o[e + 7]);
-        }
-      }
+      for (int e = 0; e < 64; ++e) merged[e] = __uint_as_float(o[e]) * fA;
+    }
+    if (nB > 0 && ok) {
+      uint32_t o[64];
+      tmem_ld32(oB, o, 0);
+      tmem_ld32(oB + 32u, o, 32);
+      tc_wait_ld();
+#pragma unroll
+      for (int e = 0; e < 64; ++e) merged[e] = fmaf(__uint_as_float(o[e]), fB, merged[e]);
     }
   }
-  cluster.sync();
-  if (threadIdx.x == 128) UTRACE(2, 8);
-  {
-    float M = -INFINITY;
-    for (int p = 0; p < workers; ++p) M = fmaxf(M, sm->ml[p][r].x);
-    float Ls = 0.f;
-    for (int p = 0; p < workers; ++p) {
-      const float2 mlp = sm->ml[p][r];
-      if (mlp.x != -INFINITY) Ls += mlp.y * ex2(mlp.x - M);
+  uint8_t* out_row = reinterpret_cast<uint8_t*>(a.out) + 2 * ((int64_t)i * a.o_stride_tok + (int64_t)h * a.o_stride_head);
+  if (a.splits == 1) {
+    if (row_valid) {
+      const float inv = 1.f / Lc;  // the row saw at least its own key, so Lc > 0
+#pragma unroll
+      for (int e = 0; e < 64; e += 8) {
+        uint4 val;
+        val.x = pack2<kBf16>(merged[e] * inv, merged[e + 1] * inv);
+        val.y = pack2<kBf16>(merged[e + 2] * inv, merged[e + 3] * inv);
+        val.z = pack2<kBf16>(merged[e + 4] * inv, merged[e + 5] * inv);
+        val.w = pack2<kBf16>(merged[e + 6] * inv, merged[e + 7] * inv);
+        *reinterpret_cast<uint4*>(out_row + 2 * (64 * chain + e)) = val;
+      }
+      if (chain == 0 && a.lse != nullptr) a.lse[(size_t)h * a.n + i] = (M + log2f(Lc)) * kLn2;
     }
-    const float inv = 1.f / Ls;  // some chain saw the row's own key, so Ls > 0
-    const float4* mine = reinterpret_cast<const float4*>(chain == 0 ? sm->k[0] : sm->v[0]);
-    for (int slot = 0, slice = me; slice < 16; ++slot, slice += workers) {
+  } else {
+    // Step 2, across the cluster (cs = 2, 4 or 8 CTAs along the key range).  The 16 slices of 8 output
+    // columns are owned round-robin: slice s by CTA s % cs, as its slot s / cs.  Every CTA pushes each
+    // 8-column piece of its merged partial into the owner's receive buffer (the K stages, dead by
+    // then), laid out as float4 planes [contributor][slot][half][row], and its (m, l) into every CTA,
+    // with plain remote stores; after a cluster barrier each owner reduces its slots locally.
+    const int cs = a.splits, slots = 16 / cs;
+    tc_fence_before();
+    cluster.sync();  // every CTA of the cluster is done with its K stages before anyone writes into them
+    if (threadIdx.x == 128) UTRACE(2, 7);
+    if (chain == 0)
+      for (int q = 0; q < cs; ++q) *cluster.map_shared_rank(&sm->ml_cta[split][r], q) = make_float2(M, Lc);
+#pragma unroll
+    for (int j = 0; j < 8; ++j) {
+      const int s_idx = 8 * chain + j;
+      uint4* dst = cluster.map_shared_rank(reinterpret_cast<uint4*>(sm->k[0]), s_idx % cs) +
+                   ((size_t)(split * slots + s_idx / cs) * 2) * kTileM + r;
+      dst[0] = make_uint4(__float_as_uint(merged[8 * j]), __float_as_uint(merged[8 * j + 1]),
+                          __float_as_uint(merged[8 * j + 2]), __float_as_uint(merged[8 * j + 3]));
+      dst[kTileM] = make_uint4(__float_as_uint(merged[8 * j + 4]), __float_as_uint(merged[8 * j + 5]),
+                               __float_as_uint(merged[8 * j + 6]), __float_as_uint(merged[8 * j + 7]));
+    }
+    cluster.sync();
+    if (threadIdx.x == 128) UTRACE(2, 8);
+    float Mg = -INFINITY;
+    for (int q = 0; q < cs; ++q) Mg = fmaxf(Mg, sm->ml_cta[q][r].x);
+    float Ls = 0.f;
+    for (int q = 0; q < cs; ++q) {
+      const float2 mlq = sm->ml_cta[q][r];
+      if (mlq.x != -INFINITY) Ls += mlq.y * ex2(mlq.x - Mg);
+    }
+    const float inv = 1.f / Ls;  // some CTA saw the row's own key, so Ls > 0
+    const float4* mine = reinterpret_cast<const float4*>(sm->k[0]);
+    for (int slot = chain; slot < slots; slot += 2) {  // the two warp groups share this CTA's slots
       float acc[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
-      for (int p = 0; p < workers; ++p) {
-        const float mp = sm->ml[p][r].x;
-        if (mp == -INFINITY) continue;
-        const float f = ex2(mp - M);
-        const float4* src = mine + ((size_t)(p * per_owner + slot) * 2) * kTileM + r;
+      for (int q = 0; q < cs; ++q) {
+        const float mq = sm->ml_cta[q][r].x;
+        if (mq == -INFINITY) continue;
+        const float f = ex2(mq - Mg);
+        const float4* src = mine + ((size_t)(q * slots + slot) * 2) * kTileM + r;
         const float4 x = src[0], y = src[kTileM];
         acc[0] = fmaf(x.x, f, acc[0]); acc[1] = fmaf(x.y, f, acc[1]); acc[2] = fmaf(x.z, f, acc[2]); acc[3] = fmaf(x.w, f, acc[3]);
         acc[4] = fmaf(y.x, f, acc[4]); acc[5] = fmaf(y.y, f, acc[5]); acc[6] = fmaf(y.z, f, acc[6]); acc[7] = fmaf(y.w, f, acc[7]);
@@ -506,11 +559,10 @@ tree_attention_umma_kernel(const __grid_constant__ CUtensorMap q_map, const __gr
         val.y = pack2<kBf16>(acc[2] * inv, acc[3] * inv);
         val.z = pack2<kBf16>(acc[4] * inv, acc[5] * inv);
         val.w = pack2<kBf16>(acc[6] * inv, acc[7] * inv);
-        *reinterpret_cast<uint4*>(reinterpret_cast<uint8_t*>(a.out) +
-                                  2 * ((int64_t)i * a.o_stride_tok + (int64_t)h * a.o_stride_head + 8 * slice)) = val;
+        *reinterpret_cast<uint4*>(out_row + 2 * (8 * (slot * cs + split))) = val;
       }
     }
-    if (me == 0 && row_valid && a.lse != nullptr) a.lse[(size_t)h * a.n + i] = (M + log2f(Ls)) * kLn2;
+    if (split == 0 && chain == 0 && row_valid && a.lse != nullptr) a.lse[(size_t)h * a.n + i] = (Mg + log2f(Ls)) * kLn2;
   }
   if (threadIdx.x == 128) UTRACE(2, 9);
   // no remote access happens after the second cluster barrier, so CTAs may leave independently
