@@ -3,19 +3,22 @@
 //
 // Work unit: one CTA = (kv head g, tile of 128 query rows, share of the key range).  A query row is
 // a (node, head-in-group) pair, r = i_local * G + hg, so under GQA the G heads that share a kv head
-// share every K/V tile.  Keys are taken in blocks of 128:
-//     S = Q K^T      128x128x128  tcgen05.mma, Q and K K-major in 128-byte-swizzled shared memory
+// share every K/V tile.  Per block of 64 keys:
+//     S = Q K^T      128x64x128   tcgen05.mma, Q and K K-major in 128-byte-swizzled shared memory
 //     P = 2^(scale*S - m) masked  one thread per row: S read from tensor memory, P written back over
 //                                 it as packed 16-bit values
-//     O += P V       128x128x128  tcgen05.mma, A = P from tensor memory, V MN-major in shared memory
+//     O += P V       128x128x64   tcgen05.mma, A = P from tensor memory, V MN-major in shared memory
 //
-// Two chains per CTA.  Even blocks of the CTA's key range belong to chain A, odd blocks to chain B.
-// Each chain has its own S/P buffer and its own accumulator O in tensor memory (4 x 128 columns),
-// its own K/V stage in shared memory, its own 128 row threads (one warp group) and its own running
-// (m, l); the chains only share Q, the TMA warp and the MMA warp.  While the row threads of one chain
-// exponentiate, the tensor pipe works for the other.  The running maximum of a row is only moved
-// when a block maximum exceeds it by more than 2^8 (the accumulator row is then rescaled in tensor
-// memory).  Registers are rebalanced with setmaxnreg: 40 for the TMA/MMA warp group, 232 for the rows.
+// Two chains per CTA, each double-buffered.  Keys are taken in blocks of 64; even blocks of the CTA's
+// key range belong to chain A, odd blocks to chain B.  Each chain has two S/P buffers (64 columns
+// each) and its own accumulator O in tensor memory (2 x (2*64 + 128) = 512 columns), two K and two V
+// stages in shared memory, its own 128 row threads (one warp group) and its own running (m, l); the
+// chains only share Q and the TMA warp; each has its own MMA-issuing warp.  S of a chain's next block is computed while
+// its row threads still work on the current one, so a chain runs at the speed of its softmax, and
+// while one chain exponentiates the tensor pipe also works for the other.  The running maximum of a
+// row is only moved when a block maximum exceeds it by more than 2^8 (the accumulator row is then
+// rescaled in tensor memory).  Registers are rebalanced with setmaxnreg: 40 for the TMA/MMA warp
+// group, 232 for the rows.
 //
 // Merge.  The CTAs that share (tile, kv head) form a thread-block cluster along the key
 // range (cs = 1, 2, 4 or 8); its 2*cs chains share the 16 slices of 8 output columns round-robin.  Every chain pushes,
@@ -54,24 +57,29 @@ __device__ unsigned long long g_utrace[4][512];
 #endif
 
 constexpr int kTileM = 128;         // query rows per CTA
-constexpr int kBlockN = 128;        // keys per block
+constexpr int kBlockN = 64;         // keys per block
 constexpr int kUmmaThreads = 384;   // warp group 0: TMA warp, MMA warp, two spare; warp groups 1, 2: rows of chains A, B
 constexpr int kRegsLight = 40, kRegsRows = 232;  // after setmaxnreg: 128*40 + 256*232 = 384*168
 constexpr int kMaxClusterSplit = 8;
 constexpr int kNumSMs = 148;
-constexpr uint32_t kTileBytes = 128 * 128 * 2;   // one 128x128 16-bit tile
-constexpr uint32_t kHalfBytes = kTileBytes / 2;  // one 128-row x 64-element sub-tile (128 B rows)
+constexpr uint32_t kTileBytes = 128 * 128 * 2;   // the Q tile: 128 rows x 128 elements of 16 bits
+constexpr uint32_t kHalfBytes = kTileBytes / 2;  // one 128-row x 64-element sub-tile of Q (128 B rows)
+constexpr uint32_t kKvBytes = kBlockN * 128 * 2; // a K or V tile: 64 keys x 128 elements
+constexpr uint32_t kKvHalf = kKvBytes / 2;       // one 64-row x 64-element sub-tile of K or V
 constexpr float kRescaleThreshold = 8.f;         // log2 units
 constexpr uint32_t kSpinLimit = 1u << 22;
 
 struct UmmaSmem {
   // all tiles 1024-byte aligned (128-byte swizzle atoms are 8 rows x 128 B)
   uint8_t q[kTileBytes];
-  uint8_t k[2][kTileBytes];  // K stage of chain A, of chain B; after the last block: chain A's 128x128 fp32 accumulator
-  uint8_t v[2][kTileBytes];  // V stage of chain A, of chain B; after the last block: chain B's accumulator
+  uint8_t k[2][2][kKvBytes];  // [chain][stage]; after the last block these 64 KB receive the cluster merge
+  uint8_t v[2][2][kKvBytes];  // [chain][stage]
   float2 ml_chain[2][kTileM];                // (m, l) of every row of the two chains of this CTA
   float2 ml_cta[kMaxClusterSplit][kTileM];   // (m, l) of every row of every CTA of the cluster, after its chains are merged
-  uint64_t q_full, k_full[2], k_empty[2], v_full[2], v_empty[2], s_full[2], p_full[2], pv_done[2];
+  uint64_t q_full;
+  uint64_t k_full[2][2], k_empty[2][2], v_full[2][2], v_empty[2][2], s_full[2][2], p_full[2][2];  // [chain][stage]
+  uint64_t pv_done[2];                       // [chain]: one phase per block of the chain
+  uint64_t all_done;                         // every MMA of the CTA has completed
   uint32_t tmem_base;
   volatile int abort_flag;
 };
@@ -134,6 +142,19 @@ __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::
 __device__ __forceinline__ void tc_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 __device__ __forceinline__ void tc_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
 __device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+
+// True in exactly one lane of a converged warp.  Code that must be issued once per warp (MMAs, commits)
+// goes under this predicate while everything around it stays warp-uniform, which keeps descriptors and
+// addresses on the uniform datapath.
+__device__ __forceinline__ bool elect_one() {
+  uint32_t pred;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "elect.sync _|p, 0xffffffff;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(pred));
+  return pred != 0;
+}
 
 __device__ __forceinline__ void tc_commit(uint64_t* bar) {
   asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar)) : "memory");
@@ -254,15 +275,19 @@ tree_attention_umma_kernel(const __grid_constant__ CUtensorMap q_map, const __gr
   if (threadIdx.x == 0) {
     mbar_init(&sm->q_full, 1);
     for (int c = 0; c < 2; ++c) {
-      mbar_init(&sm->k_full[c], 1); mbar_init(&sm->k_empty[c], 1);
-      mbar_init(&sm->v_full[c], 1); mbar_init(&sm->v_empty[c], 1);
-      mbar_init(&sm->s_full[c], 1); mbar_init(&sm->p_full[c], 128); mbar_init(&sm->pv_done[c], 1);
+      for (int b = 0; b < 2; ++b) {
+        mbar_init(&sm->k_full[c][b], 1); mbar_init(&sm->k_empty[c][b], 1);
+        mbar_init(&sm->v_full[c][b], 1); mbar_init(&sm->v_empty[c][b], 1);
+        mbar_init(&sm->s_full[c][b], 1); mbar_init(&sm->p_full[c][b], 4);
+      }
+      mbar_init(&sm->pv_done[c], 1);
     }
+    mbar_init(&sm->all_done, 2);  // one arrival per chain
     sm->abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   if (threadIdx.x == 128) UTRACE(2, 11);
-  if (warp == 1) {  // all 512 tensor-memory columns: S_A, S_B (P over them), O_A, O_B
+  if (warp == 1) {  // all 512 tensor-memory columns: per chain two S buffers of 64 (P over them), then O_A, O_B
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], 512;" ::"r"(smem_u32(&sm->tmem_base)) : "memory");
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
   }
@@ -282,62 +307,81 @@ tree_attention_umma_kernel(const __grid_constant__ CUtensorMap q_map, const __gr
         tma_load_4d(sm->q, &q_map, &sm->q_full, 0, 0, i0, g);
         tma_load_4d(sm->q + kHalfBytes, &q_map, &sm->q_full, 64, 0, i0, g);
         for (int jj = 0; jj < nblk; ++jj) {
-          const int c = jj & 1, u = jj >> 1;  // chain (= stage) and its use count
+          const int c = jj & 1, u = jj >> 1, b = u & 1, w = u >> 1;  // chain, its block index, stage, use count of the stage
           const int row = (blk_lo + jj) * kBlockN;
-          if (u > 0 && !mbar_wait(sm, &sm->k_empty[c], (u - 1) & 1, a.dev_status)) break;
+          if (w > 0 && !mbar_wait(sm, &sm->k_empty[c][b], (w - 1) & 1, a.dev_status)) break;
           UTRACE(0, 1);
-          mbar_expect_tx(&sm->k_full[c], kTileBytes);
-          tma_load_3d(sm->k[c], &k_map, &sm->k_full[c], 0, row, g);
-          tma_load_3d(sm->k[c] + kHalfBytes, &k_map, &sm->k_full[c], 64, row, g);
-          if (u > 0 && !mbar_wait(sm, &sm->v_empty[c], (u - 1) & 1, a.dev_status)) break;
+          mbar_expect_tx(&sm->k_full[c][b], kKvBytes);
+          tma_load_3d(sm->k[c][b], &k_map, &sm->k_full[c][b], 0, row, g);
+          tma_load_3d(sm->k[c][b] + kKvHalf, &k_map, &sm->k_full[c][b], 64, row, g);
+          if (w > 0 && !mbar_wait(sm, &sm->v_empty[c][b], (w - 1) & 1, a.dev_status)) break;
           UTRACE(0, 2);
-          mbar_expect_tx(&sm->v_full[c], kTileBytes);
-          tma_load_3d(sm->v[c], &v_map, &sm->v_full[c], 0, row, g);
-          tma_load_3d(sm->v[c] + kHalfBytes, &v_map, &sm->v_full[c], 64, row, g);
+          mbar_expect_tx(&sm->v_full[c][b], kKvBytes);
+          tma_load_3d(sm->v[c][b], &v_map, &sm->v_full[c][b], 0, row, g);
+          tma_load_3d(sm->v[c][b] + kKvHalf, &v_map, &sm->v_full[c][b], 64, row, g);
         }
       }
       __syncwarp();
-    } else if (warp == 1) {
-      // ---------------------------------------------------------- MMA issuer --------------------
-      if (lane == 0 && nblk > 0) {
+    } else if (warp <= 2) {
+      // ---------------------------------------------------------- MMA issuers -------------------
+      // Warp 1 issues for chain A, warp 2 for chain B.  The whole warp runs this code; only the MMAs and
+      // commits are issued by one elected lane, so descriptors and addresses stay warp-uniform.
+      const int c = warp - 1;
+      const int n_c = nblk > c ? (nblk - c + 1) >> 1 : 0;  // blocks of this chain
+      if (n_c > 0) {
         bool go = mbar_wait(sm, &sm->q_full, 0, a.dev_status);
         // A step along the contraction only moves a descriptor's 14-bit start-address field (16-byte units).
         const uint64_t qd0 = make_desc(smem_u32(sm->q), 16, 1024);
-        auto issue_qk = [&](int jj) -> bool {
-          const int c = jj & 1, u = jj >> 1;
-          if (!mbar_wait(sm, &sm->k_full[c], u & 1, a.dev_status)) return false;
+        const uint32_t tmem_o = tmem + 256u + 128u * c;
+        // S of block u of the chain: buffer u & 1
+        auto issue_qk = [&](int u) -> bool {
+          const int b = u & 1, w = u >> 1;
+          if (!mbar_wait(sm, &sm->k_full[c][b], w & 1, a.dev_status)) return false;
           tc_fence_after();
-          const uint64_t kd0 = make_desc(smem_u32(sm->k[c]), 16, 1024);
+          const uint64_t kd0 = make_desc(smem_u32(sm->k[c][b]), 16, 1024);
+          const uint32_t d = tmem + 128u * c + 64u * b;
+          if (elect_one()) {
 #pragma unroll
-          for (int ks = 0; ks < 8; ++ks) {  // 16 elements of head_dim per step: 32 bytes inside a 64-element sub-tile
-            const uint64_t off = (uint64_t)(((ks >> 2) * kHalfBytes + (ks & 3) * 32) >> 4);
-            tc_mma(tmem + 128u * c, qd0 + off, kd0 + off, a.idesc_qk, ks > 0);
+            for (int ks = 0; ks < 8; ++ks) {  // 16 elements of head_dim per step: 32 bytes inside a 64-element sub-tile
+              tc_mma(d, qd0 + (uint64_t)(((ks >> 2) * kHalfBytes + (ks & 3) * 32) >> 4),
+                     kd0 + (uint64_t)(((ks >> 2) * kKvHalf + (ks & 3) * 32) >> 4), a.idesc_qk, ks > 0);
+            }
+            tc_commit(&sm->k_empty[c][b]);
+            tc_commit(&sm->s_full[c][b]);
           }
-          tc_commit(&sm->k_empty[c]);
-          tc_commit(&sm->s_full[c]);
-          UTRACE(1, 2);
+          __syncwarp();
+          if (lane == 0) UTRACE(c == 0 ? 1 : 3, 2);
           return true;
         };
+        // two S in flight before the first P is needed
         if (go) go = issue_qk(0);
-        if (go && nblk > 1) go = issue_qk(1);
-        for (int jj = 0; jj < nblk && go; ++jj) {
-          const int c = jj & 1, u = jj >> 1;
-          if (!mbar_wait(sm, &sm->p_full[c], u & 1, a.dev_status)) break;
-          UTRACE(1, 3);
-          if (!mbar_wait(sm, &sm->v_full[c], u & 1, a.dev_status)) break;
+        if (go && n_c > 1) go = issue_qk(1);
+        for (int u = 0; u < n_c && go; ++u) {
+          const int b = u & 1, w = u >> 1;
+          if (!mbar_wait(sm, &sm->p_full[c][b], w & 1, a.dev_status)) break;
+          if (lane == 0) UTRACE(c == 0 ? 1 : 3, 3);
+          if (!mbar_wait(sm, &sm->v_full[c][b], w & 1, a.dev_status)) break;
           tc_fence_after();
-          const uint64_t vd0 = make_desc(smem_u32(sm->v[c]), kHalfBytes, 1024);
+          const uint64_t vd0 = make_desc(smem_u32(sm->v[c][b]), kKvHalf, 1024);
+          const uint32_t pa = tmem + 128u * c + 64u * b;
+          const uint32_t first = u > 0 ? 1u : 0u;
+          if (elect_one()) {
 #pragma unroll
-          for (int ks = 0; ks < 8; ++ks)  // A = 8 packed columns of P, B = 16 key rows of V per step
-            tc_mma_tmem_a(tmem + 256u + 128u * c, tmem + 128u * c + 8u * ks, vd0 + (uint64_t)(ks * (2048 >> 4)), a.idesc_pv,
-                          (u > 0 || ks > 0) ? 1u : 0u);
-          tc_commit(&sm->v_empty[c]);
-          tc_commit(&sm->pv_done[c]);
-          UTRACE(1, 5);
-          // The chain's next S goes where its P lives.  tcgen05.mma operations issued by one thread
+            for (int ks = 0; ks < 4; ++ks)  // A = 8 packed columns of P, B = 16 key rows of V per step
+              tc_mma_tmem_a(tmem_o, pa + 8u * ks, vd0 + (uint64_t)(ks * (2048 >> 4)), a.idesc_pv, ks > 0 ? 1u : first);
+            tc_commit(&sm->v_empty[c][b]);
+            tc_commit(&sm->pv_done[c]);
+          }
+          __syncwarp();
+          if (lane == 0) UTRACE(c == 0 ? 1 : 3, 5);
+          // S of block u+2 goes where P of block u lives.  tcgen05.mma operations issued by one thread
           // execute in issue order, so this QK^T cannot overtake the P.V just issued.
-          if (jj + 2 < nblk && !issue_qk(jj + 2)) break;
+          if (u + 2 < n_c && !issue_qk(u + 2)) break;
         }
+        if (elect_one()) tc_commit(&sm->all_done);  // arrives when every MMA of this chain has completed
+        __syncwarp();
+      } else if (lane == 0 && nblk > 0) {
+        mbar_arrive(&sm->all_done);  // a chain without blocks
       }
       __syncwarp();
     }
@@ -361,7 +405,7 @@ tree_attention_umma_kernel(const __grid_constant__ CUtensorMap q_map, const __gr
   const int quad = warp & 3;                  // tensor-memory lane quarter this warp may access
   const int r = quad * 32 + lane;             // row of the tile = tensor-memory lane
   const uint32_t lane_sel = (uint32_t)(quad * 32) << 16;
-  const uint32_t tmem_s = tmem + 128u * chain + lane_sel, tmem_o = tmem + 256u + 128u * chain + lane_sel;
+  const uint32_t tmem_o = tmem + 256u + 128u * chain + lane_sel;
   const int i = i0 + r / a.group;             // node of this row
   const int h = g * a.group + r % a.group;
   const bool row_valid = i < a.n;
@@ -372,28 +416,29 @@ tree_attention_umma_kernel(const __grid_constant__ CUtensorMap q_map, const __gr
   bool ok = true;
   const int n_mine = nblk > chain ? (nblk - chain + 1) >> 1 : 0;  // blocks of this chain
   for (int u = 0; u < n_mine && ok; ++u) {
-    const int jj = 2 * u + chain;
-    if (!mbar_wait(sm, &sm->s_full[chain], u & 1, a.dev_status)) { ok = false; break; }
+    const int jj = 2 * u + chain, b = u & 1, w = u >> 1;
+    const uint32_t tmem_s = tmem + 128u * chain + 64u * b + lane_sel;
+    if (!mbar_wait(sm, &sm->s_full[chain][b], w & 1, a.dev_status)) { ok = false; break; }
     if (threadIdx.x == 128) UTRACE(2, 1);
     tc_fence_after();
-    uint32_t sreg[128];
-#pragma unroll
-    for (int c = 0; c < 4; ++c) tmem_ld32(tmem_s + 32u * c, sreg, 32 * c);
+    uint32_t sreg[64];
+    tmem_ld32(tmem_s, sreg, 0);
+    tmem_ld32(tmem_s + 32u, sreg, 32);
     const int kb = (blk_lo + jj) * kBlockN;
     const bool masked = kb + kBlockN > a.L;  // the block reaches into the tree keys (or past the end)
-    uint32_t vis[4] = {0xFFFFFFFFu, 0xFFFFFFFFu, 0xFFFFFFFFu, 0xFFFFFFFFu};
+    uint32_t vis[2] = {0xFFFFFFFFu, 0xFFFFFFFFu};
     if (masked) {
-#pragma unroll
-      for (int c = 0; c < 4; ++c) vis[c] = mask_window(mrow, a.mask_wpr, a.n, kb - a.L + 32 * c);
+      vis[0] = mask_window(mrow, a.mask_wpr, a.n, kb - a.L);
+      vis[1] = mask_window(mrow, a.mask_wpr, a.n, kb - a.L + 32);
     }
     tc_wait_ld();
     if (threadIdx.x == 128) UTRACE(2, 2);
     if (masked) {  // masked scores become -inf: probability exactly 0, and they cannot raise the maximum
 #pragma unroll
-      for (int e = 0; e < 128; ++e)
+      for (int e = 0; e < 64; ++e)
         if (!(vis[e >> 5] & (1u << (e & 31)))) sreg[e] = __float_as_uint(-INFINITY);
     }
-    // P = 2^(scale*s - m) written over S as packed 16-bit values (64 columns, four stores of 16), with the
+    // P = 2^(scale*s - m) written over S as packed 16-bit values (32 columns, two stores of 16), with the
     // block maximum taken in the same sweep: the exponentials are MUFU-bound, so the comparisons ride
     // along.  The sweep first assumes the reference maximum does not have to move; if the block maximum
     // turns out to exceed it by more than the threshold (or there is no reference yet) it is redone once.
@@ -402,7 +447,7 @@ tree_attention_umma_kernel(const __grid_constant__ CUtensorMap q_map, const __gr
       float sm4[4] = {0.f, 0.f, 0.f, 0.f};
       float mx[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
 #pragma unroll
-      for (int c = 0; c < 4; ++c) {
+      for (int c = 0; c < 2; ++c) {
         uint32_t packed[16];
 #pragma unroll
         for (int e = 0; e < 16; ++e) {
@@ -430,8 +475,10 @@ tree_attention_umma_kernel(const __grid_constant__ CUtensorMap q_map, const __gr
           alpha = m_used == -INFINITY ? 0.f : ex2(m_used - m_blk);
           m_used = m_blk;
         }
-        // this S was issued after O took the chain's previous block, so O is quiescent here
         if (u > 0) {
+          // O may still be taking the chain's previous block: wait for it, then rescale this warp's rows
+          if (!mbar_wait(sm, &sm->pv_done[chain], (u - 1) & 1, a.dev_status)) { ok = false; break; }
+          tc_fence_after();
 #pragma unroll
           for (int c = 0; c < 4; ++c) {
             uint32_t o[32];
@@ -450,13 +497,12 @@ tree_attention_umma_kernel(const __grid_constant__ CUtensorMap q_map, const __gr
     if (threadIdx.x == 128) UTRACE(2, 4);
     tc_wait_st();
     tc_fence_before();
-    mbar_arrive(&sm->p_full[chain]);
+    __syncwarp();
+    if (lane == 0) mbar_arrive(&sm->p_full[chain][b]);  // one arrival per warp
   }
-  // both chains must be done with the tensor pipe before the K/V stages are reused as staging
-  for (int c = 0; c < 2; ++c) {
-    const int n_c = nblk > c ? (nblk - c + 1) >> 1 : 0;
-    if (n_c > 0 && ok) ok = mbar_wait(sm, &sm->pv_done[c], (n_c - 1) & 1, a.dev_status);
-  }
+  // Both chains must be done with the tensor pipe before O is read and the K stages are reused.  (A
+  // parity wait on pv_done could be fooled here: the other chain may be several phases behind.)
+  if (nblk > 0 && ok) ok = mbar_wait(sm, &sm->all_done, 0, a.dev_status);
   tc_fence_after();
 
   // ---------------------------------------------------------------- merge ------------------------
@@ -524,7 +570,7 @@ tree_attention_umma_kernel(const __grid_constant__ CUtensorMap q_map, const __gr
 #pragma unroll
     for (int j = 0; j < 8; ++j) {
       const int s_idx = 8 * chain + j;
-      uint4* dst = cluster.map_shared_rank(reinterpret_cast<uint4*>(sm->k[0]), s_idx % cs) +
+      uint4* dst = cluster.map_shared_rank(reinterpret_cast<uint4*>(&sm->k[0][0][0]), s_idx % cs) +
                    ((size_t)(split * slots + s_idx / cs) * 2) * kTileM + r;
       dst[0] = make_uint4(__float_as_uint(merged[8 * j]), __float_as_uint(merged[8 * j + 1]),
                           __float_as_uint(merged[8 * j + 2]), __float_as_uint(merged[8 * j + 3]));
@@ -541,7 +587,7 @@ tree_attention_umma_kernel(const __grid_constant__ CUtensorMap q_map, const __gr
       if (mlq.x != -INFINITY) Ls += mlq.y * ex2(mlq.x - Mg);
     }
     const float inv = 1.f / Ls;  // some CTA saw the row's own key, so Ls > 0
-    const float4* mine = reinterpret_cast<const float4*>(sm->k[0]);
+    const float4* mine = reinterpret_cast<const float4*>(&sm->k[0][0][0]);
     for (int slot = chain; slot < slots; slot += 2) {  // the two warp groups share this CTA's slots
       float acc[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
       for (int q = 0; q < cs; ++q) {
@@ -596,8 +642,8 @@ bool umma_supported(const seq_tree_attention_params& p) {
 }
 
 // Size of the cluster that shares one (tile, kv head): 1, 2, 4 or 8 CTAs along the key range, chosen for the
-// shortest estimated makespan with one CTA per SM (about 0.9 us per key block with both chains busy,
-// about 4 us of fixed cost per CTA).
+// shortest estimated makespan with one CTA per SM (about 0.4 us per 64-key block with both chains busy,
+// about 5 us of fixed cost per CTA).
 int umma_default_splits(const seq_tree_attention_params& p) {
   const int G = p.num_q_heads / p.num_kv_heads;
   const int nodes_per_tile = kTileM / G;
@@ -612,7 +658,7 @@ int umma_default_splits(const seq_tree_attention_params& p) {
   for (int cs = 1; cs <= kMaxClusterSplit; cs *= 2) {  // powers of two: 16 slices divide evenly among 2*cs chains
     if (cs > 1 && cs > nblk) break;
     const long waves = (units * cs + kNumSMs - 1) / kNumSMs;
-    const double cost = (double)waves * (0.9 * ((nblk + cs - 1) / cs) + 4.0);
+    const double cost = (double)waves * (0.4 * ((nblk + cs - 1) / cs) + 5.0);
     if (best_cost < 0 || cost < best_cost - 1e-9) { best = cs; best_cost = cost; }
   }
   return best;
@@ -658,9 +704,9 @@ int launch_attention_umma(const seq_tree_attention_params& p, int splits, cudaSt
   a.scale_log2 = scale * kLog2e;
   const uint32_t fmt = p.dtype == SEQ_BF16 ? 1u : 0u;
   // instruction descriptor: D fp32 (bit 4), A/B format (bits 7, 10), B major (bit 16), N>>3 (bit 17), M>>4 (bit 24)
-  const uint32_t idesc = (1u << 4) | (fmt << 7) | (fmt << 10) | ((uint32_t)(kBlockN >> 3) << 17) | ((uint32_t)(kTileM >> 4) << 24);
-  a.idesc_qk = idesc;
-  a.idesc_pv = idesc | (1u << 16);
+  const uint32_t idesc = (1u << 4) | (fmt << 7) | (fmt << 10) | ((uint32_t)(kTileM >> 4) << 24);
+  a.idesc_qk = idesc | ((uint32_t)(kBlockN >> 3) << 17);                 // S: N = 64 keys
+  a.idesc_pv = idesc | ((uint32_t)(kHeadDim >> 3) << 17) | (1u << 16);   // O: N = 128, V is MN-major
   a.mask_bits = p.mask_bits;
   a.out = p.out; a.o_stride_tok = p.o_stride_tok; a.o_stride_head = p.o_stride_head;
   a.lse = p.lse;
