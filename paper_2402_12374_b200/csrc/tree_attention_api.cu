@@ -44,10 +44,11 @@ static int choose_kernel(const seq_tree_attention_params& p) {
   const bool ok = umma_supported(p);
   if (p.kernel == 2) return ok ? 2 : 0;
   if (!ok) return 1;
-  // The tensor-core tile holds 128 (node, head-in-group) rows: below 32 rows per kv head most of
-  // each tile would be padding, and the CUDA-core kernel moves the same bytes with less set-up.
-  const int rows_per_kv_head = p.n_tree * (p.num_q_heads / p.num_kv_heads);
-  return rows_per_kv_head >= 32 ? 2 : 1;
+  // Measured on B200: even with a single query row per kv head (127 of the tile's 128 rows padding) the
+  // tensor-core kernel is faster than the CUDA-core one, because it streams K/V once per kv head with
+  // TMA while the CUDA-core kernel re-reads them for every (node, head).  The CUDA-core kernel is kept
+  // for fp32 inputs and for group sizes that do not divide 128.
+  return 2;
 }
 
 }  // namespace seqtree

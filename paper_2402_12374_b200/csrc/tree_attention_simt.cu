@@ -143,7 +143,7 @@ tree_attention_simt_kernel(const SimtArgs a) {
     if (valid) {
       const T* kr = kbase + (int64_t)j * a.kv_stride_tok;
       float d0 = 0.f, d1 = 0.f;
-#pragma unroll 4
+#pragma unroll
       for (int c0 = 0; c0 < kHeadDim; c0 += Vec16<T>::kElems) {
         float kv[Vec16<T>::kElems];
         Vec16<T>::load(kr + c0, kv);
@@ -163,14 +163,24 @@ tree_attention_simt_kernel(const SimtArgs a) {
 #pragma unroll
     for (int e = 0; e < 4; ++e) acc[e] *= alpha;
     m = m_new;
+    // all lanes walk the chunk's keys together, eight at a time so that the eight V loads are in flight
+    // at once; keys the row cannot see have p = 0 exactly and are skipped as whole groups
     const uint32_t live = __ballot_sync(0xffffffffu, p != 0.f);
-    for (uint32_t rem = live; rem != 0u; rem &= rem - 1u) {
-      const int jj = __ffs(rem) - 1;
-      const float pj = __shfl_sync(0xffffffffu, p, jj);
-      float vv[4];
-      load4<T>(vbase + (int64_t)((c << 5) + jj) * a.kv_stride_tok + lane * 4, vv);
 #pragma unroll
-      for (int e = 0; e < 4; ++e) acc[e] = fmaf(pj, vv[e], acc[e]);
+    for (int j0 = 0; j0 < 32; j0 += 8) {
+      if (((live >> j0) & 0xFFu) == 0u) continue;
+      float pj[8], vv[8][4];
+#pragma unroll
+      for (int e = 0; e < 8; ++e) {
+        pj[e] = __shfl_sync(0xffffffffu, p, j0 + e);
+        if (pj[e] != 0.f) load4<T>(vbase + (int64_t)((c << 5) + j0 + e) * a.kv_stride_tok + lane * 4, vv[e]);
+        else vv[e][0] = vv[e][1] = vv[e][2] = vv[e][3] = 0.f;
+      }
+#pragma unroll
+      for (int e = 0; e < 8; ++e) {
+#pragma unroll
+        for (int d = 0; d < 4; ++d) acc[d] = fmaf(pj[e], vv[e][d], acc[d]);
+      }
     }
   }
 

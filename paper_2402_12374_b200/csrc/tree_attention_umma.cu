@@ -302,23 +302,33 @@ tree_attention_umma_kernel(const __grid_constant__ CUtensorMap q_map, const __gr
     asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(kRegsLight));
     if (warp == 0) {
       // ---------------------------------------------------------- TMA producer ------------------
-      if (lane == 0 && nblk > 0) {
-        mbar_expect_tx(&sm->q_full, kTileBytes);
-        tma_load_4d(sm->q, &q_map, &sm->q_full, 0, 0, i0, g);
-        tma_load_4d(sm->q + kHalfBytes, &q_map, &sm->q_full, 64, 0, i0, g);
+      // The whole warp runs the loop; one elected lane issues the copies (coordinates stay warp-uniform).
+      if (nblk > 0) {
+        if (elect_one()) {
+          mbar_expect_tx(&sm->q_full, kTileBytes);
+          tma_load_4d(sm->q, &q_map, &sm->q_full, 0, 0, i0, g);
+          tma_load_4d(sm->q + kHalfBytes, &q_map, &sm->q_full, 64, 0, i0, g);
+        }
+        __syncwarp();
         for (int jj = 0; jj < nblk; ++jj) {
           const int c = jj & 1, u = jj >> 1, b = u & 1, w = u >> 1;  // chain, its block index, stage, use count of the stage
           const int row = (blk_lo + jj) * kBlockN;
           if (w > 0 && !mbar_wait(sm, &sm->k_empty[c][b], (w - 1) & 1, a.dev_status)) break;
-          UTRACE(0, 1);
-          mbar_expect_tx(&sm->k_full[c][b], kKvBytes);
-          tma_load_3d(sm->k[c][b], &k_map, &sm->k_full[c][b], 0, row, g);
-          tma_load_3d(sm->k[c][b] + kKvHalf, &k_map, &sm->k_full[c][b], 64, row, g);
+          if (elect_one()) {
+            mbar_expect_tx(&sm->k_full[c][b], kKvBytes);
+            tma_load_3d(sm->k[c][b], &k_map, &sm->k_full[c][b], 0, row, g);
+            tma_load_3d(sm->k[c][b] + kKvHalf, &k_map, &sm->k_full[c][b], 64, row, g);
+          }
+          __syncwarp();
+          if (lane == 0) UTRACE(0, 1);
           if (w > 0 && !mbar_wait(sm, &sm->v_empty[c][b], (w - 1) & 1, a.dev_status)) break;
-          UTRACE(0, 2);
-          mbar_expect_tx(&sm->v_full[c][b], kKvBytes);
-          tma_load_3d(sm->v[c][b], &v_map, &sm->v_full[c][b], 0, row, g);
-          tma_load_3d(sm->v[c][b] + kKvHalf, &v_map, &sm->v_full[c][b], 64, row, g);
+          if (elect_one()) {
+            mbar_expect_tx(&sm->v_full[c][b], kKvBytes);
+            tma_load_3d(sm->v[c][b], &v_map, &sm->v_full[c][b], 0, row, g);
+            tma_load_3d(sm->v[c][b] + kKvHalf, &v_map, &sm->v_full[c][b], 64, row, g);
+          }
+          __syncwarp();
+          if (lane == 0) UTRACE(0, 2);
         }
       }
       __syncwarp();
