@@ -579,29 +579,25 @@ __global__ void __launch_bounds__(kVThreads, 1) tree_verify_kernel(const VerifyA
   st.c2 = greedy ? 0.f : kLog2e / a.temperature;
   const int cluster_id = blockIdx.x / kVCluster, n_clusters = gridDim.x / kVCluster;
 
-  if (all_nodes) {
-    // test hook: every node gets its own run of Algorithm 2's loop; no walk, no final draw
-    for (int v = cluster_id; v < a.n; v += n_clusters) {
-      const int acc = process_node(cluster, c, a, v, st, true, false);
-      if (c.rank == 0 && c.tid == 0) a.next_child_out[v] = acc;
-      __syncthreads();
-    }
-    return;
-  }
-
-  if (a.next_child_out != nullptr && c.rank == 0)
+  if (!all_nodes && a.next_child_out != nullptr && c.rank == 0)
     for (int i = c.tid; i < a.n; i += kVThreads) a.next_child_out[i] = -2;
   __syncthreads();
-  int cur = 0, plen = 0;
-  for (int hop = 0; hop < a.n; ++hop) {  // a walk visits at most n nodes
-    if (c.rank == 0 && c.tid == 0) a.path[plen] = cur;
-    ++plen;
-    const int acc = process_node(cluster, c, a, cur, st, false, hop == 0);
+  // One loop (and one copy of the per-node code) serves both schedules: the walk from the root, and the
+  // test hook in which every node gets its own run of Algorithm 2's loop (no walk, no final draw).
+  int cur = all_nodes ? cluster_id : 0, plen = 0;
+  for (int hop = 0; hop < a.n && cur < a.n; ++hop) {  // a walk visits at most n nodes
+    if (!all_nodes) {
+      if (c.rank == 0 && c.tid == 0) a.path[plen] = cur;
+      ++plen;
+    }
+    const int acc = process_node(cluster, c, a, cur, st, all_nodes, !all_nodes && hop == 0);
     if (c.rank == 0 && c.tid == 0 && a.next_child_out != nullptr) a.next_child_out[cur] = acc;
-    if (acc < 0) break;
-    cur = acc;
+    if (all_nodes) cur += n_clusters;
+    else if (acc < 0) break;
+    else cur = acc;
     __syncthreads();  // all reads of this node's slices are done before the next copies land
   }
+  if (all_nodes) return;
   if (c.rank == 0 && c.tid == 0) *a.path_len = plen;
   TRACE(11);
   draw_bonus(c, a, st);
