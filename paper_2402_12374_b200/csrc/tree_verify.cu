@@ -127,7 +127,6 @@ __device__ __forceinline__ float resid(float pn, float qn, float Cf, float Uf) {
 template <typename F4, typename F1>
 __device__ __forceinline__ void sweep(const Ctx& c, F4 f4, F1 f1) {
   int t = c.s_lo + 4 * c.lane;
-  for (; t + 131 < c.s_hi; t += 256) { f4(t); f4(t + 128); }  // two independent steps per trip
   for (; t + 3 < c.s_hi; t += 128) f4(t);
   for (int e = t; e < c.s_hi && e < t + 4; ++e) f1(e);
 }
