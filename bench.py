@@ -36,7 +36,10 @@ L2_BYTES = 126 * 1024 * 1024
 
 # DRAM traffic per launch (dram__bytes_read.sum + dram__bytes_write.sum) of the attention kernel, from
 # the ncu captures summarised under profiles/; None where no capture exists for that workload.
-NCU_TRAFFIC_BYTES = {}
+NCU_TRAFFIC_BYTES = {
+    "llama2-7b": 18418432,    # profiles/tree_attention_umma_llama2-7b.md
+    "llama3-70b": 32649728,   # profiles/tree_attention_umma_llama3-70b.md
+}
 
 
 def measured_peaks():
@@ -345,6 +348,21 @@ def main():
         "algorithmic_bytes": attn_bytes, "algorithmic_flops": flops, "peak_source": f"of {peaks['source']}",
         "timing": f"CUDA events around each call in a replay of the same steps ({Kb} of them), mean",
     })
+    # verification: HBM-bound in principle (the target row of every visited node, the draft row of every
+    # visited node that has children), latency-bound in practice (one cluster of 8 CTAs walks the path)
+    has_child = np.zeros(n, dtype=bool)
+    has_child[parent[1:][parent[1:] >= 0]] = True
+    vbytes = []
+    for vc in ver_calls:
+        plen = int(vc.path_len.item())
+        nodes = vc.path[:plen].cpu().numpy()
+        vbytes.append(sum(4 * cfg.vocab * (2 if has_child[v] else 1) for v in nodes))
+    ver_bytes = float(np.mean(vbytes))
+    ver_gbs = ver_bytes / (ver_us * 1e-6) / 1e9
+    roofline_verify = {"bound": "hbm", "achieved": ver_gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                       "frac": ver_gbs / peaks["hbm_gbs"], "traffic": None, "kernel": "seq_tree_verify",
+                       "us_per_launch": ver_us, "algorithmic_bytes": ver_bytes,
+                       "note": "logit rows of the visited nodes only; a dependent walk on one cluster, latency-bound"}
 
     line = {
         "metric": METRIC, "value": value_us, "unit": UNIT, "n_gpus": world, "steps": K, "warmup": Wm,
@@ -359,8 +377,9 @@ def main():
                 "steps": Ke},
         "gpu_launches": K * launches_per_step,
         "roofline": roofline,
+        "roofline_verify": roofline_verify,
         "breakdown_us": {"attention": attn_us, "verify": ver_us,
-                         "verify_bytes_visited_rows_x2": None},
+                         "largest_share": "seq_tree_verify" if ver_us > attn_us else "seq_tree_attention"},
     }
     if not args.no_cpu_baseline:
         from oracle import oracle as O
