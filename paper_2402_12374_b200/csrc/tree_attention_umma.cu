@@ -44,12 +44,17 @@ namespace cg = cooperative_groups;
 namespace seqtree {
 
 #ifdef SEQ_TRACE
-__device__ unsigned long long g_utrace[4][512];
+// Debug builds only: per role (0 TMA, 1 MMA chain A, 2 rows, 3 MMA chain B) a list of (tag, clock) events of
+// CTA (0, 0, 0), one 8-byte store each.  SEQ_TRACE_ROLES (bit per role) limits which roles record.
+#ifndef SEQ_TRACE_ROLES
+#define SEQ_TRACE_ROLES 15
+#endif
+__device__ unsigned long long g_utrace[4][2048];
 #define UTRACE(role, tag)                                                       \
   do {                                                                          \
-    if (blockIdx.x == 0 && blockIdx.y == 0 && blockIdx.z == 0) {                \
-      int _i = utrace_i++;                                                      \
-      if (_i < 255) { g_utrace[role][2 * _i + 2] = (tag); g_utrace[role][2 * _i + 3] = clock64(); g_utrace[role][0] = _i + 1; } \
+    if (((SEQ_TRACE_ROLES) >> (role)) & 1) {                                    \
+      if (blockIdx.x == 0 && blockIdx.y == 0 && blockIdx.z == 0 && utrace_i < 2047) \
+        g_utrace[role][++utrace_i] = ((unsigned long long)(tag) << 56) | ((unsigned long long)clock64() & 0xFFFFFFFFFFFFFFull); \
     }                                                                           \
   } while (0)
 #else
@@ -300,35 +305,35 @@ tree_attention_umma_kernel(const __grid_constant__ CUtensorMap q_map, const __gr
   if (warp < 4) {
     // ============================ warp group 0: data movement and MMA issue, few registers =========
     asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(kRegsLight));
-    if (warp == 0) {
-      // ---------------------------------------------------------- TMA producer ------------------
+    if (warp == 0 || warp == 3) {
+      // ---------------------------------------------------------- TMA producers -----------------
+      // Warp 0 loads Q and the K tiles, warp 3 the V tiles.  A K stage is free as soon as its S has been
+      // computed, a V stage only after the block's softmax and P.V; in one queue the K loads would wait
+      // behind the V stages and arrive just in time instead of a block ahead.
       // The whole warp runs the loop; one elected lane issues the copies (coordinates stay warp-uniform).
       if (nblk > 0) {
-        if (elect_one()) {
+        const bool is_v = warp == 3;
+        if (!is_v && elect_one()) {
           mbar_expect_tx(&sm->q_full, kTileBytes);
           tma_load_4d(sm->q, &q_map, &sm->q_full, 0, 0, i0, g);
           tma_load_4d(sm->q + kHalfBytes, &q_map, &sm->q_full, 64, 0, i0, g);
         }
         __syncwarp();
+        const CUtensorMap* map = is_v ? &v_map : &k_map;
         for (int jj = 0; jj < nblk; ++jj) {
           const int c = jj & 1, u = jj >> 1, b = u & 1, w = u >> 1;  // chain, its block index, stage, use count of the stage
           const int row = (blk_lo + jj) * kBlockN;
-          if (w > 0 && !mbar_wait(sm, &sm->k_empty[c][b], (w - 1) & 1, a.dev_status)) break;
+          uint64_t* full = is_v ? &sm->v_full[c][b] : &sm->k_full[c][b];
+          uint64_t* empty = is_v ? &sm->v_empty[c][b] : &sm->k_empty[c][b];
+          uint8_t* dst = is_v ? sm->v[c][b] : sm->k[c][b];
+          if (w > 0 && !mbar_wait(sm, empty, (w - 1) & 1, a.dev_status)) break;
           if (elect_one()) {
-            mbar_expect_tx(&sm->k_full[c][b], kKvBytes);
-            tma_load_3d(sm->k[c][b], &k_map, &sm->k_full[c][b], 0, row, g);
-            tma_load_3d(sm->k[c][b] + kKvHalf, &k_map, &sm->k_full[c][b], 64, row, g);
+            mbar_expect_tx(full, kKvBytes);
+            tma_load_3d(dst, map, full, 0, row, g);
+            tma_load_3d(dst + kKvHalf, map, full, 64, row, g);
           }
           __syncwarp();
-          if (lane == 0) UTRACE(0, 1);
-          if (w > 0 && !mbar_wait(sm, &sm->v_empty[c][b], (w - 1) & 1, a.dev_status)) break;
-          if (elect_one()) {
-            mbar_expect_tx(&sm->v_full[c][b], kKvBytes);
-            tma_load_3d(sm->v[c][b], &v_map, &sm->v_full[c][b], 0, row, g);
-            tma_load_3d(sm->v[c][b] + kKvHalf, &v_map, &sm->v_full[c][b], 64, row, g);
-          }
-          __syncwarp();
-          if (lane == 0) UTRACE(0, 2);
+          if (lane == 0 && !is_v) UTRACE(0, 1);
         }
       }
       __syncwarp();
@@ -448,39 +453,17 @@ tree_attention_umma_kernel(const __grid_constant__ CUtensorMap q_map, const __gr
       for (int e = 0; e < 64; ++e)
         if (!(vis[e >> 5] & (1u << (e & 31)))) sreg[e] = __float_as_uint(-INFINITY);
     }
-    // P = 2^(scale*s - m) written over S as packed 16-bit values (32 columns, two stores of 16), with the
-    // block maximum taken in the same sweep: the exponentials are MUFU-bound, so the comparisons ride
-    // along.  The sweep first assumes the reference maximum does not have to move; if the block maximum
-    // turns out to exceed it by more than the threshold (or there is no reference yet) it is redone once.
-    // (A row without a reference that sees nothing in this block has all scores -inf: its P are 0.)
-    auto sweep = [&](float neg_m, float& m_raw) -> float {
-      float sm4[4] = {0.f, 0.f, 0.f, 0.f};
+    // Block maximum first (a pass of comparisons only, on another pipe than the exponentials), so that
+    // the reference maximum is settled before any exponential is taken.  It only moves when the block
+    // maximum exceeds it by more than the threshold, or when the row has no reference yet.
+    float alpha = 1.f;
+    {
       float mx[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
 #pragma unroll
-      for (int c = 0; c < 2; ++c) {
-        uint32_t packed[16];
-#pragma unroll
-        for (int e = 0; e < 16; ++e) {
-          const float s0 = __uint_as_float(sreg[32 * c + 2 * e]), s1 = __uint_as_float(sreg[32 * c + 2 * e + 1]);
-          mx[e & 1] = fmaxf(mx[e & 1], s0);
-          mx[2 + (e & 1)] = fmaxf(mx[2 + (e & 1)], s1);
-          const float p0 = ex2(fmaf(s0, sc, neg_m));
-          const float p1 = ex2(fmaf(s1, sc, neg_m));
-          sm4[e & 1] += p0;
-          sm4[2 + (e & 1)] += p1;
-          packed[e] = pack2<kBf16>(p0, p1);
-        }
-        tmem_st16(tmem_s + 16u * c, packed);
-      }
-      m_raw = fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3]));
-      return (sm4[0] + sm4[1]) + (sm4[2] + sm4[3]);
-    };
-    float alpha = 1.f, m_raw;
-    float sum = sweep(m_used == -INFINITY ? 0.f : -m_used, m_raw);
-    {
-      const float m_blk = m_raw * sc;  // scale > 0
+      for (int e = 0; e < 64; ++e) mx[e & 3] = fmaxf(mx[e & 3], __uint_as_float(sreg[e]));
+      const float m_blk = fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3])) * sc;  // scale > 0
       const bool move = m_blk > m_used + kRescaleThreshold || (m_used == -INFINITY && m_blk != -INFINITY);
-      if (__any_sync(0xffffffffu, move)) {  // rare: the whole warp redoes the block (rows that do not move get the same P again)
+      if (__any_sync(0xffffffffu, move)) {  // rare after the first blocks
         if (move) {
           alpha = m_used == -INFINITY ? 0.f : ex2(m_used - m_blk);
           m_used = m_blk;
@@ -499,8 +482,28 @@ tree_attention_umma_kernel(const __grid_constant__ CUtensorMap q_map, const __gr
             tmem_st32(tmem_o + 32u * c, o, 0);
           }
         }
-        sum = sweep(m_used == -INFINITY ? 0.f : -m_used, m_raw);
       }
+    }
+    // P = 2^(scale*s - m) written over S as packed 16-bit values (32 columns, two stores of 16).
+    // (A row without a reference sees nothing in this block: its scores are all -inf and its P are 0.)
+    float sum;
+    {
+      const float neg_m = m_used == -INFINITY ? 0.f : -m_used;
+      float sm4[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+      for (int c = 0; c < 2; ++c) {
+        uint32_t packed[16];
+#pragma unroll
+        for (int e = 0; e < 16; ++e) {
+          const float p0 = ex2(fmaf(__uint_as_float(sreg[32 * c + 2 * e]), sc, neg_m));
+          const float p1 = ex2(fmaf(__uint_as_float(sreg[32 * c + 2 * e + 1]), sc, neg_m));
+          sm4[e & 1] += p0;
+          sm4[2 + (e & 1)] += p1;
+          packed[e] = pack2<kBf16>(p0, p1);
+        }
+        tmem_st16(tmem_s + 16u * c, packed);
+      }
+      sum = (sm4[0] + sm4[1]) + (sm4[2] + sm4[3]);
     }
     if (threadIdx.x == 128) UTRACE(2, 3);
     l = l * alpha + sum;
@@ -750,8 +753,8 @@ int launch_attention_umma(const seq_tree_attention_params& p, int splits, cudaSt
 #ifdef SEQ_TRACE
 extern "C" int seq_debug_utrace_dump(unsigned long long* host_out) {
   cudaDeviceSynchronize();
-  cudaMemcpyFromSymbol(host_out, seqtree::g_utrace, sizeof(unsigned long long) * 4 * 512);
-  static unsigned long long zeros[4 * 512];
+  cudaMemcpyFromSymbol(host_out, seqtree::g_utrace, sizeof(unsigned long long) * 4 * 2048);
+  static unsigned long long zeros[4 * 2048];
   cudaMemcpyToSymbol(seqtree::g_utrace, zeros, sizeof(zeros));
   return 0;
 }
