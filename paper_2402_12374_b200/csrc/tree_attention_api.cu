@@ -9,6 +9,7 @@ namespace seqtree {
 bool umma_supported(const seq_tree_attention_params& p);
 int umma_default_splits(const seq_tree_attention_params& p);
 int launch_attention_umma(const seq_tree_attention_params& p, int splits, cudaStream_t stream);
+size_t umma_workspace_bytes(const seq_tree_attention_params& p);
 
 static size_t elem_size(int dtype) { return dtype == SEQ_F32 ? 4 : 2; }
 
@@ -59,7 +60,7 @@ extern "C" size_t seq_tree_attention_workspace_bytes(const seq_tree_attention_pa
   if (validate_attention_params(p) != SEQ_OK) return 0;
   const int which = choose_kernel(*p);
   if (which == 0) return 0;
-  if (which == 2) return 0;  // the tensor-core kernel merges its key-range shares on chip
+  if (which == 2) return umma_workspace_bytes(*p);  // only its stream mode (more units than SMs) needs one
   const int splits = simt_default_splits(*p);
   size_t bytes = splits > 1 ? split_workspace_bytes(splits, p->num_q_heads, p->n_tree) : 0;
   return (bytes + 255) & ~(size_t)255;

@@ -49,11 +49,16 @@ namespace seqtree {
 #ifndef SEQ_TRACE_ROLES
 #define SEQ_TRACE_ROLES 15
 #endif
+#ifndef SEQ_TRACE_CTA
+#define SEQ_TRACE_CTA 0
+#endif
 __device__ unsigned long long g_utrace[4][2048];
+__device__ unsigned long long g_cta_times[1024][2];
+__device__ __forceinline__ unsigned long long gtimer() { unsigned long long t; asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t)); return t; }
 #define UTRACE(role, tag)                                                       \
   do {                                                                          \
     if (((SEQ_TRACE_ROLES) >> (role)) & 1) {                                    \
-      if (blockIdx.x == 0 && blockIdx.y == 0 && blockIdx.z == 0 && utrace_i < 2047) \
+      if (blockIdx.x == (SEQ_TRACE_CTA) && blockIdx.y == 0 && blockIdx.z == 0 && utrace_i < 2047) \
         g_utrace[role][++utrace_i] = ((unsigned long long)(tag) << 56) | ((unsigned long long)clock64() & 0xFFFFFFFFFFFFFFull); \
     }                                                                           \
   } while (0)
@@ -67,6 +72,7 @@ constexpr int kUmmaThreads = 384;   // warp group 0: TMA warp, MMA warp, two spa
 constexpr int kRegsLight = 40, kRegsRows = 232;  // after setmaxnreg: 128*40 + 256*232 = 384*168
 constexpr int kMaxClusterSplit = 8;
 constexpr int kNumSMs = 148;
+constexpr int kMaxStreamTiles = 128;  // tiles per kv head the stream mode can index
 constexpr uint32_t kTileBytes = 128 * 128 * 2;   // the Q tile: 128 rows x 128 elements of 16 bits
 constexpr uint32_t kHalfBytes = kTileBytes / 2;  // one 128-row x 64-element sub-tile of Q (128 B rows)
 constexpr uint32_t kKvBytes = kBlockN * 128 * 2; // a K or V tile: 64 keys x 128 elements
@@ -79,18 +85,29 @@ struct UmmaSmem {
   uint8_t q[kTileBytes];
   uint8_t k[2][2][kKvBytes];  // [chain][stage]; after the last block these 64 KB receive the cluster merge
   uint8_t v[2][2][kKvBytes];  // [chain][stage]
-  float2 ml_chain[2][kTileM];                // (m, l) of every row of the two chains of this CTA
+  float2 ml_chain[2][2][kTileM];             // [segment parity][chain]: (m, l) of every row of the two chains of this CTA
   float2 ml_cta[kMaxClusterSplit][kTileM];   // (m, l) of every row of every CTA of the cluster, after its chains are merged
   uint64_t q_full;
   uint64_t k_full[2][2], k_empty[2][2], v_full[2][2], v_empty[2][2], s_full[2][2], p_full[2][2];  // [chain][stage]
   uint64_t pv_done[2];                       // [chain]: one phase per block of the chain
-  uint64_t all_done;                         // every MMA of the CTA has completed
+  uint64_t all_done;                         // every MMA of the segment has completed (one phase per segment)
+  uint64_t o_free;                           // the row threads have read both accumulators (one phase per segment)
   uint32_t tmem_base;
   volatile int abort_flag;
+  int32_t last_part;                         // stream mode: this CTA completed the tile (broadcast to the row threads)
+  int32_t tile_prefix[kMaxStreamTiles + 1];  // stream mode: 64-key blocks of a kv head before tile t
 };
 
 struct UmmaArgs {
   int32_t n, L, Hq, Hkv, group, mask_wpr, splits, nodes_per_tile, tiles;
+  // Stream mode (more (tile, kv head) units than SMs): the 64-key blocks of all units, laid end to end, are
+  // cut into gridDim.x equal ranges, one per CTA; a tile cut by a range boundary is completed by whichever
+  // of its CTAs finishes last, from partial results in the workspace.
+  int32_t stream, blocks_per_head;
+  int64_t total_blocks;
+  int32_t* ws_count;   // [Hkv * tiles] arrivals per tile, zero on entry and on exit
+  float2* ws_ml;       // [2 * gridDim.x][128] (m, l) of a partial result
+  float4* ws_o;        // [2 * gridDim.x][2][16][128] its unnormalised accumulator, thread-major
   float scale_log2;
   uint32_t idesc_qk, idesc_pv;
   const uint32_t* mask_bits;
@@ -266,18 +283,55 @@ tree_attention_umma_kernel(const __grid_constant__ CUtensorMap q_map, const __gr
 #ifdef SEQ_TRACE
   int utrace_i = 0;
 #endif
-  const int tile = blockIdx.x, g = blockIdx.y, split = blockIdx.z;  // the cluster spans blockIdx.z
+  const int split = blockIdx.z;  // the cluster spans blockIdx.z
   if (threadIdx.x == 128) UTRACE(2, 10);
+#ifdef SEQ_TRACE
+  if (threadIdx.x == 128 && blockIdx.y == 0 && blockIdx.z == 0 && blockIdx.x < 1024) g_cta_times[blockIdx.x][0] = gtimer();
+#endif
 
-  const int i0 = tile * a.nodes_per_tile;
-  const int i1 = min(i0 + a.nodes_per_tile, a.n);
-  // keys this tile can see end at L + i1 (a node sees no later node); blocks of this CTA
-  const int nblk_tile = (a.L + i1 + kBlockN - 1) / kBlockN;
-  const int blk_lo = (int)(((long)split * nblk_tile) / a.splits);
-  const int blk_hi = (int)(((long)(split + 1) * nblk_tile) / a.splits);
-  const int nblk = blk_hi - blk_lo;
-
-  if (threadIdx.x == 0) {
+  // A CTA works through segments: (kv head, tile, range of the tile's 64-key blocks).  Grid mode: the one
+  // segment (blockIdx.y, blockIdx.x, this CTA's share of the cluster's key range).  Stream mode: the pieces
+  // of the units that its range [range_lo, range_hi) of the flattened block space overlaps.
+  const int64_t range_lo = a.stream ? (a.total_blocks * (int64_t)blockIdx.x) / (int64_t)gridDim.x : 0;
+  const int64_t range_hi = a.stream ? (a.total_blocks * (int64_t)(blockIdx.x + 1)) / (int64_t)gridDim.x : 1;
+  struct Seg { int g, tile, slot_in_head, i0, i1, blk_lo, nblk, nblk_tile; int64_t next; };
+  // Stream mode lays the tiles of a kv head out alternating from both ends (0, T-1, 1, T-2, ...): late tiles
+  // have more masked blocks, which cost more, and this way every range gets its share of them.
+  auto tile_at = [&](int k) { return (k & 1) ? a.tiles - 1 - (k >> 1) : (k >> 1); };
+  auto seg_at = [&](int64_t pos) -> Seg {
+    Seg x;
+    if (!a.stream) {
+      x.tile = blockIdx.x; x.g = blockIdx.y; x.slot_in_head = x.tile;
+      x.i0 = x.tile * a.nodes_per_tile;
+      x.i1 = min(x.i0 + a.nodes_per_tile, a.n);
+      // keys this tile can see end at L + i1 (a node sees no later node); blocks of this CTA
+      x.nblk_tile = (a.L + x.i1 + kBlockN - 1) / kBlockN;
+      x.blk_lo = (int)(((long)split * x.nblk_tile) / a.splits);
+      x.nblk = (int)(((long)(split + 1) * x.nblk_tile) / a.splits) - x.blk_lo;
+      x.next = 1;
+    } else {
+      x.g = (int)(pos / a.blocks_per_head);
+      const int rem = (int)(pos % a.blocks_per_head);
+      int lo = 0, hi = a.tiles - 1;  // the last place in the head's layout whose first block is at or before rem
+      while (lo < hi) {
+        const int mid = (lo + hi + 1) >> 1;
+        if (sm->tile_prefix[mid] <= rem) lo = mid; else hi = mid - 1;
+      }
+      x.slot_in_head = lo;
+      x.tile = tile_at(lo);
+      x.i0 = x.tile * a.nodes_per_tile;
+      x.i1 = min(x.i0 + a.nodes_per_tile, a.n);
+      x.blk_lo = rem - sm->tile_prefix[lo];
+      x.nblk_tile = sm->tile_prefix[lo + 1] - sm->tile_prefix[lo];
+      x.nblk = (int)min((int64_t)(x.nblk_tile - x.blk_lo), range_hi - pos);
+      x.next = pos + x.nblk;
+    }
+    return x;
+  };
+  // The barriers are armed once.  Their phases run on from segment to segment: a stage barrier counts the
+  // blocks its chain has processed so far, q_full / all_done / o_free count segments.  So the loads and
+  // the first S of the next segment are under way while the row threads still merge and store this one.
+  auto init_barriers = [&]() {  // thread 0
     mbar_init(&sm->q_full, 1);
     for (int c = 0; c < 2; ++c) {
       for (int b = 0; b < 2; ++b) {
@@ -288,8 +342,36 @@ tree_attention_umma_kernel(const __grid_constant__ CUtensorMap q_map, const __gr
       mbar_init(&sm->pv_done[c], 1);
     }
     mbar_init(&sm->all_done, 2);  // one arrival per chain
-    sm->abort_flag = 0;
+    mbar_init(&sm->o_free, 8);    // one arrival per warp of row threads
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  };
+  if (threadIdx.x == 0) {
+    init_barriers();
+    sm->abort_flag = 0;
+  }
+  if (a.stream && warp == 2) {  // blocks of a kv head before each place of its layout: four places per lane, then a warp scan
+    const int per = (a.tiles + 31) / 32;
+    int local[kMaxStreamTiles / 32], sum = 0;
+#pragma unroll
+    for (int k = 0; k < kMaxStreamTiles / 32; ++k) {
+      const int t = lane * per + k;
+      local[k] = (k < per && t < a.tiles) ? (a.L + min((tile_at(t) + 1) * a.nodes_per_tile, a.n) + kBlockN - 1) / kBlockN : 0;
+      sum += local[k];
+    }
+    int incl = sum;
+#pragma unroll
+    for (int d = 1; d < 32; d <<= 1) {
+      const int v = __shfl_up_sync(0xffffffffu, incl, d);
+      if (lane >= d) incl += v;
+    }
+    int run = incl - sum;
+#pragma unroll
+    for (int k = 0; k < kMaxStreamTiles / 32; ++k) {
+      const int t = lane * per + k;
+      if (k < per && t < a.tiles) sm->tile_prefix[t] = run;
+      run += local[k];
+    }
+    if (lane == 31) sm->tile_prefix[a.tiles] = incl;
   }
   if (threadIdx.x == 128) UTRACE(2, 11);
   if (warp == 1) {  // all 512 tensor-memory columns: per chain two S buffers of 64 (P over them), then O_A, O_B
@@ -305,6 +387,10 @@ tree_attention_umma_kernel(const __grid_constant__ CUtensorMap q_map, const __gr
   if (warp < 4) {
     // ============================ warp group 0: data movement and MMA issue, few registers =========
     asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(kRegsLight));
+    int seg = 0, base_a = 0, base_b = 0;  // segments done; blocks chains A, B have processed in them
+    for (int64_t pos = range_lo; pos < range_hi;) {
+    const Seg sg = seg_at(pos);
+    const int g = sg.g, i0 = sg.i0, blk_lo = sg.blk_lo, nblk = sg.nblk;
     if (warp == 0 || warp == 3) {
       // ---------------------------------------------------------- TMA producers -----------------
       // Warp 0 loads Q and the K tiles, warp 3 the V tiles.  A K stage is free as soon as its S has been
@@ -313,6 +399,8 @@ tree_attention_umma_kernel(const __grid_constant__ CUtensorMap q_map, const __gr
       // The whole warp runs the loop; one elected lane issues the copies (coordinates stay warp-uniform).
       if (nblk > 0) {
         const bool is_v = warp == 3;
+        // the Q tile is free when every MMA of the previous segment has completed
+        if (!is_v && seg > 0 && !mbar_wait(sm, &sm->all_done, (seg - 1) & 1, a.dev_status)) break;
         if (!is_v && elect_one()) {
           mbar_expect_tx(&sm->q_full, kTileBytes);
           tma_load_4d(sm->q, &q_map, &sm->q_full, 0, 0, i0, g);
@@ -321,7 +409,8 @@ tree_attention_umma_kernel(const __grid_constant__ CUtensorMap q_map, const __gr
         __syncwarp();
         const CUtensorMap* map = is_v ? &v_map : &k_map;
         for (int jj = 0; jj < nblk; ++jj) {
-          const int c = jj & 1, u = jj >> 1, b = u & 1, w = u >> 1;  // chain, its block index, stage, use count of the stage
+          const int c = jj & 1, u = (c ? base_b : base_a) + (jj >> 1);  // chain, the chain's running block count
+          const int b = u & 1, w = u >> 1;                              // stage, use count of the stage
           const int row = (blk_lo + jj) * kBlockN;
           uint64_t* full = is_v ? &sm->v_full[c][b] : &sm->k_full[c][b];
           uint64_t* empty = is_v ? &sm->v_empty[c][b] : &sm->k_empty[c][b];
@@ -344,13 +433,14 @@ tree_attention_umma_kernel(const __grid_constant__ CUtensorMap q_map, const __gr
       const int c = warp - 1;
       const int n_c = nblk > c ? (nblk - c + 1) >> 1 : 0;  // blocks of this chain
       if (n_c > 0) {
-        bool go = mbar_wait(sm, &sm->q_full, 0, a.dev_status);
+        const int base = c ? base_b : base_a;
+        bool go = mbar_wait(sm, &sm->q_full, seg & 1, a.dev_status);
         // A step along the contraction only moves a descriptor's 14-bit start-address field (16-byte units).
         const uint64_t qd0 = make_desc(smem_u32(sm->q), 16, 1024);
         const uint32_t tmem_o = tmem + 256u + 128u * c;
         // S of block u of the chain: buffer u & 1
         auto issue_qk = [&](int u) -> bool {
-          const int b = u & 1, w = u >> 1;
+          const int b = (base + u) & 1, w = (base + u) >> 1;
           if (!mbar_wait(sm, &sm->k_full[c][b], w & 1, a.dev_status)) return false;
           tc_fence_after();
           const uint64_t kd0 = make_desc(smem_u32(sm->k[c][b]), 16, 1024);
@@ -372,8 +462,10 @@ tree_attention_umma_kernel(const __grid_constant__ CUtensorMap q_map, const __gr
         if (go) go = issue_qk(0);
         if (go && n_c > 1) go = issue_qk(1);
         for (int u = 0; u < n_c && go; ++u) {
-          const int b = u & 1, w = u >> 1;
+          const int b = (base + u) & 1, w = (base + u) >> 1;
           if (!mbar_wait(sm, &sm->p_full[c][b], w & 1, a.dev_status)) break;
+          // the first P.V of a segment overwrites O: the row threads must have read the previous segment's
+          if (u == 0 && seg > 0 && !mbar_wait(sm, &sm->o_free, (seg - 1) & 1, a.dev_status)) break;
           if (lane == 0) UTRACE(c == 0 ? 1 : 3, 3);
           if (!mbar_wait(sm, &sm->v_full[c][b], w & 1, a.dev_status)) break;
           tc_fence_after();
@@ -405,6 +497,10 @@ tree_attention_umma_kernel(const __grid_constant__ CUtensorMap q_map, const __gr
       cluster.sync();
     }
     if (threadIdx.x == 32) UTRACE(1, 9);
+    pos = sg.next;
+    ++seg; base_a += (nblk + 1) >> 1; base_b += nblk >> 1;
+    if (sm->abort_flag) break;
+    }  // segments
     tc_fence_before();
     __syncthreads();
     if (warp == 1) {
@@ -421,6 +517,10 @@ tree_attention_umma_kernel(const __grid_constant__ CUtensorMap q_map, const __gr
   const int r = quad * 32 + lane;             // row of the tile = tensor-memory lane
   const uint32_t lane_sel = (uint32_t)(quad * 32) << 16;
   const uint32_t tmem_o = tmem + 256u + 128u * chain + lane_sel;
+  int seg = 0, base = 0;  // segments done; blocks this chain has processed in them
+  for (int64_t pos = range_lo; pos < range_hi;) {
+  const Seg sg = seg_at(pos);
+  const int g = sg.g, i0 = sg.i0, blk_lo = sg.blk_lo, nblk = sg.nblk;
   const int i = i0 + r / a.group;             // node of this row
   const int h = g * a.group + r % a.group;
   const bool row_valid = i < a.n;
@@ -431,7 +531,7 @@ tree_attention_umma_kernel(const __grid_constant__ CUtensorMap q_map, const __gr
   bool ok = true;
   const int n_mine = nblk > chain ? (nblk - chain + 1) >> 1 : 0;  // blocks of this chain
   for (int u = 0; u < n_mine && ok; ++u) {
-    const int jj = 2 * u + chain, b = u & 1, w = u >> 1;
+    const int jj = 2 * u + chain, b = (base + u) & 1, w = (base + u) >> 1;
     const uint32_t tmem_s = tmem + 128u * chain + 64u * b + lane_sel;
     if (!mbar_wait(sm, &sm->s_full[chain][b], w & 1, a.dev_status)) { ok = false; break; }
     if (threadIdx.x == 128) UTRACE(2, 1);
@@ -470,7 +570,7 @@ tree_attention_umma_kernel(const __grid_constant__ CUtensorMap q_map, const __gr
         }
         if (u > 0) {
           // O may still be taking the chain's previous block: wait for it, then rescale this warp's rows
-          if (!mbar_wait(sm, &sm->pv_done[chain], (u - 1) & 1, a.dev_status)) { ok = false; break; }
+          if (!mbar_wait(sm, &sm->pv_done[chain], (base + u - 1) & 1, a.dev_status)) { ok = false; break; }
           tc_fence_after();
 #pragma unroll
           for (int c = 0; c < 4; ++c) {
@@ -515,7 +615,7 @@ tree_attention_umma_kernel(const __grid_constant__ CUtensorMap q_map, const __gr
   }
   // Both chains must be done with the tensor pipe before O is read and the K stages are reused.  (A
   // parity wait on pv_done could be fooled here: the other chain may be several phases behind.)
-  if (nblk > 0 && ok) ok = mbar_wait(sm, &sm->all_done, 0, a.dev_status);
+  if (nblk > 0 && ok) ok = mbar_wait(sm, &sm->all_done, seg & 1, a.dev_status);
   tc_fence_after();
 
   // ---------------------------------------------------------------- merge ------------------------
@@ -523,12 +623,12 @@ tree_attention_umma_kernel(const __grid_constant__ CUtensorMap q_map, const __gr
   // any column of its 32 lanes, so the thread of chain c and row r merges columns [64c, 64c+64) of
   // O_A and O_B itself; only (m, l) goes through shared memory.
   if (threadIdx.x == 128) UTRACE(2, 6);
-  sm->ml_chain[chain][r] = (ok && n_mine > 0) ? make_float2(m_used, l) : make_float2(-INFINITY, 0.f);
+  sm->ml_chain[seg & 1][chain][r] = (ok && n_mine > 0) ? make_float2(m_used, l) : make_float2(-INFINITY, 0.f);
   asm volatile("bar.sync 1, 256;" ::: "memory");  // the 256 row threads only
   float M, Lc;           // reference maximum and denominator of the CTA's merged partial
   float merged[64];      // its columns [64*chain, 64*chain + 64), unnormalised
   {
-    const float2 mlA = sm->ml_chain[0][r], mlB = sm->ml_chain[1][r];
+    const float2 mlA = sm->ml_chain[seg & 1][0][r], mlB = sm->ml_chain[seg & 1][1][r];
     M = fmaxf(mlA.x, mlB.x);
     const float fA = mlA.x == -INFINITY ? 0.f : ex2(mlA.x - M), fB = mlB.x == -INFINITY ? 0.f : ex2(mlB.x - M);
     Lc = mlA.y * fA + mlB.y * fB;
@@ -553,8 +653,73 @@ tree_attention_umma_kernel(const __grid_constant__ CUtensorMap q_map, const __gr
       for (int e = 0; e < 64; ++e) merged[e] = fmaf(__uint_as_float(o[e]), fB, merged[e]);
     }
   }
+  // both accumulators are in registers: the next segment's first P.V may overwrite them
+  tc_fence_before();
+  __syncwarp();
+  if (lane == 0) mbar_arrive(&sm->o_free);
   uint8_t* out_row = reinterpret_cast<uint8_t*>(a.out) + 2 * ((int64_t)i * a.o_stride_tok + (int64_t)h * a.o_stride_head);
-  if (a.splits == 1) {
+  if (a.stream && nblk < sg.nblk_tile) {
+    // A piece of a tile (stream mode).  Every piece is written to this CTA's slot of the workspace (slot 0
+    // if the piece opens the CTA's range, else 1), then counted; the CTA whose count completes the tile
+    // adds the other pieces to its own and writes the output.  Nobody waits for anybody.
+    const int64_t t0 = (int64_t)g * a.blocks_per_head + sm->tile_prefix[sg.slot_in_head], t1 = t0 + sg.nblk_tile;
+    auto cta_lo = [&](int c) { return (a.total_blocks * (int64_t)c) / (int64_t)gridDim.x; };
+    int c_first = (int)((t0 * (int64_t)gridDim.x) / a.total_blocks);  // the CTA whose range holds block t0 ...
+    while (cta_lo(c_first + 1) <= t0) ++c_first;                      // ... exactly
+    while (cta_lo(c_first) > t0) --c_first;
+    int c_last = c_first;
+    while (cta_lo(c_last + 1) < t1) ++c_last;
+    const int my_slot = 2 * (int)blockIdx.x + (pos == range_lo ? 0 : 1);
+    int* cnt = a.ws_count + (size_t)g * a.tiles + sg.tile;
+    const int parts = c_last - c_first + 1;
+    // If every other piece has been counted already (the usual case for the piece that closes a range: the
+    // others were finished long ago), this CTA completes the tile without writing its own piece.
+    if (threadIdx.x == 128) {
+      const int done = *reinterpret_cast<volatile int*>(cnt) == parts - 1;
+      if (done) *cnt = 0;  // leave the counter as it was found
+      sm->last_part = done;
+    }
+    asm volatile("bar.sync 1, 256;" ::: "memory");
+    if (!sm->last_part) {
+      if (chain == 0) a.ws_ml[(size_t)my_slot * kTileM + r] = make_float2(M, Lc);
+      float4* my_o = a.ws_o + ((size_t)(my_slot * 2 + chain) * 16) * kTileM + r;
+#pragma unroll
+      for (int j = 0; j < 16; ++j) my_o[(size_t)j * kTileM] = make_float4(merged[4 * j], merged[4 * j + 1], merged[4 * j + 2], merged[4 * j + 3]);
+      __threadfence();
+      asm volatile("bar.sync 1, 256;" ::: "memory");
+      if (threadIdx.x == 128) {
+        const int last = atomicAdd(cnt, 1) == parts - 1;
+        if (last) *cnt = 0;  // every piece has been counted
+        sm->last_part = last;
+      }
+      asm volatile("bar.sync 1, 256;" ::: "memory");
+    }
+    if (sm->last_part) {
+      __threadfence();
+      for (int c = c_first; c <= c_last; ++c) {
+        if (c == (int)blockIdx.x) continue;
+        const int slot = 2 * c + (max(t0, cta_lo(c)) == cta_lo(c) ? 0 : 1);
+        const float2 ml = __ldcg(a.ws_ml + (size_t)slot * kTileM + r);
+        if (ml.x == -INFINITY) continue;
+        const float Mn = fmaxf(M, ml.x);
+        const float f_me = M == -INFINITY ? 0.f : ex2(M - Mn), f_it = ex2(ml.x - Mn);
+        const float4* its = a.ws_o + ((size_t)(slot * 2 + chain) * 16) * kTileM + r;
+#pragma unroll
+        for (int j = 0; j < 16; ++j) {
+          const float4 x = __ldcg(its + (size_t)j * kTileM);
+          merged[4 * j] = fmaf(x.x, f_it, merged[4 * j] * f_me);
+          merged[4 * j + 1] = fmaf(x.y, f_it, merged[4 * j + 1] * f_me);
+          merged[4 * j + 2] = fmaf(x.z, f_it, merged[4 * j + 2] * f_me);
+          merged[4 * j + 3] = fmaf(x.w, f_it, merged[4 * j + 3] * f_me);
+        }
+        Lc = fmaf(ml.y, f_it, Lc * f_me);
+        M = Mn;
+      }
+    }
+  }
+  if (a.stream && nblk < sg.nblk_tile && !sm->last_part) {
+    // not the completing piece: nothing to write
+  } else if (a.splits == 1) {
     if (row_valid) {
       const float inv = 1.f / Lc;  // the row saw at least its own key, so Lc > 0
 #pragma unroll
@@ -624,6 +789,13 @@ tree_attention_umma_kernel(const __grid_constant__ CUtensorMap q_map, const __gr
     if (split == 0 && chain == 0 && row_valid && a.lse != nullptr) a.lse[(size_t)h * a.n + i] = (Mg + log2f(Ls)) * kLn2;
   }
   if (threadIdx.x == 128) UTRACE(2, 9);
+  pos = sg.next;
+  ++seg; base += n_mine;
+  if (sm->abort_flag) break;
+  }  // segments
+#ifdef SEQ_TRACE
+  if (threadIdx.x == 128 && blockIdx.y == 0 && blockIdx.z == 0 && blockIdx.x < 1024) g_cta_times[blockIdx.x][1] = gtimer();
+#endif
   // no remote access happens after the second cluster barrier, so CTAs may leave independently
   tc_fence_before();
   __syncthreads();  // pairs with warp group 0, whose MMA warp then frees the tensor memory
@@ -677,6 +849,30 @@ int umma_default_splits(const seq_tree_attention_params& p) {
   return best;
 }
 
+// Stream mode applies when one CTA per (tile, kv head) would need more than one wave of the SMs.
+static bool umma_stream_mode(const seq_tree_attention_params& p, int splits) {
+  const int G = p.num_q_heads / p.num_kv_heads;
+  const int nodes_per_tile = kTileM / G;
+  const int tiles = (p.n_tree + nodes_per_tile - 1) / nodes_per_tile;
+  return splits == 1 && tiles <= kMaxStreamTiles && (long)tiles * p.num_kv_heads > kNumSMs;
+}
+
+// Workspace of the stream mode: one arrival counter per (kv head, tile), then two slots per CTA for the
+// pieces of tiles that its range cuts: (m, l) per row and the 128 x 128 fp32 accumulator.
+static size_t stream_count_bytes(const seq_tree_attention_params& p) {
+  const int G = p.num_q_heads / p.num_kv_heads;
+  const int nodes_per_tile = kTileM / G;
+  const int tiles = (p.n_tree + nodes_per_tile - 1) / nodes_per_tile;
+  return ((size_t)tiles * p.num_kv_heads * sizeof(int32_t) + 255) & ~(size_t)255;
+}
+static constexpr size_t kStreamMlBytes = (size_t)2 * kNumSMs * kTileM * sizeof(float2);
+static constexpr size_t kStreamOBytes = (size_t)2 * kNumSMs * 2 * 16 * kTileM * sizeof(float4);
+
+size_t umma_workspace_bytes(const seq_tree_attention_params& p) {
+  if (!umma_stream_mode(p, umma_default_splits(p))) return 0;
+  return stream_count_bytes(p) + kStreamMlBytes + kStreamOBytes;
+}
+
 int launch_attention_umma(const seq_tree_attention_params& p, int splits, cudaStream_t stream) {
   EncodeTiledFn encode = encode_fn();
   if (encode == nullptr) return SEQ_ERR_CUDA;
@@ -724,10 +920,28 @@ int launch_attention_umma(const seq_tree_attention_params& p, int splits, cudaSt
   a.out = p.out; a.o_stride_tok = p.o_stride_tok; a.o_stride_head = p.o_stride_head;
   a.lse = p.lse;
   a.dev_status = p.dev_status;
+  a.stream = umma_stream_mode(p, splits) ? 1 : 0;
+  a.blocks_per_head = 0; a.total_blocks = 0;
+  a.ws_count = nullptr; a.ws_ml = nullptr; a.ws_o = nullptr;
+  if (a.stream) {
+    const size_t cnt_bytes = stream_count_bytes(p);
+    if (p.workspace == nullptr || p.workspace_bytes < cnt_bytes + kStreamMlBytes + kStreamOBytes) return SEQ_ERR_WORKSPACE;
+    if (reinterpret_cast<uintptr_t>(p.workspace) % 256 != 0) return SEQ_ERR_INVALID_ARG;
+    for (int t = 0; t < tiles; ++t) {
+      const int i1 = (t + 1) * nodes_per_tile < p.n_tree ? (t + 1) * nodes_per_tile : p.n_tree;
+      a.blocks_per_head += (p.prefix_len + i1 + kBlockN - 1) / kBlockN;
+    }
+    a.total_blocks = (int64_t)a.blocks_per_head * p.num_kv_heads;
+    uint8_t* ws = static_cast<uint8_t*>(p.workspace);
+    a.ws_count = reinterpret_cast<int32_t*>(ws);
+    a.ws_ml = reinterpret_cast<float2*>(ws + cnt_bytes);
+    a.ws_o = reinterpret_cast<float4*>(ws + cnt_bytes + kStreamMlBytes);
+    SEQ_CUDA_OK(cudaMemsetAsync(a.ws_count, 0, cnt_bytes, stream));  // the counters start at zero (the kernel leaves them at zero)
+  }
 
   const size_t smem = sizeof(UmmaSmem) + 1024;
   cudaLaunchConfig_t cfg = {};
-  cfg.gridDim = dim3(tiles, p.num_kv_heads, splits);
+  cfg.gridDim = a.stream ? dim3(kNumSMs, 1, 1) : dim3(tiles, p.num_kv_heads, splits);
   cfg.blockDim = dim3(kUmmaThreads);
   cfg.dynamicSmemBytes = smem;
   cfg.stream = stream;
@@ -751,6 +965,11 @@ int launch_attention_umma(const seq_tree_attention_params& p, int splits, cudaSt
 }  // namespace seqtree
 
 #ifdef SEQ_TRACE
+extern "C" int seq_debug_cta_times(unsigned long long* host_out) {
+  cudaDeviceSynchronize();
+  cudaMemcpyFromSymbol(host_out, seqtree::g_cta_times, sizeof(unsigned long long) * 2048);
+  return 0;
+}
 extern "C" int seq_debug_utrace_dump(unsigned long long* host_out) {
   cudaDeviceSynchronize();
   cudaMemcpyFromSymbol(host_out, seqtree::g_utrace, sizeof(unsigned long long) * 4 * 2048);
