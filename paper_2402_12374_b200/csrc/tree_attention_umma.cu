@@ -272,7 +272,7 @@ __device__ __forceinline__ uint32_t mask_window(const uint32_t* row, int wpr, in
   return bits;
 }
 
-template <bool kBf16>
+template <bool kBf16, bool kStream>
 __global__ void __launch_bounds__(kUmmaThreads, 1)
 tree_attention_umma_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant__ CUtensorMap k_map,
                            const __grid_constant__ CUtensorMap v_map, const UmmaArgs a) {
@@ -292,15 +292,15 @@ tree_attention_umma_kernel(const __grid_constant__ CUtensorMap q_map, const __gr
   // A CTA works through segments: (kv head, tile, range of the tile's 64-key blocks).  Grid mode: the one
   // segment (blockIdx.y, blockIdx.x, this CTA's share of the cluster's key range).  Stream mode: the pieces
   // of the units that its range [range_lo, range_hi) of the flattened block space overlaps.
-  const int64_t range_lo = a.stream ? (a.total_blocks * (int64_t)blockIdx.x) / (int64_t)gridDim.x : 0;
-  const int64_t range_hi = a.stream ? (a.total_blocks * (int64_t)(blockIdx.x + 1)) / (int64_t)gridDim.x : 1;
+  const int64_t range_lo = kStream ? (a.total_blocks * (int64_t)blockIdx.x) / (int64_t)gridDim.x : 0;
+  const int64_t range_hi = kStream ? (a.total_blocks * (int64_t)(blockIdx.x + 1)) / (int64_t)gridDim.x : 1;
   struct Seg { int g, tile, slot_in_head, i0, i1, blk_lo, nblk, nblk_tile; int64_t next; };
   // Stream mode lays the tiles of a kv head out alternating from both ends (0, T-1, 1, T-2, ...): late tiles
   // have more masked blocks, which cost more, and this way every range gets its share of them.
   auto tile_at = [&](int k) { return (k & 1) ? a.tiles - 1 - (k >> 1) : (k >> 1); };
   auto seg_at = [&](int64_t pos) -> Seg {
     Seg x;
-    if (!a.stream) {
+    if (!kStream) {
       x.tile = blockIdx.x; x.g = blockIdx.y; x.slot_in_head = x.tile;
       x.i0 = x.tile * a.nodes_per_tile;
       x.i1 = min(x.i0 + a.nodes_per_tile, a.n);
@@ -349,7 +349,7 @@ tree_attention_umma_kernel(const __grid_constant__ CUtensorMap q_map, const __gr
     init_barriers();
     sm->abort_flag = 0;
   }
-  if (a.stream && warp == 2) {  // blocks of a kv head before each place of its layout: four places per lane, then a warp scan
+  if (kStream && warp == 2) {  // blocks of a kv head before each place of its layout: four places per lane, then a warp scan
     const int per = (a.tiles + 31) / 32;
     int local[kMaxStreamTiles / 32], sum = 0;
 #pragma unroll
@@ -387,10 +387,11 @@ tree_attention_umma_kernel(const __grid_constant__ CUtensorMap q_map, const __gr
   if (warp < 4) {
     // ============================ warp group 0: data movement and MMA issue, few registers =========
     asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(kRegsLight));
-    int seg = 0, base_a = 0, base_b = 0;  // segments done; blocks chains A, B have processed in them
+    int seg_n = 0, base_an = 0, base_bn = 0;  // segments done; blocks chains A, B have processed in them
     for (int64_t pos = range_lo; pos < range_hi;) {
     const Seg sg = seg_at(pos);
     const int g = sg.g, i0 = sg.i0, blk_lo = sg.blk_lo, nblk = sg.nblk;
+    const int seg = kStream ? seg_n : 0, base_a = kStream ? base_an : 0, base_b = kStream ? base_bn : 0;  // grid mode: constants
     if (warp == 0 || warp == 3) {
       // ---------------------------------------------------------- TMA producers -----------------
       // Warp 0 loads Q and the K tiles, warp 3 the V tiles.  A K stage is free as soon as its S has been
@@ -498,8 +499,8 @@ tree_attention_umma_kernel(const __grid_constant__ CUtensorMap q_map, const __gr
     }
     if (threadIdx.x == 32) UTRACE(1, 9);
     pos = sg.next;
-    ++seg; base_a += (nblk + 1) >> 1; base_b += nblk >> 1;
-    if (sm->abort_flag) break;
+    ++seg_n; base_an += (nblk + 1) >> 1; base_bn += nblk >> 1;
+    if (kStream && sm->abort_flag) break;
     }  // segments
     tc_fence_before();
     __syncthreads();
@@ -517,10 +518,11 @@ tree_attention_umma_kernel(const __grid_constant__ CUtensorMap q_map, const __gr
   const int r = quad * 32 + lane;             // row of the tile = tensor-memory lane
   const uint32_t lane_sel = (uint32_t)(quad * 32) << 16;
   const uint32_t tmem_o = tmem + 256u + 128u * chain + lane_sel;
-  int seg = 0, base = 0;  // segments done; blocks this chain has processed in them
+  int seg_n = 0, base_n = 0;  // segments done; blocks this chain has processed in them
   for (int64_t pos = range_lo; pos < range_hi;) {
   const Seg sg = seg_at(pos);
   const int g = sg.g, i0 = sg.i0, blk_lo = sg.blk_lo, nblk = sg.nblk;
+  const int seg = kStream ? seg_n : 0, base = kStream ? base_n : 0;  // grid mode: constants
   const int i = i0 + r / a.group;             // node of this row
   const int h = g * a.group + r % a.group;
   const bool row_valid = i < a.n;
@@ -654,11 +656,13 @@ tree_attention_umma_kernel(const __grid_constant__ CUtensorMap q_map, const __gr
     }
   }
   // both accumulators are in registers: the next segment's first P.V may overwrite them
-  tc_fence_before();
-  __syncwarp();
-  if (lane == 0) mbar_arrive(&sm->o_free);
+  if (kStream) {
+    tc_fence_before();
+    __syncwarp();
+    if (lane == 0) mbar_arrive(&sm->o_free);
+  }
   uint8_t* out_row = reinterpret_cast<uint8_t*>(a.out) + 2 * ((int64_t)i * a.o_stride_tok + (int64_t)h * a.o_stride_head);
-  if (a.stream && nblk < sg.nblk_tile) {
+  if (kStream && nblk < sg.nblk_tile) {
     // A piece of a tile (stream mode).  Every piece is written to this CTA's slot of the workspace (slot 0
     // if the piece opens the CTA's range, else 1), then counted; the CTA whose count completes the tile
     // adds the other pieces to its own and writes the output.  Nobody waits for anybody.
@@ -717,7 +721,7 @@ tree_attention_umma_kernel(const __grid_constant__ CUtensorMap q_map, const __gr
       }
     }
   }
-  if (a.stream && nblk < sg.nblk_tile && !sm->last_part) {
+  if (kStream && nblk < sg.nblk_tile && !sm->last_part) {
     // not the completing piece: nothing to write
   } else if (a.splits == 1) {
     if (row_valid) {
@@ -790,8 +794,8 @@ tree_attention_umma_kernel(const __grid_constant__ CUtensorMap q_map, const __gr
   }
   if (threadIdx.x == 128) UTRACE(2, 9);
   pos = sg.next;
-  ++seg; base += n_mine;
-  if (sm->abort_flag) break;
+  ++seg_n; base_n += n_mine;
+  if (kStream && sm->abort_flag) break;
   }  // segments
 #ifdef SEQ_TRACE
   if (threadIdx.x == 128 && blockIdx.y == 0 && blockIdx.z == 0 && blockIdx.x < 1024) g_cta_times[blockIdx.x][1] = gtimer();
@@ -952,14 +956,14 @@ int launch_attention_umma(const seq_tree_attention_params& p, int splits, cudaSt
   attr[0].val.clusterDim.z = splits;
   cfg.attrs = attr;
   cfg.numAttrs = 1;
-  if (p.dtype == SEQ_BF16) {
-    SEQ_CUDA_OK(cudaFuncSetAttribute(tree_attention_umma_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-    SEQ_CUDA_OK(cudaLaunchKernelEx(&cfg, tree_attention_umma_kernel<true>, q_map, k_map, v_map, a));
-  } else {
-    SEQ_CUDA_OK(cudaFuncSetAttribute(tree_attention_umma_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-    SEQ_CUDA_OK(cudaLaunchKernelEx(&cfg, tree_attention_umma_kernel<false>, q_map, k_map, v_map, a));
-  }
-  return SEQ_OK;
+  // four instantiations: element type x (grid | stream) mode; the grid-mode code carries none of the stream machinery
+  auto launch = [&](auto kernel) -> int {
+    SEQ_CUDA_OK(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    SEQ_CUDA_OK(cudaLaunchKernelEx(&cfg, kernel, q_map, k_map, v_map, a));
+    return SEQ_OK;
+  };
+  if (p.dtype == SEQ_BF16) return a.stream ? launch(tree_attention_umma_kernel<true, true>) : launch(tree_attention_umma_kernel<true, false>);
+  return a.stream ? launch(tree_attention_umma_kernel<false, true>) : launch(tree_attention_umma_kernel<false, false>);
 }
 
 }  // namespace seqtree
