@@ -73,6 +73,9 @@ constexpr int kRegsLight = 40, kRegsRows = 232;  // after setmaxnreg: 128*40 + 2
 constexpr int kMaxClusterSplit = 8;
 constexpr int kNumSMs = 148;
 constexpr int kMaxStreamTiles = 128;  // tiles per kv head the stream mode can index
+// Stream mode balances cost, not block counts: every tile is laid out with this many extra positions in
+// front of its blocks, standing for what starting and finishing a tile costs (about 4 us, in 64-key blocks).
+constexpr int kStreamTileCost = 8;
 constexpr uint32_t kTileBytes = 128 * 128 * 2;   // the Q tile: 128 rows x 128 elements of 16 bits
 constexpr uint32_t kHalfBytes = kTileBytes / 2;  // one 128-row x 64-element sub-tile of Q (128 B rows)
 constexpr uint32_t kKvBytes = kBlockN * 128 * 2; // a K or V tile: 64 keys x 128 elements
@@ -95,7 +98,7 @@ struct UmmaSmem {
   uint32_t tmem_base;
   volatile int abort_flag;
   int32_t last_part;                         // stream mode: this CTA completed the tile (broadcast to the row threads)
-  int32_t tile_prefix[kMaxStreamTiles + 1];  // stream mode: 64-key blocks of a kv head before tile t
+  int32_t tile_prefix[kMaxStreamTiles + 1];  // stream mode: positions of a kv head's layout before its t-th tile
 };
 
 struct UmmaArgs {
@@ -321,10 +324,14 @@ tree_attention_umma_kernel(const __grid_constant__ CUtensorMap q_map, const __gr
       x.tile = tile_at(lo);
       x.i0 = x.tile * a.nodes_per_tile;
       x.i1 = min(x.i0 + a.nodes_per_tile, a.n);
-      x.blk_lo = rem - sm->tile_prefix[lo];
-      x.nblk_tile = sm->tile_prefix[lo + 1] - sm->tile_prefix[lo];
-      x.nblk = (int)min((int64_t)(x.nblk_tile - x.blk_lo), range_hi - pos);
-      x.next = pos + x.nblk;
+      // the tile's positions are [vs, ve): kStreamTileCost positions of overhead, then its blocks
+      const int vs = sm->tile_prefix[lo], ve = sm->tile_prefix[lo + 1];
+      const int end = (int)min((int64_t)ve, (int64_t)rem + (range_hi - pos));  // where this CTA leaves the tile
+      const int from = max(rem, vs + kStreamTileCost);
+      x.blk_lo = from - (vs + kStreamTileCost);
+      x.nblk_tile = ve - vs - kStreamTileCost;
+      x.nblk = max(end - from, 0);  // 0: the range ends in the overhead positions, the tile is the next CTA's
+      x.next = pos + (end - rem);
     }
     return x;
   };
@@ -355,7 +362,7 @@ tree_attention_umma_kernel(const __grid_constant__ CUtensorMap q_map, const __gr
 #pragma unroll
     for (int k = 0; k < kMaxStreamTiles / 32; ++k) {
       const int t = lane * per + k;
-      local[k] = (k < per && t < a.tiles) ? (a.L + min((tile_at(t) + 1) * a.nodes_per_tile, a.n) + kBlockN - 1) / kBlockN : 0;
+      local[k] = (k < per && t < a.tiles) ? kStreamTileCost + (a.L + min((tile_at(t) + 1) * a.nodes_per_tile, a.n) + kBlockN - 1) / kBlockN : 0;
       sum += local[k];
     }
     int incl = sum;
@@ -390,6 +397,7 @@ tree_attention_umma_kernel(const __grid_constant__ CUtensorMap q_map, const __gr
     int seg_n = 0, base_an = 0, base_bn = 0;  // segments done; blocks chains A, B have processed in them
     for (int64_t pos = range_lo; pos < range_hi;) {
     const Seg sg = seg_at(pos);
+    if (kStream && sg.nblk == 0) { pos = sg.next; continue; }
     const int g = sg.g, i0 = sg.i0, blk_lo = sg.blk_lo, nblk = sg.nblk;
     const int seg = kStream ? seg_n : 0, base_a = kStream ? base_an : 0, base_b = kStream ? base_bn : 0;  // grid mode: constants
     if (warp == 0 || warp == 3) {
@@ -521,6 +529,7 @@ tree_attention_umma_kernel(const __grid_constant__ CUtensorMap q_map, const __gr
   int seg_n = 0, base_n = 0;  // segments done; blocks this chain has processed in them
   for (int64_t pos = range_lo; pos < range_hi;) {
   const Seg sg = seg_at(pos);
+  if (kStream && sg.nblk == 0) { pos = sg.next; continue; }
   const int g = sg.g, i0 = sg.i0, blk_lo = sg.blk_lo, nblk = sg.nblk;
   const int seg = kStream ? seg_n : 0, base = kStream ? base_n : 0;  // grid mode: constants
   const int i = i0 + r / a.group;             // node of this row
@@ -666,14 +675,15 @@ tree_attention_umma_kernel(const __grid_constant__ CUtensorMap q_map, const __gr
     // A piece of a tile (stream mode).  Every piece is written to this CTA's slot of the workspace (slot 0
     // if the piece opens the CTA's range, else 1), then counted; the CTA whose count completes the tile
     // adds the other pieces to its own and writes the output.  Nobody waits for anybody.
-    const int64_t t0 = (int64_t)g * a.blocks_per_head + sm->tile_prefix[sg.slot_in_head], t1 = t0 + sg.nblk_tile;
+    // positions of the tile's blocks in the layout, and the CTAs whose ranges hold some of them
+    const int64_t t0 = (int64_t)g * a.blocks_per_head + sm->tile_prefix[sg.slot_in_head] + kStreamTileCost, t1 = t0 + sg.nblk_tile;
     auto cta_lo = [&](int c) { return (a.total_blocks * (int64_t)c) / (int64_t)gridDim.x; };
     int c_first = (int)((t0 * (int64_t)gridDim.x) / a.total_blocks);  // the CTA whose range holds block t0 ...
     while (cta_lo(c_first + 1) <= t0) ++c_first;                      // ... exactly
     while (cta_lo(c_first) > t0) --c_first;
     int c_last = c_first;
     while (cta_lo(c_last + 1) < t1) ++c_last;
-    const int my_slot = 2 * (int)blockIdx.x + (pos == range_lo ? 0 : 1);
+    const int my_slot = 2 * (int)blockIdx.x + (max(t0, range_lo) == range_lo ? 0 : 1);
     int* cnt = a.ws_count + (size_t)g * a.tiles + sg.tile;
     const int parts = c_last - c_first + 1;
     // If every other piece has been counted already (the usual case for the piece that closes a range: the
@@ -933,7 +943,7 @@ int launch_attention_umma(const seq_tree_attention_params& p, int splits, cudaSt
     if (reinterpret_cast<uintptr_t>(p.workspace) % 256 != 0) return SEQ_ERR_INVALID_ARG;
     for (int t = 0; t < tiles; ++t) {
       const int i1 = (t + 1) * nodes_per_tile < p.n_tree ? (t + 1) * nodes_per_tile : p.n_tree;
-      a.blocks_per_head += (p.prefix_len + i1 + kBlockN - 1) / kBlockN;
+      a.blocks_per_head += kStreamTileCost + (p.prefix_len + i1 + kBlockN - 1) / kBlockN;
     }
     a.total_blocks = (int64_t)a.blocks_per_head * p.num_kv_heads;
     uint8_t* ws = static_cast<uint8_t*>(p.workspace);
