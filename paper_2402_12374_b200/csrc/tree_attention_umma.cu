@@ -93,7 +93,7 @@ struct UmmaSmem {
   uint64_t q_full;
   uint64_t k_full[2][2], k_empty[2][2], v_full[2][2], v_empty[2][2], s_full[2][2], p_full[2][2];  // [chain][stage]
   uint64_t pv_done[2];                       // [chain]: one phase per block of the chain
-  uint64_t all_done;                         // every MMA of the segment has completed (one phase per segment)
+  uint64_t all_done[2];                      // [chain]: every MMA of the chain in this segment has completed (one phase per segment)
   uint64_t o_free;                           // the row threads have read both accumulators (one phase per segment)
   uint32_t tmem_base;
   volatile int abort_flag;
@@ -336,7 +336,7 @@ tree_attention_umma_kernel(const __grid_constant__ CUtensorMap q_map, const __gr
     return x;
   };
   // The barriers are armed once.  Their phases run on from segment to segment: a stage barrier counts the
-  // blocks its chain has processed so far, q_full / all_done / o_free count segments.  So the loads and
+  // blocks its chain has processed so far, q_full / all_done[] / o_free count segments.  So the loads and
   // the first S of the next segment are under way while the row threads still merge and store this one.
   auto init_barriers = [&]() {  // thread 0
     mbar_init(&sm->q_full, 1);
@@ -348,7 +348,7 @@ tree_attention_umma_kernel(const __grid_constant__ CUtensorMap q_map, const __gr
       }
       mbar_init(&sm->pv_done[c], 1);
     }
-    mbar_init(&sm->all_done, 2);  // one arrival per chain
+    mbar_init(&sm->all_done[0], 1); mbar_init(&sm->all_done[1], 1);  // each has one arriver: its chain's MMA warp
     mbar_init(&sm->o_free, 8);    // one arrival per warp of row threads
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   };
@@ -408,8 +408,10 @@ tree_attention_umma_kernel(const __grid_constant__ CUtensorMap q_map, const __gr
       // The whole warp runs the loop; one elected lane issues the copies (coordinates stay warp-uniform).
       if (nblk > 0) {
         const bool is_v = warp == 3;
-        // the Q tile is free when every MMA of the previous segment has completed
-        if (!is_v && seg > 0 && !mbar_wait(sm, &sm->all_done, (seg - 1) & 1, a.dev_status)) break;
+        // the Q tile is free when every MMA of the previous segment has completed: the row threads have
+        // seen that before they read O (waiting on o_free rather than all_done keeps every waiter of a
+        // barrier within one phase of its arrivers)
+        if (!is_v && seg > 0 && !mbar_wait(sm, &sm->o_free, (seg - 1) & 1, a.dev_status)) break;
         if (!is_v && elect_one()) {
           mbar_expect_tx(&sm->q_full, kTileBytes);
           tma_load_4d(sm->q, &q_map, &sm->q_full, 0, 0, i0, g);
@@ -441,9 +443,12 @@ tree_attention_umma_kernel(const __grid_constant__ CUtensorMap q_map, const __gr
       // commits are issued by one elected lane, so descriptors and addresses stay warp-uniform.
       const int c = warp - 1;
       const int n_c = nblk > c ? (nblk - c + 1) >> 1 : 0;  // blocks of this chain
+      // Both MMA warps see every phase of q_full, also in a segment in which their chain has no block: a
+      // parity wait must never be two phases behind its barrier.
+      const bool q_here = nblk > 0 && mbar_wait(sm, &sm->q_full, seg & 1, a.dev_status);
       if (n_c > 0) {
         const int base = c ? base_b : base_a;
-        bool go = mbar_wait(sm, &sm->q_full, seg & 1, a.dev_status);
+        bool go = q_here;
         // A step along the contraction only moves a descriptor's 14-bit start-address field (16-byte units).
         const uint64_t qd0 = make_desc(smem_u32(sm->q), 16, 1024);
         const uint32_t tmem_o = tmem + 256u + 128u * c;
@@ -494,10 +499,14 @@ tree_attention_umma_kernel(const __grid_constant__ CUtensorMap q_map, const __gr
           // execute in issue order, so this QK^T cannot overtake the P.V just issued.
           if (u + 2 < n_c && !issue_qk(u + 2)) break;
         }
-        if (elect_one()) tc_commit(&sm->all_done);  // arrives when every MMA of this chain has completed
+        if (elect_one()) tc_commit(&sm->all_done[c]);  // arrives when every MMA of this chain has completed
         __syncwarp();
-      } else if (lane == 0 && nblk > 0) {
-        mbar_arrive(&sm->all_done);  // a chain without blocks
+      } else if (nblk > 0) {
+        // A chain without blocks in this segment.  Its arrival must not overtake the completion of its own
+        // previous segment (an asynchronous commit), nor run a phase ahead of the row threads: it waits
+        // until they have taken the previous segment's accumulators.
+        const bool go = q_here && (seg == 0 || mbar_wait(sm, &sm->o_free, (seg - 1) & 1, a.dev_status));
+        if (go && lane == 0) mbar_arrive(&sm->all_done[c]);
       }
       __syncwarp();
     }
@@ -626,7 +635,7 @@ tree_attention_umma_kernel(const __grid_constant__ CUtensorMap q_map, const __gr
   }
   // Both chains must be done with the tensor pipe before O is read and the K stages are reused.  (A
   // parity wait on pv_done could be fooled here: the other chain may be several phases behind.)
-  if (nblk > 0 && ok) ok = mbar_wait(sm, &sm->all_done, seg & 1, a.dev_status);
+  if (nblk > 0 && ok) ok = mbar_wait(sm, &sm->all_done[0], seg & 1, a.dev_status) && mbar_wait(sm, &sm->all_done[1], seg & 1, a.dev_status);
   tc_fence_after();
 
   // ---------------------------------------------------------------- merge ------------------------
@@ -709,26 +718,46 @@ tree_attention_umma_kernel(const __grid_constant__ CUtensorMap q_map, const __gr
       asm volatile("bar.sync 1, 256;" ::: "memory");
     }
     if (sm->last_part) {
+      // The pieces are added in the order of their CTAs, this CTA's own (from registers) at its place, with one
+      // common reference maximum: the result does not depend on which CTA happened to finish last.
       __threadfence();
-      for (int c = c_first; c <= c_last; ++c) {
-        if (c == (int)blockIdx.x) continue;
-        const int slot = 2 * c + (max(t0, cta_lo(c)) == cta_lo(c) ? 0 : 1);
-        const float2 ml = __ldcg(a.ws_ml + (size_t)slot * kTileM + r);
-        if (ml.x == -INFINITY) continue;
-        const float Mn = fmaxf(M, ml.x);
-        const float f_me = M == -INFINITY ? 0.f : ex2(M - Mn), f_it = ex2(ml.x - Mn);
-        const float4* its = a.ws_o + ((size_t)(slot * 2 + chain) * 16) * kTileM + r;
+      auto slot_of = [&](int c) { return 2 * c + (max(t0, cta_lo(c)) == cta_lo(c) ? 0 : 1); };
+      float Mg = M;
+      for (int c = c_first; c <= c_last; ++c)
+        if (c != (int)blockIdx.x) Mg = fmaxf(Mg, __ldcg(a.ws_ml + (size_t)slot_of(c) * kTileM + r).x);
+      float Ls = 0.f;
 #pragma unroll
-        for (int j = 0; j < 16; ++j) {
-          const float4 x = __ldcg(its + (size_t)j * kTileM);
-          merged[4 * j] = fmaf(x.x, f_it, merged[4 * j] * f_me);
-          merged[4 * j + 1] = fmaf(x.y, f_it, merged[4 * j + 1] * f_me);
-          merged[4 * j + 2] = fmaf(x.z, f_it, merged[4 * j + 2] * f_me);
-          merged[4 * j + 3] = fmaf(x.w, f_it, merged[4 * j + 3] * f_me);
+      for (int half = 0; half < 2; ++half) {  // 32 columns at a time: the own piece must stay until its turn
+        float acc[32];
+#pragma unroll
+        for (int e = 0; e < 32; ++e) acc[e] = 0.f;
+        for (int c = c_first; c <= c_last; ++c) {
+          if (c == (int)blockIdx.x) {
+            const float f = M == -INFINITY ? 0.f : ex2(M - Mg);
+#pragma unroll
+            for (int e = 0; e < 32; ++e) acc[e] = fmaf(merged[32 * half + e], f, acc[e]);
+            if (half == 0) Ls = fmaf(Lc, f, Ls);
+          } else {
+            const int slot = slot_of(c);
+            const float2 ml = __ldcg(a.ws_ml + (size_t)slot * kTileM + r);
+            const float f = ml.x == -INFINITY ? 0.f : ex2(ml.x - Mg);
+            const float4* its = a.ws_o + ((size_t)(slot * 2 + chain) * 16 + 8 * half) * kTileM + r;
+#pragma unroll
+            for (int j = 0; j < 8; ++j) {
+              const float4 x = __ldcg(its + (size_t)j * kTileM);
+              acc[4 * j] = fmaf(x.x, f, acc[4 * j]);
+              acc[4 * j + 1] = fmaf(x.y, f, acc[4 * j + 1]);
+              acc[4 * j + 2] = fmaf(x.z, f, acc[4 * j + 2]);
+              acc[4 * j + 3] = fmaf(x.w, f, acc[4 * j + 3]);
+            }
+            if (half == 0) Ls = fmaf(ml.y, f, Ls);
+          }
         }
-        Lc = fmaf(ml.y, f_it, Lc * f_me);
-        M = Mn;
+#pragma unroll
+        for (int e = 0; e < 32; ++e) merged[32 * half + e] = acc[e];
       }
+      M = Mg;
+      Lc = Ls;
     }
   }
   if (kStream && nblk < sg.nblk_tile && !sm->last_part) {
@@ -852,6 +881,7 @@ int umma_default_splits(const seq_tree_attention_params& p) {
 #ifdef SEQ_TRACE
   if (const char* e = getenv("SEQ_DEBUG_SPLITS")) return atoi(e);  // debug builds only
 #endif
+  if (units > kNumSMs && tiles <= kMaxStreamTiles) return 1;  // the stream mode fills the SMs evenly by itself
   int best = 1;
   double best_cost = -1.0;
   for (int cs = 1; cs <= kMaxClusterSplit; cs *= 2) {  // powers of two: 16 slices divide evenly among 2*cs chains

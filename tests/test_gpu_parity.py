@@ -263,6 +263,41 @@ def test_tensor_core_attention_large_magnitude_scores_rescale_path():
     G.check_attention(dataclasses.replace(ai, k_cache=k), kernel=B.KERNEL_TENSOR_CORE)
 
 
+@pytest.mark.parametrize("dtype", ["fp16", "bf16"])
+@pytest.mark.parametrize("n,L,Hq,Hkv", [(300, 200, 64, 8),    # 19 tiles x 8 heads, tiles about as long as a CTA's range
+                                        (600, 100, 32, 2),    # 75 tiles per head (three per lane in the prefix scan)
+                                        (1024, 40, 24, 6),    # maximum tree, 32 tiles x 6 heads, ragged last blocks
+                                        (150, 3000, 128, 16)])  # 10 tiles x 16 heads, long prefix: tiles cut in three
+def test_tensor_core_attention_stream_mode(dtype, n, L, Hq, Hkv):
+    """More (tile, kv head) units than SMs: CTAs take equal ranges of the flattened block space and tiles cut
+    by a range boundary are completed from workspace pieces.  All rows against the oracle, then repeated
+    calls on the same workspace (the arrival counters must have been left at zero), bit for bit."""
+    cfg = _cfg("tiny", num_q_heads=Hq, num_kv_heads=Hkv, prefix_len=L, n_tree=n, max_depth=14)
+    ai = W.make_attention_inputs(cfg, 11, dtype=dtype)
+    d = G.dev()
+    mask, _, st = G.gpu_mask(ai.parent.numpy())
+    lse = torch.empty((Hq, n), dtype=torch.float32, device=d)
+    call = B.AttentionCall(ai.q.to(d), ai.k_cache.to(d), ai.v_cache.to(d), mask, L, lse=lse, dev_status=st,
+                           kernel=B.KERNEL_TENSOR_CORE)
+    assert call.workspace_bytes_needed > 0, "this shape is meant to take the stream mode"
+    first = call.run().clone()
+    torch.cuda.synchronize()
+    assert int(st.item()) == 0
+    ref, rlse, _ = O.tree_attention(ai.q, ai.k_cache, ai.v_cache, ai.parent, L)
+    assert np.abs(first.double().cpu().numpy() - ref).max() < G.ATTN_TOL[ai.q.dtype]
+    assert np.abs(lse.double().cpu().numpy() - rlse).max() < 2e-2
+    # Repeated calls, each after a large fill that empties the L2 and shifts the order in which the CTAs
+    # finish their pieces: the result may not depend on which CTA completes a tile.
+    junk = torch.empty(160 << 20, dtype=torch.uint8, device=d)
+    for it in range(12):
+        junk.fill_(it)
+        again = call.run()
+        if it % 2:
+            again = call.run()  # and back to back
+        torch.cuda.synchronize()
+        assert int(st.item()) == 0 and torch.equal(first, again), f"call {it} differs from the first"
+
+
 @pytest.mark.parametrize("name,rows", [("llama2-7b", [0, 1, 13, 40, 63]), ("llama2-13b", [0, 5, 64, 127]),
                                        ("vicuna-33b", [0, 100, 128, 255]), ("llama3-70b", [0, 31, 32, 400, 767])])
 def test_attention_full_size_configs_sampled_rows(name, rows):
