@@ -105,7 +105,15 @@ int seq_tree_mask_from_parents(const int32_t* parent, int32_t n, uint32_t* mask_
  * head_dim must be 128.  Base pointers and strides must keep every row
  * 16-byte aligned.  dtype selects f16/bf16/f32 for q, k, v and out alike.
  * workspace: at least seq_tree_attention_workspace_bytes(p) bytes, 256-byte
- * aligned, device; contents undefined before and after.
+ * aligned, device; contents undefined before and after.  The size depends on
+ * the shape and on p->kernel and may be 0 (workspace may then be NULL): the
+ * CUDA-core kernel keeps the partial results of its key-range splits there,
+ * the tensor-core kernel the pieces of the query tiles that its CTAs share
+ * when there are more (tile, kv head) units than SMs (about 19 MB then).  A
+ * call with a workspace that is too small returns SEQ_ERR_WORKSPACE and
+ * launches nothing.  Two calls that run concurrently need a workspace each.
+ * The results do not depend on the order in which CTAs finish: a call
+ * repeated on the same inputs returns the same bits.
  */
 typedef struct {
   int32_t n_tree, prefix_len, num_q_heads, num_kv_heads, head_dim;

@@ -1,7 +1,7 @@
 // Tree-masked attention on the 5th-generation tensor cores (tcgen05.mma, accumulators in tensor
 // memory, K/V/Q tiles staged by TMA), for 16-bit inputs.
 //
-// Work unit: one CTA = (kv head g, tile of 128 query rows, share of the key range).  A query row is
+// Work unit: (kv head g, tile of 128 query rows, range of the tile's keys).  A query row is
 // a (node, head-in-group) pair, r = i_local * G + hg, so under GQA the G heads that share a kv head
 // share every K/V tile.  Per block of 64 keys:
 //     S = Q K^T      128x64x128   tcgen05.mma, Q and K K-major in 128-byte-swizzled shared memory
@@ -12,13 +12,26 @@
 // Two chains per CTA, each double-buffered.  Keys are taken in blocks of 64; even blocks of the CTA's
 // key range belong to chain A, odd blocks to chain B.  Each chain has two S/P buffers (64 columns
 // each) and its own accumulator O in tensor memory (2 x (2*64 + 128) = 512 columns), two K and two V
-// stages in shared memory, its own 128 row threads (one warp group) and its own running (m, l); the
-// chains only share Q and the TMA warp; each has its own MMA-issuing warp.  S of a chain's next block is computed while
-// its row threads still work on the current one, so a chain runs at the speed of its softmax, and
-// while one chain exponentiates the tensor pipe also works for the other.  The running maximum of a
-// row is only moved when a block maximum exceeds it by more than 2^8 (the accumulator row is then
-// rescaled in tensor memory).  Registers are rebalanced with setmaxnreg: 40 for the TMA/MMA warp
-// group, 232 for the rows.
+// stages in shared memory, its own 128 row threads (one warp group), its own MMA-issuing warp and its
+// own running (m, l); the chains share Q and the two TMA warps (one for Q and K, one for V: a K stage
+// is free once its S is computed, a V stage only after the block's softmax, and K loads must not queue
+// behind that).  S of a chain's next block is computed while its row threads still work on the current
+// one, so a chain runs at the speed of its softmax, and while one chain exponentiates the tensor pipe
+// also works for the other.  Per block a row thread first takes the block maximum (comparisons only),
+// settles the reference maximum - it only moves when the block maximum exceeds it by more than 2^8, the
+// accumulator row is then rescaled in tensor memory - and then takes the 64 exponentials, which are
+// the bottleneck (16 per clock and SM).  Registers are rebalanced with setmaxnreg: 40 for the TMA/MMA
+// warp group, 232 for the rows.
+//
+// Work distribution.  Grid mode (at most one wave of CTAs): one CTA per (tile, kv head), or a cluster
+// of 2, 4 or 8 CTAs that split its key range.  Stream mode (more units than SMs): one CTA per SM; the
+// 64-key blocks of all units are laid end to end (each tile preceded by a few positions that stand for
+// its fixed cost, tiles of a head taken alternately from both ends) and cut into equal ranges.  A CTA
+// works through the segments of its range with barrier phases that run on from segment to segment, so
+// the next segment's loads and first S are under way while the rows still merge and store.  A tile cut
+// by a range boundary is completed by whichever of its CTAs finishes last: the others leave their
+// piece (m, l, unnormalised accumulator) in the workspace and count themselves on the tile's counter;
+// the pieces are added in CTA order, so the result does not depend on who finishes last.
 //
 // Merge.  The CTAs that share (tile, kv head) form a thread-block cluster along the key
 // range (cs = 1, 2, 4 or 8); its 2*cs chains share the 16 slices of 8 output columns round-robin.  Every chain pushes,
