@@ -198,6 +198,8 @@ def main():
     ap.add_argument("--temperature", type=float, default=0.6)
     ap.add_argument("--kernel", type=int, default=0, help="0 auto, 1 CUDA-core, 2 tensor-core attention")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--separate-mask", action="store_true",
+                    help="build the ancestor mask with a launch of its own instead of inside the attention kernel")
     args = ap.parse_args()
     cfg = W.CONFIGS[args.workload]
     T = args.temperature
@@ -234,20 +236,26 @@ def main():
     depth = torch.empty(n, dtype=torch.int32, device=dev)
     attn_calls, ver_calls = [], []
     workspace = None
+    # The ancestor mask: derived from the parent array inside the attention kernel (tensor-core kernel), or by a
+    # launch of its own before it (--separate-mask, and always for the CUDA-core kernel).
+    fused_mask = (not args.separate_mask and args.kernel != B.KERNEL_CUDA_CORE and cfg.dtype in ("fp16", "bf16")
+                  and 128 % (cfg.num_q_heads // cfg.num_kv_heads) == 0)
     for ai in attn_h:
-        call = B.AttentionCall(ai.q.to(dev), ai.k_cache.to(dev), ai.v_cache.to(dev), mask, cfg.prefix_len,
-                               workspace=workspace, dev_status=status, kernel=args.kernel)
-        workspace = call._keep[6]
+        call = B.AttentionCall(ai.q.to(dev), ai.k_cache.to(dev), ai.v_cache.to(dev), None if fused_mask else mask,
+                               cfg.prefix_len, parent=parent_d, workspace=workspace, dev_status=status, kernel=args.kernel)
+        workspace = call.workspace
         attn_calls.append(call)
     for vi in ver_h:
         ver_calls.append(B.VerifyCall(parent_d, vi.tokens.to(dev), vi.target_logits.to(dev), vi.draft_logits.to(dev),
                                       T, vi.uniforms.to(dev), dev_status=status))
-    launches_per_step = 1 + (2 if attn_calls[0].workspace_bytes_needed else 1) + 1
+    combine = args.kernel == B.KERNEL_CUDA_CORE and attn_calls[0].workspace_bytes_needed > 0  # split-KV partials merged by a second kernel
+    launches_per_step = (0 if fused_mask else 1) + (2 if combine else 1) + 1
 
     stream = torch.cuda.Stream(device=dev)
 
     def step(i, s, ev=None):
-        B.seq_tree_mask_from_parents(parent_d, mask_bits=mask, depth=depth, dev_status=status, stream=s)
+        if not fused_mask:
+            B.seq_tree_mask_from_parents(parent_d, mask_bits=mask, depth=depth, dev_status=status, stream=s)
         if ev:
             ev[0].record(s)
         attn_calls[i % na].run(s)
@@ -310,7 +318,8 @@ def main():
 
     # end to end from pinned host buffers through the public API, copies inside the timed region
     host = B.HostStep(attn_h[0].q, attn_h[0].k_cache, attn_h[0].v_cache, torch.from_numpy(parent), cfg.prefix_len,
-                      ver_h[0].tokens, ver_h[0].target_logits, ver_h[0].draft_logits, T, ver_h[0].uniforms, device=dev)
+                      ver_h[0].tokens, ver_h[0].target_logits, ver_h[0].draft_logits, T, ver_h[0].uniforms, device=dev,
+                      fused_mask=fused_mask, kernel=args.kernel)
     Ke = min(K, 20)
     with torch.cuda.stream(stream):
         for _ in range(3):
@@ -371,7 +380,8 @@ def main():
         "config": {"workload": cfg.name, "temperature": T, "n_tree": n, "prefix_len": cfg.prefix_len,
                    "heads": f"{cfg.num_q_heads}/{cfg.num_kv_heads}", "vocab": cfg.vocab, "requests_per_gpu": 1,
                    "l2": f"inputs rotate over {na} attention sets ({na * attn_bytes >> 20} MiB) and {nv} logit sets, "
-                         f"larger than the 126 MiB L2", "launch": "CUDA graph of the K steps"},
+                         f"larger than the 126 MiB L2", "launch": "CUDA graph of the K steps",
+                   "mask": "from the parent array inside the attention kernel" if fused_mask else "separate launch"},
         "clocks": clocks.summary(),
         "e2e": {"value": e2e_us, "unit": UNIT, "h2d_bytes_per_step": host.h2d_bytes, "d2h_bytes_per_step": host.d2h_bytes,
                 "steps": Ke},

@@ -104,6 +104,16 @@ int seq_tree_mask_from_parents(const int32_t* parent, int32_t n, uint32_t* mask_
  *                 sum-exp of the scaled scores of each row.
  * head_dim must be 128.  Base pointers and strides must keep every row
  * 16-byte aligned.  dtype selects f16/bf16/f32 for q, k, v and out alike.
+ * Mask from the parent array: with mask_bits == NULL and parent != NULL the
+ * tensor-core kernel derives each query tile's ancestor rows from parent[]
+ * itself (the walk of seq_tree_mask_from_parents, done in shared memory while
+ * the first tiles are in flight), so a decoding step needs no separate mask
+ * launch; a parent[i] outside {-1} u [0,i) raises SEQ_DEV_BAD_PARENT and is
+ * read as -1, as there.  The results are those of a call with the mask_bits of
+ * seq_tree_mask_from_parents(parent).  The CUDA-core kernel has no such mode:
+ * a request that needs it (fp32, a group size that does not divide 128,
+ * kernel == 1) without mask_bits returns SEQ_ERR_UNSUPPORTED.  When mask_bits
+ * is given, parent is ignored.
  * workspace: at least seq_tree_attention_workspace_bytes(p) bytes, 256-byte
  * aligned, device; contents undefined before and after.  The size depends on
  * the shape and on p->kernel and may be 0 (workspace may then be NULL): the
@@ -134,6 +144,7 @@ typedef struct {
   size_t workspace_bytes;
   int32_t* dev_status;
   int32_t kernel; /* 0 = choose; 1 = force the CUDA-core kernel; 2 = force the tensor-core kernel */
+  const int32_t* parent; /* nullable, [n_tree] int32, device: see "mask from the parent array" above */
 } seq_tree_attention_params;
 
 size_t seq_tree_attention_workspace_bytes(const seq_tree_attention_params* p);

@@ -55,6 +55,7 @@ class AttentionParams(C.Structure):
         ("out", C.c_void_p), ("o_stride_tok", C.c_int64), ("o_stride_head", C.c_int64),
         ("lse", C.c_void_p), ("workspace", C.c_void_p), ("workspace_bytes", C.c_size_t),
         ("dev_status", C.c_void_p), ("kernel", C.c_int32),
+        ("parent", C.c_void_p),
     ]
 
 
@@ -147,9 +148,11 @@ class AttentionCall:
 
     def __init__(self, q, k_cache, v_cache, mask_bits, prefix_len: int, *, out=None, lse=None,
                  softmax_scale: float = 0.0, workspace=None, dev_status=None, kernel: int = KERNEL_AUTO,
-                 noalloc: bool = False):
+                 noalloc: bool = False, parent=None):
         """``noalloc=True`` prepares a call of ``seq_tree_attention_noalloc``: no workspace tensor is
-        created or passed; the library's built-in scratch array is used (CUDA-core kernel)."""
+        created or passed; the library's built-in scratch array is used (CUDA-core kernel).
+        ``mask_bits=None`` with ``parent`` (int32 [n], device) lets the tensor-core kernel derive the
+        ancestor mask from the parent array itself."""
         if q.dtype not in _DTYPES or k_cache.dtype != q.dtype or v_cache.dtype != q.dtype:
             raise ValueError("q, k_cache, v_cache must share one of float16/bfloat16/float32")
         n, Hq, d = q.shape
@@ -169,7 +172,13 @@ class AttentionCall:
         p.q, p.q_stride_tok, p.q_stride_head = _dev(q, "q"), q.stride(0), q.stride(1)
         p.k_cache, p.v_cache = _dev(k_cache, "k_cache"), _dev(v_cache, "v_cache")
         p.kv_stride_tok, p.kv_stride_head, p.kv_capacity = k_cache.stride(1), k_cache.stride(0), cap
-        p.mask_bits, p.mask_words_per_row = _dev(mask_bits, "mask_bits", torch.int32), mask_bits.shape[1]
+        if mask_bits is not None:
+            p.mask_bits, p.mask_words_per_row = _dev(mask_bits, "mask_bits", torch.int32), mask_bits.shape[1]
+        else:
+            if parent is None:
+                raise ValueError("mask_bits or parent is required")
+            p.mask_bits, p.mask_words_per_row = None, 0
+        p.parent = _dev(parent, "parent", torch.int32)
         p.out, p.o_stride_tok, p.o_stride_head = _dev(out, "out", q.dtype), out.stride(0), out.stride(1)
         p.lse = _dev(lse, "lse", torch.float32)
         p.dev_status = _dev(dev_status, "dev_status", torch.int32)
@@ -181,7 +190,8 @@ class AttentionCall:
         p.workspace = _dev(workspace, "workspace") if workspace is not None else None
         p.workspace_bytes = workspace.numel() * workspace.element_size() if workspace is not None else 0
         self.params, self.out, self.lse, self.workspace_bytes_needed = p, out, lse, need
-        self._keep = (q, k_cache, v_cache, mask_bits, out, lse, workspace, dev_status)
+        self.workspace = workspace
+        self._keep = (q, k_cache, v_cache, mask_bits, parent, out, lse, workspace, dev_status)
 
     def run(self, stream=None):
         if self.noalloc:
@@ -256,11 +266,12 @@ def seq_tree_verify(parent, tokens, target_logits, draft_logits, temperature: fl
 
 class HostStep:
     """One whole verify step fed from pinned HOST buffers: per call it copies the step's inputs to
-    the device, builds the ancestor mask, runs attention and verification, and copies the results
-    (attention output, path, bonus token) back.  Device staging buffers are allocated once here."""
+    the device, builds the ancestor mask (inside the attention kernel with ``fused_mask``, else by a
+    launch of its own), runs attention and verification, and copies the results (attention output,
+    path, bonus token) back.  Device staging buffers are allocated once here."""
 
     def __init__(self, q, k_cache, v_cache, parent, prefix_len, tokens, target_logits, draft_logits, temperature,
-                 uniforms, device="cuda"):
+                 uniforms, device="cuda", fused_mask: bool = False, kernel: int = KERNEL_AUTO):
         self.host_in = [t if t.is_pinned() else t.pin_memory()
                         for t in (q, k_cache, v_cache, parent, tokens, target_logits, draft_logits, uniforms)]
         self.dev_in = [torch.empty_like(t, device=device) for t in self.host_in]
@@ -269,7 +280,9 @@ class HostStep:
         self.mask = torch.empty((n, (n + 31) // 32), dtype=torch.int32, device=device)
         self.depth = torch.empty(n, dtype=torch.int32, device=device)
         self.status = torch.zeros(1, dtype=torch.int32, device=device)
-        self.attn = AttentionCall(dq, dk, dv, self.mask, prefix_len, dev_status=self.status)
+        self.fused_mask = fused_mask
+        self.attn = AttentionCall(dq, dk, dv, None if fused_mask else self.mask, prefix_len, parent=dparent,
+                                  dev_status=self.status, kernel=kernel)
         self.verify = VerifyCall(dparent, dtok, dtl, ddl, temperature, du, dev_status=self.status)
         self.host_out = [torch.empty_like(self.attn.out, device="cpu").pin_memory(),
                          torch.empty(n, dtype=torch.int32).pin_memory(),
@@ -281,8 +294,9 @@ class HostStep:
     def run(self, stream=None):
         for h, d in zip(self.host_in, self.dev_in):
             d.copy_(h, non_blocking=True)
-        seq_tree_mask_from_parents(self.dev_in[3], mask_bits=self.mask, depth=self.depth, dev_status=self.status,
-                                   stream=stream)
+        if not self.fused_mask:
+            seq_tree_mask_from_parents(self.dev_in[3], mask_bits=self.mask, depth=self.depth, dev_status=self.status,
+                                       stream=stream)
         self.attn.run(stream)
         self.verify.run(stream)
         for h, d in zip(self.host_out, (self.attn.out, self.verify.path, self.verify.path_len, self.verify.bonus_token)):

@@ -16,7 +16,7 @@ static size_t elem_size(int dtype) { return dtype == SEQ_F32 ? 4 : 2; }
 int validate_attention_params(const seq_tree_attention_params* p) {
   if (p == nullptr) return SEQ_ERR_INVALID_ARG;
   if (p->q == nullptr || p->k_cache == nullptr || p->v_cache == nullptr || p->out == nullptr ||
-      p->mask_bits == nullptr)
+      (p->mask_bits == nullptr && p->parent == nullptr))
     return SEQ_ERR_INVALID_ARG;
   if (p->n_tree < 1 || p->n_tree > SEQ_MAX_TREE || p->prefix_len < 0) return SEQ_ERR_INVALID_ARG;
   if (p->num_q_heads < 1 || p->num_kv_heads < 1 || p->num_q_heads % p->num_kv_heads != 0)
@@ -25,7 +25,7 @@ int validate_attention_params(const seq_tree_attention_params* p) {
   if (p->dtype != SEQ_F16 && p->dtype != SEQ_BF16 && p->dtype != SEQ_F32) return SEQ_ERR_INVALID_ARG;
   if (p->head_dim != kHeadDim) return SEQ_ERR_UNSUPPORTED;
   if ((int64_t)p->prefix_len + p->n_tree > (int64_t)p->kv_capacity) return SEQ_ERR_INVALID_ARG;
-  if (p->mask_words_per_row < (p->n_tree + 31) / 32) return SEQ_ERR_INVALID_ARG;
+  if (p->mask_bits != nullptr && p->mask_words_per_row < (p->n_tree + 31) / 32) return SEQ_ERR_INVALID_ARG;
   if (isnan(p->softmax_scale) || isinf(p->softmax_scale)) return SEQ_ERR_INVALID_ARG;
   const size_t es = elem_size(p->dtype);
   const int64_t strides[] = {p->q_stride_tok,  p->q_stride_head, p->kv_stride_tok,
@@ -41,8 +41,9 @@ int validate_attention_params(const seq_tree_attention_params* p) {
 
 // 1 = CUDA cores, 2 = tensor cores
 static int choose_kernel(const seq_tree_attention_params& p) {
-  if (p.kernel == 1) return 1;
   const bool ok = umma_supported(p);
+  if (p.mask_bits == nullptr) return ok && p.kernel != 1 ? 2 : 0;  // only the tensor-core kernel derives the mask itself
+  if (p.kernel == 1) return 1;
   if (p.kernel == 2) return ok ? 2 : 0;
   if (!ok) return 1;
   // Measured on B200: even with a single query row per kv head (127 of the tile's 128 rows padding) the

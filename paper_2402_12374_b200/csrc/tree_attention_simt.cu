@@ -327,6 +327,7 @@ extern "C" int seq_tree_attention_noalloc(const seq_tree_attention_params* p, vo
   using namespace seqtree;
   int rc = validate_attention_params(p);
   if (rc != SEQ_OK) return rc;
+  if (p->mask_bits == nullptr) return SEQ_ERR_UNSUPPORTED;  // the CUDA-core kernel does not derive the mask itself
   const int splits = simt_default_splits(*p);
   const size_t need = splits > 1 ? split_workspace_bytes(splits, p->num_q_heads, p->n_tree) : 0;
   if (need > SEQ_NOALLOC_SCRATCH_BYTES) return SEQ_ERR_WORKSPACE;  // too large for the built-in array

@@ -111,6 +111,9 @@ struct UmmaSmem {
   uint32_t tmem_base;
   volatile int abort_flag;
   int32_t last_part;                         // stream mode: this CTA completed the tile (broadcast to the row threads)
+  // mask from the parent array: the tree, and the ancestor rows of the current tile's nodes (row stride 33 words)
+  int32_t parent[SEQ_MAX_TREE];
+  uint32_t tile_mask[kTileM][SEQ_MAX_TREE / 32 + 1];
   int32_t tile_prefix[kMaxStreamTiles + 1];  // stream mode: positions of a kv head's layout before its t-th tile
 };
 
@@ -127,6 +130,7 @@ struct UmmaArgs {
   float scale_log2;
   uint32_t idesc_qk, idesc_pv;
   const uint32_t* mask_bits;
+  const int32_t* parent;  // used when mask_bits is null
   void* out; int64_t o_stride_tok, o_stride_head;
   float* lse;
   int32_t* dev_status;
@@ -369,6 +373,8 @@ tree_attention_umma_kernel(const __grid_constant__ CUtensorMap q_map, const __gr
     init_barriers();
     sm->abort_flag = 0;
   }
+  if (a.mask_bits == nullptr)
+    for (int t = threadIdx.x; t < a.n; t += kUmmaThreads) sm->parent[t] = a.parent[t];
   if (kStream && warp == 2) {  // blocks of a kv head before each place of its layout: four places per lane, then a warp scan
     const int per = (a.tiles + 31) / 32;
     int local[kMaxStreamTiles / 32], sum = 0;
@@ -557,7 +563,28 @@ tree_attention_umma_kernel(const __grid_constant__ CUtensorMap q_map, const __gr
   const int i = i0 + r / a.group;             // node of this row
   const int h = g * a.group + r % a.group;
   const bool row_valid = i < a.n;
-  const uint32_t* mrow = a.mask_bits + (size_t)min(i, a.n - 1) * a.mask_wpr;
+  // The row's ancestor bits: the caller's mask, or rows derived from the parent array at the start of the
+  // segment by the first thread of each node (0 <= parent[j] < j, so a walk ends; anything else is flagged and
+  // read as "no parent").  In grid mode the row threads are idle at this point, waiting for the first tiles.
+  // (The previous segment's rows are out of use: every row thread has passed that segment's merge barrier.)
+  if (a.mask_bits == nullptr) {
+    if (chain == 0 && r % a.group == 0) {
+      uint32_t* row = sm->tile_mask[r / a.group];
+      const int wpr = (a.n + 31) >> 5;
+      for (int w = 0; w < wpr; ++w) row[w] = 0u;  // (nodes past the last one see no tree key)
+      int j = i;
+      for (int step = 0; step < a.n && row_valid; ++step) {
+        row[j >> 5] |= 1u << (j & 31);
+        const int pj = sm->parent[j];
+        if (pj == -1) break;
+        if (pj < -1 || pj >= j) { dev_flag(a.dev_status, SEQ_DEV_BAD_PARENT); break; }
+        j = pj;
+      }
+    }
+    asm volatile("bar.sync 1, 256;" ::: "memory");
+  }
+  const uint32_t* mrow = a.mask_bits != nullptr ? a.mask_bits + (size_t)min(i, a.n - 1) * a.mask_wpr : sm->tile_mask[r / a.group];
+  const int mask_wpr = a.mask_bits != nullptr ? a.mask_wpr : (a.n + 31) >> 5;
   const float sc = a.scale_log2;
 
   float m_used = -INFINITY, l = 0.f;
@@ -576,8 +603,8 @@ tree_attention_umma_kernel(const __grid_constant__ CUtensorMap q_map, const __gr
     const bool masked = kb + kBlockN > a.L;  // the block reaches into the tree keys (or past the end)
     uint32_t vis[2] = {0xFFFFFFFFu, 0xFFFFFFFFu};
     if (masked) {
-      vis[0] = mask_window(mrow, a.mask_wpr, a.n, kb - a.L);
-      vis[1] = mask_window(mrow, a.mask_wpr, a.n, kb - a.L + 32);
+      vis[0] = mask_window(mrow, mask_wpr, a.n, kb - a.L);
+      vis[1] = mask_window(mrow, mask_wpr, a.n, kb - a.L + 32);
     }
     tc_wait_ld();
     if (threadIdx.x == 128) UTRACE(2, 2);
@@ -974,6 +1001,7 @@ int launch_attention_umma(const seq_tree_attention_params& p, int splits, cudaSt
   a.idesc_qk = idesc | ((uint32_t)(kBlockN >> 3) << 17);                 // S: N = 64 keys
   a.idesc_pv = idesc | ((uint32_t)(kHeadDim >> 3) << 17) | (1u << 16);   // O: N = 128, V is MN-major
   a.mask_bits = p.mask_bits;
+  a.parent = p.parent;
   a.out = p.out; a.o_stride_tok = p.o_stride_tok; a.o_stride_head = p.o_stride_head;
   a.lse = p.lse;
   a.dev_status = p.dev_status;

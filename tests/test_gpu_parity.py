@@ -298,6 +298,54 @@ def test_tensor_core_attention_stream_mode(dtype, n, L, Hq, Hkv):
         assert int(st.item()) == 0 and torch.equal(first, again), f"call {it} differs from the first"
 
 
+@pytest.mark.parametrize("n,L,Hq,Hkv,tree", [(1, 0, 2, 2, "random"), (17, 33, 4, 4, "random"), (64, 1024, 32, 32, "random"),
+                                             (130, 1000, 4, 4, "chain"), (257, 5, 16, 1, "star"), (1024, 40, 24, 6, "random"),
+                                             (768, 4096, 64, 8, "random")])
+def test_tensor_core_attention_mask_from_parent_array(n, L, Hq, Hkv, tree):
+    """mask_bits = NULL, parent given: the kernel walks the parent array itself.  Same bits as with the mask
+    of seq_tree_mask_from_parents (grid mode with and without clusters, and stream mode)."""
+    cfg = _cfg("tiny", num_q_heads=Hq, num_kv_heads=Hkv, prefix_len=L, n_tree=n, max_depth=14)
+    parent = {"random": None, "chain": W.chain_tree(n), "star": W.star_tree(n)}[tree]
+    ai = W.make_attention_inputs(cfg, 13, parent=parent, dtype="bf16")
+    d = G.dev()
+    q, k, v, par = ai.q.to(d), ai.k_cache.to(d), ai.v_cache.to(d), ai.parent.to(d)
+    mask, _, _ = G.gpu_mask(ai.parent.numpy())
+    st = torch.zeros(1, dtype=torch.int32, device=d)
+    with_mask = B.seq_tree_attention(q, k, v, mask, L, kernel=B.KERNEL_TENSOR_CORE).clone()
+    lse = torch.empty((Hq, n), dtype=torch.float32, device=d)
+    fused = B.seq_tree_attention(q, k, v, None, L, parent=par, lse=lse, dev_status=st)
+    torch.cuda.synchronize()
+    assert int(st.item()) == 0 and torch.equal(with_mask, fused)
+    if n <= 300:
+        ref, rlse, _ = O.tree_attention(ai.q, ai.k_cache, ai.v_cache, ai.parent, L)
+        assert np.abs(fused.double().cpu().numpy() - ref).max() < 2e-2
+        assert np.abs(lse.double().cpu().numpy() - rlse).max() < 2e-2
+
+
+def test_attention_mask_from_parent_array_bad_parent_and_unsupported():
+    cfg = _cfg("tiny", num_q_heads=4, num_kv_heads=2, prefix_len=40, n_tree=50)
+    ai = W.make_attention_inputs(cfg, 14, dtype="bf16")
+    d = G.dev()
+    q, k, v = ai.q.to(d), ai.k_cache.to(d), ai.v_cache.to(d)
+    bad = ai.parent.clone()
+    bad[20] = 35   # a later node: flagged, read as "no parent"
+    bad[30] = -7
+    st = torch.zeros(1, dtype=torch.int32, device=d)
+    fused = B.seq_tree_attention(q, k, v, None, 40, parent=bad.to(d), dev_status=st)
+    torch.cuda.synchronize()
+    assert int(st.item()) & B.SEQ_DEV_BAD_PARENT
+    st2 = torch.zeros(1, dtype=torch.int32, device=d)
+    mask, _ = B.seq_tree_mask_from_parents(bad.to(d), dev_status=st2)   # same reading of the bad entries
+    assert torch.equal(fused, B.seq_tree_attention(q, k, v, mask, 40, kernel=B.KERNEL_TENSOR_CORE))
+    # the CUDA-core kernel needs mask_bits
+    with pytest.raises(B.SeqTreeError) as e:
+        B.seq_tree_attention(q, k, v, None, 40, parent=ai.parent.to(d), kernel=B.KERNEL_CUDA_CORE)
+    assert e.value.code == B.SEQ_ERR_UNSUPPORTED
+    with pytest.raises(B.SeqTreeError) as e:
+        B.seq_tree_attention(q.float(), k.float(), v.float(), None, 40, parent=ai.parent.to(d))
+    assert e.value.code == B.SEQ_ERR_UNSUPPORTED
+
+
 @pytest.mark.parametrize("name,rows", [("llama2-7b", [0, 1, 13, 40, 63]), ("llama2-13b", [0, 5, 64, 127]),
                                        ("vicuna-33b", [0, 100, 128, 255]), ("llama3-70b", [0, 31, 32, 400, 767])])
 def test_attention_full_size_configs_sampled_rows(name, rows):
