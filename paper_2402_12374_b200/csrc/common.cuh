@@ -24,10 +24,14 @@ __device__ __forceinline__ void dev_flag(int32_t* dev_status, int bit) {
   if (dev_status != nullptr) atomicOr(dev_status, bit);
 }
 
+// Maximum over the warp in one redux.sync: floats are mapped to integers in the same order (sign-magnitude to
+// two's complement), -inf and +inf included.  (A NaN, which fmaxf would drop, comes out as the maximum.)
 __device__ __forceinline__ float warp_max(float v) {
-#pragma unroll
-  for (int o = 16; o > 0; o >>= 1) v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, o));
-  return v;
+  int b = __float_as_int(v);
+  b ^= (b >> 31) & 0x7fffffff;
+  b = __reduce_max_sync(0xffffffffu, b);
+  b ^= (b >> 31) & 0x7fffffff;
+  return __int_as_float(b);
 }
 __device__ __forceinline__ float warp_sum(float v) {
 #pragma unroll

@@ -113,9 +113,14 @@ __device__ __forceinline__ float sanitize_logit(float x, int32_t* dev_status) {
   dev_flag(dev_status, SEQ_DEV_NONFINITE);
   return x != x ? -INFINITY : FLT_MAX;
 }
+__device__ __forceinline__ float fast_ex2(float x) {  // 2^x, relative error 2^-22; 2^-inf = 0
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
 // 2^((m - M) c2), and 0 for an empty (all -inf) part
 __device__ __forceinline__ float rel_exp(float m, float M, float c2) {
-  return m == -INFINITY ? 0.f : exp2f((m - M) * c2);
+  return m == -INFINITY ? 0.f : fast_ex2((m - M) * c2);
 }
 // unnormalised residual max(p - C q - U, 0) of one token
 __device__ __forceinline__ float resid(float pn, float qn, float Cf, float Uf) {
@@ -127,13 +132,10 @@ __device__ __forceinline__ float resid(float pn, float qn, float Cf, float Uf) {
 template <typename F4, typename F1>
 __device__ __forceinline__ void sweep(const Ctx& c, F4 f4, F1 f1) {
   int t = c.s_lo + 4 * c.lane;
+#pragma unroll 1
   for (; t + 3 < c.s_hi; t += 128) f4(t);
+#pragma unroll 1
   for (int e = t; e < c.s_hi && e < t + 4; ++e) f1(e);
-}
-__device__ __forceinline__ float fast_ex2(float x) {  // 2^x, relative error 2^-22; 2^-inf = 0
-  float y;
-  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
-  return y;
 }
 
 __device__ __forceinline__ double sum_lanes(double v, int width) {  // butterfly over `width` lanes
@@ -216,6 +218,24 @@ __device__ __forceinline__ void prefetch_slice_l2(const Ctx& c, const float* row
 }
 __device__ __forceinline__ bool node_has_child(const Ctx& c, int v) { return (c.sh->has_child[v >> 5] >> (v & 31)) & 1u; }
 
+// Rare path of the maximum sweep: this warp's segment holds a NaN or +inf logit (or mixes -inf and a huge
+// value in one group of four).  Every element is checked, offenders are flagged and replaced in place, and the
+// segment maxima are taken again.
+__device__ __noinline__ void sanitize_segment(Ctx& c, bool need_draft, int32_t* dev_status, float& mp, float& mq) {
+  mp = -INFINITY; mq = -INFINITY;
+  for (int t = c.s_lo + c.lane; t < c.s_hi; t += 32) {
+    float x = c.ps[t];
+    if (!(x < INFINITY)) { x = sanitize_logit(x, dev_status); c.ps[t] = x; }
+    mp = fmaxf(mp, x);
+    if (need_draft) {
+      float y = c.qs[t];
+      if (!(y < INFINITY)) { y = sanitize_logit(y, dev_status); c.qs[t] = y; }
+      mq = fmaxf(mq, y);
+    }
+  }
+  __syncwarp();
+}
+
 // Runs Algorithm 2's loop at node v.  Returns the accepted child's node id or -1 and leaves in
 // `st` (and in ps/qs/wseg) the state the final draw needs.
 __device__ int process_node(cg::cluster_group& cluster, Ctx& c, const VerifyArgs& a, int v, NodeState& st,
@@ -236,9 +256,11 @@ __device__ int process_node(cg::cluster_group& cluster, Ctx& c, const VerifyArgs
   TRACE(1);
   const int k = build_kids(c, v, a.n);  // overlaps the copies
   // duplicates among siblings, and L2 prefetch of the first children's rows
+#pragma unroll 1
   for (int i = c.tid; i < k; i += kVThreads) {
     const int s = c.sh->tokens[c.sh->kids[i]];
     int d = 0;
+#pragma unroll 1
     for (int j = 0; j < i; ++j) d |= c.sh->tokens[c.sh->kids[j]] == s;
     c.sh->dup[i] = (uint8_t)d;
     if (i < kPrefetchChildren) {
@@ -291,33 +313,30 @@ __device__ int process_node(cg::cluster_group& cluster, Ctx& c, const VerifyArgs
   }
 
   const float c2 = st.c2;
-  // segment maxima; a NaN or +inf logit is flagged and replaced in place (rare path)
+  // segment maxima; a NaN or +inf logit is flagged and replaced in place (rare path, out of line).  A sum of
+  // four elements is NaN or +inf exactly when one of them is NaN or +inf or they mix -inf with +inf, so one
+  // comparison per float4 finds the rows that need the slow path.
   float mp = -INFINITY, mq = -INFINITY;
   {
-    auto fix = [&](float* p) { *p = sanitize_logit(*p, a.dev_status); return *p; };
+    bool bad = false;
     auto f1 = [&](int t) {
-      float x = c.ps[t];
-      if (!(x < INFINITY)) x = fix(c.ps + t);
+      const float x = c.ps[t];
+      bad |= !(x < INFINITY);
       mp = fmaxf(mp, x);
-      if (need_draft) {
-        float y = c.qs[t];
-        if (!(y < INFINITY)) y = fix(c.qs + t);
-        mq = fmaxf(mq, y);
-      }
+      if (need_draft) { const float y = c.qs[t]; bad |= !(y < INFINITY); mq = fmaxf(mq, y); }
     };
     auto f4 = [&](int t) {
       const float4 x = *reinterpret_cast<const float4*>(c.ps + t);
-      const float m4 = fmaxf(fmaxf(x.x, x.y), fmaxf(x.z, x.w));
-      if (m4 < INFINITY && x.x == x.x && x.y == x.y && x.z == x.z && x.w == x.w) mp = fmaxf(mp, m4);
-      else { f1(t); f1(t + 1); f1(t + 2); f1(t + 3); return; }
+      bad |= !((x.x + x.y) + (x.z + x.w) < INFINITY);
+      mp = fmaxf(mp, fmaxf(fmaxf(x.x, x.y), fmaxf(x.z, x.w)));
       if (need_draft) {
         const float4 y = *reinterpret_cast<const float4*>(c.qs + t);
-        const float n4 = fmaxf(fmaxf(y.x, y.y), fmaxf(y.z, y.w));
-        if (n4 < INFINITY && y.x == y.x && y.y == y.y && y.z == y.z && y.w == y.w) mq = fmaxf(mq, n4);
-        else { f1(t); f1(t + 1); f1(t + 2); f1(t + 3); }
+        bad |= !((y.x + y.y) + (y.z + y.w) < INFINITY);
+        mq = fmaxf(mq, fmaxf(fmaxf(y.x, y.y), fmaxf(y.z, y.w)));
       }
     };
     sweep(c, f4, f1);
+    if (__any_sync(0xffffffffu, bad)) sanitize_segment(c, need_draft, a.dev_status, mp, mq);
   }
   mp = warp_max(mp);
   mq = warp_max(mq);
