@@ -590,11 +590,20 @@ tree_attention_umma_kernel(const __grid_constant__ CUtensorMap q_map, const __gr
   float m_used = -INFINITY, l = 0.f;
   bool ok = true;
   const int n_mine = nblk > chain ? (nblk - chain + 1) >> 1 : 0;  // blocks of this chain
+  // A warp whose 32 rows all lie past the tile's last node (small trees fill only part of a 128-row tile) leaves
+  // the special-function unit and the issue slots to the warps with real rows; its P rows stay whatever they are
+  // (rows of the product are independent).
+  const bool warp_live = i0 + (quad * 32) / a.group < a.n;
   for (int u = 0; u < n_mine && ok; ++u) {
     const int jj = 2 * u + chain, b = (base + u) & 1, w = (base + u) >> 1;
     const uint32_t tmem_s = tmem + 128u * chain + 64u * b + lane_sel;
     if (!mbar_wait(sm, &sm->s_full[chain][b], w & 1, a.dev_status)) { ok = false; break; }
     if (threadIdx.x == 128) UTRACE(2, 1);
+    if (!warp_live) {  // 32 padding rows: nothing to compute, only keep in step with the barriers
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&sm->p_full[chain][b]);
+      continue;
+    }
     tc_fence_after();
     uint32_t sreg[64];
     tmem_ld32(tmem_s, sreg, 0);
@@ -826,10 +835,12 @@ tree_attention_umma_kernel(const __grid_constant__ CUtensorMap q_map, const __gr
     tc_fence_before();
     cluster.sync();  // every CTA of the cluster is done with its K stages before anyone writes into them
     if (threadIdx.x == 128) UTRACE(2, 7);
-    if (chain == 0)
+    // (rows past the tile's last node are padding: nothing of theirs is pushed, reduced or stored)
+    if (chain == 0 && row_valid)
       for (int q = 0; q < cs; ++q) *cluster.map_shared_rank(&sm->ml_cta[split][r], q) = make_float2(M, Lc);
 #pragma unroll
     for (int j = 0; j < 8; ++j) {
+      if (!row_valid) break;
       const int s_idx = 8 * chain + j;
       uint4* dst = cluster.map_shared_rank(reinterpret_cast<uint4*>(&sm->k[0][0][0]), s_idx % cs) +
                    ((size_t)(split * slots + s_idx / cs) * 2) * kTileM + r;
@@ -849,7 +860,7 @@ tree_attention_umma_kernel(const __grid_constant__ CUtensorMap q_map, const __gr
     }
     const float inv = 1.f / Ls;  // some CTA saw the row's own key, so Ls > 0
     const float4* mine = reinterpret_cast<const float4*>(&sm->k[0][0][0]);
-    for (int slot = chain; slot < slots; slot += 2) {  // the two warp groups share this CTA's slots
+    for (int slot = chain; slot < slots && row_valid; slot += 2) {  // the two warp groups share this CTA's slots
       float acc[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
       for (int q = 0; q < cs; ++q) {
         const float mq = sm->ml_cta[q][r].x;
