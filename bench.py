@@ -38,7 +38,7 @@ L2_BYTES = 126 * 1024 * 1024
 # the ncu captures summarised under profiles/; None where no capture exists for that workload.
 NCU_TRAFFIC_BYTES = {
     "llama2-7b": 18418432,    # profiles/tree_attention_umma_llama2-7b.md
-    "llama3-70b": 32832000,   # profiles/tree_attention_umma_llama3-70b.md
+    "llama3-70b": 32801792,   # profiles/tree_attention_umma_llama3-70b.md
 }
 
 
