@@ -212,7 +212,15 @@ int seq_tree_attention_noalloc(const seq_tree_attention_params* p, void* stream)
  *                       every node is processed and gets its own decision.
  * workspace may be NULL when seq_tree_verify_workspace_bytes() returns 0.
  */
-enum { SEQ_VERIFY_ALL_NODES = 1 };
+enum {
+  SEQ_VERIFY_ALL_NODES = 1,
+  /* Algorithm 2 without its lines 10-16 (the lines the paper prints in blue): the draft distribution D
+   * is left as it is after a rejection -- the rejected token is neither removed from it nor is it
+   * renormalised -- which is SpecInfer's multi-round rejection sampling, the baseline the paper compares
+   * its verification with (Section 3.2.2, Algorithm 2's caption; Theorem 3.7's counter-example).  The
+   * children of a node are then draws WITH replacement from the draft row and may repeat. */
+  SEQ_VERIFY_SPECINFER = 2
+};
 
 typedef struct {
   int32_t n_tree, vocab;
@@ -232,7 +240,7 @@ typedef struct {
   void* workspace;
   size_t workspace_bytes;
   int32_t* dev_status;
-  int32_t flags; /* 0 or SEQ_VERIFY_ALL_NODES */
+  int32_t flags; /* 0 or an OR of SEQ_VERIFY_ALL_NODES, SEQ_VERIFY_SPECINFER */
 } seq_tree_verify_params;
 
 size_t seq_tree_verify_workspace_bytes(const seq_tree_verify_params* p);

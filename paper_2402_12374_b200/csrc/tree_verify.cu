@@ -241,6 +241,7 @@ __device__ __noinline__ void sanitize_segment(Ctx& c, bool need_draft, int32_t* 
 __device__ int process_node(cg::cluster_group& cluster, Ctx& c, const VerifyArgs& a, int v, NodeState& st,
                             bool skip_leaves, bool copies_started) {
   const bool greedy = a.temperature == 0.f;
+  const bool specinfer = (a.flags & SEQ_VERIFY_SPECINFER) != 0;  // D is never touched: ZD stays 1, S stays empty
   const bool has_kids = node_has_child(c, v);
   if (skip_leaves && !has_kids) return -1;
   const bool need_draft = !greedy && (has_kids || (copies_started && a.n > 1));
@@ -403,7 +404,9 @@ __device__ int process_node(cg::cluster_group& cluster, Ctx& c, const VerifyArgs
     const int ch = c.sh->kids[i];
     const int s = c.sh->tokens[ch];
     if (s < 0 || s >= a.V) { dev_flag(a.dev_status, SEQ_DEV_BAD_TOKEN); continue; }
-    const bool in_S = c.sh->dup[i] != 0;  // an earlier (hence rejected) sibling carried the same token
+    // an earlier (hence rejected) sibling carried the same token: it is in S.  (Without lines 10-16 there is no
+    // S: a repeated token is tested like any other, and its R is 0 by then.)
+    const bool in_S = !specinfer && c.sh->dup[i] != 0;
     float pn = 0.f, qn = 0.f;
     if (!in_S) {
       const float4 pq = kid_pq[i];
@@ -423,7 +426,7 @@ __device__ int process_node(cg::cluster_group& cluster, Ctx& c, const VerifyArgs
     if (st.mode == 0) Cn += st.Z / st.ZD;
     else if (a.V - st.nS > 0) Un += st.Z / (double)(a.V - st.nS);
     // lines 10-11: D[s] <- 0, S.add(s); done by the warp that owns s
-    if (!in_S) {
+    if (!in_S && !specinfer) {
       const int sl = s - c.lo;
       if (sl >= c.s_lo && sl < c.s_hi && c.lane == 0) { c.ps[sl] = 0.f; c.qs[sl] = 0.f; }
       st.nS += 1;
@@ -459,8 +462,10 @@ __device__ int process_node(cg::cluster_group& cluster, Ctx& c, const VerifyArgs
     } else {
       dev_flag(a.dev_status, SEQ_DEV_DEGENERATE);  // keep R
     }
-    st.ZD = ZDn;
-    if (st.mode == 0 && !(ZDn > 0.0)) st.mode = 1;  // lines 12-15: uniform over the non-rejected set
+    if (!specinfer) {
+      st.ZD = ZDn;
+      if (st.mode == 0 && !(ZDn > 0.0)) st.mode = 1;  // lines 12-15: uniform over the non-rejected set
+    }
   }
   return -1;
 }
@@ -633,7 +638,7 @@ static int verify_validate(const seq_tree_verify_params* p) {
   if (p->n_tree < 1 || p->n_tree > SEQ_MAX_TREE || p->vocab < 1) return SEQ_ERR_INVALID_ARG;
   if (p->parent == nullptr || p->tokens == nullptr || p->target_logits == nullptr) return SEQ_ERR_INVALID_ARG;
   if (!(p->temperature >= 0.f) || isinf(p->temperature)) return SEQ_ERR_INVALID_ARG;
-  if (p->flags & ~SEQ_VERIFY_ALL_NODES) return SEQ_ERR_INVALID_ARG;
+  if (p->flags & ~(SEQ_VERIFY_ALL_NODES | SEQ_VERIFY_SPECINFER)) return SEQ_ERR_INVALID_ARG;
   const bool all_nodes = p->flags & SEQ_VERIFY_ALL_NODES;
   if (all_nodes) {
     if (p->next_child_out == nullptr) return SEQ_ERR_INVALID_ARG;

@@ -71,7 +71,7 @@ def _path(parent, i):
     return out
 
 
-def run_verify(vi: W.VerifyInputs, all_nodes=False, want_residual=True):
+def run_verify(vi: W.VerifyInputs, all_nodes=False, want_residual=True, specinfer=False):
     d = dev()
     n, V = vi.target_logits.shape
     st = torch.zeros(1, dtype=torch.int32, device=d)
@@ -84,7 +84,7 @@ def run_verify(vi: W.VerifyInputs, all_nodes=False, want_residual=True):
     tl[:, :V], dl[:, :V] = vi.target_logits.to(d), vi.draft_logits.to(d)
     call = B.VerifyCall(vi.parent.to(d), vi.tokens.to(d), tl[:, :V], dl[:, :V],
                         vi.temperature, vi.uniforms.to(d), residual_out=residual, next_child_out=nxt,
-                        all_nodes=all_nodes, dev_status=st)
+                        all_nodes=all_nodes, dev_status=st, specinfer=specinfer)
     call.run()
     torch.cuda.synchronize()
     plen = int(call.path_len.item())
@@ -93,11 +93,12 @@ def run_verify(vi: W.VerifyInputs, all_nodes=False, want_residual=True):
                 next_child=nxt.cpu().numpy(), status=int(st.item()))
 
 
-def check_verify(vi: W.VerifyInputs):
+def check_verify(vi: W.VerifyInputs, specinfer=False):
     """Path and bonus identical to the oracle's (outside the rounding band), residual within 1e-5.
     Returns 'ok' or 'excluded'."""
-    got = run_verify(vi)
-    ref = O.tree_verify(vi.parent, vi.tokens, vi.target_logits, vi.draft_logits, vi.temperature, vi.uniforms)
+    got = run_verify(vi, specinfer=specinfer)
+    ref = O.tree_verify(vi.parent, vi.tokens, vi.target_logits, vi.draft_logits, vi.temperature, vi.uniforms,
+                        variant=O.VARIANT_SPECINFER if specinfer else O.VARIANT_SEQUOIA)
     assert got["status"] == ref["flags"] == 0
     if ref["min_gap"] < GAP:
         return "excluded"

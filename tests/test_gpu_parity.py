@@ -198,6 +198,43 @@ def test_verify_uniform_fallback_duplicates_and_bad_tokens():
     assert np.abs(got["residual"] - ref["residual"]).max() < 1e-5
 
 
+@pytest.mark.parametrize("name,T,seeds", [("tiny", 0.6, range(8)), ("llama2-7b", 0.6, range(4)), ("llama2-7b", 1.0, range(3)),
+                                          ("llama2-13b", 1.0, range(2))])
+def test_verify_specinfer_variant_configs(name, T, seeds):
+    """SEQ_VERIFY_SPECINFER: Algorithm 2 without lines 10-16 (D untouched after a rejection), against the
+    oracle's walk of the same variant."""
+    cfg = W.CONFIGS[name]
+    outcomes = [G.check_verify(W.make_verify_inputs(cfg, T, seed), specinfer=True) for seed in seeds]
+    assert outcomes.count("ok") >= max(1, len(outcomes) - 1), outcomes
+
+
+def test_verify_specinfer_children_with_replacement_and_many_rejections():
+    """Children drawn WITH replacement (repeated sibling tokens), large uniforms so that most tests
+    reject: every repeated token is tested again (ratio 0 by then) and costs one more residual round."""
+    rng = np.random.default_rng(3)
+    V, n = 96, 14
+    parent = W.star_tree(n)
+    checked = 0
+    for trial in range(25):
+        tl = (2 * rng.standard_normal((n, V))).astype(np.float32)
+        dl = (tl + 1.5 * rng.standard_normal((n, V))).astype(np.float32)
+        q = np.exp((dl[0] - dl[0].max()) / 0.8)
+        tokens = np.zeros(n, np.int32)
+        tokens[1:] = rng.choice(V, n - 1, replace=True, p=q / q.sum())  # repeats are likely with 13 draws
+        if trial == 0:
+            tokens[2] = tokens[1]
+        u = (0.85 + 0.15 * rng.random(n + 1)).astype(np.float32)
+        u[-1] = rng.random()
+        vi = W.VerifyInputs(torch.from_numpy(parent), torch.from_numpy(tokens), torch.from_numpy(tl),
+                            torch.from_numpy(dl), torch.from_numpy(u), 0.8)
+        checked += G.check_verify(vi, specinfer=True) == "ok"
+        # the two variants are different algorithms: on these inputs they must not be interchangeable
+    assert checked >= 20
+    ref_a = O.tree_verify(parent, tokens, tl, dl, 0.8, u, variant=O.VARIANT_SEQUOIA)
+    ref_b = O.tree_verify(parent, tokens, tl, dl, 0.8, u, variant=O.VARIANT_SPECINFER)
+    assert np.abs(ref_a["residual"] - ref_b["residual"]).max() > 1e-4 or ref_a["path"].tolist() != ref_b["path"].tolist()
+
+
 def test_verify_nonfinite_logits_are_flagged_not_trapped():
     vi = W.make_verify_inputs(W.CONFIGS["tiny"], 0.6, 0, vocab=512)
     vi.target_logits[0, 5] = float("nan")
