@@ -59,6 +59,7 @@ def lib():
         L.orc_softmax_T.argtypes = [pf32, i32, f64, pf64]
         L.orc_softmax_T.restype = None
         L.orc_alg2_node.argtypes = [pf64, pf64, i32, pi32, pf64, i32, i32, pi32, pf64, pf64, pf64, pf64]
+        L.orc_draft_sample.argtypes = [pf32, i32, f64, pf32, i32, pi32, pf64, pf64]
         L.orc_sample_inverse_cdf.argtypes = [pf64, i32, f64]
         L.orc_sample_inverse_cdf.restype = i32
         L.orc_tree_verify.argtypes = [i32, i32, pi32, pi32, pf32, i64, pf32, i64, f64, pf32, i32,
@@ -123,6 +124,19 @@ def softmax_T(logits, T: float) -> np.ndarray:
     out = np.empty(logits.shape[0], dtype=np.float64)
     lib().orc_softmax_T(_p(logits, C.c_float), logits.shape[0], float(T), _p(out, C.c_double))
     return out
+
+
+def draft_sample(logits, T: float, u, k: int) -> dict:
+    """k tokens drawn without replacement from softmax(logits/T) by exponential sort with the uniforms u."""
+    logits, u = _f32(logits), _f32(u)
+    V = logits.shape[0]
+    assert u.shape[0] == V and k >= 0
+    out = np.full(max(k, 1), -1, dtype=np.int32)
+    keys = np.empty(V, dtype=np.float64)
+    gap = C.c_double(0.0)
+    lib().orc_draft_sample(_p(logits, C.c_float), V, float(T), _p(u, C.c_float), k, _p(out, C.c_int32),
+                           _p(keys, C.c_double), C.byref(gap))
+    return dict(tokens=out[:k].copy(), keys=keys, min_rel_gap=float(gap.value))
 
 
 def alg2_node(P, Q, child_tok, child_u, variant: int = VARIANT_SEQUOIA) -> dict:

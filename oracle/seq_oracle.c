@@ -10,7 +10,9 @@
  *     the committed prefix and its own root-to-node path (Section 1: the
  *     whole tree is verified by one forward pass of the target model);
  *   - Algorithm 2 ("Sequoia Sampling and Verification") applied recursively
- *     from the root (Section 2.2), ending with the draw x ~ R.
+ *     from the root (Section 2.2), ending with the draw x ~ R;
+ *   - the draft side's draw of a node's children without replacement by
+ *     exponential sort (Section 5, "Implementation Details").
  *
  * Nothing here is blocked, fused or reordered: every function is the
  * definition, or the algorithm's steps in the paper's order and notation, so
@@ -24,7 +26,9 @@
  * transport closed form 1-|P-Q|_1/2 at k=1, the cover property, the lemma
  * P(reject at i) = sum max(0, t_i - d_i), reduction of a chain to Algorithm 3,
  * Monte-Carlo; attention against library causal attention (chain tree),
- * single-query decode (star tree) and explicit-sequence brute force.
+ * single-query decode (star tree) and explicit-sequence brute force; the
+ * exponential sort against the exact without-replacement law of ordered pairs
+ * (Monte-Carlo), library sorts in its two degenerate cases, and invariants.
  *
  * Build: gcc -O2 -fopenmp -shared -fPIC seq_oracle.c -o liboracle.so -lm
  */
@@ -159,6 +163,64 @@ void orc_softmax_T(const float* logits, int32_t V, double T, double* out) {
     z += out[t];
   }
   for (int32_t t = 0; t < V; ++t) out[t] /= z;
+}
+
+/*
+ * Draft-side sampling without replacement by exponential sort (Section 5,
+ * "Implementation Details": sampling without replacement is done with "the
+ * exponential-sort algorithm"; this is the draw s_i ~ D of Algorithm 2's line 5
+ * for all k children of a node at once).
+ *
+ * Every token t gets an exponential variate E_t = -log(u_t) (u_t uniform on
+ * (0,1), supplied by the caller) and the key E_t / q_t with q = softmax(logits/T).
+ * The tokens in ascending key order are a sample without replacement from q in
+ * draw order: the smallest key is a draw from q, the next one a draw from q
+ * renormalised without the first, and so on.  The first k are returned.
+ *
+ *   logits [V], u [V] (anything outside (0,1) gives that token no chance).
+ *   out [k]: the drawn tokens in draw order; -1 once no token with q_t > 0 is left.
+ *   keys_out (nullable, [V]): the keys (INFINITY where q_t = 0 or u_t is unusable).
+ *   min_rel_gap (nullable): over the k+1 smallest keys in order, the smallest
+ *       relative difference (b - a) / b between neighbours: how much room a
+ *       lower-precision computation of the keys has before the order changes.
+ * Equal keys are taken in token order.  Returns 0.
+ */
+int orc_draft_sample(const float* logits, int32_t V, double T, const float* u, int32_t k,
+                     int32_t* out, double* keys_out, double* min_rel_gap) {
+  double* q = (double*)malloc(sizeof(double) * (size_t)V);
+  double* key = (double*)malloc(sizeof(double) * (size_t)V);
+  unsigned char* taken = (unsigned char*)calloc((size_t)V, 1);
+  orc_softmax_T(logits, V, T, q);
+  for (int32_t t = 0; t < V; ++t) {
+    double ut = (double)u[t];
+    if (q[t] > 0.0 && ut > 0.0 && ut < 1.0)
+      key[t] = -log(ut) / q[t];
+    else
+      key[t] = INFINITY;
+    if (keys_out) keys_out[t] = key[t];
+  }
+  if (min_rel_gap) *min_rel_gap = INFINITY;
+  double prev = -1.0;
+  for (int32_t i = 0; i <= k; ++i) { /* one more than k, for the gap behind the last draw */
+    int32_t best = -1;
+    for (int32_t t = 0; t < V; ++t)
+      if (!taken[t] && key[t] < INFINITY && (best < 0 || key[t] < key[best])) best = t;
+    if (i < k) out[i] = best;
+    if (best < 0) {
+      for (int32_t j = i + 1; j < k; ++j) out[j] = -1;
+      break;
+    }
+    taken[best] = 1;
+    if (min_rel_gap && prev >= 0.0 && key[best] > 0.0) {
+      double g = (key[best] - prev) / key[best];
+      if (g < *min_rel_gap) *min_rel_gap = g;
+    }
+    prev = key[best];
+  }
+  free(q);
+  free(key);
+  free(taken);
+  return 0;
 }
 
 /*
