@@ -247,6 +247,43 @@ size_t seq_tree_verify_workspace_bytes(const seq_tree_verify_params* p);
 int seq_tree_verify(const seq_tree_verify_params* p, void* stream);
 
 /* Library build string ("seqtree <version> sm_100a"); static storage. */
+/*
+ * seq_tree_draft_sample -- the draft side's draw of the children of tree nodes: k tokens without
+ * replacement from softmax(draft_logits / temperature), for n_rows nodes at once (Algorithm 2, line 5,
+ * "s_i ~ D", for all children of a node; Section 5, "Implementation Details": sampling without replacement
+ * is done with the exponential-sort algorithm).  A step before the verify path: its output is the tokens[]
+ * of seq_tree_verify's children, in sibling order.
+ *
+ * Token t of a row gets the key E_t / q_t with E_t = -log(u_t) an exponential variate and q the row's
+ * softmax; the tokens in ascending key order are a sample without replacement in draw order, and the
+ * first k are returned.  Equal keys are taken in token order.
+ *
+ *   draft_logits   fp32, row r at r*logits_row_stride (elements), device.  -inf entries are legal
+ *                  (probability 0); a NaN or +inf entry raises SEQ_DEV_NONFINITE and is never drawn.
+ *   uniforms       fp32 [n_rows][vocab], row r at r*uniforms_row_stride, device: one uniform per (row,
+ *                  token); a value outside (0,1) gives its token no chance.  Caller-supplied, so that a
+ *                  draw can be repeated and checked.
+ *   temperature    > 0, finite.
+ *   k              1..64 draws per row.
+ *   tokens_out     int32 [n_rows][k], device: the drawn tokens in draw order, -1 where no token with
+ *                  positive probability was left.
+ *   dev_status     nullable.
+ * The decision is taken in fp32 (on the logarithm of the inverse key): two keys closer than fp32 resolves
+ * may come out in either order.  No workspace.  Returns SEQ_OK or SEQ_ERR_INVALID_ARG.
+ */
+typedef struct {
+  int32_t n_rows, vocab, k;
+  const float* draft_logits;
+  int64_t logits_row_stride;
+  const float* uniforms;
+  int64_t uniforms_row_stride;
+  float temperature;
+  int32_t* tokens_out;
+  int32_t* dev_status;
+} seq_tree_draft_sample_params;
+
+int seq_tree_draft_sample(const seq_tree_draft_sample_params* p, void* stream);
+
 const char* seq_tree_version(void);
 
 #ifdef __cplusplus

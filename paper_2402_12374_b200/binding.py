@@ -34,6 +34,7 @@ EXPORTED_SYMBOLS = (
     "seq_tree_attention_noalloc",
     "seq_tree_verify_workspace_bytes",
     "seq_tree_verify",
+    "seq_tree_draft_sample",
     "seq_tree_version",
 )
 
@@ -94,6 +95,8 @@ def load() -> C.CDLL:
         lib.seq_tree_attention.restype = C.c_int
         lib.seq_tree_attention_noalloc.argtypes = [C.POINTER(AttentionParams), C.c_void_p]
         lib.seq_tree_attention_noalloc.restype = C.c_int
+        lib.seq_tree_draft_sample.argtypes = [C.POINTER(DraftSampleParams), C.c_void_p]
+        lib.seq_tree_draft_sample.restype = C.c_int
         lib.seq_tree_verify_workspace_bytes.argtypes = [C.POINTER(VerifyParams)]
         lib.seq_tree_verify_workspace_bytes.restype = C.c_size_t
         lib.seq_tree_verify.argtypes = [C.POINTER(VerifyParams), C.c_void_p]
@@ -142,6 +145,35 @@ def seq_tree_mask_from_parents(parent: torch.Tensor, *, words_per_row: int | Non
                                            _stream(stream))
     _check("seq_tree_mask_from_parents", rc)
     return mask_bits, depth
+
+
+class DraftSampleParams(C.Structure):
+    _fields_ = [
+        ("n_rows", C.c_int32), ("vocab", C.c_int32), ("k", C.c_int32),
+        ("draft_logits", C.c_void_p), ("logits_row_stride", C.c_int64),
+        ("uniforms", C.c_void_p), ("uniforms_row_stride", C.c_int64),
+        ("temperature", C.c_float), ("tokens_out", C.c_void_p), ("dev_status", C.c_void_p),
+    ]
+
+
+def seq_tree_draft_sample(draft_logits, temperature: float, uniforms, k: int, *, tokens_out=None, dev_status=None,
+                          stream=None):
+    """k tokens per row drawn without replacement from softmax(draft_logits / temperature) by exponential
+    sort with the supplied uniforms; returns int32 [rows, k] (device), -1 where nothing was left to draw."""
+    rows, V = draft_logits.shape
+    if uniforms.shape != draft_logits.shape or draft_logits.stride(1) != 1 or uniforms.stride(1) != 1:
+        raise ValueError("draft_logits and uniforms must be [rows, vocab] with contiguous rows")
+    if tokens_out is None:
+        tokens_out = torch.empty((rows, k), dtype=torch.int32, device=draft_logits.device)
+    p = DraftSampleParams()
+    p.n_rows, p.vocab, p.k = rows, V, k
+    p.draft_logits, p.logits_row_stride = _dev(draft_logits, "draft_logits", torch.float32), draft_logits.stride(0)
+    p.uniforms, p.uniforms_row_stride = _dev(uniforms, "uniforms", torch.float32), uniforms.stride(0)
+    p.temperature = temperature
+    p.tokens_out = _dev(tokens_out, "tokens_out", torch.int32)
+    p.dev_status = _dev(dev_status, "dev_status", torch.int32)
+    _check("seq_tree_draft_sample", load().seq_tree_draft_sample(C.byref(p), _stream(stream)))
+    return tokens_out
 
 
 class AttentionCall:
