@@ -268,8 +268,12 @@ int seq_tree_verify(const seq_tree_verify_params* p, void* stream);
  *   tokens_out     int32 [n_rows][k], device: the drawn tokens in draw order, -1 where no token with
  *                  positive probability was left.
  *   dev_status     nullable.
+ *   workspace      seq_tree_draft_sample_workspace_bytes(p) bytes, 8-byte aligned, device, contents
+ *                  undefined before and after: the k best (score, token) pairs of every 4096-token chunk
+ *                  of every row (two launches: per-chunk draws, then the row's draws among them).
  * The decision is taken in fp32 (on the logarithm of the inverse key): two keys closer than fp32 resolves
- * may come out in either order.  No workspace.  Returns SEQ_OK or SEQ_ERR_INVALID_ARG.
+ * may come out in either order.  Returns SEQ_OK, SEQ_ERR_INVALID_ARG, SEQ_ERR_WORKSPACE, or
+ * SEQ_ERR_UNSUPPORTED (vocab/4096 * k above 25600).
  */
 typedef struct {
   int32_t n_rows, vocab, k;
@@ -280,8 +284,11 @@ typedef struct {
   float temperature;
   int32_t* tokens_out;
   int32_t* dev_status;
+  void* workspace;
+  size_t workspace_bytes;
 } seq_tree_draft_sample_params;
 
+size_t seq_tree_draft_sample_workspace_bytes(const seq_tree_draft_sample_params* p);
 int seq_tree_draft_sample(const seq_tree_draft_sample_params* p, void* stream);
 
 const char* seq_tree_version(void);

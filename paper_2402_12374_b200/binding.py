@@ -34,6 +34,7 @@ EXPORTED_SYMBOLS = (
     "seq_tree_attention_noalloc",
     "seq_tree_verify_workspace_bytes",
     "seq_tree_verify",
+    "seq_tree_draft_sample_workspace_bytes",
     "seq_tree_draft_sample",
     "seq_tree_version",
 )
@@ -95,6 +96,8 @@ def load() -> C.CDLL:
         lib.seq_tree_attention.restype = C.c_int
         lib.seq_tree_attention_noalloc.argtypes = [C.POINTER(AttentionParams), C.c_void_p]
         lib.seq_tree_attention_noalloc.restype = C.c_int
+        lib.seq_tree_draft_sample_workspace_bytes.argtypes = [C.POINTER(DraftSampleParams)]
+        lib.seq_tree_draft_sample_workspace_bytes.restype = C.c_size_t
         lib.seq_tree_draft_sample.argtypes = [C.POINTER(DraftSampleParams), C.c_void_p]
         lib.seq_tree_draft_sample.restype = C.c_int
         lib.seq_tree_verify_workspace_bytes.argtypes = [C.POINTER(VerifyParams)]
@@ -153,11 +156,12 @@ class DraftSampleParams(C.Structure):
         ("draft_logits", C.c_void_p), ("logits_row_stride", C.c_int64),
         ("uniforms", C.c_void_p), ("uniforms_row_stride", C.c_int64),
         ("temperature", C.c_float), ("tokens_out", C.c_void_p), ("dev_status", C.c_void_p),
+        ("workspace", C.c_void_p), ("workspace_bytes", C.c_size_t),
     ]
 
 
 def seq_tree_draft_sample(draft_logits, temperature: float, uniforms, k: int, *, tokens_out=None, dev_status=None,
-                          stream=None):
+                          workspace=None, stream=None):
     """k tokens per row drawn without replacement from softmax(draft_logits / temperature) by exponential
     sort with the supplied uniforms; returns int32 [rows, k] (device), -1 where nothing was left to draw."""
     rows, V = draft_logits.shape
@@ -172,6 +176,11 @@ def seq_tree_draft_sample(draft_logits, temperature: float, uniforms, k: int, *,
     p.temperature = temperature
     p.tokens_out = _dev(tokens_out, "tokens_out", torch.int32)
     p.dev_status = _dev(dev_status, "dev_status", torch.int32)
+    need = load().seq_tree_draft_sample_workspace_bytes(C.byref(p))
+    if workspace is None and need:
+        workspace = torch.empty(need, dtype=torch.uint8, device=draft_logits.device)
+    p.workspace = _dev(workspace, "workspace") if workspace is not None else None
+    p.workspace_bytes = workspace.numel() * workspace.element_size() if workspace is not None else 0
     _check("seq_tree_draft_sample", load().seq_tree_draft_sample(C.byref(p), _stream(stream)))
     return tokens_out
 
