@@ -188,6 +188,49 @@ def run_reference(args, cfg, T):
     print(json.dumps(line), flush=True)
 
 
+def draft_sample_leg(cfg, parent, ver_h, T, dev, stream, peaks) -> dict:
+    """Not part of the timed step: the draft side's draw of every internal node's children (exponential sort),
+    timed on its own in a CUDA graph over rotating logit sets.  One row per internal node, k = the tree's
+    largest fan-out, uniforms of the same shape as the logits (seeded on the device)."""
+    from paper_2402_12374_b200 import binding as B
+
+    kids = W.children_lists(parent)
+    internal = [v for v in range(len(parent)) if kids[v]]
+    k = min(64, max(len(kids[v]) for v in internal))
+    rows = torch.tensor(internal, dtype=torch.long, device=dev)
+    gen = torch.Generator(device=dev)
+    gen.manual_seed(20240212)
+    logit_sets = [vi.draft_logits.to(dev)[rows].contiguous() for vi in ver_h[:4]]
+    unif_sets = [torch.rand(ls.shape, device=dev, generator=gen).clamp_(1e-7, 1 - 1e-7) for ls in logit_sets]
+    out = torch.empty((len(internal), k), dtype=torch.int32, device=dev)
+    ws = torch.empty(len(internal) * ((cfg.vocab + 4095) // 4096) * k * 8 + 256, dtype=torch.uint8, device=dev)
+    reps = 40
+    with torch.cuda.stream(stream):
+        for i in range(3):
+            B.seq_tree_draft_sample(logit_sets[i % len(logit_sets)], T, unif_sets[i % len(logit_sets)], k, tokens_out=out,
+                                    workspace=ws, stream=stream)
+        stream.synchronize()
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g, stream=stream):
+            for i in range(reps):
+                B.seq_tree_draft_sample(logit_sets[i % len(logit_sets)], T, unif_sets[i % len(logit_sets)], k, tokens_out=out,
+                                        workspace=ws, stream=stream)
+        g.replay()
+        stream.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        g.replay()
+        e1.record(stream)
+        stream.synchronize()
+    us = e0.elapsed_time(e1) * 1e3 / reps
+    nbytes = 2 * len(internal) * cfg.vocab * 4
+    gbs = nbytes / (us * 1e-6) / 1e9
+    return {"us_per_call": us, "rows": len(internal), "k": k, "vocab": cfg.vocab, "gpu_launches_per_call": 2,
+            "roofline": {"bound": "hbm", "achieved": gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                         "frac": gbs / peaks["hbm_gbs"], "algorithmic_bytes": nbytes, "traffic": None},
+            "note": "logits + uniforms of every internal node read once; outside the timed step"}
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -391,6 +434,8 @@ def main():
         "breakdown_us": {"attention": attn_us, "verify": ver_us,
                          "largest_share": "seq_tree_verify" if ver_us > attn_us else "seq_tree_attention"},
     }
+    if T > 0:
+        line["next_rows"] = {"draft_sample": draft_sample_leg(cfg, parent, ver_h, T, dev, stream, peaks)}
     if not args.no_cpu_baseline:
         from oracle import oracle as O
 
