@@ -72,23 +72,24 @@ __device__ __forceinline__ void ds_warp_argmax(float& s, int& i) {
   b = m ^ ((m >> 31) & 0x7fffffff);
   s = __int_as_float(b);
 }
-// Block-wide arg-max.  Result in every thread.
-__device__ __forceinline__ void ds_block_argmax(float& s, int& i, float* w_s, int* w_i) {
-  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+// Block-wide arg-max.  Result in every thread.  The per-warp results go through one of two shared buffers,
+// alternating from call to call (`round`), so that one barrier per call is enough: a thread can be at most one
+// call ahead of the slowest reader, which then still reads the other buffer.
+__device__ __forceinline__ void ds_block_argmax(float& s, int& i, float (*w_s)[kDsWarps], int (*w_i)[kDsWarps], int round) {
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, buf = round & 1;
   ds_warp_argmax(s, i);
-  __syncthreads();  // the previous round's readers are done with w_s / w_i
-  if (lane == 0) { w_s[warp] = s; w_i[warp] = i; }
+  if (lane == 0) { w_s[buf][warp] = s; w_i[buf][warp] = i; }
   __syncthreads();
-  s = lane < kDsWarps ? w_s[lane] : -INFINITY;
-  i = lane < kDsWarps ? w_i[lane] : 0x7fffffff;
+  s = lane < kDsWarps ? w_s[buf][lane] : -INFINITY;
+  i = lane < kDsWarps ? w_i[buf][lane] : 0x7fffffff;
   ds_warp_argmax(s, i);
 }
 
 // (1) the k best of one chunk of one row, best first; slots past the last token with a chance: (-inf, -1)
 __global__ void __launch_bounds__(kDsThreads) draft_sample_chunk_kernel(const DraftSampleArgs a) {
   __shared__ float sc[kDsChunk];
-  __shared__ float w_s[kDsWarps];
-  __shared__ int w_i[kDsWarps];
+  __shared__ float w_s[2][kDsWarps];
+  __shared__ int w_i[2][kDsWarps];
   const int chunk = blockIdx.x, row = blockIdx.y, tid = threadIdx.x;
   const int base = chunk * kDsChunk, cnt = min(kDsChunk, a.V - base);
   const float* lrow = a.logits + (int64_t)row * a.logits_stride + base;
@@ -122,7 +123,7 @@ __global__ void __launch_bounds__(kDsThreads) draft_sample_chunk_kernel(const Dr
   for (int r = 0; r < a.k; ++r) {
     float s = bs;
     int i = bi;
-    ds_block_argmax(s, i, w_s, w_i);
+    ds_block_argmax(s, i, w_s, w_i, r);
     if (!(s > -INFINITY)) {  // nothing with a chance is left in this chunk
       for (int j = r + tid; j < a.k; j += kDsThreads) cand[j] = make_float2(-INFINITY, __int_as_float(-1));
       return;
@@ -145,8 +146,8 @@ __global__ void __launch_bounds__(kDsThreads) draft_sample_chunk_kernel(const Dr
 
 // (2) the k best of a row from its chunks' candidates (chunks * k of them), in draw order
 __global__ void __launch_bounds__(kDsThreads) draft_sample_merge_kernel(const DraftSampleArgs a) {
-  __shared__ float w_s[kDsWarps];
-  __shared__ int w_i[kDsWarps];
+  __shared__ float w_s[2][kDsWarps];
+  __shared__ int w_i[2][kDsWarps];
   extern __shared__ float2 cs[];  // the row's candidates
   const int row = blockIdx.x, tid = threadIdx.x;
   const int n = a.chunks * a.k;
@@ -168,7 +169,7 @@ __global__ void __launch_bounds__(kDsThreads) draft_sample_merge_kernel(const Dr
   for (int r = 0; r < a.k; ++r) {
     float s = bs;
     int i = bi;
-    ds_block_argmax(s, i, w_s, w_i);
+    ds_block_argmax(s, i, w_s, w_i, r);
     if (!(s > -INFINITY)) {  // the remaining draws do not exist
       for (int j = r + tid; j < a.k; j += kDsThreads) out[j] = -1;
       return;
