@@ -171,8 +171,8 @@ def seq_tree_draft_sample(draft_logits, temperature: float, uniforms, k: int, *,
         tokens_out = torch.empty((rows, k), dtype=torch.int32, device=draft_logits.device)
     p = DraftSampleParams()
     p.n_rows, p.vocab, p.k = rows, V, k
-    p.draft_logits, p.logits_row_stride = _dev(draft_logits, "draft_logits", torch.float32), draft_logits.stride(0)
-    p.uniforms, p.uniforms_row_stride = _dev(uniforms, "uniforms", torch.float32), uniforms.stride(0)
+    p.draft_logits, p.logits_row_stride = _dev(draft_logits, "draft_logits", torch.float32), (draft_logits.stride(0) if rows > 1 else V)
+    p.uniforms, p.uniforms_row_stride = _dev(uniforms, "uniforms", torch.float32), (uniforms.stride(0) if rows > 1 else V)
     p.temperature = temperature
     p.tokens_out = _dev(tokens_out, "tokens_out", torch.int32)
     p.dev_status = _dev(dev_status, "dev_status", torch.int32)
