@@ -386,7 +386,7 @@ def test_attention_mask_from_parent_array_bad_parent_and_unsupported():
 @pytest.mark.parametrize("name,rows", [("llama2-7b", [0, 1, 13, 40, 63]), ("llama2-13b", [0, 5, 64, 127]),
                                        ("vicuna-33b", [0, 100, 128, 255]), ("llama3-70b", [0, 31, 32, 400, 767])])
 def test_attention_full_size_configs_sampled_rows(name, rows):
-    """BASELINE sizes in the launch configuration the benchmark times; the oracle recomputes the
+    """The full workload sizes, in the launch configuration the benchmark times; the oracle recomputes the
     sampled nodes (and their ancestors) one by one."""
     cfg = W.CONFIGS[name]
     ai = W.make_attention_inputs(cfg, 0)
