@@ -64,6 +64,7 @@ def lib():
         L.orc_sample_inverse_cdf.restype = i32
         L.orc_tree_verify.argtypes = [i32, i32, pi32, pi32, pf32, i64, pf32, i64, f64, pf32, i32,
                                       pi32, pi32, pi32, pf64, pi32, pf64, pf64]
+        L.orc_tree_verify_target_sample.argtypes = [i32, i32, pi32, pi32, pf32, i64, f64, pf32, pi32, pi32, pi32, pf64, pi32, pf64]
         L.orc_alg3_chain.argtypes = [pf64, pf64, i32, i32, pi32, pf64, f64, pi32]
         L.orc_alg3_chain.restype = i32
         _lib = L
@@ -178,6 +179,25 @@ def tree_verify(parent, tokens, target_logits, draft_logits, T: float, uniforms,
     return dict(path=path[: plen.value].copy(), path_len=int(plen.value), bonus=int(bonus.value),
                 residual=residual, next_child=next_child, ratio=ratio, min_gap=float(gap.value),
                 flags=int(flags))
+
+
+def tree_verify_target_sample(parent, tokens, target_logits, T: float, uniforms) -> dict:
+    """Verification by sampling from the target at every visited node ("naive" / "top-k sampling")."""
+    parent, tokens = _i32(parent), _i32(tokens)
+    tl, un = _f32(target_logits), _f32(uniforms)
+    n, V = tl.shape
+    assert un.shape[0] == n + 1 and parent.shape[0] == n
+    path = np.empty(n, dtype=np.int32)
+    plen, bonus = C.c_int32(0), C.c_int32(-1)
+    residual = np.empty(V, dtype=np.float64)
+    next_child = np.empty(n, dtype=np.int32)
+    gap = C.c_double(0.0)
+    flags = lib().orc_tree_verify_target_sample(n, V, _p(parent, C.c_int32), _p(tokens, C.c_int32), _p(tl, C.c_float), V,
+                                                float(T), _p(un, C.c_float), _p(path, C.c_int32), C.byref(plen),
+                                                C.byref(bonus), _p(residual, C.c_double), _p(next_child, C.c_int32),
+                                                C.byref(gap))
+    return dict(path=path[: plen.value].copy(), path_len=int(plen.value), bonus=int(bonus.value), residual=residual,
+                next_child=next_child, min_gap=float(gap.value), flags=int(flags))
 
 
 def alg3_chain(p, q, x, r, u_final: float):

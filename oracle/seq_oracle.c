@@ -420,6 +420,81 @@ int orc_tree_verify(int32_t n, int32_t V, const int32_t* parent, const int32_t* 
 }
 
 /*
+ * Verification by sampling from the target (Section 2.2, "Naive sampling and
+ * top-k sampling": the verification algorithm "first samples from the target
+ * model's distribution P(.|x_<n) at that node, and then accepts this sample if
+ * it is equal to one of the children of that node"), applied recursively from
+ * the root like Algorithm 2.
+ *
+ * At node v: x ~ softmax(target_logits[v] / T) by inverse CDF in index order
+ * with uniforms[v]; if a child of v carries token x the walk moves to the
+ * first such child (ascending node index), else it stops and x is the token
+ * emitted there (bonus).  T = 0: x is the arg-max (lowest index on ties).
+ * The draft model plays no part.  residual_out (nullable): the distribution
+ * the last x was drawn from.  min_gap (nullable): the smallest distance of a
+ * used uniform to the two ends of the CDF interval of its x.
+ */
+int orc_tree_verify_target_sample(int32_t n, int32_t V, const int32_t* parent, const int32_t* tokens,
+                                  const float* target_logits, int64_t target_row_stride, double T,
+                                  const float* uniforms, int32_t* path, int32_t* path_len,
+                                  int32_t* bonus, double* residual_out, int32_t* next_child,
+                                  double* min_gap) {
+  int flags = 0;
+  double* P = (double*)malloc(sizeof(double) * (size_t)V);
+  if (next_child)
+    for (int32_t i = 0; i < n; ++i) next_child[i] = -2;
+  if (min_gap) *min_gap = INFINITY;
+  for (int32_t i = 1; i < n; ++i) (void)clean_parent(parent, i, &flags);
+  int32_t cur = 0, plen = 0;
+  path[plen++] = 0;
+  for (;;) {
+    const float* trow = target_logits + (size_t)cur * (size_t)target_row_stride;
+    for (int32_t t = 0; t < V; ++t)
+      if (!isfinite(trow[t]) && !(trow[t] < 0 && isinf(trow[t]))) flags |= ORC_NONFINITE;
+    int32_t x;
+    if (T == 0.0) {
+      x = 0;
+      for (int32_t t = 1; t < V; ++t)
+        if (trow[t] > trow[x]) x = t;
+      for (int32_t t = 0; t < V; ++t) P[t] = 0.0;
+      P[x] = 1.0;
+    } else {
+      orc_softmax_T(trow, V, T, P);
+      double u = (double)uniforms[cur];
+      x = orc_sample_inverse_cdf(P, V, u);
+      if (min_gap) {
+        double lo = 0.0;
+        for (int32_t t = 0; t < x; ++t) lo += P[t];
+        double g1 = fabs(u - lo), g2 = fabs(lo + P[x] - u);
+        if (g1 < *min_gap) *min_gap = g1;
+        if (g2 < *min_gap) *min_gap = g2;
+      }
+    }
+    int32_t acc = -1;
+    for (int32_t c = cur + 1; c < n && acc < 0; ++c)
+      if (parent[c] == cur) {
+        int32_t s = tokens[c];
+        if (s < 0 || s >= V) {
+          flags |= ORC_BAD_TOKEN;
+          continue;
+        }
+        if (s == x) acc = c;
+      }
+    if (next_child) next_child[cur] = acc;
+    if (acc < 0) {
+      *bonus = x;
+      if (residual_out) memcpy(residual_out, P, sizeof(double) * (size_t)V);
+      break;
+    }
+    cur = acc;
+    path[plen++] = cur;
+  }
+  *path_len = plen;
+  free(P);
+  return flags;
+}
+
+/*
  * Algorithm 3 (sequence-based speculative decoding) for one chain, with the
  * two misprints of the listing read as: the target distributions come from the
  * target model, and the final residual is taken iff fewer than gamma tokens
