@@ -219,7 +219,14 @@ enum {
    * renormalised -- which is SpecInfer's multi-round rejection sampling, the baseline the paper compares
    * its verification with (Section 3.2.2, Algorithm 2's caption; Theorem 3.7's counter-example).  The
    * children of a node are then draws WITH replacement from the draft row and may repeat. */
-  SEQ_VERIFY_SPECINFER = 2
+  SEQ_VERIFY_SPECINFER = 2,
+  /* Verification by sampling from the target (Section 2.2, "Naive sampling and top-k sampling"): at every
+   * visited node v a token x ~ softmax(target_logits[v] / T) is drawn by inverse CDF in index order with
+   * uniforms[v] (entry 0 serves the root); the walk moves to the first child of v that carries x, else it
+   * stops and x is bonus_token.  draft_logits is not read and may be NULL; residual_out receives the
+   * distribution the last x was drawn from.  At T = 0 this is the arg-max matching of the default mode.
+   * Not to be combined with SEQ_VERIFY_SPECINFER. */
+  SEQ_VERIFY_TARGET_SAMPLE = 4
 };
 
 typedef struct {
@@ -240,7 +247,7 @@ typedef struct {
   void* workspace;
   size_t workspace_bytes;
   int32_t* dev_status;
-  int32_t flags; /* 0 or an OR of SEQ_VERIFY_ALL_NODES, SEQ_VERIFY_SPECINFER */
+  int32_t flags; /* 0 or an OR of SEQ_VERIFY_ALL_NODES, SEQ_VERIFY_SPECINFER, SEQ_VERIFY_TARGET_SAMPLE */
 } seq_tree_verify_params;
 
 size_t seq_tree_verify_workspace_bytes(const seq_tree_verify_params* p);

@@ -19,6 +19,7 @@ SEQ_F16, SEQ_BF16, SEQ_F32 = 0, 1, 2
 SEQ_DEV_BAD_PARENT, SEQ_DEV_BAD_TOKEN, SEQ_DEV_NONFINITE, SEQ_DEV_DEGENERATE, SEQ_DEV_TIMEOUT = 1, 2, 4, 8, 16
 SEQ_VERIFY_ALL_NODES = 1
 SEQ_VERIFY_SPECINFER = 2
+SEQ_VERIFY_TARGET_SAMPLE = 4
 SEQ_MAX_TREE = 1024
 SEQ_NOALLOC_SCRATCH_BYTES = 384 << 10
 KERNEL_AUTO, KERNEL_CUDA_CORE, KERNEL_TENSOR_CORE = 0, 1, 2
@@ -261,7 +262,7 @@ class VerifyCall:
 
     def __init__(self, parent, tokens, target_logits, draft_logits, temperature: float, uniforms, *,
                  path=None, path_len=None, bonus_token=None, residual_out=None, next_child_out=None,
-                 all_nodes: bool = False, dev_status=None, specinfer: bool = False):
+                 all_nodes: bool = False, dev_status=None, specinfer: bool = False, target_sample: bool = False):
         n, V = target_logits.shape
         dev = target_logits.device
         if path is None:
@@ -289,7 +290,8 @@ class VerifyCall:
         p.next_child_out = _dev(next_child_out, "next_child_out", torch.int32)
         p.workspace, p.workspace_bytes = None, 0
         p.dev_status = _dev(dev_status, "dev_status", torch.int32)
-        p.flags = (SEQ_VERIFY_ALL_NODES if all_nodes else 0) | (SEQ_VERIFY_SPECINFER if specinfer else 0)
+        p.flags = ((SEQ_VERIFY_ALL_NODES if all_nodes else 0) | (SEQ_VERIFY_SPECINFER if specinfer else 0) |
+                   (SEQ_VERIFY_TARGET_SAMPLE if target_sample else 0))
         self.params = p
         self.path, self.path_len, self.bonus_token = path, path_len, bonus_token
         self.residual_out, self.next_child_out = residual_out, next_child_out

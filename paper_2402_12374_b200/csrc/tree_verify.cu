@@ -80,6 +80,7 @@ struct VShared {
   uint32_t has_child[SEQ_MAX_TREE / 32];
   float4 xbuf[2][kVParts];              // cluster exchange: one entry per (rank, warp), double-buffered
   int32_t wcnt[kVWarps];
+  int32_t drawn[2];                     // the token sampled from the target at this node (SEQ_VERIFY_TARGET_SAMPLE)
   uint64_t bar[2];                      // completion of the target / draft slice copies
 };
 
@@ -94,7 +95,7 @@ struct NodeState {
   int mode;             // 0: D proportional to q; 1: uniform over the non-rejected set
   int nS;               // |S|
   int has_q;            // qs holds this node's draft slice
-  int greedy_token;
+  int greedy_token;     // the token fixed at this node: the target arg-max (T = 0), or the sample from the target
 };
 
 struct Ctx {
@@ -238,17 +239,25 @@ __device__ __noinline__ void sanitize_segment(Ctx& c, bool need_draft, int32_t* 
 
 // Runs Algorithm 2's loop at node v.  Returns the accepted child's node id or -1 and leaves in
 // `st` (and in ps/qs/wseg) the state the final draw needs.
+__device__ int draw_token(Ctx& c, const NodeState& st, float u, float Cf, float Uf, float ipw, float iqw,
+                          const float* qsrc, double total);
+
 __device__ int process_node(cg::cluster_group& cluster, Ctx& c, const VerifyArgs& a, int v, NodeState& st,
                             bool skip_leaves, bool copies_started) {
   const bool greedy = a.temperature == 0.f;
   const bool specinfer = (a.flags & SEQ_VERIFY_SPECINFER) != 0;  // D is never touched: ZD stays 1, S stays empty
   const bool has_kids = node_has_child(c, v);
   if (skip_leaves && !has_kids) return -1;
-  const bool need_draft = !greedy && (has_kids || (copies_started && a.n > 1));
+  // verification by sampling from the target (at T = 0 that is the greedy branch): the draft plays no part
+  const bool tsample = !greedy && (a.flags & SEQ_VERIFY_TARGET_SAMPLE) != 0;
+  const bool need_draft = !greedy && !tsample && (has_kids || (copies_started && a.n > 1));
   const float* trow = a.target + (int64_t)v * a.target_stride;
   const float* drow = a.draft + (int64_t)v * a.draft_stride;
   c.npar ^= 1;
   float4* kid_pq = c.sh->kid_pq[c.npar];
+  // two slots by node parity: a thread may still be reading the previous node's slot, and cluster barriers
+  // lie between this reset and the remote write below
+  if (tsample && c.tid == 0) c.sh->drawn[c.npar] = -3;
   if (c.tid == 0 && !copies_started) {
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");  // earlier plain writes to the slices come first
     start_slice_copy(c, trow, c.ps, 0);
@@ -267,7 +276,7 @@ __device__ int process_node(cg::cluster_group& cluster, Ctx& c, const VerifyArgs
     if (i < kPrefetchChildren) {
       const int ch = c.sh->kids[i];
       prefetch_slice_l2(c, a.target + (int64_t)ch * a.target_stride);
-      if (!greedy && node_has_child(c, ch)) prefetch_slice_l2(c, a.draft + (int64_t)ch * a.draft_stride);
+      if (!greedy && !tsample && node_has_child(c, ch)) prefetch_slice_l2(c, a.draft + (int64_t)ch * a.draft_stride);
     }
   }
   TRACE(2);
@@ -400,6 +409,25 @@ __device__ int process_node(cg::cluster_group& cluster, Ctx& c, const VerifyArgs
   st.C = 0.0; st.U = 0.0; st.Z = 1.0; st.ZD = 1.0; st.nS = 0; st.has_q = need_draft;
   TRACE(7);
 
+  if (tsample) {
+    // x ~ P with this node's uniform; the warp that finds x tells every CTA; a child that carries x is taken
+    const double total = sum_lanes(st.part_sum[0] + st.part_sum[1], 32);
+    const int found = draw_token(c, st, c.sh->uniforms[v], 0.f, 0.f, st.ipw, 0.f, c.ps, total);
+    if (found >= 0)
+      for (int r = 0; r < kVCluster; ++r) *cluster.map_shared_rank(&c.sh->drawn[c.npar], r) = found;
+    cluster.sync();
+    int x = c.sh->drawn[c.npar];
+    if (x < 0) { dev_flag(a.dev_status, SEQ_DEV_DEGENERATE); x = 0; }  // a target row without mass
+    st.greedy_token = x;
+    for (int i = 0; i < k; ++i) {
+      const int ch = c.sh->kids[i];
+      const int s = c.sh->tokens[ch];
+      if (s < 0 || s >= a.V) { dev_flag(a.dev_status, SEQ_DEV_BAD_TOKEN); continue; }
+      if (s == x) return ch;
+    }
+    return -1;
+  }
+
   for (int i = 0; i < k; ++i) {
     const int ch = c.sh->kids[i];
     const int s = c.sh->tokens[ch];
@@ -470,28 +498,14 @@ __device__ int process_node(cg::cluster_group& cluster, Ctx& c, const VerifyArgs
   return -1;
 }
 
-// Line 18, x ~ R by inverse CDF in index order with uniforms[n]; optionally writes R.
-__device__ void draw_bonus(Ctx& c, const VerifyArgs& a, const NodeState& st) {
-  if (a.temperature == 0.f) {
-    if (a.residual_out != nullptr)
-      for (int t = c.tid; t < c.cnt; t += kVThreads) a.residual_out[c.lo + t] = (c.lo + t == st.greedy_token) ? 1.f : 0.f;
-    if (c.rank == 0 && c.tid == 0) *a.bonus = st.greedy_token;
-    return;
-  }
-  const float Cf = (float)st.C, Uf = (float)st.U;
-  const bool has_q = st.has_q && (st.C != 0.0);
-  const float ipw = st.ipw, iqw = has_q ? st.iqw : 0.f;
-  const float* qsrc = has_q ? c.qs : c.ps;  // never dereference a slice that was not loaded
-  const double total = sum_lanes(st.part_sum[0] + st.part_sum[1], 32);
-
-  if (a.residual_out != nullptr) {
-    const float it = total > 0.0 ? (float)(1.0 / total) : 0.f;
-    for (int t = c.s_lo + c.lane; t < c.s_hi; t += 32)
-      a.residual_out[c.lo + t] = resid(c.ps[t] * ipw, qsrc[t] * iqw, Cf, Uf) * it;
-  }
-
+// x ~ R by inverse CDF in index order with the uniform u, R being the residual max(p - C q - U, 0) of the
+// current node (the target distribution itself when C = U = 0).  Returns the token in lane 0 of the one warp of
+// the cluster whose segment holds the crossing, -1 in every other thread, and -3 in every thread when R has no
+// mass at all.
+__device__ int draw_token(Ctx& c, const NodeState& st, float u, float Cf, float Uf, float ipw, float iqw,
+                          const float* qsrc, double total) {
   // inverse CDF over the 64 (rank, warp) segments: inclusive scan across lanes, segments `lane` first
-  const double tgt = (double)c.sh->uniforms[a.n] * total;
+  const double tgt = (double)u * total;
   double inc0 = st.part_sum[0];
 #pragma unroll
   for (int o = 1; o < 32; o <<= 1) {
@@ -518,12 +532,9 @@ __device__ void draw_bonus(Ctx& c, const VerifyArgs& a, const NodeState& st) {
     take_last = true;
     if (pos1) part = 63 - __clz(pos1);
     else if (pos0) part = 31 - __clz(pos0);
-    else {           // no mass anywhere: degenerate input, defined output
-      if (c.rank == 0 && c.tid == 0) { *a.bonus = 0; dev_flag(a.dev_status, SEQ_DEV_DEGENERATE); }
-      return;
-    }
+    else return -3;  // no mass anywhere: degenerate input (every thread of the cluster sees this)
   }
-  if (part != c.rank * kVWarps + c.warp) return;
+  if (part != c.rank * kVWarps + c.warp) return -1;
   const double incl_part = part < 32 ? __shfl_sync(0xffffffffu, inc0, part & 31) : __shfl_sync(0xffffffffu, inc1, part & 31);
   const double mass_part = part < 32 ? __shfl_sync(0xffffffffu, st.part_sum[0], part & 31)
                                      : __shfl_sync(0xffffffffu, st.part_sum[1], part & 31);
@@ -548,7 +559,43 @@ __device__ void draw_bonus(Ctx& c, const VerifyArgs& a, const NodeState& st) {
     carry += __shfl_sync(0xffffffffu, incl, 31);
   }
   if (found < 0) found = last_pos;
-  if (c.lane == 0) *a.bonus = c.lo + (found < 0 ? c.s_lo : found);
+  return c.lane == 0 ? c.lo + (found < 0 ? c.s_lo : found) : -1;
+}
+
+
+// Line 18, x ~ R with uniforms[n]; optionally writes R.  (Greedy, and verification by sampling from the target:
+// the token was fixed at the last node, R is the distribution it came from.)
+__device__ void draw_bonus(Ctx& c, const VerifyArgs& a, const NodeState& st) {
+  if (a.temperature == 0.f) {
+    if (a.residual_out != nullptr)
+      for (int t = c.tid; t < c.cnt; t += kVThreads) a.residual_out[c.lo + t] = (c.lo + t == st.greedy_token) ? 1.f : 0.f;
+    if (c.rank == 0 && c.tid == 0) *a.bonus = st.greedy_token;
+    return;
+  }
+  if (a.flags & SEQ_VERIFY_TARGET_SAMPLE) {
+    if (a.residual_out != nullptr)
+      for (int t = c.s_lo + c.lane; t < c.s_hi; t += 32) a.residual_out[c.lo + t] = c.ps[t] * st.ipw;
+    if (c.rank == 0 && c.tid == 0) *a.bonus = st.greedy_token;
+    return;
+  }
+  const float Cf = (float)st.C, Uf = (float)st.U;
+  const bool has_q = st.has_q && (st.C != 0.0);
+  const float ipw = st.ipw, iqw = has_q ? st.iqw : 0.f;
+  const float* qsrc = has_q ? c.qs : c.ps;  // never dereference a slice that was not loaded
+  const double total = sum_lanes(st.part_sum[0] + st.part_sum[1], 32);
+
+  if (a.residual_out != nullptr) {
+    const float it = total > 0.0 ? (float)(1.0 / total) : 0.f;
+    for (int t = c.s_lo + c.lane; t < c.s_hi; t += 32)
+      a.residual_out[c.lo + t] = resid(c.ps[t] * ipw, qsrc[t] * iqw, Cf, Uf) * it;
+  }
+
+  const int x = draw_token(c, st, c.sh->uniforms[a.n], Cf, Uf, ipw, iqw, qsrc, total);
+  if (x == -3) {
+    if (c.rank == 0 && c.tid == 0) { *a.bonus = 0; dev_flag(a.dev_status, SEQ_DEV_DEGENERATE); }
+  } else if (x >= 0) {
+    *a.bonus = x;
+  }
 }
 
 __global__ void __launch_bounds__(kVThreads, 1) tree_verify_kernel(const VerifyArgs a) {
@@ -577,7 +624,7 @@ __global__ void __launch_bounds__(kVThreads, 1) tree_verify_kernel(const VerifyA
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     if (!all_nodes) {  // the walk always starts at the root: fetch its rows while the tree is being read
       start_slice_copy(c, a.target, c.ps, 0);
-      if (!greedy && a.n > 1) start_slice_copy(c, a.draft, c.qs, 1);  // draft row 0 is read whenever the tree has children
+      if (!greedy && a.n > 1 && !(a.flags & SEQ_VERIFY_TARGET_SAMPLE)) start_slice_copy(c, a.draft, c.qs, 1);  // draft row 0 is read whenever the tree has children
     }
   }
   if (c.tid < SEQ_MAX_TREE / 32) sh.has_child[c.tid] = 0u;
@@ -638,14 +685,16 @@ static int verify_validate(const seq_tree_verify_params* p) {
   if (p->n_tree < 1 || p->n_tree > SEQ_MAX_TREE || p->vocab < 1) return SEQ_ERR_INVALID_ARG;
   if (p->parent == nullptr || p->tokens == nullptr || p->target_logits == nullptr) return SEQ_ERR_INVALID_ARG;
   if (!(p->temperature >= 0.f) || isinf(p->temperature)) return SEQ_ERR_INVALID_ARG;
-  if (p->flags & ~(SEQ_VERIFY_ALL_NODES | SEQ_VERIFY_SPECINFER)) return SEQ_ERR_INVALID_ARG;
+  if (p->flags & ~(SEQ_VERIFY_ALL_NODES | SEQ_VERIFY_SPECINFER | SEQ_VERIFY_TARGET_SAMPLE)) return SEQ_ERR_INVALID_ARG;
+  if ((p->flags & SEQ_VERIFY_SPECINFER) && (p->flags & SEQ_VERIFY_TARGET_SAMPLE)) return SEQ_ERR_INVALID_ARG;
   const bool all_nodes = p->flags & SEQ_VERIFY_ALL_NODES;
   if (all_nodes) {
     if (p->next_child_out == nullptr) return SEQ_ERR_INVALID_ARG;
   } else if (p->path == nullptr || p->path_len == nullptr || p->bonus_token == nullptr) {
     return SEQ_ERR_INVALID_ARG;
   }
-  if (p->temperature > 0.f && (p->draft_logits == nullptr || p->uniforms == nullptr)) return SEQ_ERR_INVALID_ARG;
+  if (p->temperature > 0.f && p->uniforms == nullptr) return SEQ_ERR_INVALID_ARG;
+  if (p->temperature > 0.f && p->draft_logits == nullptr && !(p->flags & SEQ_VERIFY_TARGET_SAMPLE)) return SEQ_ERR_INVALID_ARG;
   if (p->target_row_stride < p->vocab || p->target_row_stride % 4 != 0 ||
       reinterpret_cast<uintptr_t>(p->target_logits) % 16 != 0)
     return SEQ_ERR_INVALID_ARG;

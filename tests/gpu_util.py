@@ -71,7 +71,7 @@ def _path(parent, i):
     return out
 
 
-def run_verify(vi: W.VerifyInputs, all_nodes=False, want_residual=True, specinfer=False):
+def run_verify(vi: W.VerifyInputs, all_nodes=False, want_residual=True, specinfer=False, target_sample=False):
     d = dev()
     n, V = vi.target_logits.shape
     st = torch.zeros(1, dtype=torch.int32, device=d)
@@ -80,11 +80,15 @@ def run_verify(vi: W.VerifyInputs, all_nodes=False, want_residual=True, specinfe
     # rows padded to a multiple of 4 floats (NaN in the padding) so every row stays 16-byte aligned
     Vp = (V + 3) // 4 * 4
     tl = torch.full((n, Vp), float("nan"), dtype=torch.float32, device=d)
-    dl = torch.full((n, Vp), float("nan"), dtype=torch.float32, device=d)
-    tl[:, :V], dl[:, :V] = vi.target_logits.to(d), vi.draft_logits.to(d)
-    call = B.VerifyCall(vi.parent.to(d), vi.tokens.to(d), tl[:, :V], dl[:, :V],
+    tl[:, :V] = vi.target_logits.to(d)
+    dl = None
+    if vi.draft_logits is not None:
+        dl = torch.full((n, Vp), float("nan"), dtype=torch.float32, device=d)
+        dl[:, :V] = vi.draft_logits.to(d)
+        dl = dl[:, :V]
+    call = B.VerifyCall(vi.parent.to(d), vi.tokens.to(d), tl[:, :V], dl,
                         vi.temperature, vi.uniforms.to(d), residual_out=residual, next_child_out=nxt,
-                        all_nodes=all_nodes, dev_status=st, specinfer=specinfer)
+                        all_nodes=all_nodes, dev_status=st, specinfer=specinfer, target_sample=target_sample)
     call.run()
     torch.cuda.synchronize()
     plen = int(call.path_len.item())
@@ -117,6 +121,26 @@ def check_verify(vi: W.VerifyInputs, specinfer=False):
         lo = cdf[t - 1] if t > 0 else 0.0
         assert lo - GAP <= u < cdf[t] + GAP and ref["residual"][t] > 0, (t, ref["bonus"], u, lo, cdf[t])
         return "excluded"
+    return "ok"
+
+
+def check_verify_target_sample(vi: W.VerifyInputs, with_draft=False):
+    """SEQ_VERIFY_TARGET_SAMPLE: path, per-node decisions and bonus identical to the oracle's walk that samples
+    from the target at every node (outside the rounding band of its inverse CDFs); residual_out = the target
+    distribution at the last node, within 1e-5.  Returns 'ok' or 'excluded'."""
+    if not with_draft:
+        vi = W.VerifyInputs(vi.parent, vi.tokens, vi.target_logits, None, vi.uniforms, vi.temperature)
+    got = run_verify(vi, target_sample=True)
+    ref = O.tree_verify_target_sample(vi.parent, vi.tokens, vi.target_logits, vi.temperature, vi.uniforms)
+    assert got["status"] == ref["flags"] == 0
+    if ref["min_gap"] < GAP:
+        return "excluded"
+    assert got["path"].tolist() == ref["path"].tolist(), (got["path"], ref["path"])
+    assert np.array_equal(got["next_child"], ref["next_child"]), "per-node decisions differ"
+    assert got["bonus"] == ref["bonus"]
+    rerr = np.abs(got["residual"] - ref["residual"]).max()
+    assert rerr < RESID_TOL, f"residual max abs err {rerr}"
+    assert abs(got["residual"].sum() - 1.0) < 1e-5 and (got["residual"] >= 0).all()
     return "ok"
 
 

@@ -235,6 +235,55 @@ def test_verify_specinfer_children_with_replacement_and_many_rejections():
     assert np.abs(ref_a["residual"] - ref_b["residual"]).max() > 1e-4 or ref_a["path"].tolist() != ref_b["path"].tolist()
 
 
+@pytest.mark.parametrize("name,T,seeds", [("tiny", 0.6, range(8)), ("llama2-7b", 0.6, range(4)), ("llama2-7b", 1.0, range(3)),
+                                          ("llama2-13b", 1.0, range(2)), ("llama3-70b", 0.6, range(1))])
+def test_verify_target_sample_configs(name, T, seeds):
+    """SEQ_VERIFY_TARGET_SAMPLE (Section 2.2, naive / top-k sampling): the walk that samples from the target at
+    every node, against the oracle's; no draft row is passed."""
+    cfg = W.CONFIGS[name]
+    outcomes = [G.check_verify_target_sample(W.make_verify_inputs(cfg, T, seed)) for seed in seeds]
+    assert outcomes.count("ok") >= max(1, len(outcomes) - 1), outcomes
+
+
+def _steer_tokens_to_samples(vi, every=1):
+    """Rewrites the first child's token of every `every`-th internal node to the token the oracle's inverse CDF
+    draws there, so that the walk goes deep; returns the number of nodes steered."""
+    kids = W.children_lists(vi.parent.numpy())
+    steered = 0
+    for v, ch in enumerate(kids):
+        if ch and v % every == 0:
+            P = O.softmax_T(vi.target_logits[v], vi.temperature)
+            vi.tokens[ch[0]] = O.sample_inverse_cdf(P, float(vi.uniforms[v]))
+            steered += 1
+    return steered
+
+
+@pytest.mark.parametrize("name,T,vocab", [("tiny", 0.6, None), ("llama2-7b", 1.0, None), ("llama2-7b", 0.3, 5003)])
+def test_verify_target_sample_deep_walks(name, T, vocab):
+    """Children carrying exactly the token that is drawn at their parent: the walk follows them to a leaf, one
+    cluster-wide draw per level, and the bonus is the leaf's own draw.  (Vocabulary 5003: ragged slices.)"""
+    cfg = W.CONFIGS[name]
+    ok = 0
+    for seed in range(3):
+        vi = W.make_verify_inputs(cfg, T, seed, vocab=vocab)
+        assert _steer_tokens_to_samples(vi) > 1
+        ref = O.tree_verify_target_sample(vi.parent, vi.tokens, vi.target_logits, vi.temperature, vi.uniforms)
+        assert ref["path_len"] >= 3  # the steering worked: root, its first child, that child's first child ...
+        ok += G.check_verify_target_sample(vi, with_draft=(seed == 1)) == "ok"
+    assert ok >= 2
+
+
+def test_verify_target_sample_greedy_is_argmax_matching():
+    """T = 0 with the flag set: the arg-max matching of the default mode (the draw degenerates to the arg-max)."""
+    vi = W.make_verify_inputs(W.CONFIGS["tiny"], 0.0, 2)
+    a = G.run_verify(vi, target_sample=True)
+    b = G.run_verify(vi)
+    ref = O.tree_verify_target_sample(vi.parent, vi.tokens, vi.target_logits, 0.0, vi.uniforms)
+    assert a["path"].tolist() == b["path"].tolist() == ref["path"].tolist()
+    assert a["bonus"] == b["bonus"] == ref["bonus"] and a["status"] == 0
+    assert np.array_equal(a["residual"], ref["residual"])
+
+
 def test_verify_nonfinite_logits_are_flagged_not_trapped():
     vi = W.make_verify_inputs(W.CONFIGS["tiny"], 0.6, 0, vocab=512)
     vi.target_logits[0, 5] = float("nan")
