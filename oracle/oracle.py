@@ -26,6 +26,7 @@ VARIANT_SEQUOIA = 0
 VARIANT_SPECINFER = 1
 
 BAD_PARENT, BAD_TOKEN, NONFINITE, DEGENERATE = 1, 2, 4, 8
+BAD_PATH = 32
 
 
 def build(force: bool = False) -> str:
@@ -65,6 +66,7 @@ def lib():
         L.orc_tree_verify.argtypes = [i32, i32, pi32, pi32, pf32, i64, pf32, i64, f64, pf32, i32,
                                       pi32, pi32, pi32, pf64, pi32, pf64, pf64]
         L.orc_tree_verify_target_sample.argtypes = [i32, i32, pi32, pi32, pf32, i64, f64, pf32, pi32, pi32, pi32, pf64, pi32, pf64]
+        L.orc_kv_commit.argtypes = [C.c_void_p, C.c_void_p, i64, i64, i64, i32, i32, pi32, i32]
         L.orc_alg3_chain.argtypes = [pf64, pf64, i32, i32, pi32, pf64, f64, pi32]
         L.orc_alg3_chain.restype = i32
         _lib = L
@@ -208,3 +210,17 @@ def alg3_chain(p, q, x, r, u_final: float):
     s = lib().orc_alg3_chain(_p(p, C.c_double), _p(q, C.c_double), V, gamma, _p(x, C.c_int32),
                              _p(r, C.c_double), float(u_final), C.byref(t))
     return int(s), int(t.value)
+
+
+def kv_commit(cache, prefix_len: int, n_tree: int, path):
+    """cache: numpy array [..., rows, d] of any item size (leading dimensions = planes).  Returns the committed
+    copy (row L+i <- row L+path[i]) and the flags."""
+    cache = np.ascontiguousarray(cache)
+    path = _i32(path)
+    rows, d = cache.shape[-2], cache.shape[-1]
+    assert rows >= prefix_len + n_tree
+    planes = int(np.prod(cache.shape[:-2], dtype=np.int64))
+    out = np.empty_like(cache)
+    flags = lib().orc_kv_commit(cache.ctypes.data, out.ctypes.data, planes, rows, d * cache.itemsize, prefix_len,
+                                n_tree, _p(path, C.c_int32), path.shape[0])
+    return out, int(flags)

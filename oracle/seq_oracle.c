@@ -12,7 +12,9 @@
  *   - Algorithm 2 ("Sequoia Sampling and Verification") applied recursively
  *     from the root (Section 2.2), ending with the draw x ~ R;
  *   - the draft side's draw of a node's children without replacement by
- *     exponential sort (Section 5, "Implementation Details").
+ *     exponential sort (Section 5, "Implementation Details");
+ *   - verification by sampling from the target (Section 2.2, naive / top-k
+ *     sampling), and the commit of an accepted path into the cache.
  *
  * Nothing here is blocked, fused or reordered: every function is the
  * definition, or the algorithm's steps in the paper's order and notation, so
@@ -28,7 +30,10 @@
  * Monte-Carlo; attention against library causal attention (chain tree),
  * single-query decode (star tree) and explicit-sequence brute force; the
  * exponential sort against the exact without-replacement law of ordered pairs
- * (Monte-Carlo), library sorts in its two degenerate cases, and invariants.
+ * (Monte-Carlo), library sorts in its two degenerate cases, and invariants;
+ * the commit against a library gather, hand-written cases where a row is both
+ * read and overwritten, and the identity "attention of a path node over the
+ * tree == causal attention over the committed cache".
  *
  * Build: gcc -O2 -fopenmp -shared -fPIC seq_oracle.c -o liboracle.so -lm
  */
@@ -45,6 +50,7 @@
 #define ORC_BAD_TOKEN 2
 #define ORC_NONFINITE 4
 #define ORC_DEGENERATE 8
+#define ORC_BAD_PATH 32
 
 #define ORC_VARIANT_SEQUOIA 0   /* Algorithm 2 as printed */
 #define ORC_VARIANT_SPECINFER 1 /* Algorithm 2 without its blue lines 10-16 */
@@ -528,4 +534,37 @@ int32_t orc_alg3_chain(const double* p, const double* q, int32_t V, int32_t gamm
   *t_out = orc_sample_inverse_cdf(pp, V, u_final);
   free(pp);
   return s;
+}
+
+/*
+ * Commit of an accepted path into the key/value cache: what has to happen
+ * between one verification and the next so that the accepted tokens become
+ * part of the prefix (Section 2.1: the accepted tokens are kept and decoding
+ * goes on from them; the cache itself is left to the implementation).  The
+ * tree's rows sit at [L, L+n) of every plane (one plane = the keys or the
+ * values of one head of one layer); afterwards row L+i holds what row
+ * L+path[i] held, for i in [0, path_len), so that the new prefix is
+ * L + path_len rows long.  Every other row is unchanged.  Written out of place
+ * (in -> out, both [planes][rows][row_bytes] bytes) so that the definition has
+ * no ordering in it.
+ *
+ * A path is valid iff 0 <= path_len <= n, path[0] == 0, it is strictly
+ * ascending and stays below n (a parent always precedes its child); an invalid
+ * path raises ORC_BAD_PATH and nothing moves (out == in).
+ */
+int32_t orc_kv_commit(const uint8_t* in, uint8_t* out, int64_t planes, int64_t rows,
+                      int64_t row_bytes, int32_t L, int32_t n, const int32_t* path,
+                      int32_t path_len) {
+  memcpy(out, in, (size_t)(planes * rows * row_bytes));
+  int ok = path_len >= 0 && path_len <= n;
+  for (int32_t i = 0; ok && i < path_len; ++i) {
+    if (i == 0 ? path[0] != 0 : path[i] <= path[i - 1]) ok = 0;
+    if (path[i] < 0 || path[i] >= n) ok = 0;
+  }
+  if (!ok) return ORC_BAD_PATH;
+  for (int64_t h = 0; h < planes; ++h)
+    for (int32_t i = 0; i < path_len; ++i)
+      memcpy(out + ((size_t)h * rows + (size_t)(L + i)) * row_bytes,
+             in + ((size_t)h * rows + (size_t)(L + path[i])) * row_bytes, (size_t)row_bytes);
+  return 0;
 }
