@@ -231,6 +231,61 @@ def draft_sample_leg(cfg, parent, ver_h, T, dev, stream, peaks) -> dict:
             "note": "logits + uniforms of every internal node read once; outside the timed step"}
 
 
+def kv_commit_leg(cfg, parent, dev, stream, peaks) -> dict:
+    """Not part of the timed step: the commit of an accepted path into the whole model's key/value cache (every
+    layer's planes), timed per call with event nodes inside one CUDA graph, a write of a buffer larger than L2
+    before every call.  The path: the root and, level by level, the last child that has children of its own (else
+    the last child), five nodes at most."""
+    from paper_2402_12374_b200 import binding as B
+
+    layers = W.NUM_LAYERS[cfg.name]
+    kids = W.children_lists(parent)
+    path = [0]
+    while kids[path[-1]] and len(path) < 5:
+        inner = [c for c in kids[path[-1]] if kids[c]]
+        path.append(inner[-1] if inner else kids[path[-1]][-1])
+    n, L = len(parent), cfg.prefix_len
+    planes = layers * cfg.num_kv_heads
+    dt = W.TORCH_DTYPES[cfg.dtype]
+    k = torch.zeros((planes, L + n, cfg.head_dim), dtype=dt, device=dev)
+    v = torch.zeros((planes, L + n, cfg.head_dim), dtype=dt, device=dev)
+    k[:, L:].normal_()
+    v[:, L:].normal_()
+    path_d = torch.zeros(n, dtype=torch.int32, device=dev)
+    path_d[: len(path)] = torch.tensor(path, dtype=torch.int32)
+    plen = torch.tensor([len(path)], dtype=torch.int32, device=dev)
+    status = torch.zeros(1, dtype=torch.int32, device=dev)
+    flush = torch.empty(160 << 20, dtype=torch.uint8, device=dev)
+    reps = 20
+    evs = [[torch.cuda.Event(enable_timing=True, external=True) for _ in range(2)] for _ in range(reps)]
+    with torch.cuda.stream(stream):
+        for _ in range(3):
+            B.seq_tree_kv_commit(k, v, L, n, path_d, plen, dev_status=status, stream=stream)
+        stream.synchronize()
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g, stream=stream):
+            for i in range(reps):
+                flush.fill_(i)
+                evs[i][0].record(stream)
+                B.seq_tree_kv_commit(k, v, L, n, path_d, plen, dev_status=status, stream=stream)
+                evs[i][1].record(stream)
+        g.replay()
+        stream.synchronize()
+        g.replay()
+        stream.synchronize()
+    if int(status.item()) != 0:
+        raise RuntimeError(f"kv_commit dev_status = {int(status.item())}")
+    us = float(np.median([a.elapsed_time(b) * 1e3 for a, b in evs]))
+    moved = sum(int(p != i) for i, p in enumerate(path))
+    nbytes = 2 * 2 * planes * moved * cfg.head_dim * k.element_size()
+    gbs = nbytes / (us * 1e-6) / 1e9
+    return {"us_per_call": us, "layers": layers, "planes": planes, "path_len": len(path), "rows_moved": moved,
+            "gpu_launches_per_call": 1, "l2": "flushed before every call",
+            "roofline": {"bound": "hbm", "achieved": gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                         "frac": gbs / peaks["hbm_gbs"], "algorithmic_bytes": nbytes, "traffic": None},
+            "note": "moved rows of every plane read and written once; latency-bound at this size; outside the timed step"}
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -434,8 +489,9 @@ def main():
         "breakdown_us": {"attention": attn_us, "verify": ver_us,
                          "largest_share": "seq_tree_verify" if ver_us > attn_us else "seq_tree_attention"},
     }
+    line["next_rows"] = {"kv_commit": kv_commit_leg(cfg, parent, dev, stream, peaks)}
     if T > 0:
-        line["next_rows"] = {"draft_sample": draft_sample_leg(cfg, parent, ver_h, T, dev, stream, peaks)}
+        line["next_rows"]["draft_sample"] = draft_sample_leg(cfg, parent, ver_h, T, dev, stream, peaks)
     if not args.no_cpu_baseline:
         from oracle import oracle as O
 

@@ -55,7 +55,8 @@ enum {
   SEQ_DEV_BAD_TOKEN = 2,   /* token id outside [0,vocab): the child is rejected, R and D untouched */
   SEQ_DEV_NONFINITE = 4,   /* NaN or +inf logit on a visited row */
   SEQ_DEV_DEGENERATE = 8,  /* sum max(R-D,0) == 0 after a rejection (impossible in exact arithmetic): R kept */
-  SEQ_DEV_TIMEOUT = 16     /* a bounded on-chip wait ran out; outputs of that call are undefined */
+  SEQ_DEV_TIMEOUT = 16,    /* a bounded on-chip wait ran out; outputs of that call are undefined */
+  SEQ_DEV_BAD_PATH = 32    /* seq_tree_kv_commit: path not a root-to-node path (see there); nothing was moved */
 };
 
 /*
@@ -297,6 +298,45 @@ typedef struct {
 
 size_t seq_tree_draft_sample_workspace_bytes(const seq_tree_draft_sample_params* p);
 int seq_tree_draft_sample(const seq_tree_draft_sample_params* p, void* stream);
+
+/* ---------------------------------------------------------------------------
+ * seq_tree_kv_commit -- makes the accepted path part of the prefix (Section 2.1: the accepted tokens are kept
+ * and decoding goes on after them; the key/value cache that makes this possible is the implementation's).
+ *
+ * The tree's keys and values sit at rows [prefix_len, prefix_len + n_tree) of every plane (one plane = one
+ * head of one layer, for the keys or for the values).  After the call, in every plane, row prefix_len + i holds
+ * what row prefix_len + path[i] held before it, for i in [0, *path_len); every other row is unchanged.  The
+ * next step's prefix is therefore prefix_len + *path_len rows, which is written to *new_prefix_len.  The move
+ * is in place and needs no workspace (each thread owns 16 bytes of a plane's rows, takes the rows in ascending
+ * order and reads a batch before it writes it; path[j] > path[i] >= i for j > i, so no row is overwritten
+ * before its last reader has it).
+ *
+ *   k_cache, v_cache   device, [num_planes] planes of rows of row_bytes bytes; plane_stride_bytes and
+ *                      row_stride_bytes are multiples of 16, the base pointers 16-byte aligned, row_bytes a
+ *                      multiple of 16 (<= row_stride_bytes).  v_cache may be NULL (keys only).  The two
+ *                      buffers must not overlap.
+ *   path, path_len     device, as seq_tree_verify wrote them (path has room for n_tree entries, all of them
+ *                      readable): path[0] = 0, strictly ascending, below n_tree, 0 <= *path_len <= n_tree.
+ *                      Anything else raises SEQ_DEV_BAD_PATH, moves nothing and
+ *                      leaves *new_prefix_len = prefix_len.
+ *   new_prefix_len     device, nullable.
+ *
+ * The caller keeps ownership of everything.  Asynchronous on `stream`; capturable in a CUDA graph.  Returns
+ * SEQ_OK, SEQ_ERR_INVALID_ARG (null pointer, size or alignment out of range) or SEQ_ERR_CUDA. */
+typedef struct {
+  int32_t num_planes;
+  int32_t row_bytes;
+  int32_t prefix_len, n_tree;
+  void* k_cache;
+  void* v_cache;
+  int64_t plane_stride_bytes, row_stride_bytes;
+  const int32_t* path;
+  const int32_t* path_len;
+  int32_t* new_prefix_len;
+  int32_t* dev_status;
+} seq_tree_kv_commit_params;
+
+int seq_tree_kv_commit(const seq_tree_kv_commit_params* p, void* stream);
 
 const char* seq_tree_version(void);
 

@@ -20,6 +20,7 @@ SEQ_DEV_BAD_PARENT, SEQ_DEV_BAD_TOKEN, SEQ_DEV_NONFINITE, SEQ_DEV_DEGENERATE, SE
 SEQ_VERIFY_ALL_NODES = 1
 SEQ_VERIFY_SPECINFER = 2
 SEQ_VERIFY_TARGET_SAMPLE = 4
+SEQ_DEV_BAD_PATH = 32
 SEQ_MAX_TREE = 1024
 SEQ_NOALLOC_SCRATCH_BYTES = 384 << 10
 KERNEL_AUTO, KERNEL_CUDA_CORE, KERNEL_TENSOR_CORE = 0, 1, 2
@@ -37,6 +38,7 @@ EXPORTED_SYMBOLS = (
     "seq_tree_verify",
     "seq_tree_draft_sample_workspace_bytes",
     "seq_tree_draft_sample",
+    "seq_tree_kv_commit",
     "seq_tree_version",
 )
 
@@ -105,6 +107,8 @@ def load() -> C.CDLL:
         lib.seq_tree_verify_workspace_bytes.restype = C.c_size_t
         lib.seq_tree_verify.argtypes = [C.POINTER(VerifyParams), C.c_void_p]
         lib.seq_tree_verify.restype = C.c_int
+        lib.seq_tree_kv_commit.argtypes = [C.POINTER(KvCommitParams), C.c_void_p]
+        lib.seq_tree_kv_commit.restype = C.c_int
         lib.seq_tree_version.restype = C.c_char_p
         _lib = lib
     return _lib
@@ -158,6 +162,15 @@ class DraftSampleParams(C.Structure):
         ("uniforms", C.c_void_p), ("uniforms_row_stride", C.c_int64),
         ("temperature", C.c_float), ("tokens_out", C.c_void_p), ("dev_status", C.c_void_p),
         ("workspace", C.c_void_p), ("workspace_bytes", C.c_size_t),
+    ]
+
+
+class KvCommitParams(C.Structure):
+    _fields_ = [
+        ("num_planes", C.c_int32), ("row_bytes", C.c_int32), ("prefix_len", C.c_int32), ("n_tree", C.c_int32),
+        ("k_cache", C.c_void_p), ("v_cache", C.c_void_p),
+        ("plane_stride_bytes", C.c_int64), ("row_stride_bytes", C.c_int64),
+        ("path", C.c_void_p), ("path_len", C.c_void_p), ("new_prefix_len", C.c_void_p), ("dev_status", C.c_void_p),
     ]
 
 
@@ -306,6 +319,27 @@ def seq_tree_verify(parent, tokens, target_logits, draft_logits, temperature: fl
     """Algorithm 2 walked from the root; returns device tensors (path [n], path_len [1], bonus_token [1])."""
     stream = kw.pop("stream", None)
     return VerifyCall(parent, tokens, target_logits, draft_logits, temperature, uniforms, **kw).run(stream)
+
+
+def seq_tree_kv_commit(k_cache, v_cache, prefix_len: int, n_tree: int, path, path_len, *, new_prefix_len=None,
+                       dev_status=None, stream=None):
+    """In place: row prefix_len+i of every plane <- row prefix_len+path[i], i < path_len (device tensors as
+    seq_tree_verify wrote them).  k_cache / v_cache: [planes, rows, head_dim] (v_cache may be None), rows
+    contiguous."""
+    planes, rows, d = k_cache.shape
+    for t in (k_cache, v_cache):
+        if t is not None and (t.shape != k_cache.shape or t.stride() != k_cache.stride() or t.stride(2) != 1):
+            raise ValueError("k_cache and v_cache must be [planes, rows, head_dim] with the same strides, rows contiguous")
+    e = k_cache.element_size()
+    p = KvCommitParams()
+    p.num_planes, p.row_bytes, p.prefix_len, p.n_tree = planes, d * e, prefix_len, n_tree
+    p.k_cache, p.v_cache = _dev(k_cache, "k_cache"), _dev(v_cache, "v_cache")
+    p.plane_stride_bytes = (k_cache.stride(0) if planes > 1 else rows * k_cache.stride(1)) * e
+    p.row_stride_bytes = k_cache.stride(1) * e
+    p.path, p.path_len = _dev(path, "path", torch.int32), _dev(path_len, "path_len", torch.int32)
+    p.new_prefix_len = _dev(new_prefix_len, "new_prefix_len", torch.int32)
+    p.dev_status = _dev(dev_status, "dev_status", torch.int32)
+    _check("seq_tree_kv_commit", load().seq_tree_kv_commit(C.byref(p), _stream(stream)))
 
 
 class HostStep:

@@ -57,6 +57,9 @@ CONFIGS = {
     ]
 }
 
+# decoder layers of the models the configs are named after (the whole-model key/value cache has layers x kv heads planes)
+NUM_LAYERS = {"tiny": 2, "llama2-7b": 32, "llama2-13b": 40, "vicuna-33b": 60, "llama3-70b": 80}
+
 TORCH_DTYPES = {"fp16": torch.float16, "bf16": torch.bfloat16, "fp32": torch.float32}
 
 

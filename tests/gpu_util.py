@@ -144,6 +144,19 @@ def check_verify_target_sample(vi: W.VerifyInputs, with_draft=False):
     return "ok"
 
 
+def steer_tokens_to_samples(vi, every=1):
+    """Rewrites the first child's token of every `every`-th internal node to the token the oracle's inverse CDF
+    draws there, so that the walk goes deep; returns the number of nodes steered."""
+    kids = W.children_lists(vi.parent.numpy())
+    steered = 0
+    for v, ch in enumerate(kids):
+        if ch and v % every == 0:
+            P = O.softmax_T(vi.target_logits[v], vi.temperature)
+            vi.tokens[ch[0]] = O.sample_inverse_cdf(P, float(vi.uniforms[v]))
+            steered += 1
+    return steered
+
+
 def check_verify_all_nodes(vi: W.VerifyInputs):
     """SEQ_VERIFY_ALL_NODES: every internal node's accept/reject loop against Algorithm 2 run by the
     oracle on that node's two distributions."""

@@ -44,12 +44,16 @@ def test_ctypes_structs_match_the_header(tmp_path):
 
     fields_a = [f[0] for f in binding.AttentionParams._fields_]
     fields_v = [f[0] for f in binding.VerifyParams._fields_]
+    others = (("seq_tree_draft_sample_params", binding.DraftSampleParams), ("seq_tree_kv_commit_params", binding.KvCommitParams))
     src = tmp_path / "layout.c"
     lines = ['#include <stdio.h>', '#include <stddef.h>', '#include "seq_tree.h"', "int main(void){",
              'printf("%zu\\n", sizeof(seq_tree_attention_params));']
     lines += [f'printf("%zu\\n", offsetof(seq_tree_attention_params, {f}));' for f in fields_a]
     lines += ['printf("%zu\\n", sizeof(seq_tree_verify_params));']
     lines += [f'printf("%zu\\n", offsetof(seq_tree_verify_params, {f}));' for f in fields_v]
+    for cname, st in others:
+        lines += [f'printf("%zu\\n", sizeof({cname}));']
+        lines += [f'printf("%zu\\n", offsetof({cname}, {f[0]}));' for f in st._fields_]
     lines += ["return 0;}"]
     src.write_text("\n".join(lines))
     exe = tmp_path / "layout"
@@ -59,7 +63,14 @@ def test_ctypes_structs_match_the_header(tmp_path):
     assert nums[1:1 + len(fields_a)] == [getattr(binding.AttentionParams, f).offset for f in fields_a]
     rest = nums[1 + len(fields_a):]
     assert rest[0] == C.sizeof(binding.VerifyParams)
-    assert rest[1:] == [getattr(binding.VerifyParams, f).offset for f in fields_v]
+    assert rest[1:1 + len(fields_v)] == [getattr(binding.VerifyParams, f).offset for f in fields_v]
+    rest = rest[1 + len(fields_v):]
+    for cname, st in others:
+        names = [f[0] for f in st._fields_]
+        assert rest[0] == C.sizeof(st), cname
+        assert rest[1:1 + len(names)] == [getattr(st, f).offset for f in names], cname
+        rest = rest[1 + len(names):]
+    assert not rest
 
 
 def test_host_checkable_errors_are_refused_before_launch(lib):
@@ -116,6 +127,23 @@ def test_host_checkable_errors_are_refused_before_launch(lib):
     assert lib.seq_tree_verify(C.byref(ver(vocab=400000, target_row_stride=400000, draft_row_stride=400000)), None) \
         == B.SEQ_ERR_UNSUPPORTED
     assert lib.seq_tree_verify_workspace_bytes(C.byref(ver())) == 0
+
+    def commit(**kw):
+        p = B.KvCommitParams()
+        p.num_planes, p.row_bytes, p.prefix_len, p.n_tree = 64, 256, 128, 16
+        p.k_cache = p.v_cache = p.path = p.path_len = fake
+        p.row_stride_bytes, p.plane_stride_bytes = 256, 144 * 256
+        for k, v in kw.items():
+            setattr(p, k, v)
+        return p
+
+    bad = [dict(k_cache=None), dict(path=None), dict(path_len=None), dict(num_planes=0), dict(n_tree=0), dict(n_tree=1025),
+           dict(prefix_len=-1), dict(row_bytes=8), dict(row_bytes=250), dict(row_stride_bytes=128), dict(row_stride_bytes=264),
+           dict(plane_stride_bytes=143 * 256), dict(plane_stride_bytes=144 * 256 + 8), dict(k_cache=fake + 4),
+           dict(v_cache=fake + 8)]
+    for kw in bad:
+        assert lib.seq_tree_kv_commit(C.byref(commit(**kw)), None) == B.SEQ_ERR_INVALID_ARG, kw
+    assert lib.seq_tree_kv_commit(None, None) == B.SEQ_ERR_INVALID_ARG
 
 
 def test_binding_refuses_cpu_tensors():

@@ -245,19 +245,6 @@ def test_verify_target_sample_configs(name, T, seeds):
     assert outcomes.count("ok") >= max(1, len(outcomes) - 1), outcomes
 
 
-def _steer_tokens_to_samples(vi, every=1):
-    """Rewrites the first child's token of every `every`-th internal node to the token the oracle's inverse CDF
-    draws there, so that the walk goes deep; returns the number of nodes steered."""
-    kids = W.children_lists(vi.parent.numpy())
-    steered = 0
-    for v, ch in enumerate(kids):
-        if ch and v % every == 0:
-            P = O.softmax_T(vi.target_logits[v], vi.temperature)
-            vi.tokens[ch[0]] = O.sample_inverse_cdf(P, float(vi.uniforms[v]))
-            steered += 1
-    return steered
-
-
 @pytest.mark.parametrize("name,T,vocab", [("tiny", 0.6, None), ("llama2-7b", 1.0, None), ("llama2-7b", 0.3, 5003)])
 def test_verify_target_sample_deep_walks(name, T, vocab):
     """Children carrying exactly the token that is drawn at their parent: the walk follows them to a leaf, one
@@ -266,7 +253,7 @@ def test_verify_target_sample_deep_walks(name, T, vocab):
     ok = 0
     for seed in range(3):
         vi = W.make_verify_inputs(cfg, T, seed, vocab=vocab)
-        assert _steer_tokens_to_samples(vi) > 1
+        assert G.steer_tokens_to_samples(vi) > 1
         ref = O.tree_verify_target_sample(vi.parent, vi.tokens, vi.target_logits, vi.temperature, vi.uniforms)
         assert ref["path_len"] >= 3  # the steering worked: root, its first child, that child's first child ...
         ok += G.check_verify_target_sample(vi, with_draft=(seed == 1)) == "ok"
