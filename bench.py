@@ -129,10 +129,20 @@ def n_sets(bytes_per_set: int, lo: int = 2, hi: int = 48) -> int:
     return max(lo, min(hi, math.ceil(3 * L2_BYTES / max(1, bytes_per_set))))
 
 
-def build_requests(cfg, T, rank, n_attn, n_verify):
-    """Host-side inputs for this rank: n_attn attention sets and n_verify logit sets (seeds differ by rank)."""
+def build_requests(cfg, T, rank, n_attn, n_verify, tree="random", parent=None):
+    """Host-side inputs for this rank: n_attn attention sets and n_verify logit sets (seeds differ by rank).
+    tree = "dp": the tree comes from the library's own construction (seq_tree_build, a host call) on the
+    acceptance vector the paper prints, within the config's size, depth and fan-out bounds."""
     base = rank_seed_base(rank)
-    parent = W.make_tree(cfg, base)
+    if parent is not None:
+        pass
+    elif tree == "dp":
+        from paper_2402_12374_b200 import binding as B
+
+        parent, _ = B.seq_tree_build(W.PAPER_ACCEPTANCE_VECTOR, cfg.n_tree, cfg.max_depth, cfg.max_fanout or 31)
+        assert len(parent) == cfg.n_tree
+    else:
+        parent = W.make_tree(cfg, base)
     attn = [W.make_attention_inputs(cfg, base + s, parent=parent) for s in range(n_attn)]
     ver = [W.make_verify_inputs(cfg, T, base + s, parent=parent) for s in range(n_verify)]
     return parent, attn, ver
@@ -166,7 +176,12 @@ def run_reference(args, cfg, T):
         return
     from oracle import oracle as O
 
-    parent, attn, ver = build_requests(cfg, T, 0, 1, 1)
+    parent = None
+    if args.tree == "dp":  # this arm runs none of the library: the oracle's own statement of the dynamic program
+        from oracle import tree_dp
+
+        parent, _ = tree_dp.build_tree(W.PAPER_ACCEPTANCE_VECTOR, cfg.n_tree, cfg.max_depth, cfg.max_fanout or 31)
+    parent, attn, ver = build_requests(cfg, T, 0, 1, 1, parent=parent)
     for _ in range(min(args.warmup, 2)):
         oracle_step_sample(cfg, parent, attn[0], ver[0], T)
     steps = min(args.steps, 20)
@@ -273,13 +288,26 @@ def kv_commit_leg(cfg, parent, dev, stream, peaks) -> dict:
         stream.synchronize()
         g.replay()
         stream.synchronize()
+        # and back to back, the rows still in L2 from the call before (the device clock ticks coarsely: means, not medians)
+        gw = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(gw, stream=stream):
+            for i in range(2 * reps):
+                B.seq_tree_kv_commit(k, v, L, n, path_d, plen, dev_status=status, stream=stream)
+        gw.replay()
+        stream.synchronize()
+        w0, w1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        w0.record(stream)
+        gw.replay()
+        w1.record(stream)
+        stream.synchronize()
     if int(status.item()) != 0:
         raise RuntimeError(f"kv_commit dev_status = {int(status.item())}")
-    us = float(np.median([a.elapsed_time(b) * 1e3 for a, b in evs]))
+    us = float(np.mean([a.elapsed_time(b) * 1e3 for a, b in evs]))
+    us_warm = w0.elapsed_time(w1) * 1e3 / (2 * reps)
     moved = sum(int(p != i) for i, p in enumerate(path))
     nbytes = 2 * 2 * planes * moved * cfg.head_dim * k.element_size()
     gbs = nbytes / (us * 1e-6) / 1e9
-    return {"us_per_call": us, "layers": layers, "planes": planes, "path_len": len(path), "rows_moved": moved,
+    return {"us_per_call": us, "us_per_call_l2_warm": us_warm, "layers": layers, "planes": planes, "path_len": len(path), "rows_moved": moved,
             "gpu_launches_per_call": 1, "l2": "flushed before every call",
             "roofline": {"bound": "hbm", "achieved": gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s",
                          "frac": gbs / peaks["hbm_gbs"], "algorithmic_bytes": nbytes, "traffic": None},
@@ -296,6 +324,8 @@ def main():
     ap.add_argument("--temperature", type=float, default=0.6)
     ap.add_argument("--kernel", type=int, default=0, help="0 auto, 1 CUDA-core, 2 tensor-core attention")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--tree", default="random", choices=["random", "dp"],
+                    help="random: seeded random tree within the config's bounds; dp: Sequoia's dynamic program on the paper's acceptance vector")
     ap.add_argument("--separate-mask", action="store_true",
                     help="build the ancestor mask with a launch of its own instead of inside the attention kernel")
     args = ap.parse_args()
@@ -326,7 +356,7 @@ def main():
     logits_bytes_touched = 4 * 2 * cfg.vocab * 4  # a walk reads a few rows of each matrix
     na = n_sets(attn_bytes)
     nv = min(n_sets(logits_bytes_touched), 8 if cfg.vocab * n * 8 < (1 << 28) else 3)
-    parent, attn_h, ver_h = build_requests(cfg, T, rank, na, nv)
+    parent, attn_h, ver_h = build_requests(cfg, T, rank, na, nv, args.tree)
 
     status = torch.zeros(1, dtype=torch.int32, device=dev)
     parent_d = torch.from_numpy(parent).to(dev)
@@ -479,7 +509,9 @@ def main():
                    "heads": f"{cfg.num_q_heads}/{cfg.num_kv_heads}", "vocab": cfg.vocab, "requests_per_gpu": 1,
                    "l2": f"inputs rotate over {na} attention sets ({na * attn_bytes >> 20} MiB) and {nv} logit sets, "
                          f"larger than the 126 MiB L2", "launch": "CUDA graph of the K steps",
-                   "mask": "from the parent array inside the attention kernel" if fused_mask else "separate launch"},
+                   "mask": "from the parent array inside the attention kernel" if fused_mask else "separate launch",
+                   "tree": "seeded random within the config's depth and fan-out bounds" if args.tree == "random"
+                           else "seq_tree_build on the paper's printed acceptance vector"},
         "clocks": clocks.summary(),
         "e2e": {"value": e2e_us, "unit": UNIT, "h2d_bytes_per_step": host.h2d_bytes, "d2h_bytes_per_step": host.d2h_bytes,
                 "steps": Ke},

@@ -338,6 +338,49 @@ typedef struct {
 
 int seq_tree_kv_commit(const seq_tree_kv_commit_params* p, void* stream);
 
+/* ---------------------------------------------------------------------------
+ * seq_tree_build -- Sequoia's tree construction (Section 3.1: score function, F(tree) = sum of the nodes' scores,
+ * Algorithm 1; appendix "Dynamic programming details": the bound on the depth and one acceptance vector per
+ * depth).  HOST function, all pointers are host memory; it launches nothing.  Run once, offline: the tree is
+ * then fixed for the whole run.
+ *
+ * Finds a tree with at most max_size nodes, depth (in edges) <= max_depth and at most max_branch children per
+ * node that maximises the expected number of generated tokens F under positional acceptance:
+ *   acc_rates   [acc_rows][max_branch] doubles in [0, 1]; entry [r][b-1] = probability that the b-th child of a
+ *               node at depth r is accepted, given that the node was reached and its earlier children were
+ *               rejected.  acc_rows == 1: the same vector at every depth; else acc_rows >= max_depth.
+ *   parent_out  [max_size] int32: the tree in level order (parent[0] = -1, parent[i] < i, siblings contiguous
+ *               and in rank order), the numbering every other call of this library expects.
+ *   size_out    number of nodes of the tree (max_size unless the bounds admit fewer).
+ *   expected_out nullable: F of the returned tree.  Several trees can attain it; only F is unique.
+ *   table_out   nullable, [(max_size+1)][(max_depth+1)] doubles: entry [n][d] = G(n, d), the largest F over trees
+ *               of exactly n nodes and depth <= d; -inf where no such tree exists (and in row 0).  With
+ *               acc_rows > 1 column d < max_depth holds the value of the best subtree hanging at depth
+ *               max_depth - d instead (only the last column is a whole tree's value).
+ * Cost: O(max_size^2 * max_depth * max_branch) time.  Returns SEQ_OK, SEQ_ERR_INVALID_ARG (null pointer, size
+ * out of range, max_size above SEQ_MAX_TREE, a rate outside [0, 1] or NaN) or SEQ_ERR_UNSUPPORTED (tables above
+ * 10^8 entries). */
+typedef struct {
+  int32_t max_size, max_depth, max_branch, acc_rows;
+  const double* acc_rates;
+  int32_t* parent_out;
+  int32_t* size_out;
+  double* expected_out;
+  double* table_out;
+} seq_tree_build_params;
+
+int seq_tree_build(const seq_tree_build_params* p);
+
+/* seq_tree_speedup_search -- the hardware-aware choice of the tree's size and depth (Section 4.1): maximises
+ * Speedup(n, d) = G(n, d) / (t(n) + d * c) over 1 <= n <= max_size, 0 <= d <= max_depth.  HOST function.
+ *   table    [(max_size+1)][(max_depth+1)] as seq_tree_build writes it (-inf entries are skipped);
+ *   t_of_n   [max_size+1]: time for the target model to verify n tokens / time to verify one (entry 0 unused),
+ *            all > 0, measured by the caller on its hardware;  c: time to draft one token / time to verify one.
+ * Ties go to the smaller n, then the smaller d.  speedup_out is nullable.  Returns SEQ_OK or
+ * SEQ_ERR_INVALID_ARG. */
+int seq_tree_speedup_search(const double* table, int32_t max_size, int32_t max_depth, const double* t_of_n, double c,
+                            int32_t* n_out, int32_t* d_out, double* speedup_out);
+
 const char* seq_tree_version(void);
 
 #ifdef __cplusplus

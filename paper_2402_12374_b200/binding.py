@@ -39,6 +39,8 @@ EXPORTED_SYMBOLS = (
     "seq_tree_draft_sample_workspace_bytes",
     "seq_tree_draft_sample",
     "seq_tree_kv_commit",
+    "seq_tree_build",
+    "seq_tree_speedup_search",
     "seq_tree_version",
 )
 
@@ -109,6 +111,11 @@ def load() -> C.CDLL:
         lib.seq_tree_verify.restype = C.c_int
         lib.seq_tree_kv_commit.argtypes = [C.POINTER(KvCommitParams), C.c_void_p]
         lib.seq_tree_kv_commit.restype = C.c_int
+        lib.seq_tree_build.argtypes = [C.POINTER(TreeBuildParams)]
+        lib.seq_tree_build.restype = C.c_int
+        lib.seq_tree_speedup_search.argtypes = [C.c_void_p, C.c_int32, C.c_int32, C.c_void_p, C.c_double, C.POINTER(C.c_int32),
+                                                C.POINTER(C.c_int32), C.POINTER(C.c_double)]
+        lib.seq_tree_speedup_search.restype = C.c_int
         lib.seq_tree_version.restype = C.c_char_p
         _lib = lib
     return _lib
@@ -319,6 +326,52 @@ def seq_tree_verify(parent, tokens, target_logits, draft_logits, temperature: fl
     """Algorithm 2 walked from the root; returns device tensors (path [n], path_len [1], bonus_token [1])."""
     stream = kw.pop("stream", None)
     return VerifyCall(parent, tokens, target_logits, draft_logits, temperature, uniforms, **kw).run(stream)
+
+
+class TreeBuildParams(C.Structure):
+    _fields_ = [
+        ("max_size", C.c_int32), ("max_depth", C.c_int32), ("max_branch", C.c_int32), ("acc_rows", C.c_int32),
+        ("acc_rates", C.c_void_p), ("parent_out", C.c_void_p), ("size_out", C.c_void_p), ("expected_out", C.c_void_p),
+        ("table_out", C.c_void_p),
+    ]
+
+
+def seq_tree_build(acc_rates, max_size: int, max_depth: int, max_branch: int | None = None, *, want_table: bool = False):
+    """Host call: Sequoia's dynamic program.  acc_rates: [B] or [rows][B] array-like of acceptance probabilities.
+    Returns (parent int32 numpy array in level order, F) or (parent, F, table [max_size+1][max_depth+1])."""
+    import numpy as np
+
+    rates = np.ascontiguousarray(np.atleast_2d(np.asarray(acc_rates, dtype=np.float64)))
+    B = max_branch if max_branch is not None else rates.shape[1]
+    if B > rates.shape[1]:
+        raise ValueError("max_branch exceeds the number of acceptance rates per row")
+    rates = np.ascontiguousarray(rates[:, :B])
+    parent = np.empty(max(max_size, 1), dtype=np.int32)
+    size, F = C.c_int32(0), C.c_double(0.0)
+    table = np.empty((max_size + 1, max_depth + 1), dtype=np.float64) if want_table else None
+    p = TreeBuildParams()
+    p.max_size, p.max_depth, p.max_branch, p.acc_rows = max_size, max_depth, B, rates.shape[0]
+    p.acc_rates, p.parent_out = rates.ctypes.data, parent.ctypes.data
+    p.size_out, p.expected_out = C.addressof(size), C.addressof(F)
+    p.table_out = table.ctypes.data if want_table else None
+    _check("seq_tree_build", load().seq_tree_build(C.byref(p)))
+    out = (parent[: size.value].copy(), float(F.value))
+    return out + (table,) if want_table else out
+
+
+def seq_tree_speedup_search(table, t_of_n, c: float):
+    """Host call: (n, d, speedup) maximising G(n, d) / (t(n) + d c)."""
+    import numpy as np
+
+    table = np.ascontiguousarray(table, dtype=np.float64)
+    t = np.ascontiguousarray(t_of_n, dtype=np.float64)
+    if t.shape[0] != table.shape[0]:
+        raise ValueError("t_of_n needs one entry per row of the table (entry 0 unused)")
+    n, d, s = C.c_int32(0), C.c_int32(0), C.c_double(0.0)
+    _check("seq_tree_speedup_search",
+           load().seq_tree_speedup_search(table.ctypes.data, table.shape[0] - 1, table.shape[1] - 1, t.ctypes.data, float(c),
+                                          C.byref(n), C.byref(d), C.byref(s)))
+    return int(n.value), int(d.value), float(s.value)
 
 
 def seq_tree_kv_commit(k_cache, v_cache, prefix_len: int, n_tree: int, path, path_len, *, new_prefix_len=None,

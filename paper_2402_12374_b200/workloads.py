@@ -60,6 +60,15 @@ CONFIGS = {
 # decoder layers of the models the configs are named after (the whole-model key/value cache has layers x kv heads planes)
 NUM_LAYERS = {"tiny": 2, "llama2-7b": 32, "llama2-13b": 40, "vicuna-33b": 60, "llama3-70b": 80}
 
+# Acceptance-rate vector the paper prints (appendix "Examples of Sequoia trees": target Llama3-70B-Instruct, draft
+# Llama3-8B-Instruct, CNN daily news): entry b-1 = probability that a node's b-th child is accepted.  Input data for
+# the tree construction; nothing here computes with it.
+PAPER_ACCEPTANCE_VECTOR = (
+    0.7732, 0.1039, 0.0402, 0.0206, 0.0128, 0.0081, 0.0064, 0.0043, 0.0035, 0.0026, 0.0025, 0.0021, 0.0016, 0.0014,
+    0.0010, 0.0010, 0.0010, 0.0007, 0.0007, 0.0006, 0.0007, 0.0006, 0.0004, 0.0004, 0.0005, 0.0006, 0.0004, 0.0003,
+    0.0002, 0.0004, 0.0001,
+)
+
 TORCH_DTYPES = {"fp16": torch.float16, "bf16": torch.bfloat16, "fp32": torch.float32}
 
 

@@ -427,3 +427,49 @@ def test_attention_full_size_configs_sampled_rows(name, rows):
     cfg = W.CONFIGS[name]
     ai = W.make_attention_inputs(cfg, 0)
     G.check_attention(ai, rows=rows)
+
+
+# ---------------------------------------------------------------- trees from the dynamic program ----
+def _dp_parent(cfg):
+    parent, _ = B.seq_tree_build(W.PAPER_ACCEPTANCE_VECTOR, cfg.n_tree, cfg.max_depth, cfg.max_fanout or 31)
+    assert len(parent) == cfg.n_tree
+    return parent
+
+
+@pytest.mark.parametrize("name", ["tiny", "llama2-7b", "llama2-13b", "vicuna-33b"])
+def test_attention_on_dp_shaped_trees(name):
+    """Trees from seq_tree_build on the paper's acceptance vector (wide near the root, long first-child chains):
+    attention with the mask given and with the mask derived in the kernel, against the oracle."""
+    cfg = W.CONFIGS[name]
+    parent = _dp_parent(cfg)
+    ai = W.make_attention_inputs(cfg, 0, parent=parent)
+    G.check_attention(ai)
+    out, _, st = G.run_attention(ai)
+    d = G.dev()
+    fused = B.seq_tree_attention(ai.q.to(d), ai.k_cache.to(d), ai.v_cache.to(d), None, ai.prefix_len,
+                                 parent=ai.parent.to(d))
+    torch.cuda.synchronize()
+    assert st == 0 and torch.equal(fused, out)
+
+
+def test_attention_on_the_768_node_dp_tree_sampled_rows():
+    cfg = W.CONFIGS["llama3-70b"]
+    parent = _dp_parent(cfg)
+    ai = W.make_attention_inputs(cfg, 0, parent=parent)
+    depth = np.zeros(len(parent), int)
+    for i in range(1, len(parent)):
+        depth[i] = depth[parent[i]] + 1
+    rows = [0, 1, 63, 64, 300, 767, int(np.argmax(depth))]
+    G.check_attention(ai, rows=rows)
+
+
+@pytest.mark.parametrize("name,T", [("tiny", 0.6), ("llama2-7b", 0.6), ("llama2-7b", 1.0), ("llama2-13b", 1.0), ("llama3-70b", 0.6)])
+def test_verify_on_dp_shaped_trees(name, T):
+    cfg = W.CONFIGS[name]
+    parent = _dp_parent(cfg)
+    outcomes = []
+    for seed in range(3 if cfg.vocab < 100000 else 1):
+        vi = W.make_verify_inputs(cfg, T, seed, parent=parent)
+        outcomes.append(G.check_verify(vi))
+        outcomes.append(G.check_verify_target_sample(vi))
+    assert outcomes.count("ok") >= len(outcomes) - 1, outcomes
