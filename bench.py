@@ -314,6 +314,82 @@ def kv_commit_leg(cfg, parent, dev, stream, peaks) -> dict:
             "note": "moved rows of every plane read and written once; latency-bound at this size; outside the timed step"}
 
 
+def tree_search_leg(cfg, T, dev, stream) -> dict:
+    """Not part of the timed step: t(n) of this library's verify step (attention + verification; NOT a whole model
+    forward, which a caller measures for itself) on trees from seq_tree_build of growing size, and the
+    Speedup(n, d) = G(n, d) / (t(n) + d c) search of Section 4.1 on it for two draft costs c.  Inputs are drawn on
+    the device; each size is timed as a CUDA graph of calls rotating over sets larger than L2."""
+    from paper_2402_12374_b200 import binding as B
+
+    Bmax = cfg.max_fanout or 31
+    N, Dmax = cfg.n_tree, cfg.max_depth
+    sizes = sorted({n for n in (1, 4, 16, 32, 64, 128, 256, 512, 768, 1024) if n < N} | {N})
+    dt = W.TORCH_DTYPES[cfg.dtype]
+    gen = torch.Generator(device=dev)
+    gen.manual_seed(7)
+    V = cfg.vocab
+    status = torch.zeros(1, dtype=torch.int32, device=dev)
+    times = {}
+    for n in sizes:
+        parent, _ = B.seq_tree_build(W.PAPER_ACCEPTANCE_VECTOR, n, Dmax, Bmax)
+        n = len(parent)
+        kv_bytes = 2 * cfg.num_kv_heads * (cfg.prefix_len + n) * cfg.head_dim * 2
+        sets = max(2, min(16, math.ceil(2 * L2_BYTES / kv_bytes)))
+        parent_d = torch.from_numpy(parent).to(dev)
+        kids = W.children_lists(parent)
+        calls = []
+        for s in range(sets):
+            q = torch.randn((n, cfg.num_q_heads, cfg.head_dim), device=dev, generator=gen).to(dt)
+            k = torch.randn((cfg.num_kv_heads, cfg.prefix_len + n, cfg.head_dim), device=dev, generator=gen).to(dt)
+            v_ = torch.randn((cfg.num_kv_heads, cfg.prefix_len + n, cfg.head_dim), device=dev, generator=gen).to(dt)
+            tl = 3.0 * torch.randn((n, V), device=dev, generator=gen)
+            dl = tl + torch.randn((n, V), device=dev, generator=gen)
+            u = torch.rand(n + 1, device=dev, generator=gen)
+            # children = the first draws without replacement from the draft's distribution (Gumbel top-k), as in the
+            # host-side recipe of the timed step
+            tokens = torch.zeros(n, dtype=torch.int32, device=dev)
+            for node, ch in enumerate(kids):
+                if ch:
+                    gum = -torch.log(-torch.log(torch.rand(V, device=dev, generator=gen).clamp_(1e-9, 1 - 1e-7)))
+                    tokens[ch] = torch.topk(dl[node] / T + gum, len(ch)).indices.to(torch.int32)
+            calls.append((B.AttentionCall(q, k, v_, None, cfg.prefix_len, parent=parent_d, dev_status=status),
+                          B.VerifyCall(parent_d, tokens, tl, dl, T, u, dev_status=status)))
+        reps = 4 * sets
+        with torch.cuda.stream(stream):
+            for a, vcall in calls[:2]:
+                a.run(stream)
+                vcall.run(stream)
+            stream.synchronize()
+            g = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(g, stream=stream):
+                for i in range(reps):
+                    calls[i % sets][0].run(stream)
+                    calls[i % sets][1].run(stream)
+            g.replay()
+            stream.synchronize()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record(stream)
+            g.replay()
+            e1.record(stream)
+            stream.synchronize()
+        times[n] = e0.elapsed_time(e1) * 1e3 / reps
+        del calls
+    if int(status.item()) != 0:
+        raise RuntimeError(f"tree_search dev_status = {int(status.item())}")
+    ns = sorted(times)
+    t_of_n = np.interp(np.arange(N + 1), ns, [times[n] / times[1] for n in ns])
+    t_of_n[0] = 1.0
+    _, _, table = B.seq_tree_build(W.PAPER_ACCEPTANCE_VECTOR, N, Dmax, Bmax, want_table=True)
+    chosen = {}
+    for c in (0.02, 0.2):
+        n_s, d_s, s = B.seq_tree_speedup_search(table, t_of_n, c)
+        chosen[f"c={c}"] = {"n": n_s, "d": d_s, "speedup": s, "G": float(table[n_s, d_s])}
+    return {"us_per_step_by_tree_size": {str(n): times[n] for n in ns}, "t_of_n": {str(n): times[n] / times[1] for n in ns},
+            "bounds": {"max_size": N, "max_depth": Dmax, "max_branch": Bmax}, "speedup_search": chosen,
+            "note": "t(n) of attention + verification only, sizes in between interpolated; acceptance vector: the one the "
+                    "paper prints; outside the timed step"}
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -326,6 +402,8 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--tree", default="random", choices=["random", "dp"],
                     help="random: seeded random tree within the config's bounds; dp: Sequoia's dynamic program on the paper's acceptance vector")
+    ap.add_argument("--tree-search", action="store_true",
+                    help="also time the step on trees of growing size and run the Speedup(n, d) search on that t(n)")
     ap.add_argument("--separate-mask", action="store_true",
                     help="build the ancestor mask with a launch of its own instead of inside the attention kernel")
     args = ap.parse_args()
@@ -522,6 +600,8 @@ def main():
                          "largest_share": "seq_tree_verify" if ver_us > attn_us else "seq_tree_attention"},
     }
     line["next_rows"] = {"kv_commit": kv_commit_leg(cfg, parent, dev, stream, peaks)}
+    if T > 0 and args.tree_search:
+        line["next_rows"]["tree_search"] = tree_search_leg(cfg, T, dev, stream)
     if T > 0:
         line["next_rows"]["draft_sample"] = draft_sample_leg(cfg, parent, ver_h, T, dev, stream, peaks)
     if not args.no_cpu_baseline:
