@@ -66,6 +66,8 @@ def lib():
         L.orc_tree_verify.argtypes = [i32, i32, pi32, pi32, pf32, i64, pf32, i64, f64, pf32, i32,
                                       pi32, pi32, pi32, pf64, pi32, pf64, pf64]
         L.orc_tree_verify_target_sample.argtypes = [i32, i32, pi32, pi32, pf32, i64, f64, pf32, pi32, pi32, pi32, pf64, pi32, pf64]
+        L.orc_top_p.argtypes = [pf32, i32, f64, f64, C.c_void_p, pf64, pi32]
+        L.orc_top_p.restype = i32
         L.orc_kv_commit.argtypes = [C.c_void_p, C.c_void_p, i64, i64, i64, i32, i32, pi32, i32]
         L.orc_alg3_chain.argtypes = [pf64, pf64, i32, i32, pi32, pf64, f64, pi32]
         L.orc_alg3_chain.restype = i32
@@ -224,3 +226,16 @@ def kv_commit(cache, prefix_len: int, n_tree: int, path):
     flags = lib().orc_kv_commit(cache.ctypes.data, out.ctypes.data, planes, rows, d * cache.itemsize, prefix_len,
                                 n_tree, _p(path, C.c_int32), path.shape[0])
     return out, int(flags)
+
+
+def top_p(logits, T: float, top_p: float) -> dict:
+    """Nucleus truncation of softmax(logits/T): keep mask [V] (bool), the filtered logits (-inf outside), the
+    closeness of the decision and the flags."""
+    logits = _f32(logits)
+    V = logits.shape[0]
+    keep = np.zeros(V, dtype=np.uint8)
+    gap, flags = C.c_double(0.0), C.c_int32(0)
+    kept = lib().orc_top_p(_p(logits, C.c_float), V, float(T), float(top_p), keep.ctypes.data, C.byref(gap), C.byref(flags))
+    keep = keep.astype(bool)
+    return dict(keep=keep, kept=int(kept), filtered=np.where(keep, logits, np.float32(-np.inf)), min_gap=float(gap.value),
+                flags=int(flags.value))

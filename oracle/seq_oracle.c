@@ -14,7 +14,8 @@
  *   - the draft side's draw of a node's children without replacement by
  *     exponential sort (Section 5, "Implementation Details");
  *   - verification by sampling from the target (Section 2.2, naive / top-k
- *     sampling), and the commit of an accepted path into the cache.
+ *     sampling), the commit of an accepted path into the cache, and the nucleus
+ *     (top-p) truncation of a distribution (Section 4.2's robustness study).
  *
  * Nothing here is blocked, fused or reordered: every function is the
  * definition, or the algorithm's steps in the paper's order and notation, so
@@ -33,7 +34,8 @@
  * (Monte-Carlo), library sorts in its two degenerate cases, and invariants;
  * the commit against a library gather, hand-written cases where a row is both
  * read and overwritten, and the identity "attention of a path node over the
- * tree == causal attention over the committed cache".
+ * tree == causal attention over the committed cache"; the nucleus against the
+ * three properties that characterise it, a library sort + cumsum, closed forms.
  *
  * Build: gcc -O2 -fopenmp -shared -fPIC seq_oracle.c -o liboracle.so -lm
  */
@@ -567,4 +569,83 @@ int32_t orc_kv_commit(const uint8_t* in, uint8_t* out, int64_t planes, int64_t r
       memcpy(out + ((size_t)h * rows + (size_t)(L + i)) * row_bytes,
              in + ((size_t)h * rows + (size_t)(L + path[i])) * row_bytes, (size_t)row_bytes);
   return 0;
+}
+
+/*
+ * Nucleus ("top-p") truncation of a distribution: the hyperparameter of the
+ * robustness study (Section 4.2, table "robustness to the top-p
+ * hyperparameter").  The paper names the hyperparameter only; the operation is
+ * taken as the usual one: with p = softmax(logits / T), order the tokens by
+ * decreasing probability (equal probabilities in token order) and keep the
+ * shortest prefix of that order whose probabilities add up to at least top_p;
+ * every other token gets probability 0 (logit -inf), and the survivors are
+ * renormalised by whoever takes the softmax next.  top_p >= 1 keeps every
+ * token.  At least one token is always kept.
+ *
+ *   keep [V]: 1 for tokens inside the nucleus, else 0.  Returns their number.
+ *   min_gap (nullable): how close the decision was -- the smaller of
+ *       (cumulative mass up to and including the last kept token) - top_p and
+ *       top_p - (the same without it), and, as a relative figure, of the
+ *       difference between the last kept and the first dropped probability
+ *       over the former.  A lower-precision computation may differ only when
+ *       this is small.
+ * A NaN or +inf logit counts as -inf (never kept) and raises ORC_NONFINITE in
+ * *flags (nullable).
+ */
+typedef struct {
+  double p;
+  int32_t t;
+} orc_pt;
+
+static int orc_pt_desc(const void* a, const void* b) {
+  const orc_pt *x = (const orc_pt*)a, *y = (const orc_pt*)b;
+  if (x->p > y->p) return -1;
+  if (x->p < y->p) return 1;
+  return x->t < y->t ? -1 : (x->t > y->t ? 1 : 0);
+}
+
+int32_t orc_top_p(const float* logits, int32_t V, double T, double top_p, uint8_t* keep,
+                  double* min_gap, int32_t* flags) {
+  float* clean = (float*)malloc(sizeof(float) * (size_t)V);
+  double* p = (double*)malloc(sizeof(double) * (size_t)V);
+  orc_pt* order = (orc_pt*)malloc(sizeof(orc_pt) * (size_t)V);
+  int32_t fl = 0;
+  for (int32_t t = 0; t < V; ++t) {
+    clean[t] = logits[t];
+    if (isnan(logits[t]) || (isinf(logits[t]) && logits[t] > 0)) {
+      clean[t] = -INFINITY;
+      fl |= ORC_NONFINITE;
+    }
+  }
+  orc_softmax_T(clean, V, T, p);
+  for (int32_t t = 0; t < V; ++t) {
+    order[t].p = p[t];
+    order[t].t = t;
+    keep[t] = 0;
+  }
+  qsort(order, (size_t)V, sizeof(orc_pt), orc_pt_desc);
+  int32_t kept = 0;
+  double cum = 0.0, gap = INFINITY;
+  if (top_p >= 1.0) {
+    for (int32_t t = 0; t < V; ++t) keep[t] = 1;
+    kept = V;
+  } else {
+    for (int32_t i = 0; i < V; ++i) {
+      double before = cum;
+      cum += order[i].p;
+      keep[order[i].t] = 1;
+      ++kept;
+      if (cum >= top_p) {
+        gap = fmin(cum - top_p, top_p - before);
+        if (i + 1 < V && order[i].p > 0.0) gap = fmin(gap, (order[i].p - order[i + 1].p) / order[i].p);
+        break;
+      }
+    }
+  }
+  if (min_gap) *min_gap = gap;
+  if (flags) *flags = fl;
+  free(clean);
+  free(p);
+  free(order);
+  return kept;
 }
