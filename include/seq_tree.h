@@ -381,6 +381,37 @@ int seq_tree_build(const seq_tree_build_params* p);
 int seq_tree_speedup_search(const double* table, int32_t max_size, int32_t max_depth, const double* t_of_n, double c,
                             int32_t* n_out, int32_t* d_out, double* speedup_out);
 
+/* ---------------------------------------------------------------------------
+ * seq_tree_top_p_filter -- nucleus ("top-p") truncation of softmax(logits / T), row by row: the top-p
+ * hyperparameter of the robustness study (Section 4.2, table "robustness to the top-p hyperparameter"; the paper
+ * names the hyperparameter only, the operation is the usual one).  Per row, with p = softmax(logits / T): order
+ * the tokens by decreasing p (equal logits in token order) and keep the shortest prefix whose probabilities add
+ * up to at least top_p; out[t] = logits[t] for kept tokens (the same bits), -inf for the others, so that a later
+ * softmax renormalises over the nucleus.  Apply it to the target rows before seq_tree_verify (the output law is
+ * then the truncated target distribution, whatever the draft) and/or to draft rows before seq_tree_draft_sample.
+ *
+ *   logits, out   device fp32 [n_rows][vocab], rows 16-byte aligned (strides in elements, multiples of 4, >= vocab);
+ *                 out may be the same buffer as logits (in place), else the two must not overlap.
+ *   temperature   > 0, finite;  top_p > 0 (top_p >= 1: every token is kept, rows are copied unchanged).
+ *   kept_out      device, nullable, [n_rows]: the nucleus size of each row.
+ * At least one token is kept.  A NaN or +inf logit raises SEQ_DEV_NONFINITE, counts as -inf and comes out as
+ * -inf; a row of -inf only raises SEQ_DEV_DEGENERATE and stays -inf (kept 0).  The decision is taken on exact
+ * fixed-point sums of fp32 exponentials: it can differ from an exact computation only where the cumulative mass
+ * passes top_p within about 1e-6.  Deterministic.  No workspace.  Asynchronous on `stream`; capturable.  Returns
+ * SEQ_OK, SEQ_ERR_INVALID_ARG or SEQ_ERR_CUDA. */
+typedef struct {
+  int32_t n_rows, vocab;
+  const float* logits;
+  int64_t logits_row_stride;
+  float* out;
+  int64_t out_row_stride;
+  float temperature, top_p;
+  int32_t* kept_out;
+  int32_t* dev_status;
+} seq_tree_top_p_params;
+
+int seq_tree_top_p_filter(const seq_tree_top_p_params* p, void* stream);
+
 const char* seq_tree_version(void);
 
 #ifdef __cplusplus

@@ -229,13 +229,13 @@ def kv_commit(cache, prefix_len: int, n_tree: int, path):
 
 
 def top_p(logits, T: float, top_p: float) -> dict:
-    """Nucleus truncation of softmax(logits/T): keep mask [V] (bool), the filtered logits (-inf outside), the
-    closeness of the decision and the flags."""
+    """Nucleus truncation of softmax(logits/T): keep mask [V] (bool), the filtered logits (-inf outside), the two
+    margins of the decision (mass above top_p with the last kept token, mass below it without) and the flags."""
     logits = _f32(logits)
     V = logits.shape[0]
     keep = np.zeros(V, dtype=np.uint8)
-    gap, flags = C.c_double(0.0), C.c_int32(0)
-    kept = lib().orc_top_p(_p(logits, C.c_float), V, float(T), float(top_p), keep.ctypes.data, C.byref(gap), C.byref(flags))
+    margins, flags = (C.c_double * 2)(), C.c_int32(0)
+    kept = lib().orc_top_p(_p(logits, C.c_float), V, float(T), float(top_p), keep.ctypes.data, margins, C.byref(flags))
     keep = keep.astype(bool)
-    return dict(keep=keep, kept=int(kept), filtered=np.where(keep, logits, np.float32(-np.inf)), min_gap=float(gap.value),
-                flags=int(flags.value))
+    return dict(keep=keep, kept=int(kept), filtered=np.where(keep, logits, np.float32(-np.inf)), over=float(margins[0]),
+                under=float(margins[1]), min_gap=float(min(margins[0], margins[1])), flags=int(flags.value))

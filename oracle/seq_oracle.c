@@ -583,12 +583,12 @@ int32_t orc_kv_commit(const uint8_t* in, uint8_t* out, int64_t planes, int64_t r
  * token.  At least one token is always kept.
  *
  *   keep [V]: 1 for tokens inside the nucleus, else 0.  Returns their number.
- *   min_gap (nullable): how close the decision was -- the smaller of
- *       (cumulative mass up to and including the last kept token) - top_p and
- *       top_p - (the same without it), and, as a relative figure, of the
- *       difference between the last kept and the first dropped probability
- *       over the former.  A lower-precision computation may differ only when
- *       this is small.
+ *   margins (nullable, [2]): how close the decision was -- [0] = (cumulative
+ *       mass up to and including the last kept token) - top_p, [1] = top_p -
+ *       (the same without that token); both >= 0, +inf when top_p >= 1.  The
+ *       ORDER of the tokens is that of the fp32 logits themselves and leaves
+ *       no room for rounding; a lower-precision computation of the masses can
+ *       move the cut by one token only when one of the two margins is small.
  * A NaN or +inf logit counts as -inf (never kept) and raises ORC_NONFINITE in
  * *flags (nullable).
  */
@@ -605,7 +605,7 @@ static int orc_pt_desc(const void* a, const void* b) {
 }
 
 int32_t orc_top_p(const float* logits, int32_t V, double T, double top_p, uint8_t* keep,
-                  double* min_gap, int32_t* flags) {
+                  double* margins, int32_t* flags) {
   float* clean = (float*)malloc(sizeof(float) * (size_t)V);
   double* p = (double*)malloc(sizeof(double) * (size_t)V);
   orc_pt* order = (orc_pt*)malloc(sizeof(orc_pt) * (size_t)V);
@@ -625,7 +625,7 @@ int32_t orc_top_p(const float* logits, int32_t V, double T, double top_p, uint8_
   }
   qsort(order, (size_t)V, sizeof(orc_pt), orc_pt_desc);
   int32_t kept = 0;
-  double cum = 0.0, gap = INFINITY;
+  double cum = 0.0, over = INFINITY, under = INFINITY;
   if (top_p >= 1.0) {
     for (int32_t t = 0; t < V; ++t) keep[t] = 1;
     kept = V;
@@ -636,13 +636,16 @@ int32_t orc_top_p(const float* logits, int32_t V, double T, double top_p, uint8_
       keep[order[i].t] = 1;
       ++kept;
       if (cum >= top_p) {
-        gap = fmin(cum - top_p, top_p - before);
-        if (i + 1 < V && order[i].p > 0.0) gap = fmin(gap, (order[i].p - order[i + 1].p) / order[i].p);
+        over = cum - top_p;
+        under = top_p - before;
         break;
       }
     }
   }
-  if (min_gap) *min_gap = gap;
+  if (margins) {
+    margins[0] = over;
+    margins[1] = under;
+  }
   if (flags) *flags = fl;
   free(clean);
   free(p);

@@ -39,6 +39,7 @@ EXPORTED_SYMBOLS = (
     "seq_tree_draft_sample_workspace_bytes",
     "seq_tree_draft_sample",
     "seq_tree_kv_commit",
+    "seq_tree_top_p_filter",
     "seq_tree_build",
     "seq_tree_speedup_search",
     "seq_tree_version",
@@ -111,6 +112,8 @@ def load() -> C.CDLL:
         lib.seq_tree_verify.restype = C.c_int
         lib.seq_tree_kv_commit.argtypes = [C.POINTER(KvCommitParams), C.c_void_p]
         lib.seq_tree_kv_commit.restype = C.c_int
+        lib.seq_tree_top_p_filter.argtypes = [C.POINTER(TopPParams), C.c_void_p]
+        lib.seq_tree_top_p_filter.restype = C.c_int
         lib.seq_tree_build.argtypes = [C.POINTER(TreeBuildParams)]
         lib.seq_tree_build.restype = C.c_int
         lib.seq_tree_speedup_search.argtypes = [C.c_void_p, C.c_int32, C.c_int32, C.c_void_p, C.c_double, C.POINTER(C.c_int32),
@@ -326,6 +329,37 @@ def seq_tree_verify(parent, tokens, target_logits, draft_logits, temperature: fl
     """Algorithm 2 walked from the root; returns device tensors (path [n], path_len [1], bonus_token [1])."""
     stream = kw.pop("stream", None)
     return VerifyCall(parent, tokens, target_logits, draft_logits, temperature, uniforms, **kw).run(stream)
+
+
+class TopPParams(C.Structure):
+    _fields_ = [
+        ("n_rows", C.c_int32), ("vocab", C.c_int32),
+        ("logits", C.c_void_p), ("logits_row_stride", C.c_int64),
+        ("out", C.c_void_p), ("out_row_stride", C.c_int64),
+        ("temperature", C.c_float), ("top_p", C.c_float),
+        ("kept_out", C.c_void_p), ("dev_status", C.c_void_p),
+    ]
+
+
+def seq_tree_top_p_filter(logits, temperature: float, top_p: float, *, out=None, kept_out=None, dev_status=None,
+                          stream=None):
+    """Nucleus truncation of softmax(logits / temperature) per row: returns logits with -inf outside the nucleus
+    (``out=logits`` works in place)."""
+    rows, V = logits.shape
+    if out is None:
+        out = torch.empty_like(logits)
+    for t, nm in ((logits, "logits"), (out, "out")):
+        if t.shape != logits.shape or t.stride(1) != 1:
+            raise ValueError(f"{nm} must be [rows, vocab] with contiguous rows")
+    p = TopPParams()
+    p.n_rows, p.vocab = rows, V
+    p.logits, p.logits_row_stride = _dev(logits, "logits", torch.float32), (logits.stride(0) if rows > 1 else (V + 3) // 4 * 4)
+    p.out, p.out_row_stride = _dev(out, "out", torch.float32), (out.stride(0) if rows > 1 else (V + 3) // 4 * 4)
+    p.temperature, p.top_p = temperature, top_p
+    p.kept_out = _dev(kept_out, "kept_out", torch.int32)
+    p.dev_status = _dev(dev_status, "dev_status", torch.int32)
+    _check("seq_tree_top_p_filter", load().seq_tree_top_p_filter(C.byref(p), _stream(stream)))
+    return out
 
 
 class TreeBuildParams(C.Structure):

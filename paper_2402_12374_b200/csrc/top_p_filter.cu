@@ -1,0 +1,274 @@
+// seq_tree_top_p_filter: nucleus truncation of softmax(logits / T), row by row (the top-p hyperparameter of the
+// robustness study, Section 4.2).  One CTA per row.  The nucleus is found by a radix select on the logits' bit
+// patterns (11 + 11 + 10 bits) in which every bin carries the probability MASS of its tokens, as 2^-40 fixed point in
+// 64-bit integers: sums are exact and independent of the order of the atomic adds, so the kept set is reproducible
+// bit for bit.  A row is read five times (maximum, three select levels, the write), once from HBM and then from L2.
+#include <climits>
+
+#include "common.cuh"
+
+namespace seqtree {
+
+constexpr int kTpThreads = 1024;
+constexpr int kTpWarps = kTpThreads / 32;
+constexpr float kTpScale = 1099511627776.f;  // 2^40
+
+struct TopPArgs {
+  const float* logits; int64_t in_stride;
+  float* out; int64_t out_stride;
+  int32_t V;
+  float c2;       // log2(e) / T
+  double top_p;
+  int32_t* kept_out; int32_t* dev_status;
+};
+
+struct TpShared {
+  unsigned long long hist[2048];
+  uint32_t count[1024];
+  unsigned long long warp_tot[kTpWarps];
+  float warp_max[kTpWarps];
+  // results of a level's search
+  uint32_t sel_bin; unsigned long long sel_above; unsigned long long sel_mass; uint32_t sel_count;
+  int32_t tie_limit;
+  int32_t bad, kept;
+};
+
+// order-preserving map float -> uint32 (ascending)
+__device__ __forceinline__ uint32_t tp_key(float x) {
+  const uint32_t b = __float_as_uint(x);
+  return (b & 0x80000000u) ? ~b : (b | 0x80000000u);
+}
+// NaN and +inf count as -inf (never kept)
+__device__ __forceinline__ float tp_clean(float x, int& bad) {
+  if (!(x < INFINITY)) { bad = 1; return -INFINITY; }
+  return x;
+}
+__device__ __forceinline__ float tp_ex2(float x) {
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
+__device__ __forceinline__ unsigned long long tp_mass(float x, float M, float c2) {
+  return __float2ull_rn(tp_ex2((x - M) * c2) * kTpScale);  // (-inf - M) * c2 = -inf -> 0
+}
+
+// calls f(index, value) for every element of the row: float4 body, scalar tail
+template <typename F>
+__device__ __forceinline__ void tp_for_each(const float* row, int V, F f) {
+  const int V4 = V & ~3;
+  for (int i = threadIdx.x * 4; i < V4; i += kTpThreads * 4) {
+    const float4 x = *reinterpret_cast<const float4*>(row + i);
+    f(i, x.x); f(i + 1, x.y); f(i + 2, x.z); f(i + 3, x.w);
+  }
+  for (int i = V4 + threadIdx.x; i < V; i += kTpThreads) f(i, row[i]);
+}
+
+// Exclusive prefix sum over the block's threads in thread order; every thread also gets the total.
+__device__ __forceinline__ unsigned long long tp_block_scan(unsigned long long v, TpShared& sh, unsigned long long& total) {
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  unsigned long long inc = v;
+#pragma unroll
+  for (int o = 1; o < 32; o <<= 1) {
+    const unsigned long long up = __shfl_up_sync(0xffffffffu, inc, o);
+    if (lane >= o) inc += up;
+  }
+  __syncthreads();  // warp_tot free for reuse
+  if (lane == 31) sh.warp_tot[warp] = inc;
+  __syncthreads();
+  unsigned long long before = 0, all = 0;
+#pragma unroll 1
+  for (int w = 0; w < kTpWarps; ++w) {
+    const unsigned long long t = sh.warp_tot[w];
+    if (w < warp) before += t;
+    all += t;
+  }
+  total = all;
+  return before + inc - v;
+}
+
+// Among `bins` bins of sh.hist taken from the highest index down, finds the one in which the running mass reaches
+// `target` (> 0, <= the bins' total); leaves its index, the mass above it, its own mass (and token count when
+// `with_count`) in sh.sel_*.  bins is 2048 or 1024: two or one bin per thread.
+__device__ __forceinline__ void tp_find_crossing(TpShared& sh, int bins, unsigned long long target, bool with_count) {
+  const int per = bins / kTpThreads;  // 2 or 1
+  const int hi = bins - 1 - (int)threadIdx.x * per;  // this thread's highest bin
+  unsigned long long m0 = sh.hist[hi], m1 = per == 2 ? sh.hist[hi - 1] : 0ull;
+  unsigned long long total;
+  const unsigned long long above = tp_block_scan(m0 + m1, sh, total);
+  if (above < target && target <= above + m0) {
+    sh.sel_bin = hi; sh.sel_above = above; sh.sel_mass = m0; sh.sel_count = with_count ? sh.count[hi] : 0u;
+  } else if (per == 2 && above + m0 < target && target <= above + m0 + m1) {
+    sh.sel_bin = hi - 1; sh.sel_above = above + m0; sh.sel_mass = m1; sh.sel_count = with_count ? sh.count[hi - 1] : 0u;
+  }
+  __syncthreads();
+}
+
+__global__ void __launch_bounds__(kTpThreads, 1) top_p_filter_kernel(const TopPArgs a) {
+  __shared__ TpShared sh;
+  const float* row = a.logits + (int64_t)blockIdx.x * a.in_stride;
+  float* orow = a.out + (int64_t)blockIdx.x * a.out_stride;
+  const int V = a.V, lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+
+  // ---- the row maximum (NaN / +inf flagged and read as -inf), histogram cleared meanwhile
+  for (int i = threadIdx.x; i < 2048; i += kTpThreads) sh.hist[i] = 0ull;
+  if (threadIdx.x == 0) { sh.bad = 0; sh.kept = 0; sh.tie_limit = INT_MAX; }
+  int bad = 0;
+  float m = -INFINITY;
+  tp_for_each(row, V, [&](int, float x) { m = fmaxf(m, tp_clean(x, bad)); });
+  m = warp_max(m);
+  if (lane == 0) sh.warp_max[warp] = m;
+  __syncthreads();
+  float M = -INFINITY;
+#pragma unroll 1
+  for (int w = 0; w < kTpWarps; ++w) M = fmaxf(M, sh.warp_max[w]);
+  if (bad) sh.bad = 1;
+  if (M == -INFINITY) {  // no token with any mass: nothing to keep
+    tp_for_each(row, V, [&](int i, float) { orow[i] = -INFINITY; });
+    bad = __syncthreads_or(bad);
+    if (threadIdx.x == 0) {
+      dev_flag(a.dev_status, SEQ_DEV_DEGENERATE | (bad ? SEQ_DEV_NONFINITE : 0));
+      if (a.kept_out != nullptr) a.kept_out[blockIdx.x] = 0;
+    }
+    return;
+  }
+
+  // ---- level 0: every token, bins = the key's top 11 bits
+  tp_for_each(row, V, [&](int, float x) {
+    int b2 = 0;
+    x = tp_clean(x, b2);
+    const unsigned long long w = tp_mass(x, M, a.c2);
+    if (w) atomicAdd(&sh.hist[tp_key(x) >> 21], w);
+  });
+  __syncthreads();
+  unsigned long long target;
+  {
+    // the whole mass, then the mass the nucleus has to reach (rounded up, at least one unit)
+    const unsigned long long mine = sh.hist[2 * threadIdx.x] + sh.hist[2 * threadIdx.x + 1];
+    unsigned long long S;
+    tp_block_scan(mine, sh, S);
+    const double want = ceil(a.top_p * (double)S);
+    target = want < 1.0 ? 1ull : (want >= (double)S ? S : (unsigned long long)want);
+  }
+  tp_find_crossing(sh, 2048, target, false);
+  const uint32_t p0 = sh.sel_bin;
+  const unsigned long long above0 = sh.sel_above;
+  __syncthreads();
+
+  // ---- level 1: tokens whose key starts with p0, bins = the next 11 bits
+  for (int i = threadIdx.x; i < 2048; i += kTpThreads) sh.hist[i] = 0ull;
+  __syncthreads();
+  tp_for_each(row, V, [&](int, float x) {
+    int b2 = 0;
+    x = tp_clean(x, b2);
+    const uint32_t k = tp_key(x);
+    if ((k >> 21) == p0) {
+      const unsigned long long w = tp_mass(x, M, a.c2);
+      if (w) atomicAdd(&sh.hist[(k >> 10) & 0x7ffu], w);
+    }
+  });
+  __syncthreads();
+  tp_find_crossing(sh, 2048, target - above0, false);
+  const uint32_t p1 = (p0 << 11) | sh.sel_bin;
+  const unsigned long long above1 = above0 + sh.sel_above;
+  __syncthreads();
+
+  // ---- level 2: tokens whose key starts with p1, bins = the last 10 bits, with token counts
+  for (int i = threadIdx.x; i < 1024; i += kTpThreads) { sh.hist[i] = 0ull; sh.count[i] = 0u; }
+  __syncthreads();
+  tp_for_each(row, V, [&](int, float x) {
+    int b2 = 0;
+    x = tp_clean(x, b2);
+    const uint32_t k = tp_key(x);
+    if ((k >> 10) == p1) {
+      const unsigned long long w = tp_mass(x, M, a.c2);
+      if (w) { atomicAdd(&sh.hist[k & 0x3ffu], w); atomicAdd(&sh.count[k & 0x3ffu], 1u); }
+    }
+  });
+  __syncthreads();
+  tp_find_crossing(sh, 1024, target - above1, true);
+  const uint32_t tau = (p1 << 10) | sh.sel_bin;  // the key of the least probable kept token
+  // tokens with exactly that logit share one mass: the first `need` of them in token order are kept
+  const uint32_t ties = sh.sel_count;
+  const unsigned long long each = sh.sel_mass / (ties ? ties : 1u);
+  const unsigned long long rest = target - above1 - sh.sel_above;
+  uint32_t need = each ? (uint32_t)((rest + each - 1) / each) : ties;
+  need = need < 1u ? 1u : (need > ties ? ties : need);
+  __syncthreads();
+  if (need < ties) {
+    // rare: the cut falls inside a run of equal logits.  Contiguous chunks per thread, a scan of the tie counts,
+    // and the thread whose chunk holds the need-th tie finds its index.
+    const int len = (V + kTpThreads - 1) / kTpThreads;
+    const int lo = min((int)threadIdx.x * len, V), hi = min(lo + len, V);
+    unsigned long long cnt = 0;
+    for (int i = lo; i < hi; ++i) {
+      int b2 = 0;
+      cnt += tp_key(tp_clean(row[i], b2)) == tau;
+    }
+    unsigned long long total;
+    const unsigned long long before = tp_block_scan(cnt, sh, total);
+    if (before < need && need <= before + cnt) {
+      unsigned long long seen = before;
+      for (int i = lo; i < hi; ++i) {
+        int b2 = 0;
+        if (tp_key(tp_clean(row[i], b2)) == tau && ++seen == need) { sh.tie_limit = i; break; }
+      }
+    }
+    __syncthreads();
+  }
+  const int tie_limit = sh.tie_limit;
+
+  // ---- write: the logit itself inside the nucleus, -inf outside
+  int kept = 0;
+  tp_for_each(row, V, [&](int i, float x) {
+    int b2 = 0;
+    const float c = tp_clean(x, b2);
+    const uint32_t k = tp_key(c);
+    const bool keep = c > -INFINITY && (k > tau || (k == tau && i <= tie_limit));
+    orow[i] = keep ? x : -INFINITY;
+    kept += keep;
+  });
+  kept = __reduce_add_sync(0xffffffffu, kept);
+  if (lane == 0) atomicAdd(&sh.kept, kept);
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    if (a.kept_out != nullptr) a.kept_out[blockIdx.x] = sh.kept;
+    if (sh.bad) dev_flag(a.dev_status, SEQ_DEV_NONFINITE);
+  }
+}
+
+// top_p >= 1: every token stays (rows copied when the call is not in place)
+__global__ void top_p_copy_kernel(const TopPArgs a) {
+  const float* row = a.logits + (int64_t)blockIdx.x * a.in_stride;
+  float* orow = a.out + (int64_t)blockIdx.x * a.out_stride;
+  if (row != orow)
+    for (int i = threadIdx.x; i < a.V; i += blockDim.x) orow[i] = row[i];
+  if (threadIdx.x == 0 && a.kept_out != nullptr) a.kept_out[blockIdx.x] = a.V;
+}
+
+}  // namespace seqtree
+
+using namespace seqtree;
+
+extern "C" int seq_tree_top_p_filter(const seq_tree_top_p_params* p, void* stream) {
+  if (p == nullptr || p->logits == nullptr || p->out == nullptr) return SEQ_ERR_INVALID_ARG;
+  if (p->n_rows < 1 || p->vocab < 1 || p->vocab > (1 << 22)) return SEQ_ERR_INVALID_ARG;
+  if (!(p->temperature > 0.f) || isinf(p->temperature) || !(p->top_p > 0.f)) return SEQ_ERR_INVALID_ARG;
+  if (p->logits_row_stride < p->vocab || p->out_row_stride < p->vocab || p->logits_row_stride % 4 != 0 ||
+      p->out_row_stride % 4 != 0 || reinterpret_cast<uintptr_t>(p->logits) % 16 != 0 ||
+      reinterpret_cast<uintptr_t>(p->out) % 16 != 0)
+    return SEQ_ERR_INVALID_ARG;
+  TopPArgs a;
+  a.logits = p->logits; a.in_stride = p->logits_row_stride;
+  a.out = p->out; a.out_stride = p->out_row_stride;
+  a.V = p->vocab;
+  a.c2 = kLog2e / p->temperature;
+  a.top_p = (double)p->top_p;
+  a.kept_out = p->kept_out; a.dev_status = p->dev_status;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  if (p->top_p >= 1.f)
+    top_p_copy_kernel<<<p->n_rows, 256, 0, s>>>(a);
+  else
+    top_p_filter_kernel<<<p->n_rows, kTpThreads, 0, s>>>(a);
+  SEQ_CUDA_OK(cudaGetLastError());
+  return SEQ_OK;
+}

@@ -44,7 +44,8 @@ def test_ctypes_structs_match_the_header(tmp_path):
 
     fields_a = [f[0] for f in binding.AttentionParams._fields_]
     fields_v = [f[0] for f in binding.VerifyParams._fields_]
-    others = (("seq_tree_draft_sample_params", binding.DraftSampleParams), ("seq_tree_kv_commit_params", binding.KvCommitParams))
+    others = (("seq_tree_draft_sample_params", binding.DraftSampleParams), ("seq_tree_kv_commit_params", binding.KvCommitParams),
+              ("seq_tree_top_p_params", binding.TopPParams), ("seq_tree_build_params", binding.TreeBuildParams))
     src = tmp_path / "layout.c"
     lines = ['#include <stdio.h>', '#include <stddef.h>', '#include "seq_tree.h"', "int main(void){",
              'printf("%zu\\n", sizeof(seq_tree_attention_params));']
@@ -144,6 +145,21 @@ def test_host_checkable_errors_are_refused_before_launch(lib):
     for kw in bad:
         assert lib.seq_tree_kv_commit(C.byref(commit(**kw)), None) == B.SEQ_ERR_INVALID_ARG, kw
     assert lib.seq_tree_kv_commit(None, None) == B.SEQ_ERR_INVALID_ARG
+
+    def topp(**kw):
+        p = B.TopPParams()
+        p.n_rows, p.vocab, p.temperature, p.top_p = 4, 32000, 0.6, 0.9
+        p.logits = p.out = fake
+        p.logits_row_stride = p.out_row_stride = 32000
+        for k, v in kw.items():
+            setattr(p, k, v)
+        return p
+
+    bad = [dict(logits=None), dict(out=None), dict(n_rows=0), dict(vocab=0), dict(temperature=0.0), dict(temperature=float("nan")),
+           dict(temperature=float("inf")), dict(top_p=0.0), dict(top_p=-0.5), dict(top_p=float("nan")),
+           dict(logits_row_stride=31996), dict(out_row_stride=32002), dict(logits=fake + 4), dict(out=fake + 8)]
+    for kw in bad:
+        assert lib.seq_tree_top_p_filter(C.byref(topp(**kw)), None) == B.SEQ_ERR_INVALID_ARG, kw
 
 
 def test_binding_refuses_cpu_tensors():

@@ -96,5 +96,7 @@ def test_min_gap_reports_the_margin():
     assert r["keep"].tolist() == [True, True, False] and r["min_gap"] == pytest.approx(0.01, abs=1e-6)
     r = O.top_p(logits, 1.0, 0.51)
     assert r["keep"].tolist() == [True, True, False] and r["min_gap"] == pytest.approx(0.01, abs=1e-6)
+    assert r["over"] == pytest.approx(0.29, abs=1e-6) and r["under"] == pytest.approx(0.01, abs=1e-6)
     r = O.top_p(logits, 1.0, 0.4)
     assert r["keep"].tolist() == [True, False, False] and r["min_gap"] == pytest.approx(0.1, abs=1e-6)
+    assert r["over"] == pytest.approx(0.1, abs=1e-6) and r["under"] == pytest.approx(0.4, abs=1e-6)
