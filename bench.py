@@ -390,6 +390,44 @@ def tree_search_leg(cfg, T, dev, stream) -> dict:
                     "paper prints; outside the timed step"}
 
 
+def top_p_leg(cfg, ver_h, T, dev, stream, peaks, top_p=0.9) -> dict:
+    """Not part of the timed step: the nucleus filter over the target rows of every tree node, timed on its own in a
+    CUDA graph over rotating logit sets (out of place)."""
+    from paper_2402_12374_b200 import binding as B
+
+    sets = [vi.target_logits.to(dev) for vi in ver_h[:4]]
+    out = torch.empty_like(sets[0])
+    kept = torch.empty(sets[0].shape[0], dtype=torch.int32, device=dev)
+    status = torch.zeros(1, dtype=torch.int32, device=dev)
+    reps = 24
+    with torch.cuda.stream(stream):
+        for i in range(3):
+            B.seq_tree_top_p_filter(sets[i % len(sets)], T, top_p, out=out, kept_out=kept, dev_status=status, stream=stream)
+        stream.synchronize()
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g, stream=stream):
+            for i in range(reps):
+                B.seq_tree_top_p_filter(sets[i % len(sets)], T, top_p, out=out, kept_out=kept, dev_status=status, stream=stream)
+        g.replay()
+        stream.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        g.replay()
+        e1.record(stream)
+        stream.synchronize()
+    if int(status.item()) != 0:
+        raise RuntimeError(f"top_p dev_status = {int(status.item())}")
+    us = e0.elapsed_time(e1) * 1e3 / reps
+    rows, V = sets[0].shape
+    nbytes = 2 * rows * V * 4
+    gbs = nbytes / (us * 1e-6) / 1e9
+    return {"us_per_call": us, "rows": rows, "vocab": V, "top_p": top_p, "mean_kept": float(kept.float().mean().item()),
+            "gpu_launches_per_call": 1,
+            "roofline": {"bound": "hbm", "achieved": gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                         "frac": gbs / peaks["hbm_gbs"], "algorithmic_bytes": nbytes, "traffic": None},
+            "note": "every row read once and written once (the four re-reads of the select come from L2); outside the timed step"}
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -603,6 +641,7 @@ def main():
     if T > 0 and args.tree_search:
         line["next_rows"]["tree_search"] = tree_search_leg(cfg, T, dev, stream)
     if T > 0:
+        line["next_rows"]["top_p_filter"] = top_p_leg(cfg, ver_h, T, dev, stream, peaks)
         line["next_rows"]["draft_sample"] = draft_sample_leg(cfg, parent, ver_h, T, dev, stream, peaks)
     if not args.no_cpu_baseline:
         from oracle import oracle as O

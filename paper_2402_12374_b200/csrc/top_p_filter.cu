@@ -1,8 +1,11 @@
 // seq_tree_top_p_filter: nucleus truncation of softmax(logits / T), row by row (the top-p hyperparameter of the
-// robustness study, Section 4.2).  One CTA per row.  The nucleus is found by a radix select on the logits' bit
-// patterns (11 + 11 + 10 bits) in which every bin carries the probability MASS of its tokens, as 2^-40 fixed point in
-// 64-bit integers: sums are exact and independent of the order of the atomic adds, so the kept set is reproducible
-// bit for bit.  A row is read five times (maximum, three select levels, the write), once from HBM and then from L2.
+// robustness study, Section 4.2).  One CTA per row.  A histogram of the probability MASS over 2048 equal steps of the
+// exponent argument finds the bin in which the cut falls; the tokens of that bin (a few dozen on the paper's shapes)
+// are ordered exactly in shared memory by (logit bits, token id); a flat row or a long run of equal logits, whose bin
+// holds more than 1024 tokens, takes a radix select on the logit bits (11 + 11 + 10) instead.  Masses are 2^-40 fixed
+// point in 64-bit integers: sums are exact and independent of the order of the atomic adds, so the kept set is
+// reproducible bit for bit.  A row is read four times (maximum, histogram, collect, write), once from HBM and then
+// from L2.
 #include <climits>
 
 #include "common.cuh"
@@ -12,6 +15,7 @@ namespace seqtree {
 constexpr int kTpThreads = 1024;
 constexpr int kTpWarps = kTpThreads / 32;
 constexpr float kTpScale = 1099511627776.f;  // 2^40
+constexpr int kTpCand = 1024;  // tokens of the cut's bin that are ordered in shared memory (more: radix select)
 
 struct TopPArgs {
   const float* logits; int64_t in_stride;
@@ -30,7 +34,9 @@ struct TpShared {
   // results of a level's search
   uint32_t sel_bin; unsigned long long sel_above; unsigned long long sel_mass; uint32_t sel_count;
   int32_t tie_limit;
-  int32_t bad, kept;
+  int32_t bad, kept, ncand;
+  unsigned long long tau_comp;
+  unsigned long long sorted_c[kTpCand], sorted_w[kTpCand];  // the cut's bin in order: (key, ~index) and mass
 };
 
 // order-preserving map float -> uint32 (ascending)
@@ -52,15 +58,36 @@ __device__ __forceinline__ unsigned long long tp_mass(float x, float M, float c2
   return __float2ull_rn(tp_ex2((x - M) * c2) * kTpScale);  // (-inf - M) * c2 = -inf -> 0
 }
 
-// calls f(index, value) for every element of the row: float4 body, scalar tail
+// calls f(index, value) for every element of the row: float4 body with four independent loads in flight per
+// thread (the passes are latency-bound otherwise), scalar tail
 template <typename F>
 __device__ __forceinline__ void tp_for_each(const float* row, int V, F f) {
   const int V4 = V & ~3;
-  for (int i = threadIdx.x * 4; i < V4; i += kTpThreads * 4) {
-    const float4 x = *reinterpret_cast<const float4*>(row + i);
-    f(i, x.x); f(i + 1, x.y); f(i + 2, x.z); f(i + 3, x.w);
+  constexpr int kStride = kTpThreads * 4;
+  int i = threadIdx.x * 4;
+  for (; i + 3 * kStride < V4; i += 4 * kStride) {
+    float4 x[4];
+#pragma unroll
+    for (int k = 0; k < 4; ++k) x[k] = *reinterpret_cast<const float4*>(row + i + k * kStride);
+#pragma unroll
+    for (int k = 0; k < 4; ++k) {
+      const int j = i + k * kStride;
+      f(j, x[k].x); f(j + 1, x[k].y); f(j + 2, x[k].z); f(j + 3, x[k].w);
+    }
   }
-  for (int i = V4 + threadIdx.x; i < V; i += kTpThreads) f(i, row[i]);
+  {  // up to three more, again loaded together
+    float4 x[3];
+#pragma unroll
+    for (int k = 0; k < 3; ++k)
+      if (i + k * kStride < V4) x[k] = *reinterpret_cast<const float4*>(row + i + k * kStride);
+#pragma unroll
+    for (int k = 0; k < 3; ++k)
+      if (i + k * kStride < V4) {
+        const int j = i + k * kStride;
+        f(j, x[k].x); f(j + 1, x[k].y); f(j + 2, x[k].z); f(j + 3, x[k].w);
+      }
+  }
+  for (int t = V4 + threadIdx.x; t < V; t += kTpThreads) f(t, row[t]);
 }
 
 // Exclusive prefix sum over the block's threads in thread order; every thread also gets the total.
@@ -103,6 +130,14 @@ __device__ __forceinline__ void tp_find_crossing(TpShared& sh, int bins, unsigne
   __syncthreads();
 }
 
+// First-level bin of a (cleaned) logit: 2048 equal steps of the exponent argument d = (M - x) * log2(e) / T over
+// [0, 40), most probable tokens in the highest bin; -1 beyond (mass below one unit of the fixed point: never kept).
+// Sub, multiply by a positive constant and truncation are monotone, so a higher bin never holds a smaller logit.
+__device__ __forceinline__ int tp_lbin(float x, float M, float c2) {
+  const float d = (M - x) * c2;
+  return d < 40.f ? 2047 - (int)(d * 51.2f) : -1;
+}
+
 __global__ void __launch_bounds__(kTpThreads, 1) top_p_filter_kernel(const TopPArgs a) {
   __shared__ TpShared sh;
   const float* row = a.logits + (int64_t)blockIdx.x * a.in_stride;
@@ -111,7 +146,7 @@ __global__ void __launch_bounds__(kTpThreads, 1) top_p_filter_kernel(const TopPA
 
   // ---- the row maximum (NaN / +inf flagged and read as -inf), histogram cleared meanwhile
   for (int i = threadIdx.x; i < 2048; i += kTpThreads) sh.hist[i] = 0ull;
-  if (threadIdx.x == 0) { sh.bad = 0; sh.kept = 0; sh.tie_limit = INT_MAX; }
+  if (threadIdx.x == 0) { sh.bad = 0; sh.kept = 0; sh.tie_limit = INT_MAX; sh.ncand = 0; sh.tau_comp = 0ull; }
   int bad = 0;
   float m = -INFINITY;
   tp_for_each(row, V, [&](int, float x) { m = fmaxf(m, tp_clean(x, bad)); });
@@ -132,12 +167,13 @@ __global__ void __launch_bounds__(kTpThreads, 1) top_p_filter_kernel(const TopPA
     return;
   }
 
-  // ---- level 0: every token, bins = the key's top 11 bits
+  // ---- first level: every token with mass, equal steps of the exponent argument (tokens spread over many bins:
+  // few collisions between the atomic adds, and the bin of the cut holds few tokens)
   tp_for_each(row, V, [&](int, float x) {
     int b2 = 0;
     x = tp_clean(x, b2);
-    const unsigned long long w = tp_mass(x, M, a.c2);
-    if (w) atomicAdd(&sh.hist[tp_key(x) >> 21], w);
+    const int lb = tp_lbin(x, M, a.c2);
+    if (lb >= 0) atomicAdd(&sh.hist[lb], tp_mass(x, M, a.c2));
   });
   __syncthreads();
   unsigned long long target;
@@ -150,80 +186,128 @@ __global__ void __launch_bounds__(kTpThreads, 1) top_p_filter_kernel(const TopPA
     target = want < 1.0 ? 1ull : (want >= (double)S ? S : (unsigned long long)want);
   }
   tp_find_crossing(sh, 2048, target, false);
-  const uint32_t p0 = sh.sel_bin;
-  const unsigned long long above0 = sh.sel_above;
+  const int B0 = (int)sh.sel_bin;                    // the bin in which the cut falls
+  const unsigned long long rest0 = target - sh.sel_above;  // mass still to find inside it
   __syncthreads();
 
-  // ---- level 1: tokens whose key starts with p0, bins = the next 11 bits
-  for (int i = threadIdx.x; i < 2048; i += kTpThreads) sh.hist[i] = 0ull;
-  __syncthreads();
-  tp_for_each(row, V, [&](int, float x) {
+  // ---- the tokens of that bin, as (key, ~index) so that a larger value means "earlier in the order"
+  unsigned long long* cand = sh.hist;               // [kTpCand]   (the histogram is no longer needed)
+  unsigned long long* cand_w = sh.hist + kTpCand;   // [kTpCand]
+  tp_for_each(row, V, [&](int i, float x) {
     int b2 = 0;
     x = tp_clean(x, b2);
-    const uint32_t k = tp_key(x);
-    if ((k >> 21) == p0) {
-      const unsigned long long w = tp_mass(x, M, a.c2);
-      if (w) atomicAdd(&sh.hist[(k >> 10) & 0x7ffu], w);
-    }
-  });
-  __syncthreads();
-  tp_find_crossing(sh, 2048, target - above0, false);
-  const uint32_t p1 = (p0 << 11) | sh.sel_bin;
-  const unsigned long long above1 = above0 + sh.sel_above;
-  __syncthreads();
-
-  // ---- level 2: tokens whose key starts with p1, bins = the last 10 bits, with token counts
-  for (int i = threadIdx.x; i < 1024; i += kTpThreads) { sh.hist[i] = 0ull; sh.count[i] = 0u; }
-  __syncthreads();
-  tp_for_each(row, V, [&](int, float x) {
-    int b2 = 0;
-    x = tp_clean(x, b2);
-    const uint32_t k = tp_key(x);
-    if ((k >> 10) == p1) {
-      const unsigned long long w = tp_mass(x, M, a.c2);
-      if (w) { atomicAdd(&sh.hist[k & 0x3ffu], w); atomicAdd(&sh.count[k & 0x3ffu], 1u); }
-    }
-  });
-  __syncthreads();
-  tp_find_crossing(sh, 1024, target - above1, true);
-  const uint32_t tau = (p1 << 10) | sh.sel_bin;  // the key of the least probable kept token
-  // tokens with exactly that logit share one mass: the first `need` of them in token order are kept
-  const uint32_t ties = sh.sel_count;
-  const unsigned long long each = sh.sel_mass / (ties ? ties : 1u);
-  const unsigned long long rest = target - above1 - sh.sel_above;
-  uint32_t need = each ? (uint32_t)((rest + each - 1) / each) : ties;
-  need = need < 1u ? 1u : (need > ties ? ties : need);
-  __syncthreads();
-  if (need < ties) {
-    // rare: the cut falls inside a run of equal logits.  Contiguous chunks per thread, a scan of the tie counts,
-    // and the thread whose chunk holds the need-th tie finds its index.
-    const int len = (V + kTpThreads - 1) / kTpThreads;
-    const int lo = min((int)threadIdx.x * len, V), hi = min(lo + len, V);
-    unsigned long long cnt = 0;
-    for (int i = lo; i < hi; ++i) {
-      int b2 = 0;
-      cnt += tp_key(tp_clean(row[i], b2)) == tau;
-    }
-    unsigned long long total;
-    const unsigned long long before = tp_block_scan(cnt, sh, total);
-    if (before < need && need <= before + cnt) {
-      unsigned long long seen = before;
-      for (int i = lo; i < hi; ++i) {
-        int b2 = 0;
-        if (tp_key(tp_clean(row[i], b2)) == tau && ++seen == need) { sh.tie_limit = i; break; }
+    if (tp_lbin(x, M, a.c2) == B0) {
+      const int pos = atomicAdd(&sh.ncand, 1);
+      if (pos < kTpCand) {
+        cand[pos] = ((unsigned long long)tp_key(x) << 32) | (uint32_t)~(uint32_t)i;
+        cand_w[pos] = tp_mass(x, M, a.c2);
       }
     }
+  });
+  __syncthreads();
+  const int ncand = sh.ncand;
+  uint32_t tau = 0;          // fallback only: key of the least probable kept token
+  bool exact = ncand <= kTpCand;
+  if (exact) {
+    // rank every candidate among the others (all distinct), lay them out in order, scan the masses
+    unsigned long long my_w = 0, my_c = 0;
+    if ((int)threadIdx.x < ncand) {
+      my_c = cand[threadIdx.x];
+      my_w = cand_w[threadIdx.x];
+      int rank = 0;
+#pragma unroll 4
+      for (int j = 0; j < ncand; ++j) rank += cand[j] > my_c;
+      sh.sorted_c[rank] = my_c;
+      sh.sorted_w[rank] = my_w;
+    }
     __syncthreads();
+    const unsigned long long w = (int)threadIdx.x < ncand ? sh.sorted_w[threadIdx.x] : 0ull;
+    unsigned long long total;
+    const unsigned long long before = tp_block_scan(w, sh, total);
+    if ((int)threadIdx.x < ncand && before < rest0 && rest0 <= before + w) sh.tau_comp = sh.sorted_c[threadIdx.x];
+    __syncthreads();
+  } else {
+    // ---- many tokens in one bin (a flat row, runs of equal logits): radix select on the key bits inside the bin
+    __syncthreads();
+    for (int i = threadIdx.x; i < 2048; i += kTpThreads) sh.hist[i] = 0ull;
+    __syncthreads();
+    tp_for_each(row, V, [&](int, float x) {
+      int b2 = 0;
+      x = tp_clean(x, b2);
+      if (tp_lbin(x, M, a.c2) == B0) atomicAdd(&sh.hist[tp_key(x) >> 21], tp_mass(x, M, a.c2));
+    });
+    __syncthreads();
+    tp_find_crossing(sh, 2048, rest0, false);
+    const uint32_t p0 = sh.sel_bin;
+    const unsigned long long above0 = sh.sel_above;
+    __syncthreads();
+    for (int i = threadIdx.x; i < 2048; i += kTpThreads) sh.hist[i] = 0ull;
+    __syncthreads();
+    tp_for_each(row, V, [&](int, float x) {
+      int b2 = 0;
+      x = tp_clean(x, b2);
+      const uint32_t k = tp_key(x);
+      if ((k >> 21) == p0 && tp_lbin(x, M, a.c2) == B0) atomicAdd(&sh.hist[(k >> 10) & 0x7ffu], tp_mass(x, M, a.c2));
+    });
+    __syncthreads();
+    tp_find_crossing(sh, 2048, rest0 - above0, false);
+    const uint32_t p1 = (p0 << 11) | sh.sel_bin;
+    const unsigned long long above1 = above0 + sh.sel_above;
+    __syncthreads();
+    for (int i = threadIdx.x; i < 1024; i += kTpThreads) { sh.hist[i] = 0ull; sh.count[i] = 0u; }
+    __syncthreads();
+    tp_for_each(row, V, [&](int, float x) {
+      int b2 = 0;
+      x = tp_clean(x, b2);
+      const uint32_t k = tp_key(x);
+      if ((k >> 10) == p1 && tp_lbin(x, M, a.c2) == B0) {
+        atomicAdd(&sh.hist[k & 0x3ffu], tp_mass(x, M, a.c2));
+        atomicAdd(&sh.count[k & 0x3ffu], 1u);
+      }
+    });
+    __syncthreads();
+    tp_find_crossing(sh, 1024, rest0 - above1, true);
+    tau = (p1 << 10) | sh.sel_bin;
+    // tokens with exactly that logit share one mass: the first `need` of them in token order are kept
+    const uint32_t ties = sh.sel_count;
+    const unsigned long long each = sh.sel_mass / (ties ? ties : 1u);
+    const unsigned long long rest = rest0 - above1 - sh.sel_above;
+    uint32_t need = each ? (uint32_t)((rest + each - 1) / each) : ties;
+    need = need < 1u ? 1u : (need > ties ? ties : need);
+    __syncthreads();
+    if (need < ties) {
+      // the cut falls inside a run of equal logits: contiguous chunks per thread, a scan of the tie counts, and the
+      // thread whose chunk holds the need-th tie finds its index
+      const int len = (V + kTpThreads - 1) / kTpThreads;
+      const int lo = min((int)threadIdx.x * len, V), hi = min(lo + len, V);
+      unsigned long long cnt = 0;
+      for (int i = lo; i < hi; ++i) {
+        int b2 = 0;
+        cnt += tp_key(tp_clean(row[i], b2)) == tau;
+      }
+      unsigned long long total;
+      const unsigned long long before = tp_block_scan(cnt, sh, total);
+      if (before < need && need <= before + cnt) {
+        unsigned long long seen = before;
+        for (int i = lo; i < hi; ++i) {
+          int b2 = 0;
+          if (tp_key(tp_clean(row[i], b2)) == tau && ++seen == need) { sh.tie_limit = i; break; }
+        }
+      }
+      __syncthreads();
+    }
   }
-  const int tie_limit = sh.tie_limit;
+  const unsigned long long tau_comp = exact ? sh.tau_comp : (((unsigned long long)tau << 32) | (uint32_t)~(uint32_t)min(sh.tie_limit, V - 1));
 
-  // ---- write: the logit itself inside the nucleus, -inf outside
+  // ---- write: the logit itself inside the nucleus, -inf outside.  Inside: a more probable bin, or the cut's bin
+  // and not behind the last kept token in the order (key descending, index ascending).
   int kept = 0;
   tp_for_each(row, V, [&](int i, float x) {
     int b2 = 0;
     const float c = tp_clean(x, b2);
-    const uint32_t k = tp_key(c);
-    const bool keep = c > -INFINITY && (k > tau || (k == tau && i <= tie_limit));
+    const int lb = tp_lbin(c, M, a.c2);
+    const unsigned long long comp = ((unsigned long long)tp_key(c) << 32) | (uint32_t)~(uint32_t)i;
+    const bool keep = lb > B0 || (lb == B0 && comp >= tau_comp);
     orow[i] = keep ? x : -INFINITY;
     kept += keep;
   });
