@@ -28,6 +28,9 @@ struct TopPArgs {
 
 struct TpShared {
   unsigned long long hist[2048];
+  // first-level histogram as three 32-bit limbs per bin (native 32-bit shared-memory adds; a 64-bit add is a
+  // compare-and-swap loop): mass = lo + hi * 2^21 + top * 2^53, carries moved up when an add wraps
+  uint32_t lo[2048], hi[2048], top[2048];
   uint32_t count[1024];
   unsigned long long warp_tot[kTpWarps];
   float warp_max[kTpWarps];
@@ -139,13 +142,14 @@ __device__ __forceinline__ int tp_lbin(float x, float M, float c2) {
 }
 
 __global__ void __launch_bounds__(kTpThreads, 1) top_p_filter_kernel(const TopPArgs a) {
-  __shared__ TpShared sh;
+  extern __shared__ __align__(16) uint8_t tp_smem[];
+  TpShared& sh = *reinterpret_cast<TpShared*>(tp_smem);
   const float* row = a.logits + (int64_t)blockIdx.x * a.in_stride;
   float* orow = a.out + (int64_t)blockIdx.x * a.out_stride;
   const int V = a.V, lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
 
   // ---- the row maximum (NaN / +inf flagged and read as -inf), histogram cleared meanwhile
-  for (int i = threadIdx.x; i < 2048; i += kTpThreads) sh.hist[i] = 0ull;
+  for (int i = threadIdx.x; i < 2048; i += kTpThreads) { sh.lo[i] = 0u; sh.hi[i] = 0u; sh.top[i] = 0u; }
   if (threadIdx.x == 0) { sh.bad = 0; sh.kept = 0; sh.tie_limit = INT_MAX; sh.ncand = 0; sh.tau_comp = 0ull; }
   int bad = 0;
   float m = -INFINITY;
@@ -173,8 +177,23 @@ __global__ void __launch_bounds__(kTpThreads, 1) top_p_filter_kernel(const TopPA
     int b2 = 0;
     x = tp_clean(x, b2);
     const int lb = tp_lbin(x, M, a.c2);
-    if (lb >= 0) atomicAdd(&sh.hist[lb], tp_mass(x, M, a.c2));
+    if (lb >= 0) {
+      const unsigned long long w = tp_mass(x, M, a.c2);
+      const uint32_t l = (uint32_t)w & 0x1fffffu, h = (uint32_t)(w >> 21);
+      uint32_t carry = h;
+      if (l) {
+        const uint32_t old = atomicAdd(&sh.lo[lb], l);
+        carry += (old + l < old) ? 2048u : 0u;  // a wrap of lo is 2^32 = 2048 units of hi
+      }
+      if (carry) {
+        const uint32_t old = atomicAdd(&sh.hi[lb], carry);
+        if (old + carry < old) atomicAdd(&sh.top[lb], 1u);
+      }
+    }
   });
+  __syncthreads();
+  for (int i = threadIdx.x; i < 2048; i += kTpThreads)
+    sh.hist[i] = (unsigned long long)sh.lo[i] + ((unsigned long long)sh.hi[i] << 21) + ((unsigned long long)sh.top[i] << 53);
   __syncthreads();
   unsigned long long target;
   {
@@ -351,8 +370,11 @@ extern "C" int seq_tree_top_p_filter(const seq_tree_top_p_params* p, void* strea
   cudaStream_t s = static_cast<cudaStream_t>(stream);
   if (p->top_p >= 1.f)
     top_p_copy_kernel<<<p->n_rows, 256, 0, s>>>(a);
-  else
-    top_p_filter_kernel<<<p->n_rows, kTpThreads, 0, s>>>(a);
+  else {
+    // above the 48 KB a kernel gets without asking; set on every call (cheap, and correct on every device)
+    SEQ_CUDA_OK(cudaFuncSetAttribute(top_p_filter_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sizeof(TpShared)));
+    top_p_filter_kernel<<<p->n_rows, kTpThreads, sizeof(TpShared), s>>>(a);
+  }
   SEQ_CUDA_OK(cudaGetLastError());
   return SEQ_OK;
 }
