@@ -428,6 +428,56 @@ def top_p_leg(cfg, ver_h, T, dev, stream, peaks, top_p=0.9) -> dict:
             "note": "every row read once and written once (the four re-reads of the select come from L2); outside the timed step"}
 
 
+def verify_batch_leg(cfg, parent, ver_h, T, dev, stream) -> dict:
+    """Not part of the timed step: R requests verified by one launch (one cluster per request; 18 clusters fit the
+    GPU at a time), against R launches of the single-request call; both as CUDA graphs, logits beyond L2."""
+    from paper_2402_12374_b200 import binding as B
+
+    per_req = 2 * cfg.n_tree * cfg.vocab * 4
+    R = 18 if per_req < (100 << 20) else 4
+    pick = [ver_h[i % len(ver_h)] for i in range(R)]
+    stack = lambda f: torch.stack([f(v).to(dev) for v in pick])
+    par = torch.from_numpy(parent).to(dev).unsqueeze(0).repeat(R, 1).contiguous()
+    tok, tl, dl, un = stack(lambda v: v.tokens), stack(lambda v: v.target_logits), stack(lambda v: v.draft_logits), stack(lambda v: v.uniforms)
+    status = torch.zeros(1, dtype=torch.int32, device=dev)
+    singles = [B.VerifyCall(par[r], tok[r], tl[r], dl[r], T, un[r], dev_status=status) for r in range(R)]
+    reps = 10
+
+    def timed(fn):
+        with torch.cuda.stream(stream):
+            fn()
+            stream.synchronize()
+            g = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(g, stream=stream):
+                for _ in range(reps):
+                    fn()
+            g.replay()
+            stream.synchronize()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record(stream)
+            g.replay()
+            e1.record(stream)
+            stream.synchronize()
+        return e0.elapsed_time(e1) * 1e3 / reps
+
+    outs = {}
+
+    def batched():
+        outs["b"] = B.seq_tree_verify_batch(par, tok, tl, dl, T, un, dev_status=status, stream=stream)
+
+    def one_by_one():
+        for c in singles:
+            c.run(stream)
+
+    us_b, us_s = timed(batched), timed(one_by_one)
+    torch.cuda.synchronize()
+    same = all(int(outs["b"][2][r].item()) == int(singles[r].bonus_token.item()) for r in range(R))
+    if int(status.item()) != 0 or not same:
+        raise RuntimeError(f"verify_batch: dev_status {int(status.item())}, identical to single launches: {same}")
+    return {"requests": R, "us_per_launch": us_b, "us_per_request": us_b / R, "us_per_request_single_launches": us_s / R,
+            "gpu_launches_per_call": 1, "note": "same results as R single-request launches (checked); outside the timed step"}
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -640,6 +690,7 @@ def main():
     line["next_rows"] = {"kv_commit": kv_commit_leg(cfg, parent, dev, stream, peaks)}
     if T > 0 and args.tree_search:
         line["next_rows"]["tree_search"] = tree_search_leg(cfg, T, dev, stream)
+    line["next_rows"]["verify_batch"] = verify_batch_leg(cfg, parent, ver_h, T, dev, stream)
     if T > 0:
         line["next_rows"]["top_p_filter"] = top_p_leg(cfg, ver_h, T, dev, stream, peaks)
         line["next_rows"]["draft_sample"] = draft_sample_leg(cfg, parent, ver_h, T, dev, stream, peaks)

@@ -254,6 +254,24 @@ typedef struct {
 size_t seq_tree_verify_workspace_bytes(const seq_tree_verify_params* p);
 int seq_tree_verify(const seq_tree_verify_params* p, void* stream);
 
+/* seq_tree_verify_batch -- `batch` independent requests in one launch, one cluster of 8 CTAs per request (18
+ * clusters run at a time on 148 SMs).  Every request is verified exactly as seq_tree_verify would verify it: same
+ * sizes, temperature and flags for all (SEQ_VERIFY_ALL_NODES is not allowed), each with its own tree, tokens,
+ * logits and uniforms.  request0 describes request 0; request r's arrays start r strides further:
+ *   tree_stride      elements between the requests' parent / tokens / path / next_child_out arrays (>= n_tree);
+ *   logits_stride    elements between their target matrices, and between their draft matrices (a multiple of 4,
+ *                    large enough for n_tree rows);
+ *   uniforms_stride  >= n_tree + 1;   residual_stride  >= vocab (unused when residual_out is NULL).
+ * path_len and bonus_token are arrays of `batch` entries; dev_status is one word for all requests.  Returns what
+ * seq_tree_verify returns; SEQ_ERR_INVALID_ARG also for a stride that is too small. */
+typedef struct {
+  seq_tree_verify_params request0;
+  int32_t batch;
+  int64_t tree_stride, logits_stride, uniforms_stride, residual_stride;
+} seq_tree_verify_batch_params;
+
+int seq_tree_verify_batch(const seq_tree_verify_batch_params* p, void* stream);
+
 /* Library build string ("seqtree <version> sm_100a"); static storage. */
 /*
  * seq_tree_draft_sample -- the draft side's draw of the children of tree nodes: k tokens without

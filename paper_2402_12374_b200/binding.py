@@ -36,6 +36,7 @@ EXPORTED_SYMBOLS = (
     "seq_tree_attention_noalloc",
     "seq_tree_verify_workspace_bytes",
     "seq_tree_verify",
+    "seq_tree_verify_batch",
     "seq_tree_draft_sample_workspace_bytes",
     "seq_tree_draft_sample",
     "seq_tree_kv_commit",
@@ -110,6 +111,8 @@ def load() -> C.CDLL:
         lib.seq_tree_verify_workspace_bytes.restype = C.c_size_t
         lib.seq_tree_verify.argtypes = [C.POINTER(VerifyParams), C.c_void_p]
         lib.seq_tree_verify.restype = C.c_int
+        lib.seq_tree_verify_batch.argtypes = [C.POINTER(VerifyBatchParams), C.c_void_p]
+        lib.seq_tree_verify_batch.restype = C.c_int
         lib.seq_tree_kv_commit.argtypes = [C.POINTER(KvCommitParams), C.c_void_p]
         lib.seq_tree_kv_commit.restype = C.c_int
         lib.seq_tree_top_p_filter.argtypes = [C.POINTER(TopPParams), C.c_void_p]
@@ -323,6 +326,47 @@ class VerifyCall:
     def run(self, stream=None):
         _check("seq_tree_verify", load().seq_tree_verify(C.byref(self.params), _stream(stream)))
         return self.path, self.path_len, self.bonus_token
+
+
+class VerifyBatchParams(C.Structure):
+    _fields_ = [
+        ("request0", VerifyParams), ("batch", C.c_int32),
+        ("tree_stride", C.c_int64), ("logits_stride", C.c_int64), ("uniforms_stride", C.c_int64),
+        ("residual_stride", C.c_int64),
+    ]
+
+
+def seq_tree_verify_batch(parent, tokens, target_logits, draft_logits, temperature: float, uniforms, *, residual_out=None,
+                          next_child_out=None, dev_status=None, specinfer: bool = False, target_sample: bool = False,
+                          stream=None):
+    """R requests in one launch.  parent, tokens [R, n]; target_logits, draft_logits [R, n, V]; uniforms [R, n+1];
+    residual_out [R, V] and next_child_out [R, n] optional.  Returns path [R, n], path_len [R], bonus_token [R]."""
+    R, n, V = target_logits.shape
+    dev = target_logits.device
+    path = torch.empty((R, n), dtype=torch.int32, device=dev)
+    path_len = torch.zeros(R, dtype=torch.int32, device=dev)
+    bonus = torch.full((R,), -1, dtype=torch.int32, device=dev)
+    for t, nm in ((parent, "parent"), (tokens, "tokens"), (uniforms, "uniforms"), (target_logits, "target_logits"),
+                  (draft_logits, "draft_logits"), (residual_out, "residual_out"), (next_child_out, "next_child_out")):
+        if t is not None and (t.shape[0] != R or t.stride(-1) != 1):
+            raise ValueError(f"{nm}: one entry per request, innermost dimension contiguous")
+    if draft_logits is not None and draft_logits.stride(0) != target_logits.stride(0):
+        raise ValueError("target_logits and draft_logits must have the same stride between requests")
+    if parent.stride(0) != tokens.stride(0) or parent.stride(0) != n or (next_child_out is not None and next_child_out.stride(0) != n):
+        raise ValueError("parent, tokens and next_child_out must be [R, n] contiguous")
+    one = VerifyCall(parent[0], tokens[0], target_logits[0], None if draft_logits is None else draft_logits[0], temperature,
+                     uniforms[0], path=path[0], path_len=path_len, bonus_token=bonus,
+                     residual_out=None if residual_out is None else residual_out[0],
+                     next_child_out=None if next_child_out is None else next_child_out[0], dev_status=dev_status,
+                     specinfer=specinfer, target_sample=target_sample)
+    p = VerifyBatchParams()
+    p.request0 = one.params
+    p.batch = R
+    p.tree_stride, p.logits_stride = n, target_logits.stride(0)
+    p.uniforms_stride = uniforms.stride(0)
+    p.residual_stride = residual_out.stride(0) if residual_out is not None else 0
+    _check("seq_tree_verify_batch", load().seq_tree_verify_batch(C.byref(p), _stream(stream)))
+    return path, path_len, bonus
 
 
 def seq_tree_verify(parent, tokens, target_logits, draft_logits, temperature: float, uniforms, **kw):

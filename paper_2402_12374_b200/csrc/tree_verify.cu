@@ -65,6 +65,8 @@ struct VerifyArgs {
   const float* uniforms;
   int32_t* path; int32_t* path_len; int32_t* bonus;
   float* residual_out; int32_t* next_child_out; int32_t* dev_status;
+  // batched launch: request r = cluster r; elements between consecutive requests' arrays
+  int64_t tree_stride, logits_stride, unif_stride, resid_stride;
 };
 
 struct VShared {
@@ -598,7 +600,21 @@ __device__ void draw_bonus(Ctx& c, const VerifyArgs& a, const NodeState& st) {
   }
 }
 
-__global__ void __launch_bounds__(kVThreads, 1) tree_verify_kernel(const VerifyArgs a) {
+template <bool kBatch>
+__global__ void __launch_bounds__(kVThreads, 1) tree_verify_kernel(const VerifyArgs a_in) {
+  // One request per cluster in a batched launch: the same code on that request's arrays.
+  VerifyArgs a_req;
+  if (kBatch) {
+    const int64_t r = blockIdx.x / kVCluster;
+    a_req = a_in;
+    a_req.parent += r * a_in.tree_stride; a_req.tokens += r * a_in.tree_stride;
+    a_req.target += r * a_in.logits_stride; a_req.draft += r * a_in.logits_stride;
+    a_req.uniforms += r * a_in.unif_stride;
+    a_req.path += r * a_in.tree_stride; a_req.path_len += r; a_req.bonus += r;
+    if (a_in.residual_out != nullptr) a_req.residual_out += r * a_in.resid_stride;
+    if (a_in.next_child_out != nullptr) a_req.next_child_out += r * a_in.tree_stride;
+  }
+  const VerifyArgs& a = kBatch ? a_req : a_in;
   cg::cluster_group cluster = cg::this_cluster();
   extern __shared__ __align__(16) uint8_t dyn_smem[];  // VShared, then the two slices
   VShared& sh = *reinterpret_cast<VShared*>(dyn_smem);
@@ -647,7 +663,7 @@ __global__ void __launch_bounds__(kVThreads, 1) tree_verify_kernel(const VerifyA
   NodeState st;
   st.greedy_token = 0;
   st.c2 = greedy ? 0.f : kLog2e / a.temperature;
-  const int cluster_id = blockIdx.x / kVCluster, n_clusters = gridDim.x / kVCluster;
+  const int cluster_id = kBatch ? 0 : blockIdx.x / kVCluster, n_clusters = kBatch ? 1 : gridDim.x / kVCluster;
 
   if (!all_nodes && a.next_child_out != nullptr && c.rank == 0)
     for (int i = c.tid; i < a.n; i += kVThreads) a.next_child_out[i] = -2;
@@ -710,9 +726,8 @@ extern "C" size_t seq_tree_verify_workspace_bytes(const seq_tree_verify_params* 
   return 0;  // all scratch lives in (distributed) shared memory
 }
 
-extern "C" int seq_tree_verify(const seq_tree_verify_params* p, void* stream) {
-  int rc = verify_validate(p);
-  if (rc != SEQ_OK) return rc;
+static int verify_launch(const seq_tree_verify_params* p, int batch, int64_t tree_stride, int64_t logits_stride,
+                         int64_t unif_stride, int64_t resid_stride, void* stream) {
   VerifyArgs a;
   a.n = p->n_tree; a.V = p->vocab; a.flags = p->flags;
   a.slice_cap = (((p->vocab + kVCluster - 1) / kVCluster) + 3) & ~3;
@@ -723,13 +738,15 @@ extern "C" int seq_tree_verify(const seq_tree_verify_params* p, void* stream) {
   a.temperature = p->temperature; a.uniforms = p->uniforms;
   a.path = p->path; a.path_len = p->path_len; a.bonus = p->bonus_token;
   a.residual_out = p->residual_out; a.next_child_out = p->next_child_out; a.dev_status = p->dev_status;
+  a.tree_stride = tree_stride; a.logits_stride = logits_stride; a.unif_stride = unif_stride; a.resid_stride = resid_stride;
 
   static_assert(sizeof(VShared) % 16 == 0, "the slices behind VShared must stay 16-byte aligned");
   const size_t dyn = sizeof(VShared) + (size_t)2 * a.slice_cap * sizeof(float);
   if (dyn > 227 * 1024) return SEQ_ERR_UNSUPPORTED;  // vocabulary too large for 8 slices
-  SEQ_CUDA_OK(cudaFuncSetAttribute(tree_verify_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)dyn));
+  auto kernel = batch > 0 ? tree_verify_kernel<true> : tree_verify_kernel<false>;
+  SEQ_CUDA_OK(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)dyn));
 
-  int n_clusters = 1;
+  int n_clusters = batch > 0 ? batch : 1;
   if (p->flags & SEQ_VERIFY_ALL_NODES) n_clusters = p->n_tree < 18 ? p->n_tree : 18;  // 18 * 8 = 144 CTAs <= 148 SMs
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3(n_clusters * kVCluster);
@@ -743,8 +760,28 @@ extern "C" int seq_tree_verify(const seq_tree_verify_params* p, void* stream) {
   attr[0].val.clusterDim.z = 1;
   cfg.attrs = attr;
   cfg.numAttrs = 1;
-  SEQ_CUDA_OK(cudaLaunchKernelEx(&cfg, tree_verify_kernel, a));
+  SEQ_CUDA_OK(cudaLaunchKernelEx(&cfg, kernel, a));
   return SEQ_OK;
+}
+
+extern "C" int seq_tree_verify(const seq_tree_verify_params* p, void* stream) {
+  int rc = verify_validate(p);
+  if (rc != SEQ_OK) return rc;
+  return verify_launch(p, 0, 0, 0, 0, 0, stream);
+}
+
+extern "C" int seq_tree_verify_batch(const seq_tree_verify_batch_params* bp, void* stream) {
+  if (bp == nullptr) return SEQ_ERR_INVALID_ARG;
+  const seq_tree_verify_params* p = &bp->request0;
+  int rc = verify_validate(p);
+  if (rc != SEQ_OK) return rc;
+  if (bp->batch < 1 || bp->batch > 65535 / kVCluster || (p->flags & SEQ_VERIFY_ALL_NODES)) return SEQ_ERR_INVALID_ARG;
+  if (bp->tree_stride < p->n_tree || bp->uniforms_stride < p->n_tree + 1 || bp->logits_stride % 4 != 0 ||
+      bp->logits_stride < (int64_t)(p->n_tree - 1) * p->target_row_stride + p->vocab ||
+      (p->draft_logits != nullptr && bp->logits_stride < (int64_t)(p->n_tree - 1) * p->draft_row_stride + p->vocab) ||
+      (p->residual_out != nullptr && bp->residual_stride < p->vocab))
+    return SEQ_ERR_INVALID_ARG;
+  return verify_launch(p, bp->batch, bp->tree_stride, bp->logits_stride, bp->uniforms_stride, bp->residual_stride, stream);
 }
 
 #ifdef SEQ_TRACE

@@ -45,7 +45,8 @@ def test_ctypes_structs_match_the_header(tmp_path):
     fields_a = [f[0] for f in binding.AttentionParams._fields_]
     fields_v = [f[0] for f in binding.VerifyParams._fields_]
     others = (("seq_tree_draft_sample_params", binding.DraftSampleParams), ("seq_tree_kv_commit_params", binding.KvCommitParams),
-              ("seq_tree_top_p_params", binding.TopPParams), ("seq_tree_build_params", binding.TreeBuildParams))
+              ("seq_tree_top_p_params", binding.TopPParams), ("seq_tree_build_params", binding.TreeBuildParams),
+              ("seq_tree_verify_batch_params", binding.VerifyBatchParams))
     src = tmp_path / "layout.c"
     lines = ['#include <stdio.h>', '#include <stddef.h>', '#include "seq_tree.h"', "int main(void){",
              'printf("%zu\\n", sizeof(seq_tree_attention_params));']
@@ -128,6 +129,20 @@ def test_host_checkable_errors_are_refused_before_launch(lib):
     assert lib.seq_tree_verify(C.byref(ver(vocab=400000, target_row_stride=400000, draft_row_stride=400000)), None) \
         == B.SEQ_ERR_UNSUPPORTED
     assert lib.seq_tree_verify_workspace_bytes(C.byref(ver())) == 0
+
+    def verb(**kw):
+        p = B.VerifyBatchParams()
+        p.request0 = ver()
+        p.batch, p.tree_stride, p.logits_stride, p.uniforms_stride = 4, 16, 16 * 32000, 17
+        for k, v in kw.items():
+            setattr(p, k, v)
+        return p
+
+    for kw in (dict(batch=0), dict(tree_stride=15), dict(logits_stride=15 * 32000), dict(logits_stride=16 * 32000 + 2),
+               dict(uniforms_stride=16), dict(request0=ver(flags=1, next_child_out=fake)), dict(request0=ver(vocab=0)),
+               dict(request0=ver(residual_out=fake), residual_stride=31999)):
+        assert lib.seq_tree_verify_batch(C.byref(verb(**kw)), None) == B.SEQ_ERR_INVALID_ARG, kw
+    assert lib.seq_tree_verify_batch(None, None) == B.SEQ_ERR_INVALID_ARG
 
     def commit(**kw):
         p = B.KvCommitParams()

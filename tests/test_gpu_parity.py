@@ -473,3 +473,42 @@ def test_verify_on_dp_shaped_trees(name, T):
         outcomes.append(G.check_verify(vi))
         outcomes.append(G.check_verify_target_sample(vi))
     assert outcomes.count("ok") >= len(outcomes) - 1, outcomes
+
+
+# ---------------------------------------------------------------- batched verification --------------
+@pytest.mark.parametrize("name,T,R,mode", [("tiny", 0.6, 5, "sequoia"), ("llama2-7b", 0.6, 20, "sequoia"), ("llama2-7b", 1.0, 7, "specinfer"),
+                                           ("llama2-7b", 0.6, 6, "target"), ("llama2-7b", 0.0, 4, "sequoia")])
+def test_verify_batch_equals_one_request_at_a_time(name, T, R, mode):
+    """R requests (own tree, tokens, logits, uniforms) in one launch: every request's path, bonus and residual are
+    the oracle's, and bit-identical to what a launch of its own returns."""
+    cfg = W.CONFIGS[name]
+    d = G.dev()
+    vis = [W.make_verify_inputs(cfg, T, seed) for seed in range(R)]
+    stack = lambda f: torch.stack([f(v) for v in vis]).to(d)
+    parent, tokens = stack(lambda v: v.parent), stack(lambda v: v.tokens)
+    tl, dl, un = stack(lambda v: v.target_logits), stack(lambda v: v.draft_logits), stack(lambda v: v.uniforms)
+    n, V = cfg.n_tree, cfg.vocab
+    resid = torch.full((R, V), float("nan"), dtype=torch.float32, device=d)
+    nxt = torch.full((R, n), -9, dtype=torch.int32, device=d)
+    st = torch.zeros(1, dtype=torch.int32, device=d)
+    path, plen, bonus = B.seq_tree_verify_batch(parent, tokens, tl, None if mode == "target" else dl, T, un, residual_out=resid,
+                                                next_child_out=nxt, dev_status=st, specinfer=mode == "specinfer",
+                                                target_sample=mode == "target")
+    torch.cuda.synchronize()
+    assert int(st.item()) == 0
+    checked = 0
+    for r, vi in enumerate(vis):
+        one = G.run_verify(vi, specinfer=mode == "specinfer", target_sample=mode == "target")
+        k = int(plen[r].item())
+        assert path[r, :k].cpu().tolist() == one["path"].tolist() and int(bonus[r].item()) == one["bonus"]
+        assert np.array_equal(resid[r].double().cpu().numpy(), one["residual"]) and np.array_equal(nxt[r].cpu().numpy(), one["next_child"])
+        if mode == "target":
+            ref = O.tree_verify_target_sample(vi.parent, vi.tokens, vi.target_logits, T, vi.uniforms)
+        else:
+            ref = O.tree_verify(vi.parent, vi.tokens, vi.target_logits, vi.draft_logits, T, vi.uniforms,
+                                variant=O.VARIANT_SPECINFER if mode == "specinfer" else O.VARIANT_SEQUOIA)
+        if ref["min_gap"] >= G.GAP and one["bonus"] == ref["bonus"]:
+            assert one["path"].tolist() == ref["path"].tolist()
+            assert np.abs(one["residual"] - ref["residual"]).max() < G.RESID_TOL
+            checked += 1
+    assert checked >= R - 2
