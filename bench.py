@@ -604,6 +604,25 @@ def main():
         t_attn = [evs[i][0].elapsed_time(evs[i][1]) * 1e3 for i in range(Kb)]
         t_ver = [evs[i][1].elapsed_time(evs[i][2]) * 1e3 for i in range(Kb)]
 
+        # each kernel's average launch duration: Kb launches of that kernel alone, back to back in one graph, between
+        # two events (the event nodes of graph B add a few microseconds to every call they bracket)
+        def alone(run_one):
+            g = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(g, stream=stream):
+                for i in range(Kb):
+                    run_one(Wm + i)
+            g.replay()
+            stream.synchronize()
+            a0, a1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a0.record(stream)
+            g.replay()
+            a1.record(stream)
+            stream.synchronize()
+            return a0.elapsed_time(a1) * 1e3 / Kb
+
+        attn_alone_us = alone(lambda i: attn_calls[i % na].run(stream))
+        ver_alone_us = alone(lambda i: ver_calls[i % nv].run(stream))
+
     if int(status.item()) != 0:
         raise RuntimeError(f"dev_status = {int(status.item())} after the timed region")
     ms_total = max_over_ranks(ms_total, dev)
@@ -633,8 +652,8 @@ def main():
         return
 
     peaks = measured_peaks()
-    attn_us = statistics.mean(t_attn)
-    ver_us = statistics.mean(t_ver)
+    attn_ev_us, ver_ev_us = statistics.mean(t_attn), statistics.mean(t_ver)
+    attn_us, ver_us = attn_alone_us, ver_alone_us
     flops = W.attention_algorithmic_flops(cfg, parent)
     hbm_time = attn_bytes / (peaks["hbm_gbs"] * 1e9)
     tensor_time = flops / (peaks["bf16_tflops"] * 1e12)
@@ -649,7 +668,9 @@ def main():
     roofline.update({
         "traffic": NCU_TRAFFIC_BYTES.get(cfg.name), "kernel": "seq_tree_attention", "us_per_launch": attn_us,
         "algorithmic_bytes": attn_bytes, "algorithmic_flops": flops, "peak_source": f"of {peaks['source']}",
-        "timing": f"CUDA events around each call in a replay of the same steps ({Kb} of them), mean",
+        "us_per_launch_between_event_nodes": attn_ev_us,
+        "timing": f"{Kb} launches of the kernel alone, back to back in one CUDA graph over the rotating inputs, between two "
+                  f"CUDA events; between event nodes inside the replayed steps the same call reads {attn_ev_us:.1f} us",
     })
     # verification: HBM-bound in principle (the target row of every visited node, the draft row of every
     # visited node that has children), latency-bound in practice (one cluster of 8 CTAs walks the path)
@@ -684,7 +705,8 @@ def main():
         "gpu_launches": K * launches_per_step,
         "roofline": roofline,
         "roofline_verify": roofline_verify,
-        "breakdown_us": {"attention": attn_us, "verify": ver_us,
+        "breakdown_us": {"attention": attn_us, "verify": ver_us, "attention_between_event_nodes": attn_ev_us,
+                         "verify_between_event_nodes": ver_ev_us,
                          "largest_share": "seq_tree_verify" if ver_us > attn_us else "seq_tree_attention"},
     }
     line["next_rows"] = {"kv_commit": kv_commit_leg(cfg, parent, dev, stream, peaks)}

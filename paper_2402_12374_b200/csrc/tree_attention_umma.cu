@@ -306,7 +306,8 @@ tree_attention_umma_kernel(const __grid_constant__ CUtensorMap q_map, const __gr
   const int split = blockIdx.z;  // the cluster spans blockIdx.z
   if (threadIdx.x == 128) UTRACE(2, 10);
 #ifdef SEQ_TRACE
-  if (threadIdx.x == 128 && blockIdx.y == 0 && blockIdx.z == 0 && blockIdx.x < 1024) g_cta_times[blockIdx.x][0] = gtimer();
+  const unsigned cta_lin = (blockIdx.z * gridDim.y + blockIdx.y) * gridDim.x + blockIdx.x;
+  if (threadIdx.x == 128 && cta_lin < 1024) g_cta_times[cta_lin][0] = gtimer();
 #endif
 
   // A CTA works through segments: (kv head, tile, range of the tile's 64-key blocks).  Grid mode: the one
@@ -888,7 +889,7 @@ tree_attention_umma_kernel(const __grid_constant__ CUtensorMap q_map, const __gr
   if (kStream && sm->abort_flag) break;
   }  // segments
 #ifdef SEQ_TRACE
-  if (threadIdx.x == 128 && blockIdx.y == 0 && blockIdx.z == 0 && blockIdx.x < 1024) g_cta_times[blockIdx.x][1] = gtimer();
+  if (threadIdx.x == 128 && cta_lin < 1024) g_cta_times[cta_lin][1] = gtimer();
 #endif
   // no remote access happens after the second cluster barrier, so CTAs may leave independently
   tc_fence_before();
