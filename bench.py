@@ -478,6 +478,56 @@ def verify_batch_leg(cfg, parent, ver_h, T, dev, stream) -> dict:
             "gpu_launches_per_call": 1, "note": "same results as R single-request launches (checked); outside the timed step"}
 
 
+def attention_batch_leg(cfg, parent, attn_h, dev, stream, peaks) -> dict:
+    """Not part of the timed step: R requests that share the tree and the prefix length in ONE attention launch, as R
+    times the heads (q [n, R, Hq, d], caches concatenated along the kv-head axis); sets rotate beyond L2."""
+    from paper_2402_12374_b200 import binding as B
+
+    R = 4 if cfg.n_tree <= 256 else 2
+    n, Hq = cfg.n_tree, cfg.num_q_heads
+    per = W.attention_algorithmic_bytes(cfg)
+    sets = max(2, min(len(attn_h) // R, math.ceil(2 * L2_BYTES / (R * per))))
+    parent_d = torch.from_numpy(parent).to(dev)
+    status = torch.zeros(1, dtype=torch.int32, device=dev)
+    calls = []
+    for s in range(sets):
+        grp = [attn_h[(s * R + r) % len(attn_h)] for r in range(R)]
+        q = torch.stack([a.q for a in grp], dim=1).reshape(n, R * Hq, cfg.head_dim).contiguous().to(dev)
+        k = torch.cat([a.k_cache for a in grp], dim=0).contiguous().to(dev)
+        v = torch.cat([a.v_cache for a in grp], dim=0).contiguous().to(dev)
+        calls.append(B.AttentionCall(q, k, v, None, cfg.prefix_len, parent=parent_d, dev_status=status))
+    reps = 8 * sets
+    with torch.cuda.stream(stream):
+        for c in calls[:2]:
+            c.run(stream)
+        stream.synchronize()
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g, stream=stream):
+            for i in range(reps):
+                calls[i % sets].run(stream)
+        g.replay()
+        stream.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        g.replay()
+        e1.record(stream)
+        stream.synchronize()
+    if int(status.item()) != 0:
+        raise RuntimeError(f"attention_batch dev_status = {int(status.item())}")
+    us = e0.elapsed_time(e1) * 1e3 / reps
+    nbytes = R * per
+    flops = R * W.attention_algorithmic_flops(cfg, parent)
+    hbm_t, ten_t = nbytes / (peaks["hbm_gbs"] * 1e9), flops / (peaks["bf16_tflops"] * 1e12)
+    if hbm_t >= ten_t:
+        ach = nbytes / (us * 1e-6) / 1e9
+        roof = {"bound": "hbm", "achieved": ach, "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": ach / peaks["hbm_gbs"]}
+    else:
+        ach = flops / (us * 1e-6) / 1e12
+        roof = {"bound": "tensor", "achieved": ach, "peak": peaks["bf16_tflops"], "unit": "TFLOP/s", "frac": ach / peaks["bf16_tflops"]}
+    return {"requests": R, "us_per_launch": us, "us_per_request": us / R, "sets": sets, "roofline": roof,
+            "note": "one launch for R requests with a common tree and prefix length; outside the timed step"}
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -712,6 +762,7 @@ def main():
     line["next_rows"] = {"kv_commit": kv_commit_leg(cfg, parent, dev, stream, peaks)}
     if T > 0 and args.tree_search:
         line["next_rows"]["tree_search"] = tree_search_leg(cfg, T, dev, stream)
+    line["next_rows"]["attention_batch"] = attention_batch_leg(cfg, parent, attn_h, dev, stream, peaks)
     line["next_rows"]["verify_batch"] = verify_batch_leg(cfg, parent, ver_h, T, dev, stream)
     if T > 0:
         line["next_rows"]["top_p_filter"] = top_p_leg(cfg, ver_h, T, dev, stream, peaks)

@@ -144,7 +144,8 @@ typedef struct {
   void* workspace;
   size_t workspace_bytes;
   int32_t* dev_status;
-  int32_t kernel; /* 0 = choose; 1 = force the CUDA-core kernel; 2 = force the tensor-core kernel */
+  int32_t kernel; /* 0 = choose; 1 = force the CUDA-core kernel; 2 = force the tensor-core kernel; 3, 4 = the tensor-core
+                     kernel with its stream / grid schedule forced (tuning and tests; results do not depend on it) */
   const int32_t* parent; /* nullable, [n_tree] int32, device: see "mask from the parent array" above */
 } seq_tree_attention_params;
 

@@ -24,6 +24,7 @@ SEQ_DEV_BAD_PATH = 32
 SEQ_MAX_TREE = 1024
 SEQ_NOALLOC_SCRATCH_BYTES = 384 << 10
 KERNEL_AUTO, KERNEL_CUDA_CORE, KERNEL_TENSOR_CORE = 0, 1, 2
+KERNEL_TENSOR_CORE_STREAM, KERNEL_TENSOR_CORE_GRID = 3, 4  # the tensor-core kernel with one of its two schedules forced
 
 _STATUS_NAMES = {0: "SEQ_OK", -1: "SEQ_ERR_INVALID_ARG", -2: "SEQ_ERR_UNSUPPORTED", -3: "SEQ_ERR_WORKSPACE",
                  -4: "SEQ_ERR_CUDA"}

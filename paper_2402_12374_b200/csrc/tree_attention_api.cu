@@ -35,7 +35,7 @@ int validate_attention_params(const seq_tree_attention_params* p) {
   const void* ptrs[] = {p->q, p->k_cache, p->v_cache, p->out};
   for (const void* q : ptrs)
     if (reinterpret_cast<uintptr_t>(q) % 16 != 0) return SEQ_ERR_INVALID_ARG;
-  if (p->kernel < 0 || p->kernel > 2) return SEQ_ERR_INVALID_ARG;
+  if (p->kernel < 0 || p->kernel > 4) return SEQ_ERR_INVALID_ARG;
   return SEQ_OK;
 }
 
@@ -44,7 +44,7 @@ static int choose_kernel(const seq_tree_attention_params& p) {
   const bool ok = umma_supported(p);
   if (p.mask_bits == nullptr) return ok && p.kernel != 1 ? 2 : 0;  // only the tensor-core kernel derives the mask itself
   if (p.kernel == 1) return 1;
-  if (p.kernel == 2) return ok ? 2 : 0;
+  if (p.kernel >= 2) return ok ? 2 : 0;
   if (!ok) return 1;
   // Measured on B200: even with a single query row per kv head (127 of the tile's 128 rows padding) the
   // tensor-core kernel is faster than the CUDA-core one, because it streams K/V once per kv head with

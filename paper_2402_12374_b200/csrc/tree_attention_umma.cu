@@ -89,6 +89,7 @@ constexpr int kMaxStreamTiles = 128;  // tiles per kv head the stream mode can i
 // Stream mode balances cost, not block counts: every tile is laid out with this many extra positions in
 // front of its blocks, standing for what starting and finishing a tile costs (about 4 us, in 64-key blocks).
 constexpr int kStreamTileCost = 8;
+
 constexpr uint32_t kTileBytes = 128 * 128 * 2;   // the Q tile: 128 rows x 128 elements of 16 bits
 constexpr uint32_t kHalfBytes = kTileBytes / 2;  // one 128-row x 64-element sub-tile of Q (128 B rows)
 constexpr uint32_t kKvBytes = kBlockN * 128 * 2; // a K or V tile: 64 keys x 128 elements
@@ -924,16 +925,30 @@ bool umma_supported(const seq_tree_attention_params& p) {
 // Size of the cluster that shares one (tile, kv head): 1, 2, 4 or 8 CTAs along the key range, chosen for the
 // shortest estimated makespan with one CTA per SM (about 0.4 us per 64-key block with both chains busy,
 // about 5 us of fixed cost per CTA).
-int umma_default_splits(const seq_tree_attention_params& p) {
+// How the tiles are spread over the SMs.  Grid schedule: one CTA (or a cluster of `splits` CTAs along the key
+// range) per (tile, kv head), in as many waves as that takes.  Stream schedule: 148 CTAs take equal ranges of the
+// flattened block space and share the tiles that a range boundary cuts.  p.kernel = 3 / 4 force one of them.
+struct UmmaPlan { int splits; bool stream; };
+static UmmaPlan umma_plan(const seq_tree_attention_params& p) {
   const int G = p.num_q_heads / p.num_kv_heads;
   const int nodes_per_tile = kTileM / G;
   const int tiles = (p.n_tree + nodes_per_tile - 1) / nodes_per_tile;
   const long units = (long)tiles * p.num_kv_heads;
   const int nblk = (p.prefix_len + p.n_tree + kBlockN - 1) / kBlockN;
+  const bool can_stream = tiles <= kMaxStreamTiles;
 #ifdef SEQ_TRACE
-  if (const char* e = getenv("SEQ_DEBUG_SPLITS")) return atoi(e);  // debug builds only
+  if (const char* e = getenv("SEQ_DEBUG_SPLITS")) return {atoi(e), false};  // debug builds only
 #endif
-  if (units > kNumSMs && tiles <= kMaxStreamTiles) return 1;  // the stream mode fills the SMs evenly by itself
+  if (p.kernel == 3 && can_stream) return {1, true};
+  // More units than SMs.  Measured over batches of the paper's shapes (5 to 32 requests stacked as heads): plain
+  // waves of one CTA per unit win by 5-50 % when tiles are short (a tile cut by a range boundary costs a trip
+  // through the workspace, and every CTA starts and finishes two tiles more), the stream schedule wins by 5-15 %
+  // when tiles are long (72 blocks and more) or when the last wave would be at most 60 % full.
+  if (p.kernel != 4 && can_stream && units > kNumSMs) {
+    const long waves = (units + kNumSMs - 1) / kNumSMs;
+    const bool last_wave_thin = units * 10 <= waves * kNumSMs * 6;
+    if (nblk >= 32 && (last_wave_thin || nblk >= 72)) return {1, true};
+  }
   int best = 1;
   double best_cost = -1.0;
   for (int cs = 1; cs <= kMaxClusterSplit; cs *= 2) {  // powers of two: 16 slices divide evenly among 2*cs chains
@@ -942,15 +957,14 @@ int umma_default_splits(const seq_tree_attention_params& p) {
     const double cost = (double)waves * (0.4 * ((nblk + cs - 1) / cs) + 5.0);
     if (best_cost < 0 || cost < best_cost - 1e-9) { best = cs; best_cost = cost; }
   }
-  return best;
+  return {best, false};
 }
 
-// Stream mode applies when one CTA per (tile, kv head) would need more than one wave of the SMs.
+int umma_default_splits(const seq_tree_attention_params& p) { return umma_plan(p).splits; }
+
 static bool umma_stream_mode(const seq_tree_attention_params& p, int splits) {
-  const int G = p.num_q_heads / p.num_kv_heads;
-  const int nodes_per_tile = kTileM / G;
-  const int tiles = (p.n_tree + nodes_per_tile - 1) / nodes_per_tile;
-  return splits == 1 && tiles <= kMaxStreamTiles && (long)tiles * p.num_kv_heads > kNumSMs;
+  (void)splits;
+  return umma_plan(p).stream;
 }
 
 // Workspace of the stream mode: one arrival counter per (kv head, tile), then two slots per CTA for the

@@ -351,8 +351,8 @@ def test_tensor_core_attention_stream_mode(dtype, n, L, Hq, Hkv):
     mask, _, st = G.gpu_mask(ai.parent.numpy())
     lse = torch.empty((Hq, n), dtype=torch.float32, device=d)
     call = B.AttentionCall(ai.q.to(d), ai.k_cache.to(d), ai.v_cache.to(d), mask, L, lse=lse, dev_status=st,
-                           kernel=B.KERNEL_TENSOR_CORE)
-    assert call.workspace_bytes_needed > 0, "this shape is meant to take the stream mode"
+                           kernel=B.KERNEL_TENSOR_CORE_STREAM)
+    assert call.workspace_bytes_needed > 0, "the stream schedule was asked for"
     first = call.run().clone()
     torch.cuda.synchronize()
     assert int(st.item()) == 0
@@ -389,6 +389,14 @@ def test_tensor_core_attention_mask_from_parent_array(n, L, Hq, Hkv, tree):
     fused = B.seq_tree_attention(q, k, v, None, L, parent=par, lse=lse, dev_status=st)
     torch.cuda.synchronize()
     assert int(st.item()) == 0 and torch.equal(with_mask, fused)
+    # both schedules of the kernel, whichever of them the shape gets by default: same bits with either mask source
+    # (between the schedules the key range is cut differently, so the rounding differs: oracle tolerance)
+    for forced in (B.KERNEL_TENSOR_CORE_STREAM, B.KERNEL_TENSOR_CORE_GRID):
+        a = B.seq_tree_attention(q, k, v, mask, L, kernel=forced)
+        b = B.seq_tree_attention(q, k, v, None, L, parent=par, kernel=forced, dev_status=st)
+        torch.cuda.synchronize()
+        assert int(st.item()) == 0 and torch.equal(a, b)
+        assert (a.float() - fused.float()).abs().max().item() < 2e-2
     if n <= 300:
         ref, rlse, _ = O.tree_attention(ai.q, ai.k_cache, ai.v_cache, ai.parent, L)
         assert np.abs(fused.double().cpu().numpy() - ref).max() < 2e-2
@@ -512,3 +520,38 @@ def test_verify_batch_equals_one_request_at_a_time(name, T, R, mode):
             assert np.abs(one["residual"] - ref["residual"]).max() < G.RESID_TOL
             checked += 1
     assert checked >= R - 2
+
+
+# ---------------------------------------------------------------- a batch of requests in one attention launch ----
+@pytest.mark.parametrize("name,R", [("tiny", 3), ("llama2-7b", 5), ("llama3-70b", 2)])
+def test_attention_batch_of_requests_as_stacked_heads(name, R):  # (llama2-7b x 5: 160 units in two waves of the grid schedule)
+    """Requests that share the tree and the prefix length (Sequoia's tree is fixed in advance) go through one launch
+    as R times the heads: q laid out [n, R, Hq, d], the caches concatenated along the kv-head axis.  Every request's
+    rows against the oracle on that request alone."""
+    cfg = W.CONFIGS[name]
+    d = G.dev()
+    parent = W.make_tree(cfg, 0)
+    ais = [W.make_attention_inputs(cfg, seed, parent=parent) for seed in range(R)]
+    n, Hq = cfg.n_tree, cfg.num_q_heads
+    q = torch.stack([a.q for a in ais], dim=1).reshape(n, R * Hq, cfg.head_dim).contiguous().to(d)
+    k = torch.cat([a.k_cache for a in ais], dim=0).contiguous().to(d)
+    v = torch.cat([a.v_cache for a in ais], dim=0).contiguous().to(d)
+    st = torch.zeros(1, dtype=torch.int32, device=d)
+    out = B.seq_tree_attention(q, k, v, None, cfg.prefix_len, parent=torch.from_numpy(parent).to(d), dev_status=st)
+    torch.cuda.synchronize()
+    assert int(st.item()) == 0
+    out = out.view(n, R, Hq, cfg.head_dim)
+    rows = None if n <= 64 else [0, 1, n // 2, n - 1]
+    for r, ai in enumerate(ais):
+        if rows is None:
+            ref, _, _ = O.tree_attention(ai.q, ai.k_cache, ai.v_cache, ai.parent, ai.prefix_len)
+            got = out[:, r].double().cpu().numpy()
+        else:
+            keep = sorted(set(int(a) for i in rows for a in G._path(parent, i)))
+            idx = {a: j for j, a in enumerate(keep)}
+            psub = np.array([-1 if parent[a] < 0 else idx[int(parent[a])] for a in keep], np.int32)
+            L = ai.prefix_len
+            sel = torch.tensor(list(range(L)) + [L + a for a in keep])
+            ref, _, _ = O.tree_attention(ai.q[keep], ai.k_cache[:, sel], ai.v_cache[:, sel], psub, L)
+            got = out[keep, r].double().cpu().numpy()
+        assert np.abs(got - ref).max() < G.ATTN_TOL[ai.q.dtype]
