@@ -374,7 +374,13 @@ tree_attention_umma_kernel(const __grid_constant__ CUtensorMap q_map, const __gr
   if (threadIdx.x == 0) {
     init_barriers();
     sm->abort_flag = 0;
+    // programmatic dependent launch: the next kernel in the stream may be scheduled onto free SMs from now on (it
+    // waits, as this one does below, before it touches memory); without the launch attribute this does nothing
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
   }
+  // ... and everything above ran while the previous kernel in the stream was still finishing.  Nothing before this
+  // line reads or writes global memory.
+  asm volatile("griddepcontrol.wait;" ::: "memory");
   if (a.mask_bits == nullptr)
     for (int t = threadIdx.x; t < a.n; t += kUmmaThreads) sm->parent[t] = a.parent[t];
   if (kStream && warp == 2) {  // blocks of a kv head before each place of its layout: four places per lane, then a warp scan
@@ -1056,13 +1062,15 @@ int launch_attention_umma(const seq_tree_attention_params& p, int splits, cudaSt
   cfg.blockDim = dim3(kUmmaThreads);
   cfg.dynamicSmemBytes = smem;
   cfg.stream = stream;
-  cudaLaunchAttribute attr[1];
+  cudaLaunchAttribute attr[2];
   attr[0].id = cudaLaunchAttributeClusterDimension;
   attr[0].val.clusterDim.x = 1;
   attr[0].val.clusterDim.y = 1;
   attr[0].val.clusterDim.z = splits;
+  attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;  // start under the previous kernel's tail (see the kernel)
+  attr[1].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
-  cfg.numAttrs = 1;
+  cfg.numAttrs = 2;
   // four instantiations: element type x (grid | stream) mode; the grid-mode code carries none of the stream machinery
   auto launch = [&](auto kernel) -> int {
     SEQ_CUDA_OK(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));

@@ -638,6 +638,12 @@ __global__ void __launch_bounds__(kVThreads, 1) tree_verify_kernel(const VerifyA
     asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(vsmem_u32(&sh.bar[0])) : "memory");
     asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(vsmem_u32(&sh.bar[1])) : "memory");
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    // programmatic dependent launch: the next kernel in the stream may be scheduled onto free SMs from now on
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+  }
+  // nothing above touches global memory; everything below may read what the previous kernel in the stream wrote
+  asm volatile("griddepcontrol.wait;" ::: "memory");
+  if (c.tid == 0) {
     if (!all_nodes) {  // the walk always starts at the root: fetch its rows while the tree is being read
       start_slice_copy(c, a.target, c.ps, 0);
       if (!greedy && a.n > 1 && !(a.flags & SEQ_VERIFY_TARGET_SAMPLE)) start_slice_copy(c, a.draft, c.qs, 1);  // draft row 0 is read whenever the tree has children
@@ -753,13 +759,15 @@ static int verify_launch(const seq_tree_verify_params* p, int batch, int64_t tre
   cfg.blockDim = dim3(kVThreads);
   cfg.dynamicSmemBytes = dyn;
   cfg.stream = (cudaStream_t)stream;
-  cudaLaunchAttribute attr[1];
+  cudaLaunchAttribute attr[2];
   attr[0].id = cudaLaunchAttributeClusterDimension;
   attr[0].val.clusterDim.x = kVCluster;
   attr[0].val.clusterDim.y = 1;
   attr[0].val.clusterDim.z = 1;
+  attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;  // start under the previous kernel's tail (see the kernel)
+  attr[1].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
-  cfg.numAttrs = 1;
+  cfg.numAttrs = 2;
   SEQ_CUDA_OK(cudaLaunchKernelEx(&cfg, kernel, a));
   return SEQ_OK;
 }
