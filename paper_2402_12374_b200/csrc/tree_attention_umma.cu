@@ -174,6 +174,11 @@ __device__ __forceinline__ void tma_load_3d(void* dst, const CUtensorMap* map, u
       "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];"
       ::"r"(smem_u32(dst)), "l"(map), "r"(smem_u32(bar)), "r"(c0), "r"(c1), "r"(c2) : "memory");
 }
+__device__ __forceinline__ void tma_load_5d(void* dst, const CUtensorMap* map, uint64_t* bar, int c0, int c1, int c2, int c3, int c4) {
+  asm volatile(
+      "cp.async.bulk.tensor.5d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6, %7}], [%2];"
+      ::"r"(smem_u32(dst)), "l"(map), "r"(smem_u32(bar)), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "r"(c4) : "memory");
+}
 __device__ __forceinline__ void tma_load_4d(void* dst, const CUtensorMap* map, uint64_t* bar, int c0, int c1, int c2, int c3) {
   asm volatile(
       "cp.async.bulk.tensor.4d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6}], [%2];"
@@ -441,8 +446,7 @@ tree_attention_umma_kernel(const __grid_constant__ CUtensorMap q_map, const __gr
         if (!is_v && seg > 0 && !mbar_wait(sm, &sm->o_free, (seg - 1) & 1, a.dev_status)) break;
         if (!is_v && elect_one()) {
           mbar_expect_tx(&sm->q_full, kTileBytes);
-          tma_load_4d(sm->q, &q_map, &sm->q_full, 0, 0, i0, g);
-          tma_load_4d(sm->q + kHalfBytes, &q_map, &sm->q_full, 64, 0, i0, g);
+          tma_load_5d(sm->q, &q_map, &sm->q_full, 0, 0, i0, 0, g);  // both 64-element halves by one copy
         }
         __syncwarp();
         const CUtensorMap* map = is_v ? &v_map : &k_map;
@@ -456,8 +460,7 @@ tree_attention_umma_kernel(const __grid_constant__ CUtensorMap q_map, const __gr
           if (w > 0 && !mbar_wait(sm, empty, (w - 1) & 1, a.dev_status)) break;
           if (elect_one()) {
             mbar_expect_tx(full, kKvBytes);
-            tma_load_3d(dst, map, full, 0, row, g);
-            tma_load_3d(dst + kKvHalf, map, full, 64, row, g);
+            tma_load_4d(dst, map, full, 0, row, 0, g);  // both 64-element halves by one copy
           }
           __syncwarp();
           if (lane == 0 && !is_v) UTRACE(0, 1);
@@ -1000,23 +1003,25 @@ int launch_attention_umma(const seq_tree_attention_params& p, int splits, cudaSt
   CUtensorMap q_map, k_map, v_map;
   {
     // q viewed as [kv head][node][head in group][head_dim]
-    cuuint64_t dims[4] = {(cuuint64_t)kHeadDim, (cuuint64_t)G, (cuuint64_t)p.n_tree, (cuuint64_t)p.num_kv_heads};
-    cuuint64_t strides[3] = {(cuuint64_t)p.q_stride_head * 2, (cuuint64_t)p.q_stride_tok * 2,
+    // head_dim is split into its two 64-element halves (a dimension of its own, 128 bytes apart) so that one copy
+    // brings the tile as [half][row][64 elements], the layout of two 128-byte-swizzled sub-tiles
+    cuuint64_t dims[5] = {64, (cuuint64_t)G, (cuuint64_t)p.n_tree, 2, (cuuint64_t)p.num_kv_heads};
+    cuuint64_t strides[4] = {(cuuint64_t)p.q_stride_head * 2, (cuuint64_t)p.q_stride_tok * 2, 128,
                              (cuuint64_t)p.q_stride_head * 2 * G};
-    cuuint32_t box[4] = {64, (cuuint32_t)G, (cuuint32_t)nodes_per_tile, 1};
-    cuuint32_t estr[4] = {1, 1, 1, 1};
-    if (encode(&q_map, dt, 4, const_cast<void*>(p.q), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+    cuuint32_t box[5] = {64, (cuuint32_t)G, (cuuint32_t)nodes_per_tile, 2, 1};
+    cuuint32_t estr[5] = {1, 1, 1, 1, 1};
+    if (encode(&q_map, dt, 5, const_cast<void*>(p.q), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
                CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
       return SEQ_ERR_CUDA;
   }
   for (int which = 0; which < 2; ++which) {
     // only the live rows [0, prefix_len + n_tree) are mapped: anything past them reads as zero
-    cuuint64_t dims[3] = {(cuuint64_t)kHeadDim, (cuuint64_t)(p.prefix_len + p.n_tree), (cuuint64_t)p.num_kv_heads};
-    cuuint64_t strides[2] = {(cuuint64_t)p.kv_stride_tok * 2, (cuuint64_t)p.kv_stride_head * 2};
-    cuuint32_t box[3] = {64, (cuuint32_t)kBlockN, 1};
-    cuuint32_t estr[3] = {1, 1, 1};
-    if (encode(which == 0 ? &k_map : &v_map, dt, 3, const_cast<void*>(which == 0 ? p.k_cache : p.v_cache), dims,
+    cuuint64_t dims[4] = {64, (cuuint64_t)(p.prefix_len + p.n_tree), 2, (cuuint64_t)p.num_kv_heads};
+    cuuint64_t strides[3] = {(cuuint64_t)p.kv_stride_tok * 2, 128, (cuuint64_t)p.kv_stride_head * 2};
+    cuuint32_t box[4] = {64, (cuuint32_t)kBlockN, 2, 1};
+    cuuint32_t estr[4] = {1, 1, 1, 1};
+    if (encode(which == 0 ? &k_map : &v_map, dt, 4, const_cast<void*>(which == 0 ? p.k_cache : p.v_cache), dims,
                strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
                CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
       return SEQ_ERR_CUDA;
