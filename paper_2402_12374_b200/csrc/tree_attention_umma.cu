@@ -386,6 +386,20 @@ tree_attention_umma_kernel(const __grid_constant__ CUtensorMap q_map, const __gr
   // ... and everything above ran while the previous kernel in the stream was still finishing.  Nothing before this
   // line reads or writes global memory.
   asm volatile("griddepcontrol.wait;" ::: "memory");
+  // Grid schedule: the one segment of this CTA is known from its block index, so the thread that armed the barriers
+  // requests the Q tile and the first K tile of each chain right away, before the CTA-wide barrier below and the
+  // hand-over to the producer warps (which skip what has been requested here).
+  if (!kStream && threadIdx.x == 0) {
+    const Seg s0 = seg_at(range_lo);
+    if (s0.nblk > 0) {
+      mbar_expect_tx(&sm->q_full, kTileBytes);
+      tma_load_5d(sm->q, &q_map, &sm->q_full, 0, 0, s0.i0, 0, s0.g);
+      for (int jj = 0; jj < 2 && jj < s0.nblk; ++jj) {
+        mbar_expect_tx(&sm->k_full[jj][0], kKvBytes);
+        tma_load_4d(sm->k[jj][0], &k_map, &sm->k_full[jj][0], 0, (s0.blk_lo + jj) * kBlockN, 0, s0.g);
+      }
+    }
+  }
   if (a.mask_bits == nullptr)
     for (int t = threadIdx.x; t < a.n; t += kUmmaThreads) sm->parent[t] = a.parent[t];
   if (kStream && warp == 2) {  // blocks of a kv head before each place of its layout: four places per lane, then a warp scan
@@ -444,13 +458,13 @@ tree_attention_umma_kernel(const __grid_constant__ CUtensorMap q_map, const __gr
         // seen that before they read O (waiting on o_free rather than all_done keeps every waiter of a
         // barrier within one phase of its arrivers)
         if (!is_v && seg > 0 && !mbar_wait(sm, &sm->o_free, (seg - 1) & 1, a.dev_status)) break;
-        if (!is_v && elect_one()) {
+        if (kStream && !is_v && elect_one()) {  // (grid schedule: requested before the roles split, see above)
           mbar_expect_tx(&sm->q_full, kTileBytes);
           tma_load_5d(sm->q, &q_map, &sm->q_full, 0, 0, i0, 0, g);  // both 64-element halves by one copy
         }
         __syncwarp();
         const CUtensorMap* map = is_v ? &v_map : &k_map;
-        for (int jj = 0; jj < nblk; ++jj) {
+        for (int jj = (!kStream && !is_v) ? min(2, nblk) : 0; jj < nblk; ++jj) {
           const int c = jj & 1, u = (c ? base_b : base_a) + (jj >> 1);  // chain, the chain's running block count
           const int b = u & 1, w = u >> 1;                              // stage, use count of the stage
           const int row = (blk_lo + jj) * kBlockN;
