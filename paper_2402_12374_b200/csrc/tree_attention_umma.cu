@@ -23,8 +23,9 @@
 // the bottleneck (16 per clock and SM).  Registers are rebalanced with setmaxnreg: 40 for the TMA/MMA
 // warp group, 232 for the rows.
 //
-// Work distribution.  Grid mode (at most one wave of CTAs): one CTA per (tile, kv head), or a cluster
-// of 2, 4 or 8 CTAs that split its key range.  Stream mode (more units than SMs): one CTA per SM; the
+// Work distribution.  Grid mode: one CTA per (tile, kv head), in as many waves as that takes, or (up to one wave) a
+// cluster of 2, 4 or 8 CTAs that split its key range; the thread that arms the barriers requests the Q tile and the
+// first K tiles itself, before the CTA-wide barrier.  Stream mode (many units of long tiles): one CTA per SM; the
 // 64-key blocks of all units are laid end to end (each tile preceded by a few positions that stand for
 // its fixed cost, tiles of a head taken alternately from both ends) and cut into equal ranges.  A CTA
 // works through the segments of its range with barrier phases that run on from segment to segment, so
@@ -46,6 +47,9 @@
 // the rest of a tile with zeros.
 //
 // Every mbarrier wait is bounded; a wait that runs out raises SEQ_DEV_TIMEOUT and the CTA drains.
+//
+// The kernel is launched with programmatic stream serialisation: its set-up runs under the previous kernel's tail,
+// griddepcontrol.wait precedes its first access to global memory.
 #include <cooperative_groups.h>
 #include <cuda.h>
 #include <stdlib.h>
