@@ -37,7 +37,10 @@ L2_BYTES = 126 * 1024 * 1024
 # DRAM traffic per launch (dram__bytes_read.sum + dram__bytes_write.sum) of the attention kernel, from
 # the ncu captures summarised under profiles/; None where no capture exists for that workload.
 NCU_TRAFFIC_BYTES = {
+    "tiny": 2560000,          # profiles/tree_attention_umma_traffic.md
     "llama2-7b": 18418432,    # profiles/tree_attention_umma_llama2-7b.md
+    "llama2-13b": 45945856,   # profiles/tree_attention_umma_traffic.md
+    "vicuna-33b": 65200128,   # profiles/tree_attention_umma_traffic.md
     "llama3-70b": 32801792,   # profiles/tree_attention_umma_llama3-70b.md
 }
 
