@@ -976,7 +976,10 @@ static UmmaPlan umma_plan(const seq_tree_attention_params& p) {
   for (int cs = 1; cs <= kMaxClusterSplit; cs *= 2) {  // powers of two: 16 slices divide evenly among 2*cs chains
     if (cs > 1 && cs > nblk) break;
     const long waves = (units * cs + kNumSMs - 1) / kNumSMs;
-    const double cost = (double)waves * (0.4 * ((nblk + cs - 1) / cs) + 5.0);
+    // microseconds per wave, fitted to measured launches of the paper's shapes with every split forced: 0.65 per
+    // block of a CTA's key range, 4.7 fixed, and 1.6 / 2.7 / 4 for the merge across 2 / 4 / 8 CTAs
+    const double merge = cs == 1 ? 0.0 : (cs == 2 ? 1.6 : (cs == 4 ? 2.7 : 4.0));
+    const double cost = (double)waves * (0.65 * ((nblk + cs - 1) / cs) + 4.7 + merge);
     if (best_cost < 0 || cost < best_cost - 1e-9) { best = cs; best_cost = cost; }
   }
   return {best, false};
