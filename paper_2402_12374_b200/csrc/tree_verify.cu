@@ -51,9 +51,10 @@ __shared__ int s_trace_i;
 constexpr int kVThreads = 256;
 constexpr int kVWarps = kVThreads / 32;
 constexpr int kVCluster = 8;
-constexpr int kVParts = kVCluster * kVWarps;  // 64 (rank, warp) segments cover the vocabulary
+constexpr int kVParts = kVCluster * kVWarps;  // (rank, warp) segments cover the vocabulary
+constexpr int kVPPL = kVParts / 32;           // segments per lane in an exchange: lane l reads segments l, l + 32, ...
 constexpr uint32_t kVSpinLimit = 1u << 22;
-static_assert(kVParts == 64, "the exchange reads two entries per lane");
+static_assert(kVParts % 32 == 0 && kVCluster <= 32, "an exchange reads whole groups of 32 segments; one lane per CTA writes");
 
 struct VerifyArgs {
   int32_t n, V, slice_cap, flags;
@@ -92,7 +93,7 @@ struct NodeState {
   float invSp, invSq;   // 1 / sum of exponentials relative to the global maxima
   float ipw, iqw;       // this warp's factors turning its stored exponentials into probabilities
   double C, U, Z, ZD;
-  double part_sum[2];   // residual mass of segments `lane` and `lane + 32` (probability units)
+  double part_sum[kVPPL];  // residual mass of segments `lane`, `lane + 32`, ... (probability units)
   int mode;             // 0: D proportional to q; 1: uniform over the non-rejected set
   int nS;               // |S|
   int has_q;            // qs holds this node's draft slice
@@ -145,14 +146,22 @@ __device__ __forceinline__ double sum_lanes(double v, int width) {  // butterfly
   return v;
 }
 
-// Every warp of every CTA publishes one float4 to every CTA of the cluster.  On return e0/e1 hold the
-// entries of segments `lane` and `lane + 32` (segment index = rank * 8 + warp).  One cluster barrier.
-__device__ __forceinline__ void cluster_exchange(cg::cluster_group& cluster, Ctx& c, float4 mine, float4& e0, float4& e1) {
+// Every warp of every CTA publishes one float4 to every CTA of the cluster.  On return x.e[m] holds the entry of
+// segment lane + 32 m (segments are numbered rank-major, i.e. in vocabulary order).
+struct Exch { float4 e[kVPPL]; };
+__device__ __forceinline__ void cluster_exchange(cg::cluster_group& cluster, Ctx& c, float4 mine, Exch& x) {
   if (c.lane < kVCluster) *cluster.map_shared_rank(&c.sh->xbuf[c.xpar][c.rank * kVWarps + c.warp], c.lane) = mine;
   cluster.sync();
-  e0 = c.sh->xbuf[c.xpar][c.lane];
-  e1 = c.sh->xbuf[c.xpar][c.lane + 32];
+#pragma unroll
+  for (int m = 0; m < kVPPL; ++m) x.e[m] = c.sh->xbuf[c.xpar][c.lane + 32 * m];
   c.xpar ^= 1;
+}
+
+__device__ __forceinline__ double part_total(const double* part_sum) {
+  double t = part_sum[0];
+#pragma unroll
+  for (int m = 1; m < kVPPL; ++m) t += part_sum[m];
+  return sum_lanes(t, 32);
 }
 
 // Children of v in ascending node order -> sh->kids; returns their count.  Two barriers.
@@ -295,11 +304,12 @@ __device__ int process_node(cg::cluster_group& cluster, Ctx& c, const VerifyArgs
       const int oi = __shfl_xor_sync(0xffffffffu, best_idx, o);
       if (oi != 0x7fffffff && (best_idx == 0x7fffffff || ob > best || (ob == best && oi < best_idx))) { best = ob; best_idx = oi; }
     }
-    float4 e0, e1;
-    cluster_exchange(cluster, c, make_float4(best, __int_as_float(best_idx), 0.f, 0.f), e0, e1);
-    float gb = e0.x; int gi = __float_as_int(e0.y);
-    {
-      const float ob = e1.x; const int oi = __float_as_int(e1.y);
+    Exch x;
+    cluster_exchange(cluster, c, make_float4(best, __int_as_float(best_idx), 0.f, 0.f), x);
+    float gb = x.e[0].x; int gi = __float_as_int(x.e[0].y);
+#pragma unroll
+    for (int m = 1; m < kVPPL; ++m) {
+      const float ob = x.e[m].x; const int oi = __float_as_int(x.e[m].y);
       if (oi != 0x7fffffff && (gi == 0x7fffffff || ob > gb || (ob == gb && oi < gi))) { gb = ob; gi = oi; }
     }
 #pragma unroll
@@ -384,20 +394,28 @@ __device__ int process_node(cg::cluster_group& cluster, Ctx& c, const VerifyArgs
     }
   }
   TRACE(5);
-  float4 e0, e1;
-  cluster_exchange(cluster, c, make_float4(mp, sp, mq, sq), e0, e1);
+  Exch x;
+  cluster_exchange(cluster, c, make_float4(mp, sp, mq, sq), x);
   TRACE(6);
   {
-    float Mp = warp_max(fmaxf(e0.x, e1.x)), Mq = warp_max(fmaxf(e0.z, e1.z));
-    const double a0 = (double)e0.y * (double)rel_exp(e0.x, Mp, c2), a1 = (double)e1.y * (double)rel_exp(e1.x, Mp, c2);
-    const double b0 = (double)e0.w * (double)rel_exp(e0.z, Mq, c2), b1 = (double)e1.w * (double)rel_exp(e1.z, Mq, c2);
-    const double Sp = sum_lanes(a0 + a1, 32), Sq = sum_lanes(b0 + b1, 32);
+    float Mp = x.e[0].x, Mq = x.e[0].z;
+#pragma unroll
+    for (int m = 1; m < kVPPL; ++m) { Mp = fmaxf(Mp, x.e[m].x); Mq = fmaxf(Mq, x.e[m].z); }
+    Mp = warp_max(Mp); Mq = warp_max(Mq);
+    double am[kVPPL], asum = 0.0, bsum = 0.0;
+#pragma unroll
+    for (int m = 0; m < kVPPL; ++m) {
+      am[m] = (double)x.e[m].y * (double)rel_exp(x.e[m].x, Mp, c2);
+      asum += am[m];
+      bsum += (double)x.e[m].w * (double)rel_exp(x.e[m].z, Mq, c2);
+    }
+    const double Sp = sum_lanes(asum, 32), Sq = sum_lanes(bsum, 32);
     if (!(Sp > 0.0)) dev_flag(a.dev_status, SEQ_DEV_DEGENERATE);
     st.Mp = Mp; st.Mq = Mq;
     st.invSp = Sp > 0.0 ? (float)(1.0 / Sp) : 0.f;
     st.invSq = (need_draft && Sq > 0.0) ? (float)(1.0 / Sq) : 0.f;
-    st.part_sum[0] = a0 * (double)st.invSp;
-    st.part_sum[1] = a1 * (double)st.invSp;
+#pragma unroll
+    for (int m = 0; m < kVPPL; ++m) st.part_sum[m] = am[m] * (double)st.invSp;
     st.mode = (need_draft && !(Sq > 0.0)) ? 1 : 0;  // a draft row without mass: the fallback from the start
   }
   st.ipw = rel_exp(mp, st.Mp, c2) * st.invSp;
@@ -407,7 +425,7 @@ __device__ int process_node(cg::cluster_group& cluster, Ctx& c, const VerifyArgs
 
   if (tsample) {
     // x ~ P with this node's uniform; the warp that finds x tells every CTA; a child that carries x is taken
-    const double total = sum_lanes(st.part_sum[0] + st.part_sum[1], 32);
+    const double total = part_total(st.part_sum);
     const int found = draw_token(c, st, c.sh->uniforms[v], 0.f, 0.f, st.ipw, 0.f, c.ps, total);
     if (found >= 0)
       for (int r = 0; r < kVCluster; ++r) *cluster.map_shared_rank(&c.sh->drawn[c.npar], r) = found;
@@ -477,12 +495,16 @@ __device__ int process_node(cg::cluster_group& cluster, Ctx& c, const VerifyArgs
     zr = warp_sum(zr);
     zd = warp_sum(zd);
     TRACE(9);
-    cluster_exchange(cluster, c, make_float4(zr, zd, 0.f, 0.f), e0, e1);
+    cluster_exchange(cluster, c, make_float4(zr, zd, 0.f, 0.f), x);
     TRACE(10);
-    const double Zn = sum_lanes((double)e0.x + (double)e1.x, 32), ZDn = sum_lanes((double)e0.y + (double)e1.y, 32);
+    double zsum = 0.0, zdsum = 0.0;
+#pragma unroll
+    for (int m = 0; m < kVPPL; ++m) { zsum += (double)x.e[m].x; zdsum += (double)x.e[m].y; }
+    const double Zn = sum_lanes(zsum, 32), ZDn = sum_lanes(zdsum, 32);
     if (Zn > 0.0) {
       st.C = Cn; st.U = Un; st.Z = Zn;
-      st.part_sum[0] = (double)e0.x; st.part_sum[1] = (double)e1.x;
+#pragma unroll
+      for (int m = 0; m < kVPPL; ++m) st.part_sum[m] = (double)x.e[m].x;
     } else {
       dev_flag(a.dev_status, SEQ_DEV_DEGENERATE);  // keep R
     }
@@ -502,38 +524,41 @@ __device__ int draw_token(Ctx& c, const NodeState& st, float u, float Cf, float 
                           const float* qsrc, double total) {
   // inverse CDF over the 64 (rank, warp) segments: inclusive scan across lanes, segments `lane` first
   const double tgt = (double)u * total;
-  double inc0 = st.part_sum[0];
+  // inclusive scan over the segments in vocabulary order: across lanes within a group of 32, groups in turn
+  double inc[kVPPL], before = 0.0;
+  uint32_t hit[kVPPL], pos[kVPPL];
 #pragma unroll
-  for (int o = 1; o < 32; o <<= 1) {
-    const double up = __shfl_up_sync(0xffffffffu, inc0, o);
-    if (c.lane >= o) inc0 += up;
-  }
-  const double half = __shfl_sync(0xffffffffu, inc0, 31);
-  double inc1 = st.part_sum[1];
+  for (int m = 0; m < kVPPL; ++m) {
+    double v = st.part_sum[m];
 #pragma unroll
-  for (int o = 1; o < 32; o <<= 1) {
-    const double up = __shfl_up_sync(0xffffffffu, inc1, o);
-    if (c.lane >= o) inc1 += up;
+    for (int o = 1; o < 32; o <<= 1) {
+      const double up = __shfl_up_sync(0xffffffffu, v, o);
+      if (c.lane >= o) v += up;
+    }
+    inc[m] = v + before;
+    before = __shfl_sync(0xffffffffu, inc[m], 31);
+    hit[m] = __ballot_sync(0xffffffffu, st.part_sum[m] > 0.0 && inc[m] > tgt);
+    pos[m] = __ballot_sync(0xffffffffu, st.part_sum[m] > 0.0);
   }
-  inc1 += half;
-  const uint32_t hit0 = __ballot_sync(0xffffffffu, st.part_sum[0] > 0.0 && inc0 > tgt);
-  const uint32_t hit1 = __ballot_sync(0xffffffffu, st.part_sum[1] > 0.0 && inc1 > tgt);
-  const uint32_t pos0 = __ballot_sync(0xffffffffu, st.part_sum[0] > 0.0);
-  const uint32_t pos1 = __ballot_sync(0xffffffffu, st.part_sum[1] > 0.0);
-  int part;          // segment holding the crossing
+  int part = -1;     // segment holding the crossing
   bool take_last = false;
-  if (hit0) part = __ffs(hit0) - 1;
-  else if (hit1) part = 32 + __ffs(hit1) - 1;
-  else {             // rounding left the total at or below the target: the last segment with mass
+#pragma unroll
+  for (int m = 0; m < kVPPL; ++m)
+    if (part < 0 && hit[m]) part = 32 * m + __ffs(hit[m]) - 1;
+  if (part < 0) {    // rounding left the total at or below the target: the last segment with mass
     take_last = true;
-    if (pos1) part = 63 - __clz(pos1);
-    else if (pos0) part = 31 - __clz(pos0);
-    else return -3;  // no mass anywhere: degenerate input (every thread of the cluster sees this)
+#pragma unroll
+    for (int m = kVPPL - 1; m >= 0; --m)
+      if (part < 0 && pos[m]) part = 32 * m + 31 - __clz(pos[m]);
+    if (part < 0) return -3;  // no mass anywhere: degenerate input (every thread of the cluster sees this)
   }
   if (part != c.rank * kVWarps + c.warp) return -1;
-  const double incl_part = part < 32 ? __shfl_sync(0xffffffffu, inc0, part & 31) : __shfl_sync(0xffffffffu, inc1, part & 31);
-  const double mass_part = part < 32 ? __shfl_sync(0xffffffffu, st.part_sum[0], part & 31)
-                                     : __shfl_sync(0xffffffffu, st.part_sum[1], part & 31);
+  double incl_part = 0.0, mass_part = 0.0;
+#pragma unroll
+  for (int m = 0; m < kVPPL; ++m) {  // (every lane of the owning warp takes part in the shuffles)
+    const double i_m = __shfl_sync(0xffffffffu, inc[m], part & 31), s_m = __shfl_sync(0xffffffffu, st.part_sum[m], part & 31);
+    if ((part >> 5) == m) { incl_part = i_m; mass_part = s_m; }
+  }
   const double tl = tgt - (incl_part - mass_part);  // target within this warp's segment
   double carry = 0.0;
   int found = -1, last_pos = -1;
@@ -578,7 +603,7 @@ __device__ void draw_bonus(Ctx& c, const VerifyArgs& a, const NodeState& st) {
   const bool has_q = st.has_q && (st.C != 0.0);
   const float ipw = st.ipw, iqw = has_q ? st.iqw : 0.f;
   const float* qsrc = has_q ? c.qs : c.ps;  // never dereference a slice that was not loaded
-  const double total = sum_lanes(st.part_sum[0] + st.part_sum[1], 32);
+  const double total = part_total(st.part_sum);
 
   if (a.residual_out != nullptr) {
     const float it = total > 0.0 ? (float)(1.0 / total) : 0.f;
