@@ -256,9 +256,10 @@ size_t seq_tree_verify_workspace_bytes(const seq_tree_verify_params* p);
 int seq_tree_verify(const seq_tree_verify_params* p, void* stream);
 
 /* seq_tree_verify_batch -- `batch` independent requests in one launch, one cluster of 8 CTAs per request (18
- * clusters run at a time on 148 SMs).  Every request is verified exactly as seq_tree_verify would verify it: same
- * sizes, temperature and flags for all (SEQ_VERIFY_ALL_NODES is not allowed), each with its own tree, tokens,
- * logits and uniforms.  request0 describes request 0; request r's arrays start r strides further:
+ * clusters run at a time on 148 SMs).  Every request is verified as seq_tree_verify would verify it (the same
+ * algorithm; seq_tree_verify may spread one request over a larger cluster, so vocabulary-wide sums can round
+ * differently and a decision inside the 1e-5 band can differ): same sizes, temperature and flags for all
+ * (SEQ_VERIFY_ALL_NODES is not allowed), each with its own tree, tokens, logits and uniforms.  request0 describes request 0; request r's arrays start r strides further:
  *   tree_stride      elements between the requests' parent / tokens / path / next_child_out arrays (>= n_tree);
  *   logits_stride    elements between their target matrices, and between their draft matrices (a multiple of 4,
  *                    large enough for n_tree rows);
