@@ -51,6 +51,7 @@
 // The kernel is launched with programmatic stream serialisation: its set-up runs under the previous kernel's tail,
 // griddepcontrol.wait precedes its first access to global memory.
 #include <cooperative_groups.h>
+#include <cstddef>
 #include <cuda.h>
 #include <stdlib.h>
 
@@ -121,6 +122,8 @@ struct UmmaSmem {
   uint32_t tile_mask[kTileM][SEQ_MAX_TREE / 32 + 1];
   int32_t tile_prefix[kMaxStreamTiles + 1];  // stream mode: positions of a kv head's layout before its t-th tile
 };
+
+static_assert(offsetof(UmmaSmem, v) == offsetof(UmmaSmem, k) + sizeof(UmmaSmem::k), "the cluster merge receives into k and v as one buffer");
 
 struct UmmaArgs {
   int32_t n, L, Hq, Hkv, group, mask_wpr, splits, nodes_per_tile, tiles;
@@ -850,14 +853,15 @@ tree_attention_umma_kernel(const __grid_constant__ CUtensorMap q_map, const __gr
       if (chain == 0 && a.lse != nullptr) a.lse[(size_t)h * a.n + i] = (M + log2f(Lc)) * kLn2;
     }
   } else {
-    // Step 2, across the cluster (cs = 2, 4 or 8 CTAs along the key range).  The 16 slices of 8 output
+    // Step 2, across the cluster (cs = 2 .. 8 CTAs along the key range).  The 16 slices of 8 output
     // columns are owned round-robin: slice s by CTA s % cs, as its slot s / cs.  Every CTA pushes each
-    // 8-column piece of its merged partial into the owner's receive buffer (the K stages, dead by
-    // then), laid out as float4 planes [contributor][slot][half][row], and its (m, l) into every CTA,
-    // with plain remote stores; after a cluster barrier each owner reduces its slots locally.
-    const int cs = a.splits, slots = 16 / cs;
+    // 8-column piece of its merged partial into the owner's receive buffer (the K and V stages, adjacent in
+    // shared memory and dead by then: cs * ceil(16 / cs) * 4 KB <= 84 KB of their 128 KB), laid out as float4
+    // planes [contributor][slot][half][row], and its (m, l) into every CTA, with plain remote stores; after a
+    // cluster barrier each owner reduces its slots locally.
+    const int cs = a.splits, slots = (16 + cs - 1) / cs;  // (any cs from 2 to 8; the last slots of some CTAs may be empty)
     tc_fence_before();
-    cluster.sync();  // every CTA of the cluster is done with its K stages before anyone writes into them
+    cluster.sync();  // every CTA of the cluster is done with its K and V stages before anyone writes into them
     if (threadIdx.x == 128) UTRACE(2, 7);
     // (rows past the tile's last node are padding: nothing of theirs is pushed, reduced or stored)
     if (chain == 0 && row_valid)
@@ -885,6 +889,7 @@ tree_attention_umma_kernel(const __grid_constant__ CUtensorMap q_map, const __gr
     const float inv = 1.f / Ls;  // some CTA saw the row's own key, so Ls > 0
     const float4* mine = reinterpret_cast<const float4*>(&sm->k[0][0][0]);
     for (int slot = chain; slot < slots && row_valid; slot += 2) {  // the two warp groups share this CTA's slots
+      if (slot * cs + split >= 16) break;  // (cs does not divide 16: this CTA owns one slice fewer)
       float acc[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
       for (int q = 0; q < cs; ++q) {
         const float mq = sm->ml_cta[q][r].x;
@@ -973,12 +978,12 @@ static UmmaPlan umma_plan(const seq_tree_attention_params& p) {
   }
   int best = 1;
   double best_cost = -1.0;
-  for (int cs = 1; cs <= kMaxClusterSplit; cs *= 2) {  // powers of two: 16 slices divide evenly among 2*cs chains
+  for (int cs = 1; cs <= kMaxClusterSplit; ++cs) {
     if (cs > 1 && cs > nblk) break;
     const long waves = (units * cs + kNumSMs - 1) / kNumSMs;
     // microseconds per wave, fitted to measured launches of the paper's shapes with every split forced: 0.65 per
-    // block of a CTA's key range, 4.7 fixed, and 1.6 / 2.7 / 4 for the merge across 2 / 4 / 8 CTAs
-    const double merge = cs == 1 ? 0.0 : (cs == 2 ? 1.6 : (cs == 4 ? 2.7 : 4.0));
+    // block of a CTA's key range, 4.7 fixed, and 1.6 + 0.5 per CTA beyond two for the merge across the cluster
+    const double merge = cs == 1 ? 0.0 : 1.6 + 0.5 * (cs - 2);
     const double cost = (double)waves * (0.65 * ((nblk + cs - 1) / cs) + 4.7 + merge);
     if (best_cost < 0 || cost < best_cost - 1e-9) { best = cs; best_cost = cost; }
   }
