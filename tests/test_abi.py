@@ -184,3 +184,32 @@ def test_binding_refuses_cpu_tensors():
 
     with pytest.raises(ValueError, match="no CPU path"):
         B.seq_tree_mask_from_parents(torch.tensor([-1, 0], dtype=torch.int32))
+
+
+def test_attention_schedule_choice_is_visible_through_the_workspace_size(lib):
+    """Host logic of the tensor-core kernel's plan, observable without a GPU: only its stream schedule needs a
+    workspace.  Taken for long tiles on many (tile, kv head) units (the llama3-70b shape) or when the last wave of
+    plain waves would be thin; never for short tiles; forced either way by kernel = 3 / 4."""
+    from paper_2402_12374_b200 import binding as B
+
+    fake = 0x1000
+
+    def shape(n, L, Hq, Hkv, kernel=0):
+        p = B.AttentionParams()
+        p.n_tree, p.prefix_len, p.num_q_heads, p.num_kv_heads, p.head_dim, p.dtype = n, L, Hq, Hkv, 128, B.SEQ_BF16
+        p.q = p.k_cache = p.v_cache = p.out = fake
+        p.parent = fake
+        p.q_stride_tok, p.q_stride_head = Hq * 128, 128
+        p.o_stride_tok, p.o_stride_head = Hq * 128, 128
+        p.kv_stride_tok, p.kv_stride_head, p.kv_capacity = 128, (L + n) * 128, L + n
+        p.mask_words_per_row = (n + 31) // 32
+        p.kernel = kernel
+        return lib.seq_tree_attention_workspace_bytes(C.byref(p))
+
+    assert shape(768, 4096, 64, 8) > 0             # 384 units of 76 blocks: stream schedule
+    assert shape(64, 1024, 32, 32) == 0            # 32 units: a cluster per unit
+    assert shape(64, 1024, 8 * 32, 8 * 32) == 0    # 256 units of 17 blocks (8 requests as heads): plain waves
+    assert shape(128, 2048, 4 * 40, 4 * 40) > 0    # 160 units of 34 blocks: the second wave would hold 12 CTAs
+    assert shape(128, 2048, 6 * 40, 6 * 40) == 0   # 240 units: waves
+    assert shape(64, 1024, 8 * 32, 8 * 32, kernel=3) > 0 and shape(768, 4096, 64, 8, kernel=4) == 0
+    assert shape(64, 1024, 32, 32, kernel=3) > 0   # forced even where one wave would do
