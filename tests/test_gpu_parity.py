@@ -560,3 +560,24 @@ def test_attention_batch_of_requests_as_stacked_heads(name, R):  # (llama2-7b x 
             ref, _, _ = O.tree_attention(ai.q[keep], ai.k_cache[:, sel], ai.v_cache[:, sel], psub, L)
             got = out[keep, r].double().cpu().numpy()
         assert np.abs(got - ref).max() < G.ATTN_TOL[ai.q.dtype]
+
+
+@pytest.mark.parametrize("heads", [20, 24, 28, 40, 44])
+def test_tensor_core_attention_clusters_of_odd_sizes(heads):
+    """(tile, kv head) unit counts for which the plan takes clusters of 7, 6, 5 and 3 CTAs along the key range (the 16
+    output slices of the merge do not divide evenly among them): sampled rows against the oracle, and repeated
+    calls after L2-emptying fills bit for bit."""
+    cfg = _cfg("llama2-13b", num_q_heads=heads, num_kv_heads=heads, prefix_len=2048, n_tree=128)
+    ai = W.make_attention_inputs(cfg, 21, dtype="bf16")
+    G.check_attention(ai, kernel=B.KERNEL_TENSOR_CORE, rows=[0, 1, 63, 64, 100, 127])
+    d = G.dev()
+    st = torch.zeros(1, dtype=torch.int32, device=d)
+    call = B.AttentionCall(ai.q.to(d), ai.k_cache.to(d), ai.v_cache.to(d), None, 2048, parent=ai.parent.to(d), dev_status=st)
+    assert call.workspace_bytes_needed == 0  # a cluster per unit, not the stream schedule
+    first = call.run().clone()
+    junk = torch.empty(160 << 20, dtype=torch.uint8, device=d)
+    for it in range(6):
+        junk.fill_(it)
+        again = call.run()
+        torch.cuda.synchronize()
+        assert int(st.item()) == 0 and torch.equal(first, again)
