@@ -10,7 +10,11 @@
  * Conventions shared by every entry point
  *   - All data pointers are DEVICE pointers owned by the caller, valid on the
  *     device that is current when the call is made.  The library allocates
- *     nothing, keeps no state between calls and never synchronises the host.
+ *     no device memory and never synchronises the host.  Between calls it keeps
+ *     only per-device facts that it looks up once (a driver entry point, whether
+ *     a 16-CTA cluster can be placed, function attributes already set, the
+ *     address of the built-in scratch array); those lookups are guarded, so
+ *     calls may come from several host threads.
  *   - `stream` is a cudaStream_t passed as void* (NULL = the legacy default
  *     stream).  Work is enqueued on it and the call returns at once.
  *   - Problems the host can see (null pointers, sizes out of range, bad
@@ -22,8 +26,8 @@
  *     defined outputs.  Kernels never trap and never wait without a bound;
  *     a bounded wait that runs out sets SEQ_DEV_TIMEOUT.
  *     *dev_status is only ever OR-ed into: the caller zeroes it.
- *   - Trees: n nodes, node 0 is the root (the last committed token, Section
- *     2.1: "the tree root corresponds to the current prefix"); parent[0] = -1
+ *   - Trees: n nodes, node 0 is the root (the last committed token: in Section
+ *     2.1 the root stands for the current prefix); parent[0] = -1
  *     and 0 <= parent[i] < i.  Siblings are ordered by node index, which is
  *     the order they were drawn in.  1 <= n <= SEQ_MAX_TREE.
  */
@@ -63,9 +67,9 @@ enum {
  * seq_tree_mask_from_parents -- ancestor bitmasks of a token tree.
  *
  * Defines which tree tokens a tree token may attend to: itself and the nodes
- * on its path to the root (Section 2.2: verification walks "starting at the
- * root of the tree"; Algorithm 2's input P(.|x_<n) at a node is conditioned on
- * exactly that path).  Bit j of row i is set iff j is i or an ancestor of i.
+ * on its path to the root (Section 2.2: the verification walks the tree from
+ * its root; Algorithm 2's input P(.|x_<n) at a node is conditioned on exactly
+ * that path).  Bit j of row i is set iff j is i or an ancestor of i.
  *
  *   parent        [n] int32, device.  parent[i] = -1 also allowed for i > 0
  *                 (a node with no ancestors).
@@ -74,9 +78,8 @@ enum {
  *   depth         [n] int32, device, nullable: number of parent links from i
  *                 to its root (callers use prefix_len + depth as position id).
  *   dev_status    nullable.
- * Returns SEQ_OK or SEQ_ERR_INVALID_ARG.  Run once per tree: the tree is fixed
- * across decoding steps (Section 4.1, "we determine the optimal tree structure
- * in advance").
+ * Returns SEQ_OK or SEQ_ERR_INVALID_ARG.  Run once per tree: the tree's shape
+ * is chosen ahead of time and kept for all decoding steps (Section 4.1).
  */
 int seq_tree_mask_from_parents(const int32_t* parent, int32_t n, uint32_t* mask_bits,
                                int32_t words_per_row, int32_t* depth, int32_t* dev_status,
@@ -84,8 +87,8 @@ int seq_tree_mask_from_parents(const int32_t* parent, int32_t n, uint32_t* mask_
 
 /*
  * seq_tree_attention -- attention of the n tree tokens in one target forward
- * pass (Section 1: "the speculated tokens are then verified in parallel
- * through a single forward pass of the target model").
+ * pass (Section 1: the whole speculated tree is verified by a single forward
+ * pass of the target model).
  *
  * For query head h (kv head h / (num_q_heads/num_kv_heads)) and node i:
  *     out[i,h,:] = sum_j softmax_j(softmax_scale * q[i,h,:].k[g,j,:]) * v[g,j,:]
@@ -100,7 +103,11 @@ int seq_tree_mask_from_parents(const int32_t* parent, int32_t n, uint32_t* mask_
  *   v_cache       rows [0,prefix_len) hold the prefix, rows [prefix_len,
  *                 prefix_len+n_tree) the tree tokens in node order; rows
  *                 beyond that (up to kv_capacity) are never read into the
- *                 result and may hold anything, NaN included.
+ *                 result and may hold anything, NaN included.  The rows below
+ *                 prefix_len + n_tree must be finite: a masked key's
+ *                 probability is exactly 0, but on the tensor-core path its V
+ *                 row still enters the product, and 0 * inf is NaN for every
+ *                 row of that 128-row tile.
  *   lse           nullable, [num_q_heads][n_tree] fp32: natural-log
  *                 sum-exp of the scaled scores of each row.
  * head_dim must be 128.  Base pointers and strides must keep every row
@@ -216,7 +223,7 @@ int seq_tree_attention_noalloc(const seq_tree_attention_params* p, void* stream)
  */
 enum {
   SEQ_VERIFY_ALL_NODES = 1,
-  /* Algorithm 2 without its lines 10-16 (the lines the paper prints in blue): the draft distribution D
+  /* Algorithm 2 without its draft update (the steps the paper highlights as Sequoia's addition): the draft distribution D
    * is left as it is after a rejection -- the rejected token is neither removed from it nor is it
    * renormalised -- which is SpecInfer's multi-round rejection sampling, the baseline the paper compares
    * its verification with (Section 3.2.2, Algorithm 2's caption; Theorem 3.7's counter-example).  The
@@ -274,12 +281,11 @@ typedef struct {
 
 int seq_tree_verify_batch(const seq_tree_verify_batch_params* p, void* stream);
 
-/* Library build string ("seqtree <version> sm_100a"); static storage. */
 /*
  * seq_tree_draft_sample -- the draft side's draw of the children of tree nodes: k tokens without
- * replacement from softmax(draft_logits / temperature), for n_rows nodes at once (Algorithm 2, line 5,
- * "s_i ~ D", for all children of a node; Section 5, "Implementation Details": sampling without replacement
- * is done with the exponential-sort algorithm).  A step before the verify path: its output is the tokens[]
+ * replacement from softmax(draft_logits / temperature), for n_rows nodes at once (the draw s_i ~ D inside
+ * Algorithm 2's loop, for all children of a node; Section 5, implementation details: the exponential-sort
+ * algorithm is the paper's choice for sampling without replacement).  A step before the verify path: its output is the tokens[]
  * of seq_tree_verify's children, in sibling order.
  *
  * Token t of a row gets the key E_t / q_t with E_t = -log(u_t) an exponential variate and q the row's
@@ -432,6 +438,7 @@ typedef struct {
 
 int seq_tree_top_p_filter(const seq_tree_top_p_params* p, void* stream);
 
+/* Library build string ("seqtree <version> sm_100a"); static storage. */
 const char* seq_tree_version(void);
 
 #ifdef __cplusplus

@@ -55,7 +55,7 @@
 #define ORC_BAD_PATH 32
 
 #define ORC_VARIANT_SEQUOIA 0   /* Algorithm 2 as printed */
-#define ORC_VARIANT_SPECINFER 1 /* Algorithm 2 without its blue lines 10-16 */
+#define ORC_VARIANT_SPECINFER 1 /* Algorithm 2 without its draft update (the steps that are Sequoia's addition) */
 
 int orc_num_threads(void) {
 #ifdef _OPENMP
@@ -78,7 +78,7 @@ static int32_t clean_parent(const int32_t* parent, int32_t i, int* flags) {
 }
 
 /*
- * Ancestor relation (Section 2.2, "starting at the root of the tree"):
+ * Ancestor relation (Section 2.2: the verification walks the tree from its root):
  * bit j of row i is set iff j lies on the walk i, parent[i], parent[parent[i]], ...
  * depth[i] = number of parent links on that walk.
  */
@@ -175,8 +175,8 @@ void orc_softmax_T(const float* logits, int32_t V, double T, double* out) {
 
 /*
  * Draft-side sampling without replacement by exponential sort (Section 5,
- * "Implementation Details": sampling without replacement is done with "the
- * exponential-sort algorithm"; this is the draw s_i ~ D of Algorithm 2's line 5
+ * implementation details: the paper names the exponential-sort algorithm for
+ * sampling without replacement; this is the draw s_i ~ D inside Algorithm 2's loop
  * for all k children of a node at once).
  *
  * Every token t gets an exponential variate E_t = -log(u_t) (u_t uniform on
@@ -232,16 +232,21 @@ int orc_draft_sample(const float* logits, int32_t V, double T, const float* u, i
 }
 
 /*
- * Algorithm 2, lines 3-17, for ONE node whose k children were already drawn
- * (the draws s_i ~ D of line 5 are the caller's: child_tok[i] in draw order)
- * and whose uniforms r_i are supplied.
+ * Algorithm 2's loop for ONE node whose k children were already drawn (the
+ * draws s_i ~ D are the caller's: child_tok[i] in draw order) and whose
+ * uniforms r_i are supplied.  Per child, in the algorithm's order: the
+ * acceptance test r_i < R[s_i]/D[s_i]; on rejection the residual update
+ * R <- norm(max(R - D, 0)); then the draft update, which is what Sequoia adds
+ * to multi-round rejection sampling: s_i leaves D and joins S, D falls back to
+ * the uniform distribution over the tokens outside S once it has no mass left,
+ * and D is renormalised.
  *
  *   R, D       in: P and Q (length V); out: the residual and draft after the
- *              last executed line, i.e. R is what line 18 (x ~ R) samples if
+ *              last executed step, i.e. R is what the final draw x ~ R samples if
  *              no child was accepted.
  *   accepted   index i (0-based) of the accepted child, or -1.
  *   ratio/rnum/dden (nullable, length k): R[s_i]/D[s_i], R[s_i], D[s_i] as
- *              seen by the test of line 6 (NaN where the test never ran).
+ *              seen by the acceptance test (NaN where the test never ran).
  *   min_gap    (nullable) min over executed tests of |r_i - ratio_i|.
  * Returns flags.
  */
@@ -251,7 +256,7 @@ int orc_alg2_node(double* R, double* D, int32_t V, const int32_t* child_tok,
                   double* dden_out, double* min_gap) {
   int flags = 0;
   *accepted = -1;
-  unsigned char* S = (unsigned char*)calloc((size_t)V, 1); /* line 3: S = {} */
+  unsigned char* S = (unsigned char*)calloc((size_t)V, 1); /* S = {} */
   double* Rn = (double*)malloc(sizeof(double) * (size_t)V);
   if (min_gap) *min_gap = INFINITY;
   for (int32_t i = 0; i < k; ++i) {
@@ -260,13 +265,13 @@ int orc_alg2_node(double* R, double* D, int32_t V, const int32_t* child_tok,
     if (dden_out) dden_out[i] = NAN;
   }
   int32_t n_rejected = 0;
-  for (int32_t i = 0; i < k; ++i) { /* line 4 */
+  for (int32_t i = 0; i < k; ++i) { /* one iteration per speculated child */
     int32_t s = child_tok[i];
     if (s < 0 || s >= V) { /* not a token: cannot be accepted, touches nothing */
       flags |= ORC_BAD_TOKEN;
       continue;
     }
-    double ratio; /* line 6: R[s]/D[s] */
+    double ratio; /* acceptance test: R[s]/D[s] */
     if (D[s] > 0.0)
       ratio = R[s] / D[s];
     else
@@ -278,11 +283,11 @@ int orc_alg2_node(double* R, double* D, int32_t V, const int32_t* child_tok,
       double gap = fabs(child_u[i] - ratio);
       if (gap < *min_gap) *min_gap = gap;
     }
-    if (child_u[i] < ratio) { /* line 6, strict */
-      *accepted = i;          /* line 7 */
+    if (child_u[i] < ratio) { /* strict comparison */
+      *accepted = i;
       break;
     }
-    /* line 9: R <- norm(max(R - D, 0)), with D as it stands (s not yet removed) */
+    /* residual update: R <- norm(max(R - D, 0)), with D as it stands (s not yet removed) */
     double Z = 0.0;
     for (int32_t t = 0; t < V; ++t) {
       double x = R[t] - D[t];
@@ -295,18 +300,18 @@ int orc_alg2_node(double* R, double* D, int32_t V, const int32_t* child_tok,
       flags |= ORC_DEGENERATE; /* impossible in exact arithmetic; keep R */
     }
     if (variant == ORC_VARIANT_SEQUOIA) {
-      D[s] = 0.0; /* line 10 */
-      if (!S[s]) { /* line 11 */
+      D[s] = 0.0; /* draft update: s leaves D ... */
+      if (!S[s]) { /* ... and joins S */
         S[s] = 1;
         ++n_rejected;
       }
-      double sumD = 0.0; /* line 12 */
+      double sumD = 0.0; /* mass left in D */
       for (int32_t t = 0; t < V; ++t) sumD += D[t];
-      if (sumD == 0.0) { /* lines 13-15: uniform over the non-rejected set */
+      if (sumD == 0.0) { /* none: uniform over the non-rejected set */
         for (int32_t t = 0; t < V; ++t) D[t] = S[t] ? 0.0 : 1.0;
         sumD = (double)(V - n_rejected);
       }
-      if (sumD > 0.0) /* line 16 (nothing left to normalise once S is everything) */
+      if (sumD > 0.0) /* renormalise (nothing left to normalise once S is everything) */
         for (int32_t t = 0; t < V; ++t) D[t] /= sumD;
     }
   }
@@ -315,7 +320,7 @@ int orc_alg2_node(double* R, double* D, int32_t V, const int32_t* child_tok,
   return flags;
 }
 
-/* Line 18, x ~ R, realised by inverse CDF in index order with one uniform:
+/* Algorithm 2's final draw, x ~ R, realised by inverse CDF in index order with one uniform:
  * the first t whose inclusive cumulative sum exceeds u; if rounding leaves the
  * total at or below u, the last t with R[t] > 0. */
 int32_t orc_sample_inverse_cdf(const double* R, int32_t V, double u) {
@@ -332,7 +337,7 @@ int32_t orc_sample_inverse_cdf(const double* R, int32_t V, double u) {
 /*
  * The whole verification of one tree (Section 2.2: start at the root, apply
  * the per-node algorithm, recurse into the accepted child), Algorithm 2 at
- * every visited node, then line 18 at the node where the walk stops.
+ * every visited node, then the final draw x ~ R at the node where the walk stops.
  *
  *   parent, tokens        [n]; node 0 is the root (parent[0] = -1), tokens[0] unused.
  *   target_logits         row v = next-token logits after node v.
@@ -340,8 +345,8 @@ int32_t orc_sample_inverse_cdf(const double* R, int32_t V, double u) {
  *                         (rows of leaves are never read).
  *   T                     temperature of both distributions; 0 = greedy.
  *   uniforms              [n+1]: entry c tests child node c, entry n draws the bonus.
- *   path/path_len/bonus   visited nodes (root first), their count, the token from line 18.
- *   residual_out          nullable [V]: R at line 18.
+ *   path/path_len/bonus   visited nodes (root first), their count, the token of the final draw.
+ *   residual_out          nullable [V]: R at the final draw.
  *   next_child            nullable [n]: accepted child of each visited node,
  *                         -1 if none, -2 for nodes the walk never reached.
  *   ratio_out             nullable [n]: ratio tested for child node c (NaN if untested).
@@ -395,10 +400,10 @@ int orc_tree_verify(int32_t n, int32_t V, const int32_t* parent, const int32_t* 
         if (s == a) acc = i;
       }
     } else {
-      orc_softmax_T(trow, V, T, R); /* line 3: R <- P */
+      orc_softmax_T(trow, V, T, R); /* R <- P */
       if (k > 0) {
         const float* drow = draft_logits + (size_t)cur * (size_t)draft_row_stride;
-        orc_softmax_T(drow, V, T, D); /* line 3: D <- Q */
+        orc_softmax_T(drow, V, T, D); /* D <- Q */
         for (int32_t i = 0; i < k; ++i) {
           ktok[i] = tokens[kids[i]];
           ku[i] = (double)uniforms[kids[i]];
@@ -416,7 +421,7 @@ int orc_tree_verify(int32_t n, int32_t V, const int32_t* parent, const int32_t* 
     path[plen++] = cur;
   }
   *path_len = plen;
-  *bonus = orc_sample_inverse_cdf(R, V, (double)uniforms[n]); /* line 18 */
+  *bonus = orc_sample_inverse_cdf(R, V, (double)uniforms[n]); /* x ~ R */
   if (residual_out) memcpy(residual_out, R, sizeof(double) * (size_t)V);
   free(R);
   free(D);
@@ -428,11 +433,10 @@ int orc_tree_verify(int32_t n, int32_t V, const int32_t* parent, const int32_t* 
 }
 
 /*
- * Verification by sampling from the target (Section 2.2, "Naive sampling and
- * top-k sampling": the verification algorithm "first samples from the target
- * model's distribution P(.|x_<n) at that node, and then accepts this sample if
- * it is equal to one of the children of that node"), applied recursively from
- * the root like Algorithm 2.
+ * Verification by sampling from the target (Section 2.2, the paragraph on
+ * naive and top-k sampling: a token is sampled from the target distribution
+ * at the node and accepted when one of the node's children carries it),
+ * applied recursively from the root like Algorithm 2.
  *
  * At node v: x ~ softmax(target_logits[v] / T) by inverse CDF in index order
  * with uniforms[v]; if a child of v carries token x the walk moves to the

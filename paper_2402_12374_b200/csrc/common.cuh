@@ -82,6 +82,23 @@ inline SplitLayout split_layout(void* workspace, int splits, int Hq, int n) {
   return s;
 }
 
+// Number of SMs of the current device (asked once per device, then remembered; safe from several host threads).
+int device_sm_count();
+
+// One-time set-up of a kernel function on a device (its opt-in shared-memory size and the like): `done` is a
+// per-device array of flags owned by the call site; `setup` runs once per device, races resolved by repetition
+// (the attribute calls are idempotent).
+template <typename F>
+inline int once_per_device(int* done, F setup) {
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess) return SEQ_ERR_CUDA;
+  if (dev < 0 || dev >= 64) return setup();
+  if (__atomic_load_n(&done[dev], __ATOMIC_ACQUIRE)) return SEQ_OK;
+  const int rc = setup();
+  if (rc == SEQ_OK) __atomic_store_n(&done[dev], 1, __ATOMIC_RELEASE);
+  return rc;
+}
+
 // attention: argument checks shared by the entry points, and the kernels' host launchers
 int validate_attention_params(const seq_tree_attention_params* p);
 int launch_attention_simt(const seq_tree_attention_params& p, int splits, cudaStream_t stream);

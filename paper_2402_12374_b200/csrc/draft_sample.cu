@@ -1,6 +1,6 @@
 // seq_tree_draft_sample: the draft side's draw of a node's children, k tokens without replacement from
 // softmax(logits / T), by exponential sort (Section 5, "Implementation Details": the exponential-sort
-// algorithm; Algorithm 2's line 5 for all children of a node at once).
+// algorithm; the draw s_i ~ D of Algorithm 2's loop, for all children of a node at once).
 //
 // Token t gets the key E_t / q_t with E_t = -log(u_t); ascending keys are the draw order.  The kernels work
 // with the logarithm of the inverse key, logit_t / T - log(-log u_t) (the softmax normaliser is the same for

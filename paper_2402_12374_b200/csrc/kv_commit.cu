@@ -84,7 +84,8 @@ extern "C" int seq_tree_kv_commit(const seq_tree_kv_commit_params* p, void* stre
   a.new_prefix_len = p->new_prefix_len; a.dev_status = p->dev_status;
   const int64_t total = (int64_t)a.planes * a.cols * (a.cache[1] != nullptr ? 2 : 1);
   const int64_t want = (total + kCommitThreads - 1) / kCommitThreads;
-  const int grid = (int)(want < 148 * 8 ? want : 148 * 8);  // at most one wave of 8 CTAs per SM; larger caches loop
+  const long cap = (long)device_sm_count() * 8;
+  const int grid = (int)(want < cap ? want : cap);  // at most one wave of 8 CTAs per SM; larger caches loop
   kv_commit_kernel<<<grid, kCommitThreads, 0, static_cast<cudaStream_t>(stream)>>>(a);
   SEQ_CUDA_OK(cudaGetLastError());
   return SEQ_OK;

@@ -13,6 +13,23 @@ size_t umma_workspace_bytes(const seq_tree_attention_params& p);
 
 static size_t elem_size(int dtype) { return dtype == SEQ_F32 ? 4 : 2; }
 
+int device_sm_count() {
+  static int cached[64];  // 0 = not asked yet
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess) return 148;
+  if (dev >= 0 && dev < 64) {
+    const int c = __atomic_load_n(&cached[dev], __ATOMIC_RELAXED);
+    if (c > 0) return c;
+  }
+  int sms = 0;
+  if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms < 1) {
+    cudaGetLastError();
+    return 148;  // no device to ask (a host without a GPU sizing a workspace): B200's count
+  }
+  if (dev >= 0 && dev < 64) __atomic_store_n(&cached[dev], sms, __ATOMIC_RELAXED);
+  return sms;
+}
+
 int validate_attention_params(const seq_tree_attention_params* p) {
   if (p == nullptr) return SEQ_ERR_INVALID_ARG;
   if (p->q == nullptr || p->k_cache == nullptr || p->v_cache == nullptr || p->out == nullptr ||

@@ -252,7 +252,7 @@ int simt_default_splits(const seq_tree_attention_params& p) {
   const long rows = (long)p.n_tree * p.num_q_heads;
   const int chunks = (p.prefix_len + p.n_tree + 31) / 32;
   int splits = 1;
-  while (rows * splits < 148 * 4 && chunks / (splits * 2 * kSimtWarps) >= 4 && splits < 16) splits *= 2;
+  while (rows * splits < device_sm_count() * 4 && chunks / (splits * 2 * kSimtWarps) >= 4 && splits < 16) splits *= 2;
   return splits;
 }
 

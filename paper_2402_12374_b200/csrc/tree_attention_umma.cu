@@ -24,7 +24,7 @@
 // warp group, 232 for the rows.
 //
 // Work distribution.  Grid mode: one CTA per (tile, kv head), in as many waves as that takes, or (up to one wave) a
-// cluster of 2, 4 or 8 CTAs that split its key range; the thread that arms the barriers requests the Q tile and the
+// cluster of 2 to 8 CTAs that split its key range; the thread that arms the barriers requests the Q tile and the
 // first K tiles itself, before the CTA-wide barrier.  Stream mode (many units of long tiles): one CTA per SM; the
 // 64-key blocks of all units are laid end to end (each tile preceded by a few positions that stand for
 // its fixed cost, tiles of a head taken alternately from both ends) and cut into equal ranges.  A CTA
@@ -35,7 +35,7 @@
 // the pieces are added in CTA order, so the result does not depend on who finishes last.
 //
 // Merge.  The CTAs that share (tile, kv head) form a thread-block cluster along the key
-// range (cs = 1, 2, 4 or 8); its 2*cs chains share the 16 slices of 8 output columns round-robin.  Every chain pushes,
+// range (cs = 1 .. 8); its 2*cs chains share the 16 slices of 8 output columns round-robin.  Every chain pushes,
 // for every row, each 8-column piece of its unnormalised fp32 accumulator into the shared memory of
 // the chain that owns that slice (the K/V stages, dead by then) and its (m, l) into every CTA, with
 // plain remote stores over distributed shared memory; after one cluster barrier each owner reduces
@@ -89,7 +89,6 @@ constexpr int kBlockN = 64;         // keys per block
 constexpr int kUmmaThreads = 384;   // warp group 0: TMA warp, MMA warp, two spare; warp groups 1, 2: rows of chains A, B
 constexpr int kRegsLight = 40, kRegsRows = 232;  // after setmaxnreg: 128*40 + 256*232 = 384*168
 constexpr int kMaxClusterSplit = 8;
-constexpr int kNumSMs = 148;
 constexpr int kMaxStreamTiles = 128;  // tiles per kv head the stream mode can index
 // Stream mode balances cost, not block counts: every tile is laid out with this many extra positions in
 // front of its blocks, standing for what starting and finishing a tile costs (about 4 us, in 64-key blocks).
@@ -116,6 +115,7 @@ struct UmmaSmem {
   uint64_t o_free;                           // the row threads have read both accumulators (one phase per segment)
   uint32_t tmem_base;
   volatile int abort_flag;
+  int32_t abort_seen[2];                     // [segment parity]: abort_flag as one row thread saw it, so that all 256 leave together
   int32_t last_part;                         // stream mode: this CTA completed the tile (broadcast to the row threads)
   // mask from the parent array: the tree, and the ancestor rows of the current tile's nodes (row stride 33 words)
   int32_t parent[SEQ_MAX_TREE];
@@ -720,7 +720,11 @@ tree_attention_umma_kernel(const __grid_constant__ CUtensorMap q_map, const __gr
   // O_A and O_B itself; only (m, l) goes through shared memory.
   if (threadIdx.x == 128) UTRACE(2, 6);
   sm->ml_chain[seg & 1][chain][r] = (ok && n_mine > 0) ? make_float2(m_used, l) : make_float2(-INFINITY, 0.f);
+  // Whether to stop after this segment is decided once for all row threads: a flag raised between two threads' own
+  // reads would send some to the closing barrier and the rest into the next segment's bar.sync, which has no bound.
+  if (kStream && threadIdx.x == 128) sm->abort_seen[seg & 1] = sm->abort_flag;
   asm volatile("bar.sync 1, 256;" ::: "memory");  // the 256 row threads only
+  const bool stop_here = kStream && sm->abort_seen[seg & 1] != 0;
   float M, Lc;           // reference maximum and denominator of the CTA's merged partial
   float merged[64];      // its columns [64*chain, 64*chain + 64), unnormalised
   {
@@ -914,7 +918,7 @@ tree_attention_umma_kernel(const __grid_constant__ CUtensorMap q_map, const __gr
   if (threadIdx.x == 128) UTRACE(2, 9);
   pos = sg.next;
   ++seg_n; base_n += n_mine;
-  if (kStream && sm->abort_flag) break;
+  if (stop_here) break;
   }  // segments
 #ifdef SEQ_TRACE
   if (threadIdx.x == 128 && cta_lin < 1024) g_cta_times[cta_lin][1] = gtimer();
@@ -930,16 +934,16 @@ typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t,
                                   CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
 
 static EncodeTiledFn encode_fn() {
-  static EncodeTiledFn fn = nullptr;
-  if (fn == nullptr) {
-    void* p = nullptr;
+  static void* cached = nullptr;  // the driver's entry point, looked up once (the same answer from every thread)
+  void* p = __atomic_load_n(&cached, __ATOMIC_ACQUIRE);
+  if (p == nullptr) {
     cudaDriverEntryPointQueryResult qres;
     if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &qres) != cudaSuccess ||
-        qres != cudaDriverEntryPointSuccess)
+        qres != cudaDriverEntryPointSuccess || p == nullptr)
       return nullptr;
-    fn = reinterpret_cast<EncodeTiledFn>(p);
+    __atomic_store_n(&cached, p, __ATOMIC_RELEASE);
   }
-  return fn;
+  return reinterpret_cast<EncodeTiledFn>(p);
 }
 
 bool umma_supported(const seq_tree_attention_params& p) {
@@ -949,11 +953,8 @@ bool umma_supported(const seq_tree_attention_params& p) {
   return true;
 }
 
-// Size of the cluster that shares one (tile, kv head): 1, 2, 4 or 8 CTAs along the key range, chosen for the
-// shortest estimated makespan with one CTA per SM (about 0.4 us per 64-key block with both chains busy,
-// about 5 us of fixed cost per CTA).
 // How the tiles are spread over the SMs.  Grid schedule: one CTA (or a cluster of `splits` CTAs along the key
-// range) per (tile, kv head), in as many waves as that takes.  Stream schedule: 148 CTAs take equal ranges of the
+// range) per (tile, kv head), in as many waves as that takes.  Stream schedule: one CTA per SM, each with an equal range of the
 // flattened block space and share the tiles that a range boundary cuts.  p.kernel = 3 / 4 force one of them.
 struct UmmaPlan { int splits; bool stream; };
 static UmmaPlan umma_plan(const seq_tree_attention_params& p) {
@@ -963,6 +964,7 @@ static UmmaPlan umma_plan(const seq_tree_attention_params& p) {
   const long units = (long)tiles * p.num_kv_heads;
   const int nblk = (p.prefix_len + p.n_tree + kBlockN - 1) / kBlockN;
   const bool can_stream = tiles <= kMaxStreamTiles;
+  const int kNumSMs = device_sm_count();
 #ifdef SEQ_TRACE
   if (const char* e = getenv("SEQ_DEBUG_SPLITS")) return {atoi(e), false};  // debug builds only
 #endif
@@ -1005,12 +1007,12 @@ static size_t stream_count_bytes(const seq_tree_attention_params& p) {
   const int tiles = (p.n_tree + nodes_per_tile - 1) / nodes_per_tile;
   return ((size_t)tiles * p.num_kv_heads * sizeof(int32_t) + 255) & ~(size_t)255;
 }
-static constexpr size_t kStreamMlBytes = (size_t)2 * kNumSMs * kTileM * sizeof(float2);
-static constexpr size_t kStreamOBytes = (size_t)2 * kNumSMs * 2 * 16 * kTileM * sizeof(float4);
+static size_t stream_ml_bytes() { return (size_t)2 * device_sm_count() * kTileM * sizeof(float2); }
+static size_t stream_o_bytes() { return (size_t)2 * device_sm_count() * 2 * 16 * kTileM * sizeof(float4); }
 
 size_t umma_workspace_bytes(const seq_tree_attention_params& p) {
   if (!umma_stream_mode(p, umma_default_splits(p))) return 0;
-  return stream_count_bytes(p) + kStreamMlBytes + kStreamOBytes;
+  return stream_count_bytes(p) + stream_ml_bytes() + stream_o_bytes();
 }
 
 int launch_attention_umma(const seq_tree_attention_params& p, int splits, cudaStream_t stream) {
@@ -1068,7 +1070,7 @@ int launch_attention_umma(const seq_tree_attention_params& p, int splits, cudaSt
   a.ws_count = nullptr; a.ws_ml = nullptr; a.ws_o = nullptr;
   if (a.stream) {
     const size_t cnt_bytes = stream_count_bytes(p);
-    if (p.workspace == nullptr || p.workspace_bytes < cnt_bytes + kStreamMlBytes + kStreamOBytes) return SEQ_ERR_WORKSPACE;
+    if (p.workspace == nullptr || p.workspace_bytes < cnt_bytes + stream_ml_bytes() + stream_o_bytes()) return SEQ_ERR_WORKSPACE;
     if (reinterpret_cast<uintptr_t>(p.workspace) % 256 != 0) return SEQ_ERR_INVALID_ARG;
     for (int t = 0; t < tiles; ++t) {
       const int i1 = (t + 1) * nodes_per_tile < p.n_tree ? (t + 1) * nodes_per_tile : p.n_tree;
@@ -1078,13 +1080,17 @@ int launch_attention_umma(const seq_tree_attention_params& p, int splits, cudaSt
     uint8_t* ws = static_cast<uint8_t*>(p.workspace);
     a.ws_count = reinterpret_cast<int32_t*>(ws);
     a.ws_ml = reinterpret_cast<float2*>(ws + cnt_bytes);
-    a.ws_o = reinterpret_cast<float4*>(ws + cnt_bytes + kStreamMlBytes);
+    a.ws_o = reinterpret_cast<float4*>(ws + cnt_bytes + stream_ml_bytes());
     SEQ_CUDA_OK(cudaMemsetAsync(a.ws_count, 0, cnt_bytes, stream));  // the counters start at zero (the kernel leaves them at zero)
   }
 
   const size_t smem = sizeof(UmmaSmem) + 1024;
   cudaLaunchConfig_t cfg = {};
-  cfg.gridDim = a.stream ? dim3(kNumSMs, 1, 1) : dim3(tiles, p.num_kv_heads, splits);
+  // Stream schedule: one CTA per SM, but never more CTAs than positions in the layout: a range must not be empty
+  // (the CTAs that share a cut tile are counted from the ranges, and each of them has to arrive).
+  const int sms = device_sm_count();
+  const int stream_ctas = a.total_blocks < sms ? (int)a.total_blocks : sms;
+  cfg.gridDim = a.stream ? dim3(stream_ctas, 1, 1) : dim3(tiles, p.num_kv_heads, splits);
   cfg.blockDim = dim3(kUmmaThreads);
   cfg.dynamicSmemBytes = smem;
   cfg.stream = stream;
@@ -1098,13 +1104,18 @@ int launch_attention_umma(const seq_tree_attention_params& p, int splits, cudaSt
   cfg.attrs = attr;
   cfg.numAttrs = 2;
   // four instantiations: element type x (grid | stream) mode; the grid-mode code carries none of the stream machinery
-  auto launch = [&](auto kernel) -> int {
-    SEQ_CUDA_OK(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+  auto launch = [&](auto kernel, int which) -> int {
+    static int attr_done[4][64];  // the opt-in shared-memory size is set once per kernel and device
+    const int rc = once_per_device(attr_done[which], [&]() -> int {
+      SEQ_CUDA_OK(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+      return SEQ_OK;
+    });
+    if (rc != SEQ_OK) return rc;
     SEQ_CUDA_OK(cudaLaunchKernelEx(&cfg, kernel, q_map, k_map, v_map, a));
     return SEQ_OK;
   };
-  if (p.dtype == SEQ_BF16) return a.stream ? launch(tree_attention_umma_kernel<true, true>) : launch(tree_attention_umma_kernel<true, false>);
-  return a.stream ? launch(tree_attention_umma_kernel<false, true>) : launch(tree_attention_umma_kernel<false, false>);
+  if (p.dtype == SEQ_BF16) return a.stream ? launch(tree_attention_umma_kernel<true, true>, 0) : launch(tree_attention_umma_kernel<true, false>, 1);
+  return a.stream ? launch(tree_attention_umma_kernel<false, true>, 2) : launch(tree_attention_umma_kernel<false, false>, 3);
 }
 
 }  // namespace seqtree

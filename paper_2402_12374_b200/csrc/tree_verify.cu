@@ -16,9 +16,9 @@
 // number of rejections is
 //     R[t] = max(p[t] - C q[t] - U, 0) / Z ,     D[t] = q[t] / ZD   (or 1/(V-|S|) once the
 //                                                                   uniform fallback has fired)
-// for scalars C, U, Z, ZD: line 9's  R <- norm(max(R - D, 0))  becomes  C += Z/ZD  (or
+// for scalars C, U, Z, ZD: the residual update  R <- norm(max(R - D, 0))  becomes  C += Z/ZD  (or
 // U += Z/(V-|S|) after the fallback) followed by one vocabulary-wide sum for the new Z, and
-// line 12's sum(D) is the direct sum ZD of the surviving q, never a subtraction.
+// the test sum(D) = 0 is taken on the direct sum ZD of the surviving q, never a subtraction.
 //
 // Each warp owns a contiguous segment of its CTA's slice and keeps its exponentials relative to
 // the segment's own maximum (no block-wide maximum is needed); the per-warp sums of the last pass
@@ -115,14 +115,23 @@ extern "C" size_t seq_tree_verify_workspace_bytes(const seq_tree_verify_params* 
 }
 
 // One instance (cluster size) of the launch.
-template <int CL, typename Shared, typename Kernel>
+// Slot: a number of its own for every kernel function (two kernels can share a pointer type, hence a template instance).
+template <int CL, typename Shared, int Slot, typename Kernel>
 static int verify_launch_with(Kernel kernel, VerifyArgs a, int vocab, int n_clusters, bool check_only, cudaStream_t stream) {
   a.slice_cap = (((vocab + CL - 1) / CL) + 3) & ~3;
   static_assert(sizeof(Shared) % 16 == 0, "the slices behind the shared block must stay 16-byte aligned");
   const size_t dyn = sizeof(Shared) + (size_t)2 * a.slice_cap * sizeof(float);
   if (dyn > 227 * 1024) return SEQ_ERR_UNSUPPORTED;  // vocabulary too large for CL slices
-  SEQ_CUDA_OK(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)dyn));
-  if (CL > 8) SEQ_CUDA_OK(cudaFuncSetAttribute(kernel, cudaFuncAttributeNonPortableClusterSizeAllowed, 1));
+  {
+    // function attributes once per (kernel instance, device): the largest shared-memory size any vocabulary can ask for
+    static int attr_done[64];  // (one array per instantiation of this template, i.e. per Slot)
+    const int rc = once_per_device(attr_done, [&]() -> int {
+      SEQ_CUDA_OK(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024));
+      if (CL > 8) SEQ_CUDA_OK(cudaFuncSetAttribute(kernel, cudaFuncAttributeNonPortableClusterSizeAllowed, 1));
+      return SEQ_OK;
+    });
+    if (rc != SEQ_OK) return rc;
+  }
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3(n_clusters * CL);
   cfg.blockDim = dim3(kVThreads);
@@ -167,19 +176,22 @@ static int verify_launch(const seq_tree_verify_params* p, int batch, int64_t tre
     if (!fits8 && (!fits16 || batch > 0 || (p->flags & SEQ_VERIFY_ALL_NODES))) return SEQ_ERR_UNSUPPORTED;
   }
 
-  if (batch > 0) return verify_launch_with<8, vcl8::VShared>(vcl8::tree_verify_kernel<true>, a, p->vocab, batch, false, s);
+  if (batch > 0) return verify_launch_with<8, vcl8::VShared, 0>(vcl8::tree_verify_kernel<true>, a, p->vocab, batch, false, s);
   if (p->flags & SEQ_VERIFY_ALL_NODES)  // 18 * 8 = 144 CTAs <= 148 SMs
-    return verify_launch_with<8, vcl8::VShared>(vcl8::tree_verify_kernel<false>, a, p->vocab, p->n_tree < 18 ? p->n_tree : 18, false, s);
+    return verify_launch_with<8, vcl8::VShared, 1>(vcl8::tree_verify_kernel<false>, a, p->vocab, p->n_tree < 18 ? p->n_tree : 18, false, s);
   // One request: the cluster of 16 where the device can place one (asked once per device), else the cluster of 8.
   // Vocabularies below 8192 tokens gain nothing from more CTAs.
   static int wide_ok[64];  // per device: 0 = not asked yet, 1 = yes, 2 = no
   int dev = 0;
   SEQ_CUDA_OK(cudaGetDevice(&dev));
-  if (dev >= 0 && dev < 64 && wide_ok[dev] == 0)
-    wide_ok[dev] = verify_launch_with<16, vcl16::VShared>(vcl16::tree_verify_kernel<false>, a, 32000, 1, true, s) == SEQ_OK ? 1 : 2;
-  if (dev >= 0 && dev < 64 && wide_ok[dev] == 1 && p->vocab >= 8192)
-    return verify_launch_with<16, vcl16::VShared>(vcl16::tree_verify_kernel<false>, a, p->vocab, 1, false, s);
-  return verify_launch_with<8, vcl8::VShared>(vcl8::tree_verify_kernel<false>, a, p->vocab, 1, false, s);
+  int wide = (dev >= 0 && dev < 64) ? __atomic_load_n(&wide_ok[dev], __ATOMIC_ACQUIRE) : 2;
+  if (wide == 0) {  // (two threads asking at once get the same answer)
+    wide = verify_launch_with<16, vcl16::VShared, 2>(vcl16::tree_verify_kernel<false>, a, 32000, 1, true, s) == SEQ_OK ? 1 : 2;
+    __atomic_store_n(&wide_ok[dev], wide, __ATOMIC_RELEASE);
+  }
+  if (wide == 1 && p->vocab >= 8192)
+    return verify_launch_with<16, vcl16::VShared, 2>(vcl16::tree_verify_kernel<false>, a, p->vocab, 1, false, s);
+  return verify_launch_with<8, vcl8::VShared, 1>(vcl8::tree_verify_kernel<false>, a, p->vocab, 1, false, s);
 }
 
 extern "C" int seq_tree_verify(const seq_tree_verify_params* p, void* stream) {

@@ -75,3 +75,50 @@ def test_invariants_on_a_config_shaped_tree():
         last_kids = [c for c in range(len(par)) if par[c] == path[-1]]
         assert all(int(vi.tokens[c]) != r["bonus"] for c in last_kids)
         assert abs(r["residual"].sum() - 1) < 1e-12 and r["flags"] == 0
+
+
+def _accept_measure(parent, tokens, tl, T, N=20000):
+    """Lebesgue measure of the root uniforms for which some child is accepted: the walk is a deterministic
+    function of uniforms[0], so the measure is read off a midpoint grid (exact when the CDF steps lie on it)."""
+    n = len(parent)
+    hits = 0
+    for j in range(N):
+        u = np.zeros(n + 1, np.float32)
+        u[0] = (j + 0.5) / N
+        hits += O.tree_verify_target_sample(parent, tokens, tl, T, u)["path_len"] > 1
+    return hits / N
+
+
+def test_printed_top_k_example_accepts_with_probability_0_6():
+    """The value the paper prints for this verifier (appendix, proof of the robustness theorem, item on top-k
+    naive sampling and optimal transport): P = Q = [0.6, 0.4], one speculated token (the draft's top-1, token 0)
+    is accepted with probability 0.6, although 1 - |P - Q|_1 / 2 = 1."""
+    import json
+    import os
+
+    g = json.load(open(os.path.join(os.path.dirname(__file__), "golden", "paper_examples.json")))["top_k_naive_sampling"]
+    P, Q, k = np.array(g["P"]), np.array(g["Q"]), g["k"]
+    top = np.argsort(-Q, kind="stable")[:k]                 # the draft's top-k tokens are the children
+    parent = W.star_tree(1 + k)
+    tokens = np.concatenate([[0], top]).astype(np.int32)
+    tl = np.tile(np.log(P).astype(np.float32), (1 + k, 1))
+    assert abs(_accept_measure(parent, tokens, tl, 1.0) - g["naive_acceptance"]) < 1e-9
+    assert abs((1 - np.abs(P - Q).sum() / 2) - g["optimal_transport_acceptance"]) < 1e-12
+    # Algorithm 2 on the same pair accepts always (optimal transport at k = 1)
+    st = O.alg2_node(P, Q, top, [0.999999])
+    assert st["accepted"] == 0
+
+
+def test_top_k_cover_property_of_sampling_from_the_target():
+    """Same proof, next item: when the k children are the draft's top-k and contain the target's support, or
+    k = V, the sample from the target is always among them."""
+    P = np.array([0.5, 0.0, 0.3, 0.0, 0.2])
+    tl = np.log(np.maximum(P, 1e-300)).astype(np.float32)
+    tl[P == 0] = -np.inf
+    for kids in ([0, 2, 4], [4, 2, 0, 1], [0, 1, 2, 3, 4]):
+        parent = W.star_tree(1 + len(kids))
+        tokens = np.array([0] + kids, np.int32)
+        assert _accept_measure(parent, tokens, np.tile(tl, (len(parent), 1)), 1.0, N=2000) == 1.0
+    # one token of the support missing: accepted exactly with the mass that is covered
+    parent = W.star_tree(3)
+    assert abs(_accept_measure(parent, np.array([0, 0, 4], np.int32), np.tile(tl, (3, 1)), 1.0, N=2000) - 0.7) < 1e-9

@@ -119,6 +119,30 @@ def test_rejection_lemma_and_residual_definition():
     np.testing.assert_allclose(st["D"], expect_D / expect_D.sum(), atol=1e-15)
 
 
+def test_inverse_cdf_when_the_cumulative_sum_never_exceeds_the_uniform():
+    """x ~ R by inverse CDF (Algorithm 2's last line, reading: first index whose inclusive sum exceeds u, else
+    the LAST index with R > 0).  The second branch by hand: trailing zeros must not be returned, nor -1, nor V-1."""
+    assert O.sample_inverse_cdf([0.5, 0.5, 0.0, 0.0], 1.0) == 1          # total == u, two trailing zeros
+    assert O.sample_inverse_cdf([0.0, 0.3, 0.0], 0.9) == 1               # total well below u, zeros on both sides
+    assert O.sample_inverse_cdf([0.25, 0.0, 0.25, 0.25, 0.0], 0.75) == 3  # c == u is not "exceeds"
+    assert O.sample_inverse_cdf([1.0], 1.0) == 0
+    assert O.sample_inverse_cdf([0.0, 0.0], 0.5) == -1                   # no mass at all: nothing to return
+    # a total that rounding left below 1 (ten times 0.1 sums to 0.9999999999999999) and u just above it
+    R = [0.1] * 10 + [0.0, 0.0]
+    c = 0.0
+    for x in R:  # the sequential sum (Python's built-in sum compensates)
+        c += x
+    assert c < 1.0 and O.sample_inverse_cdf(R, float(np.nextafter(c, 2.0))) == 9 and O.sample_inverse_cdf(R, c) == 9
+    # and the first branch for contrast: strict crossing, zeros are never chosen
+    assert O.sample_inverse_cdf([0.5, 0.0, 0.5], 0.5) == 2
+    assert O.sample_inverse_cdf([0.5, 0.0, 0.5], 0.4999) == 0
+    # the whole walk reaches that branch too: a single node whose uniform is 1 (outside [0,1), legal for the oracle)
+    tl = np.log(np.array([[0.5, 0.5, 1e-300, 1e-300]])).astype(np.float32)
+    tl[0, 2:] = -np.inf
+    r = O.tree_verify(np.array([-1], np.int32), np.array([0], np.int32), tl, tl, 1.0, np.array([0.0, 1.0], np.float32))
+    assert r["bonus"] == 1 and r["path"].tolist() == [0]
+
+
 def test_hand_checked_three_token_example():
     P, Q = [0.5, 0.3, 0.2], [0.2, 0.5, 0.3]
     st = O.alg2_node(P, Q, [1, 2], [0.7, 0.1])
