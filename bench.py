@@ -1,14 +1,21 @@
 #!/usr/bin/env python
 """Benchmark of the token-tree verify step (ancestor mask -> tree attention -> Algorithm 2 walk).
 
-    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload NAME] [--temperature T]
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload all|NAME] [--temperature T]
     python bench.py --impl reference ...      # the fp64 CPU oracle on the host cores, same metric
 
-One "step" is one pass of the whole hot path over one synthetic request.  The K timed steps are
-captured in one CUDA graph and replayed between two CUDA events; inputs rotate over enough
-independent copies that every step reads memory that is not in L2.  One JSON line is printed by
-rank 0.  With N > 1 (torchrun) every rank verifies its own requests (weak scaling, no data-path
-collective) and the time is the maximum over ranks.
+One "step" is one pass of the whole hot path over one synthetic request.  By default all five
+workloads are measured in one run: the headline (`value`, `config`, `roofline`, `e2e`,
+`cpu_baseline`) is the largest single-GPU one, llama3-70b, and `per_workload` carries the same
+figures for each of the five.  The K steps of a workload are captured in one CUDA graph; the graph
+is replayed 25 times, each replay between its own pair of CUDA events (median, minimum and maximum
+are printed; the median is the value); inputs rotate over enough independent copies that every
+step reads memory that is not in L2.  One JSON line is printed by rank 0.  With N > 1 (torchrun)
+every rank verifies its own requests (weak scaling, no data-path collective) and every time is the
+maximum over ranks.
+
+    python bench.py --ncu-traffic-csv FILE    # no GPU work: turn an ncu --csv log of DRAM byte
+                                              # counters into profiles/tree_attention_umma_traffic.json
 """
 from __future__ import annotations
 
@@ -34,22 +41,55 @@ METRIC = "us_per_tree_verify_step"
 UNIT = "us/step"
 L2_BYTES = 126 * 1024 * 1024
 
-# DRAM traffic per launch (dram__bytes_read.sum + dram__bytes_write.sum) of the attention kernel, from
-# the ncu captures summarised under profiles/; None where no capture exists for that workload.
-NCU_TRAFFIC_BYTES = {
-    "tiny": 2560000,          # profiles/tree_attention_umma_traffic.md
-    "llama2-7b": 18418432,    # profiles/tree_attention_umma_llama2-7b.md
-    "llama2-13b": 45945856,   # profiles/tree_attention_umma_traffic.md
-    "vicuna-33b": 65200128,   # profiles/tree_attention_umma_traffic.md
-    "llama3-70b": 32801792,   # profiles/tree_attention_umma_llama3-70b.md
-}
+HEADLINE = "llama3-70b"                     # the largest configuration that fits one GPU
+ALL_WORKLOADS = ["tiny", "llama2-7b", "llama2-13b", "vicuna-33b", "llama3-70b"]
+SPEC_HBM_GBS, SPEC_BF16_TFLOPS = 8000.0, 2250.0   # nominal figures, printed beside the measured ones
+REPLAYS = 25                                 # timed replays of a workload's graph
+TRAFFIC_FILE = os.path.join(ROOT, "profiles", "tree_attention_umma_traffic.json")
+
+
+def ncu_traffic_bytes(workload: str):
+    """DRAM bytes per launch of the attention kernel (dram__bytes_read.sum + dram__bytes_write.sum) from the ncu
+    capture recorded in profiles/ (written by `bench.py --ncu-traffic-csv`); None without a capture."""
+    try:
+        return json.load(open(TRAFFIC_FILE))["bytes_per_launch"].get(workload)
+    except (OSError, ValueError, KeyError):
+        return None
+
+
+def write_traffic_file(csv_path: str, workload: str, command: str) -> None:
+    """Parses an `ncu --csv` log that holds dram__bytes_read.sum and dram__bytes_write.sum per captured launch
+    and records the attention kernel's mean bytes per launch for `workload`."""
+    import csv
+
+    per_launch = {}
+    with open(csv_path, newline="") as f:
+        rows = [r for r in csv.reader(f) if len(r) > 5]
+    header = next(r for r in rows if "Metric Name" in r)
+    col = {name: header.index(name) for name in ("ID", "Kernel Name", "Metric Name", "Metric Unit", "Metric Value")}
+    scale = {"byte": 1.0, "Kbyte": 1e3, "Mbyte": 1e6, "Gbyte": 1e9}
+    for r in rows:
+        if r is header or len(r) <= max(col.values()) or "tree_attention_umma" not in r[col["Kernel Name"]]:
+            continue
+        if r[col["Metric Name"]] in ("dram__bytes_read.sum", "dram__bytes_write.sum"):
+            val = float(r[col["Metric Value"]].replace(",", "")) * scale.get(r[col["Metric Unit"]], 1.0)
+            per_launch[r[col["ID"]]] = per_launch.get(r[col["ID"]], 0.0) + val
+    if not per_launch:
+        raise SystemExit(f"{csv_path}: no dram byte counters of the attention kernel found")
+    data = {"bytes_per_launch": {}, "source": {}}
+    if os.path.exists(TRAFFIC_FILE):
+        data = json.load(open(TRAFFIC_FILE))
+    data["bytes_per_launch"][workload] = int(round(sum(per_launch.values()) / len(per_launch)))
+    data["source"][workload] = {"launches": len(per_launch), "command": command}
+    json.dump(data, open(TRAFFIC_FILE, "w"), indent=1, sort_keys=True)
+    print(f"{TRAFFIC_FILE}: {workload} -> {data['bytes_per_launch'][workload]} B per launch over {len(per_launch)} launches")
 
 
 def measured_peaks():
     path = os.path.join(ROOT, "MEASURED_PEAKS.json")
     if os.path.exists(path):
         d = json.load(open(path))
-        return dict(hbm_gbs=d["hbm_gbs"], bf16_tflops=d["bf16_tflops"], source="measured")
+        return dict(hbm_gbs=d["hbm_gbs"], bf16_tflops=d["bf16_tflops"], source="measured")  # burst figure: kernels are timed alone
     return dict(hbm_gbs=6650.0, bf16_tflops=1590.0, source="fallback")
 
 
@@ -151,7 +191,7 @@ def build_requests(cfg, T, rank, n_attn, n_verify, tree="random", parent=None):
     return parent, attn, ver
 
 
-def oracle_step_sample(cfg, parent, ai, vi, T, budget_flops=1.5e9):
+def oracle_step_sample(cfg, parent, ai, vi, T, budget_flops=3e10):
     """Times the oracle on one step, attention restricted to a leading block of nodes (closed under
     'parent') when the whole tree would take too long; returns (seconds scaled to a full step, note)."""
     from oracle import oracle as O
@@ -172,8 +212,16 @@ def oracle_step_sample(cfg, parent, ai, vi, T, budget_flops=1.5e9):
     return t_attn + t_ver, note
 
 
+def config_dict(cfg, T, tree):
+    """The workload's description, the same in both arms."""
+    return {"workload": cfg.name, "temperature": T, "n_tree": cfg.n_tree, "prefix_len": cfg.prefix_len,
+            "heads": f"{cfg.num_q_heads}/{cfg.num_kv_heads}", "vocab": cfg.vocab, "requests_per_gpu": 1,
+            "tree": "seeded random within the config's depth and fan-out bounds" if tree == "random"
+                    else "seq_tree_build on the paper's printed acceptance vector"}
+
+
 def run_reference(args, cfg, T):
-    """--impl reference: the oracle, as it stands, on the host cores."""
+    """--impl reference: the oracle, as it stands, on the host cores; every step a bounded sample of the workload."""
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
         return
@@ -185,20 +233,19 @@ def run_reference(args, cfg, T):
 
         parent, _ = tree_dp.build_tree(W.PAPER_ACCEPTANCE_VECTOR, cfg.n_tree, cfg.max_depth, cfg.max_fanout or 31)
     parent, attn, ver = build_requests(cfg, T, 0, 1, 1, parent=parent)
-    for _ in range(min(args.warmup, 2)):
+    for _ in range(args.warmup):
         oracle_step_sample(cfg, parent, attn[0], ver[0], T)
-    steps = min(args.steps, 20)
     times, note = [], ""
-    for _ in range(steps):
+    for _ in range(args.steps):
         t, note = oracle_step_sample(cfg, parent, attn[0], ver[0], T)
         times.append(t)
     us = 1e6 * sum(times) / len(times)
     cores = O.num_threads()
     line = {
-        "impl": "reference", "metric": METRIC, "value": us, "unit": UNIT, "n_gpus": args.gpus, "steps": steps,
-        "warmup": min(args.warmup, 2), "ms_per_step": us / 1e3, "higher_is_better": False, "scaling": "weak",
+        "impl": "reference", "metric": METRIC, "value": us, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": us / 1e3, "higher_is_better": False, "scaling": "weak",
         "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-        "config": {"workload": cfg.name, "temperature": T},
+        "config": config_dict(cfg, T, args.tree),
         "cpu_baseline": {"value": us, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": note},
         "e2e": {"value": us, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
         "gpu_launches": 0,
@@ -532,27 +579,298 @@ def attention_batch_leg(cfg, parent, attn_h, dev, stream, peaks) -> dict:
             "note": "one launch for R requests with a common tree and prefix length; outside the timed step"}
 
 
+def device_verify_sets(cfg, parent, T, count, dev, seed):
+    """Further logit sets of a workload, drawn on the device with the host recipe's distributions (target N(0, sigma^2),
+    draft = target + noise, children's tokens by a Gumbel top-k draw from the draft at T, uniforms in [0, 1)): the
+    first set of every workload comes from the host (it is the one the oracle is timed on); these only serve to
+    rotate the verification's inputs through more memory than the L2 holds."""
+    n, V = len(parent), cfg.vocab
+    gen = torch.Generator(device=dev)
+    gen.manual_seed(W.BASE_SEED + 7919 * cfg.config_id + seed)
+    kids = W.children_lists(parent)
+    sets = []
+    for _ in range(count):
+        tl = cfg.target_sigma * torch.randn((n, V), device=dev, generator=gen)
+        dl = tl + cfg.draft_noise_sigma * torch.randn((n, V), device=dev, generator=gen)
+        tokens = torch.zeros(n, dtype=torch.int32, device=dev)
+        for node, ch in enumerate(kids):
+            if ch:
+                key = dl[node] / T if T > 0 else dl[node].clone()
+                if T > 0:
+                    key = key - torch.log(-torch.log(torch.rand(V, device=dev, generator=gen).clamp_(1e-9, 1 - 1e-7)))
+                tokens[ch] = torch.topk(key, len(ch)).indices.to(torch.int32)
+        u = torch.rand(n + 1, device=dev, generator=gen)
+        sets.append((tokens, tl, dl, u))
+    return sets
+
+
+def timed_replays(graph, stream, replays, world, dev):
+    """`replays` replays of one CUDA graph, each between its own pair of events after a barrier; per replay the
+    maximum over ranks.  Returns the list of milliseconds."""
+    import torch.distributed as dist
+
+    out = []
+    for _ in range(replays):
+        torch.cuda.synchronize()
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        graph.replay()
+        e1.record(stream)
+        stream.synchronize()
+        out.append(e0.elapsed_time(e1))
+    if world > 1:
+        t = torch.tensor(out, dtype=torch.float64, device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        out = t.tolist()
+    return out
+
+
+def spread(ms_list, per):
+    us = sorted(1e3 * m / per for m in ms_list)
+    return {"median": statistics.median(us), "min": us[0], "max": us[-1], "replays": len(us)}
+
+
+def floors_leg(dev, stream) -> dict:
+    """What the device gives to a kernel that only reads (GB/s over a buffer far larger than L2) and to a launch
+    that does next to nothing (one warp, one dependent load from memory that is not in L2), both through this
+    library's probe kernels, as CUDA graphs."""
+    from paper_2402_12374_b200 import binding as B
+
+    buf = torch.empty(1 << 30, dtype=torch.uint8, device=dev)
+    buf.random_(0, 255)
+    sink = torch.zeros(4096, dtype=torch.int64, device=dev)
+    src = buf.view(torch.int32)
+    dst = torch.zeros(1, dtype=torch.int32, device=dev)
+    reps = 10
+    with torch.cuda.stream(stream):
+        B.seq_tree_probe_stream_read(buf, sink, stream)
+        B.seq_tree_probe_dependent_load(src, dst, stream)
+        stream.synchronize()
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g, stream=stream):
+            for _ in range(reps):
+                B.seq_tree_probe_stream_read(buf, sink, stream)
+        n_small = 200
+        g2 = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g2, stream=stream):
+            for i in range(n_small):  # addresses 4 MiB apart: every launch misses the L2 (the pass above evicted them)
+                B.seq_tree_probe_dependent_load(src[i * (1 << 20):], dst, stream)
+        out = {}
+        for name, graph, per in (("read", g, reps), ("small", g2, n_small)):
+            graph.replay()
+            stream.synchronize()
+            if name == "small":
+                g.replay()  # evict
+                stream.synchronize()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record(stream)
+            graph.replay()
+            e1.record(stream)
+            stream.synchronize()
+            out[name] = e0.elapsed_time(e1) * 1e3 / per
+    del buf
+    return {"stream_read_gbs": (1 << 30) / (out["read"] * 1e-6) / 1e9, "stream_read_bytes": 1 << 30,
+            "launch_with_one_dependent_load_us": out["small"],
+            "note": "seq_tree_probe_stream_read over 1 GiB (10 passes in one graph) and seq_tree_probe_dependent_load "
+                    "(200 launches in one graph, each on an address that is not in L2)"}
+
+
+def run_workload(cfg, T, args, rank, local_rank, world, dev, stream, peaks, with_legs):
+    """Everything measured on one workload; returns (result dict, state for the e2e / cpu legs)."""
+    from paper_2402_12374_b200 import binding as B
+
+    K, Wm = args.steps, max(3, args.warmup)
+    n = cfg.n_tree
+    attn_bytes = W.attention_algorithmic_bytes(cfg)
+    na = n_sets(attn_bytes)
+    logits_set_bytes = 2 * n * cfg.vocab * 4
+    nv = 4 if logits_set_bytes < (1 << 28) else 3
+    parent, attn_h, ver_h = build_requests(cfg, T, rank, na, 1, args.tree)
+
+    status = torch.zeros(1, dtype=torch.int32, device=dev)
+    parent_d = torch.from_numpy(parent).to(dev)
+    mask = torch.empty((n, (n + 31) // 32), dtype=torch.int32, device=dev)
+    depth = torch.empty(n, dtype=torch.int32, device=dev)
+    fused_mask = (not args.separate_mask and args.kernel != B.KERNEL_CUDA_CORE and cfg.dtype in ("fp16", "bf16")
+                  and 128 % (cfg.num_q_heads // cfg.num_kv_heads) == 0)
+    attn_calls, ver_calls, workspace = [], [], None
+    for ai in attn_h:
+        call = B.AttentionCall(ai.q.to(dev), ai.k_cache.to(dev), ai.v_cache.to(dev), None if fused_mask else mask,
+                               cfg.prefix_len, parent=parent_d, workspace=workspace, dev_status=status, kernel=args.kernel)
+        workspace = call.workspace
+        attn_calls.append(call)
+    vi0 = ver_h[0]
+    ver_sets = [(vi0.tokens.to(dev), vi0.target_logits.to(dev), vi0.draft_logits.to(dev), vi0.uniforms.to(dev))]
+    ver_sets += device_verify_sets(cfg, parent, T, nv - 1, dev, rank_seed_base(rank))
+    for tok, tl, dl, u in ver_sets:
+        ver_calls.append(B.VerifyCall(parent_d, tok, tl, dl, T, u, dev_status=status))
+    combine = args.kernel == B.KERNEL_CUDA_CORE and attn_calls[0].workspace_bytes_needed > 0
+    launches_per_step = (0 if fused_mask else 1) + (2 if combine else 1) + 1
+
+    def step(i, s):
+        if not fused_mask:
+            B.seq_tree_mask_from_parents(parent_d, mask_bits=mask, depth=depth, dev_status=status, stream=s)
+        attn_calls[i % na].run(s)
+        ver_calls[i % nv].run(s)
+
+    flush = torch.empty(160 << 20, dtype=torch.uint8, device=dev)
+    Kb = max(K, 4 * na)   # launches per graph of the per-kernel timings: every attention set a few times
+
+    def graph_of(body, count):
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g, stream=stream):
+            for i in range(count):
+                body(Wm + i)
+        g.replay()  # untimed replay: uploads the graph
+        stream.synchronize()
+        return g
+
+    with torch.cuda.stream(stream):
+        for i in range(Wm):
+            step(i, stream)
+        stream.synchronize()
+        g_step = graph_of(lambda i: step(i, stream), K)
+        g_attn = graph_of(lambda i: attn_calls[i % na].run(stream), Kb)
+        g_ver_warm = graph_of(lambda i: ver_calls[i % nv].run(stream), Kb)
+        # verification with its logits out of the L2: a write larger than the L2 before every launch, and the same
+        # graph without the launches to subtract
+        Kc = 12
+        g_ver_cold = graph_of(lambda i: (flush.fill_(i & 127), ver_calls[i % nv].run(stream)), Kc)
+        g_flush = graph_of(lambda i: flush.fill_(i & 127), Kc)
+
+        with ClockSampler(local_rank) as clocks:
+            ms_steps = timed_replays(g_step, stream, REPLAYS, world, dev)
+            t_end = time.time() + 0.2  # keep the GPU under the same load a little longer: short regions still see clocks
+            while time.time() < t_end:
+                g_step.replay()
+                stream.synchronize()
+        ms_attn = timed_replays(g_attn, stream, 9, world, dev)
+        ms_ver_warm = timed_replays(g_ver_warm, stream, 9, world, dev)
+        ms_cold = timed_replays(g_ver_cold, stream, 9, world, dev)
+        ms_flush = timed_replays(g_flush, stream, 9, world, dev)
+    if int(status.item()) != 0:
+        raise RuntimeError(f"{cfg.name}: dev_status = {int(status.item())} after the timed region")
+
+    step_us = spread(ms_steps, K)
+    attn_us = statistics.median(ms_attn) * 1e3 / Kb
+    ver_warm_us = statistics.median(ms_ver_warm) * 1e3 / Kb
+    ver_cold_us = (statistics.median(ms_cold) - statistics.median(ms_flush)) * 1e3 / Kc
+    flops = W.attention_algorithmic_flops(cfg, parent)
+    hbm_time = attn_bytes / (peaks["hbm_gbs"] * 1e9)
+    tensor_time = flops / (peaks["bf16_tflops"] * 1e12)
+    if hbm_time >= tensor_time:
+        achieved = attn_bytes / (attn_us * 1e-6) / 1e9
+        roofline = {"bound": "hbm", "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                    "frac": achieved / peaks["hbm_gbs"], "frac_of_spec": achieved / SPEC_HBM_GBS, "spec_peak": SPEC_HBM_GBS}
+    else:
+        achieved = flops / (attn_us * 1e-6) / 1e12
+        roofline = {"bound": "tensor", "achieved": achieved, "peak": peaks["bf16_tflops"], "unit": "TFLOP/s",
+                    "frac": achieved / peaks["bf16_tflops"], "frac_of_spec": achieved / SPEC_BF16_TFLOPS,
+                    "spec_peak": SPEC_BF16_TFLOPS}
+    roofline.update({
+        "traffic": ncu_traffic_bytes(cfg.name), "kernel": "seq_tree_attention", "us_per_launch": attn_us,
+        "algorithmic_bytes": attn_bytes, "algorithmic_flops": flops, "peak_source": f"of {peaks['source']}",
+        "hbm_gbs": attn_bytes / (attn_us * 1e-6) / 1e9,
+        "timing": f"{Kb} launches of the kernel alone, back to back in one CUDA graph over {na} rotating input sets "
+                  f"({na * attn_bytes >> 20} MiB, L2-cold), median of 9 replays",
+    })
+    # verification: the rows of the visited nodes are the algorithmic minimum (B_path); what the schedule moved on
+    # top of that is speculative work
+    has_child = np.zeros(n, dtype=bool)
+    has_child[parent[1:][parent[1:] >= 0]] = True
+    torch.cuda.synchronize()
+    path_bytes, visited = [], []
+    for vc in ver_calls:
+        plen = int(vc.path_len.item())
+        nodes = vc.path[:plen].cpu().numpy()
+        visited.append(plen)
+        path_bytes.append(sum(4 * cfg.vocab * (2 if has_child[v] else 1) for v in nodes))
+    b_path = float(np.mean(path_bytes))
+    moved = ver_calls[0].bytes_moved_estimate(b_path) if hasattr(ver_calls[0], "bytes_moved_estimate") else b_path
+    ver_gbs = moved / (ver_cold_us * 1e-6) / 1e9
+    roofline_verify = {"bound": "hbm", "achieved": ver_gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                       "frac": ver_gbs / peaks["hbm_gbs"], "frac_of_spec": ver_gbs / SPEC_HBM_GBS, "traffic": None,
+                       "kernel": "seq_tree_verify", "us_per_launch": ver_cold_us, "us_per_launch_l2_warm": ver_warm_us,
+                       "b_path_bytes": b_path, "bytes_moved": moved, "b_path_over_bytes_moved": b_path / moved,
+                       "visited_nodes_mean": float(np.mean(visited)),
+                       "timing": f"L2-cold: {Kc} launches in one graph, a 160 MiB write before each, minus the same graph "
+                                 f"without the launches; L2-warm: {Kb} launches back to back over {nv} logit sets",
+                       "note": "a dependent walk: latency-bound, its HBM fraction says little"}
+    res = {
+        "us_per_step": step_us, "ms_per_step": step_us["median"] / 1e3,
+        "attention_us": attn_us, "verify_us": ver_cold_us, "verify_us_l2_warm": ver_warm_us,
+        "verify_us_in_step": step_us["median"] - attn_us,
+        "roofline": roofline, "roofline_verify": roofline_verify, "clocks": clocks.summary(),
+        "dtype": cfg.dtype, "gpu_launches": K * launches_per_step * (REPLAYS + 1),
+        "config": dict(config_dict(cfg, T, args.tree),
+                       l2=f"inputs rotate over {na} attention sets ({na * attn_bytes >> 20} MiB) and {nv} logit sets",
+                       launch="CUDA graph of the K steps",
+                       mask="from the parent array inside the attention kernel" if fused_mask else "separate launch"),
+        "largest_share": "seq_tree_verify" if ver_cold_us > attn_us else "seq_tree_attention",
+    }
+    state = dict(parent=parent, attn_h=attn_h, ver_h=ver_h, fused_mask=fused_mask)
+    if with_legs:
+        legs = {"kv_commit": kv_commit_leg(cfg, parent, dev, stream, peaks)}
+        if T > 0 and args.tree_search:
+            legs["tree_search"] = tree_search_leg(cfg, T, dev, stream)
+        legs["attention_batch"] = attention_batch_leg(cfg, parent, attn_h, dev, stream, peaks)
+        ver_like = [_HostLike(*s) for s in ver_sets]
+        legs["verify_batch"] = verify_batch_leg(cfg, parent, ver_like, T, dev, stream)
+        if T > 0:
+            legs["top_p_filter"] = top_p_leg(cfg, ver_like, T, dev, stream, peaks)
+            legs["draft_sample"] = draft_sample_leg(cfg, parent, ver_like, T, dev, stream, peaks)
+        res["next_rows"] = legs
+    del attn_calls, ver_calls, ver_sets, flush
+    torch.cuda.empty_cache()
+    return res, state
+
+
+class _HostLike:
+    """The fields of a logit set that the legs around the step read (tensors may live on either side)."""
+
+    def __init__(self, tokens, target_logits, draft_logits, uniforms):
+        self.tokens, self.target_logits, self.draft_logits, self.uniforms = tokens, target_logits, draft_logits, uniforms
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=500)
+    ap.add_argument("--steps", type=int, default=100)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", default="llama2-7b", choices=sorted(W.CONFIGS))
-    ap.add_argument("--temperature", type=float, default=0.6)
+    ap.add_argument("--workload", default="all", choices=["all"] + sorted(W.CONFIGS),
+                    help="all: the five workloads in one run, llama3-70b as the headline; or one of them alone")
+    ap.add_argument("--temperature", type=float, default=None, help="default: the workload's own (0.6; 1.0 for llama2-13b)")
     ap.add_argument("--kernel", type=int, default=0, help="0 auto, 1 CUDA-core, 2 tensor-core attention")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-legs", action="store_true", help="skip the calls around the step (next_rows) and the floors")
     ap.add_argument("--tree", default="random", choices=["random", "dp"],
                     help="random: seeded random tree within the config's bounds; dp: Sequoia's dynamic program on the paper's acceptance vector")
     ap.add_argument("--tree-search", action="store_true",
                     help="also time the step on trees of growing size and run the Speedup(n, d) search on that t(n)")
     ap.add_argument("--separate-mask", action="store_true",
                     help="build the ancestor mask with a launch of its own instead of inside the attention kernel")
+    ap.add_argument("--ncu-traffic-csv", default=None,
+                    help="no GPU work: parse this ncu --csv log (dram byte counters) into profiles/ for --workload")
+    ap.add_argument("--ncu-command", default="", help="with --ncu-traffic-csv: the capture command, recorded beside the numbers")
     args = ap.parse_args()
-    cfg = W.CONFIGS[args.workload]
-    T = args.temperature
+    if args.ncu_traffic_csv:
+        write_traffic_file(args.ncu_traffic_csv, HEADLINE if args.workload == "all" else args.workload, args.ncu_command)
+        return
+    names = ALL_WORKLOADS if args.workload == "all" else [args.workload]
+    head_name = HEADLINE if args.workload == "all" else args.workload
+
+    def temp_of(cfg):
+        if args.temperature is not None:
+            return args.temperature
+        return 0.6 if 0.6 in cfg.temperatures else cfg.temperatures[-1]
+
     if args.impl == "reference":
-        run_reference(args, cfg, T)
+        cfg = W.CONFIGS[head_name]
+        run_reference(args, cfg, temp_of(cfg))
         return
 
     from paper_2402_12374_b200 import binding as B
@@ -569,125 +887,29 @@ def main():
         import torch.distributed as dist
 
         dist.init_process_group("nccl", device_id=dev)
-    K, Wm = args.steps, max(3, args.warmup)
-
-    attn_bytes = W.attention_algorithmic_bytes(cfg)
-    n = cfg.n_tree
-    logits_bytes_touched = 4 * 2 * cfg.vocab * 4  # a walk reads a few rows of each matrix
-    na = n_sets(attn_bytes)
-    nv = min(n_sets(logits_bytes_touched), 8 if cfg.vocab * n * 8 < (1 << 28) else 3)
-    parent, attn_h, ver_h = build_requests(cfg, T, rank, na, nv, args.tree)
-
-    status = torch.zeros(1, dtype=torch.int32, device=dev)
-    parent_d = torch.from_numpy(parent).to(dev)
-    mask = torch.empty((n, (n + 31) // 32), dtype=torch.int32, device=dev)
-    depth = torch.empty(n, dtype=torch.int32, device=dev)
-    attn_calls, ver_calls = [], []
-    workspace = None
-    # The ancestor mask: derived from the parent array inside the attention kernel (tensor-core kernel), or by a
-    # launch of its own before it (--separate-mask, and always for the CUDA-core kernel).
-    fused_mask = (not args.separate_mask and args.kernel != B.KERNEL_CUDA_CORE and cfg.dtype in ("fp16", "bf16")
-                  and 128 % (cfg.num_q_heads // cfg.num_kv_heads) == 0)
-    for ai in attn_h:
-        call = B.AttentionCall(ai.q.to(dev), ai.k_cache.to(dev), ai.v_cache.to(dev), None if fused_mask else mask,
-                               cfg.prefix_len, parent=parent_d, workspace=workspace, dev_status=status, kernel=args.kernel)
-        workspace = call.workspace
-        attn_calls.append(call)
-    for vi in ver_h:
-        ver_calls.append(B.VerifyCall(parent_d, vi.tokens.to(dev), vi.target_logits.to(dev), vi.draft_logits.to(dev),
-                                      T, vi.uniforms.to(dev), dev_status=status))
-    combine = args.kernel == B.KERNEL_CUDA_CORE and attn_calls[0].workspace_bytes_needed > 0  # split-KV partials merged by a second kernel
-    launches_per_step = (0 if fused_mask else 1) + (2 if combine else 1) + 1
-
+    peaks = measured_peaks()
     stream = torch.cuda.Stream(device=dev)
 
-    def step(i, s, ev=None):
-        if not fused_mask:
-            B.seq_tree_mask_from_parents(parent_d, mask_bits=mask, depth=depth, dev_status=status, stream=s)
-        if ev:
-            ev[0].record(s)
-        attn_calls[i % na].run(s)
-        if ev:
-            ev[1].record(s)
-        ver_calls[i % nv].run(s)
-        if ev:
-            ev[2].record(s)
-
-    with torch.cuda.stream(stream):
-        for i in range(Wm):
-            step(i, stream)
-        stream.synchronize()
-        # graph A: the K timed steps, nothing else
-        graph = torch.cuda.CUDAGraph()
-        with torch.cuda.graph(graph, stream=stream):
-            for i in range(K):
-                step(Wm + i, stream)
-        # graph B: the same K steps with event nodes around the kernels (per-kernel durations)
-        Kb = min(K, 200)
-        evs = [[torch.cuda.Event(enable_timing=True, external=True) for _ in range(3)] for _ in range(Kb)]
-        graph_b = torch.cuda.CUDAGraph()
-        with torch.cuda.graph(graph_b, stream=stream):
-            for i in range(Kb):
-                step(Wm + i, stream, evs[i])
-        graph.replay()  # untimed replay: uploads the graph
-        graph_b.replay()
-        stream.synchronize()
-
-        def barrier():
-            torch.cuda.synchronize()
-            if world > 1:
-                dist.barrier()
-            torch.cuda.synchronize()
-
-        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        barrier()
-        with ClockSampler(local_rank) as clocks:
-            e0.record(stream)
-            graph.replay()
-            e1.record(stream)
-            stream.synchronize()
-            # keep sampling over a few more replays so that short regions still see clocks under load
-            t_end = time.time() + 0.25
-            while time.time() < t_end:
-                graph.replay()
-                stream.synchronize()
-        barrier()
-        ms_total = e0.elapsed_time(e1)
-        graph_b.replay()
-        stream.synchronize()
-        t_attn = [evs[i][0].elapsed_time(evs[i][1]) * 1e3 for i in range(Kb)]
-        t_ver = [evs[i][1].elapsed_time(evs[i][2]) * 1e3 for i in range(Kb)]
-
-        # each kernel's average launch duration: Kb launches of that kernel alone, back to back in one graph, between
-        # two events (the event nodes of graph B add a few microseconds to every call they bracket)
-        def alone(run_one):
-            g = torch.cuda.CUDAGraph()
-            with torch.cuda.graph(g, stream=stream):
-                for i in range(Kb):
-                    run_one(Wm + i)
-            g.replay()
-            stream.synchronize()
-            a0, a1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-            a0.record(stream)
-            g.replay()
-            a1.record(stream)
-            stream.synchronize()
-            return a0.elapsed_time(a1) * 1e3 / Kb
-
-        attn_alone_us = alone(lambda i: attn_calls[i % na].run(stream))
-        ver_alone_us = alone(lambda i: ver_calls[i % nv].run(stream))
-
-    if int(status.item()) != 0:
-        raise RuntimeError(f"dev_status = {int(status.item())} after the timed region")
-    ms_total = max_over_ranks(ms_total, dev)
-    ms_per_step = ms_total / K
-    value_us = whole_job_us_per_step(ms_total, K, world)
+    per, head_state = {}, None
+    for name in names:
+        cfg = W.CONFIGS[name]
+        res, state = run_workload(cfg, temp_of(cfg), args, rank, local_rank, world, dev, stream, peaks,
+                                  with_legs=(name == head_name and not args.no_legs))
+        per[name] = res
+        if name == head_name:
+            head_state = state
+        else:
+            del state
+    cfg = W.CONFIGS[head_name]
+    T = temp_of(cfg)
+    head = per[head_name]
 
     # end to end from pinned host buffers through the public API, copies inside the timed region
-    host = B.HostStep(attn_h[0].q, attn_h[0].k_cache, attn_h[0].v_cache, torch.from_numpy(parent), cfg.prefix_len,
-                      ver_h[0].tokens, ver_h[0].target_logits, ver_h[0].draft_logits, T, ver_h[0].uniforms, device=dev,
-                      fused_mask=fused_mask, kernel=args.kernel)
-    Ke = min(K, 20)
+    a0, v0 = head_state["attn_h"][0], head_state["ver_h"][0]
+    host = B.HostStep(a0.q, a0.k_cache, a0.v_cache, torch.from_numpy(head_state["parent"]), cfg.prefix_len,
+                      v0.tokens, v0.target_logits, v0.draft_logits, T, v0.uniforms, device=dev,
+                      fused_mask=head_state["fused_mask"], kernel=args.kernel)
+    Ke = max(3, min(args.steps, 10))
     with torch.cuda.stream(stream):
         for _ in range(3):
             host.run(stream)
@@ -705,76 +927,33 @@ def main():
             dist.destroy_process_group()
         return
 
-    peaks = measured_peaks()
-    attn_ev_us, ver_ev_us = statistics.mean(t_attn), statistics.mean(t_ver)
-    attn_us, ver_us = attn_alone_us, ver_alone_us
-    flops = W.attention_algorithmic_flops(cfg, parent)
-    hbm_time = attn_bytes / (peaks["hbm_gbs"] * 1e9)
-    tensor_time = flops / (peaks["bf16_tflops"] * 1e12)
-    if hbm_time >= tensor_time:
-        achieved = attn_bytes / (attn_us * 1e-6) / 1e9
-        roofline = {"bound": "hbm", "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s",
-                    "frac": achieved / peaks["hbm_gbs"]}
-    else:
-        achieved = flops / (attn_us * 1e-6) / 1e12
-        roofline = {"bound": "tensor", "achieved": achieved, "peak": peaks["bf16_tflops"], "unit": "TFLOP/s",
-                    "frac": achieved / peaks["bf16_tflops"]}
-    roofline.update({
-        "traffic": NCU_TRAFFIC_BYTES.get(cfg.name), "kernel": "seq_tree_attention", "us_per_launch": attn_us,
-        "algorithmic_bytes": attn_bytes, "algorithmic_flops": flops, "peak_source": f"of {peaks['source']}",
-        "us_per_launch_between_event_nodes": attn_ev_us,
-        "timing": f"{Kb} launches of the kernel alone, back to back in one CUDA graph over the rotating inputs, between two "
-                  f"CUDA events; between event nodes inside the replayed steps the same call reads {attn_ev_us:.1f} us",
-    })
-    # verification: HBM-bound in principle (the target row of every visited node, the draft row of every
-    # visited node that has children), latency-bound in practice (one cluster of 8 CTAs walks the path)
-    has_child = np.zeros(n, dtype=bool)
-    has_child[parent[1:][parent[1:] >= 0]] = True
-    vbytes = []
-    for vc in ver_calls:
-        plen = int(vc.path_len.item())
-        nodes = vc.path[:plen].cpu().numpy()
-        vbytes.append(sum(4 * cfg.vocab * (2 if has_child[v] else 1) for v in nodes))
-    ver_bytes = float(np.mean(vbytes))
-    ver_gbs = ver_bytes / (ver_us * 1e-6) / 1e9
-    roofline_verify = {"bound": "hbm", "achieved": ver_gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s",
-                       "frac": ver_gbs / peaks["hbm_gbs"], "traffic": None, "kernel": "seq_tree_verify",
-                       "us_per_launch": ver_us, "algorithmic_bytes": ver_bytes,
-                       "note": "logit rows of the visited nodes only; a dependent walk on one cluster, latency-bound"}
-
+    K = args.steps
+    value_us = head["us_per_step"]["median"] / world  # every rank verifies its own request per step (weak scaling)
     line = {
-        "metric": METRIC, "value": value_us, "unit": UNIT, "n_gpus": world, "steps": K, "warmup": Wm,
-        "ms_per_step": ms_per_step, "higher_is_better": False, "scaling": "weak", "vs_baseline": None,
+        "metric": METRIC, "value": value_us, "unit": UNIT, "n_gpus": world, "steps": K, "warmup": max(3, args.warmup),
+        "ms_per_step": head["ms_per_step"], "higher_is_better": False, "scaling": "weak", "vs_baseline": None,
         "dtype": cfg.dtype, "data": "synthetic",
-        "config": {"workload": cfg.name, "temperature": T, "n_tree": n, "prefix_len": cfg.prefix_len,
-                   "heads": f"{cfg.num_q_heads}/{cfg.num_kv_heads}", "vocab": cfg.vocab, "requests_per_gpu": 1,
-                   "l2": f"inputs rotate over {na} attention sets ({na * attn_bytes >> 20} MiB) and {nv} logit sets, "
-                         f"larger than the 126 MiB L2", "launch": "CUDA graph of the K steps",
-                   "mask": "from the parent array inside the attention kernel" if fused_mask else "separate launch",
-                   "tree": "seeded random within the config's depth and fan-out bounds" if args.tree == "random"
-                           else "seq_tree_build on the paper's printed acceptance vector"},
-        "clocks": clocks.summary(),
+        "config": head["config"],
+        "us_per_step_spread": head["us_per_step"],
+        "clocks": head["clocks"],
         "e2e": {"value": e2e_us, "unit": UNIT, "h2d_bytes_per_step": host.h2d_bytes, "d2h_bytes_per_step": host.d2h_bytes,
                 "steps": Ke},
-        "gpu_launches": K * launches_per_step,
-        "roofline": roofline,
-        "roofline_verify": roofline_verify,
-        "breakdown_us": {"attention": attn_us, "verify": ver_us, "attention_between_event_nodes": attn_ev_us,
-                         "verify_between_event_nodes": ver_ev_us,
-                         "largest_share": "seq_tree_verify" if ver_us > attn_us else "seq_tree_attention"},
+        "gpu_launches": sum(p["gpu_launches"] for p in per.values()),
+        "roofline": head["roofline"],
+        "roofline_verify": head["roofline_verify"],
+        "breakdown_us": {"attention": head["attention_us"], "verify": head["verify_us"],
+                         "verify_l2_warm": head["verify_us_l2_warm"], "verify_in_step": head["verify_us_in_step"],
+                         "largest_share": head["largest_share"]},
+        "per_workload": {k: {kk: vv for kk, vv in v.items() if kk != "next_rows"} for k, v in per.items()},
     }
-    line["next_rows"] = {"kv_commit": kv_commit_leg(cfg, parent, dev, stream, peaks)}
-    if T > 0 and args.tree_search:
-        line["next_rows"]["tree_search"] = tree_search_leg(cfg, T, dev, stream)
-    line["next_rows"]["attention_batch"] = attention_batch_leg(cfg, parent, attn_h, dev, stream, peaks)
-    line["next_rows"]["verify_batch"] = verify_batch_leg(cfg, parent, ver_h, T, dev, stream)
-    if T > 0:
-        line["next_rows"]["top_p_filter"] = top_p_leg(cfg, ver_h, T, dev, stream, peaks)
-        line["next_rows"]["draft_sample"] = draft_sample_leg(cfg, parent, ver_h, T, dev, stream, peaks)
+    if "next_rows" in head:
+        line["next_rows"] = head["next_rows"]
+    if not args.no_legs:
+        line["floors"] = floors_leg(dev, stream)
     if not args.no_cpu_baseline:
         from oracle import oracle as O
 
-        t, note = oracle_step_sample(cfg, parent, attn_h[0], ver_h[0], T)
+        t, note = oracle_step_sample(cfg, head_state["parent"], a0, v0, T, budget_flops=2e11)  # the whole tree on every config
         line["cpu_baseline"] = {"value": 1e6 * t, "unit": UNIT, "cores": O.num_threads(), "kind": "oracle", "sample": note}
     print(json.dumps(line), flush=True)
     if world > 1:

@@ -438,6 +438,22 @@ typedef struct {
 
 int seq_tree_top_p_filter(const seq_tree_top_p_params* p, void* stream);
 
+/* ---------------------------------------------------------------------------
+ * Measurement aids (the paper has no counterpart; Section 4.1 only says that decoding is bound by memory traffic
+ * and by launch overhead, which is what these two numbers quantify on the device at hand).  bench.py prints both
+ * beside its results.
+ *
+ * seq_tree_probe_stream_read -- a kernel that only READS `bytes` bytes (16-byte aligned, device) once, eight
+ * 16-byte loads in flight per thread, 4 CTAs of 512 threads per SM; one word per CTA is written to sink
+ * (device, sink_words >= 4 * the device's SM count, else SEQ_ERR_WORKSPACE).  bytes / its duration is the read
+ * bandwidth a key/value stream can hope for.
+ * seq_tree_probe_dependent_load -- one warp that loads *src and stores *src + 1 to *dst: the floor of a launch
+ * with one dependent trip to memory.
+ * Both are asynchronous on `stream`, allocate nothing, and return SEQ_OK, SEQ_ERR_INVALID_ARG, SEQ_ERR_WORKSPACE
+ * or SEQ_ERR_CUDA. */
+int seq_tree_probe_stream_read(const void* src, size_t bytes, unsigned long long* sink, size_t sink_words, void* stream);
+int seq_tree_probe_dependent_load(const int32_t* src, int32_t* dst, void* stream);
+
 /* Library build string ("seqtree <version> sm_100a"); static storage. */
 const char* seq_tree_version(void);
 

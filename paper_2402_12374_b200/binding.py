@@ -44,6 +44,8 @@ EXPORTED_SYMBOLS = (
     "seq_tree_top_p_filter",
     "seq_tree_build",
     "seq_tree_speedup_search",
+    "seq_tree_probe_stream_read",
+    "seq_tree_probe_dependent_load",
     "seq_tree_version",
 )
 
@@ -124,6 +126,10 @@ def load() -> C.CDLL:
                                                 C.POINTER(C.c_int32), C.POINTER(C.c_double)]
         lib.seq_tree_speedup_search.restype = C.c_int
         lib.seq_tree_version.restype = C.c_char_p
+        lib.seq_tree_probe_stream_read.argtypes = [C.c_void_p, C.c_size_t, C.c_void_p, C.c_size_t, C.c_void_p]
+        lib.seq_tree_probe_stream_read.restype = C.c_int
+        lib.seq_tree_probe_dependent_load.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p]
+        lib.seq_tree_probe_dependent_load.restype = C.c_int
         _lib = lib
     return _lib
 
@@ -512,3 +518,17 @@ class HostStep:
         for h, d in zip(self.host_out, (self.attn.out, self.verify.path, self.verify.path_len, self.verify.bonus_token)):
             h.copy_(d, non_blocking=True)
         return self.host_out
+
+
+def seq_tree_probe_stream_read(buf: torch.Tensor, sink: torch.Tensor, stream=None) -> None:
+    """Measurement aid: one read-only pass over ``buf`` (device, contiguous); ``sink`` int64 device scratch of at
+    least 4 x SM count words."""
+    nbytes = buf.numel() * buf.element_size()
+    _check("seq_tree_probe_stream_read",
+           load().seq_tree_probe_stream_read(_dev(buf, "buf"), nbytes, _dev(sink, "sink", torch.int64), sink.numel(), _stream(stream)))
+
+
+def seq_tree_probe_dependent_load(src: torch.Tensor, dst: torch.Tensor, stream=None) -> None:
+    """Measurement aid: a one-warp kernel that loads src[0] and stores it, plus one, to dst[0]."""
+    _check("seq_tree_probe_dependent_load",
+           load().seq_tree_probe_dependent_load(_dev(src, "src", torch.int32), _dev(dst, "dst", torch.int32), _stream(stream)))

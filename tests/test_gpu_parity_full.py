@@ -99,6 +99,8 @@ def _chi2_ok(counts, probs, trials):
     keep = exp >= 5
     stat = ((counts[keep] - exp[keep]) ** 2 / exp[keep]).sum()
     dof = keep.sum() - 1
+    if dof < 2:  # a distribution this peaked leaves too few cells for a chi-square: every token within 6 binomial sigmas
+        return bool((np.abs(counts - exp) <= 6 * np.sqrt(exp * (1 - probs)) + 1).all()), stat, dof
     return stat < dof + 6 * np.sqrt(2 * dof), stat, dof
 
 
@@ -143,7 +145,8 @@ def test_monte_carlo_on_gpu_outputs_follows_the_target(T, V, k):
     assert ok, (stat, dof)
     if k == V:
         assert accepted == trials  # k = vocabulary size: some child is always accepted
-    assert not _chi2_ok(counts, q / q.sum(), trials)[0], "the check cannot tell the target from the draft"
+    if np.abs(p / p.sum() - q / q.sum()).sum() > 0.1:  # (at T = 0.2 the two can share one dominant token)
+        assert not _chi2_ok(counts, q / q.sum(), trials)[0], "the check cannot tell the target from the draft"
 
 
 def test_monte_carlo_on_gpu_outputs_single_launch_kernel():
