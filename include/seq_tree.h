@@ -219,7 +219,9 @@ int seq_tree_attention_noalloc(const seq_tree_attention_params* p, void* stream)
  *   next_child_out      nullable [n] int32: accepted child of each visited node, -1 if none,
  *                       -2 for nodes the walk did not visit.  With SEQ_VERIFY_ALL_NODES
  *                       every node is processed and gets its own decision.
- * workspace may be NULL when seq_tree_verify_workspace_bytes() returns 0.
+ * workspace: seq_tree_verify_workspace_bytes(p) bytes, 16-byte aligned, device, contents undefined before the call
+ * (the call clears what it needs); afterwards its first int32 holds the number of logit rows the call read (a
+ * diagnostic: the walk's own rows are the algorithmic minimum).  May be NULL: the call then runs the walk.
  */
 enum {
   SEQ_VERIFY_ALL_NODES = 1,
@@ -235,7 +237,19 @@ enum {
    * stops and x is bonus_token.  draft_logits is not read and may be NULL; residual_out receives the
    * distribution the last x was drawn from.  At T = 0 this is the arg-max matching of the default mode.
    * Not to be combined with SEQ_VERIFY_SPECINFER. */
-  SEQ_VERIFY_TARGET_SAMPLE = 4
+  SEQ_VERIFY_TARGET_SAMPLE = 4,
+  /* Schedule of a single request (results are those of Algorithm 2 either way; vocabulary-wide sums are taken in
+   * another order, so a decision inside the 1e-5 band of its uniform can differ between the two):
+   *   node-parallel (the default wherever it applies: vocabulary up to 131072, not with SEQ_VERIFY_ALL_NODES) -- one
+   *     cluster per tree node, rows kept in registers, first the nodes 0 .. clusters-1, then whatever is unclaimed
+   *     at and below the deepest node known to be on the path; the path is assembled from the nodes' decisions by
+   *     atomics, nobody waits.  It reads the rows of nodes the walk never visits (speculative work) and needs
+   *     seq_tree_verify_workspace_bytes() of workspace.  Data problems are reported for visited nodes only.
+   *   walk -- one cluster follows the path from the root and reads only the visited nodes' rows; no workspace.
+   * Neither flag: node-parallel if it applies and enough workspace is given, else the walk.  SCHED_NODES without
+   * enough workspace returns SEQ_ERR_WORKSPACE, where it does not apply SEQ_ERR_UNSUPPORTED. */
+  SEQ_VERIFY_SCHED_WALK = 16,
+  SEQ_VERIFY_SCHED_NODES = 32
 };
 
 typedef struct {
@@ -256,7 +270,7 @@ typedef struct {
   void* workspace;
   size_t workspace_bytes;
   int32_t* dev_status;
-  int32_t flags; /* 0 or an OR of SEQ_VERIFY_ALL_NODES, SEQ_VERIFY_SPECINFER, SEQ_VERIFY_TARGET_SAMPLE */
+  int32_t flags; /* 0 or an OR of the SEQ_VERIFY_* values above */
 } seq_tree_verify_params;
 
 size_t seq_tree_verify_workspace_bytes(const seq_tree_verify_params* p);

@@ -20,6 +20,7 @@ SEQ_DEV_BAD_PARENT, SEQ_DEV_BAD_TOKEN, SEQ_DEV_NONFINITE, SEQ_DEV_DEGENERATE, SE
 SEQ_VERIFY_ALL_NODES = 1
 SEQ_VERIFY_SPECINFER = 2
 SEQ_VERIFY_TARGET_SAMPLE = 4
+SEQ_VERIFY_SCHED_WALK, SEQ_VERIFY_SCHED_NODES = 16, 32
 SEQ_DEV_BAD_PATH = 32
 SEQ_MAX_TREE = 1024
 SEQ_NOALLOC_SCRATCH_BYTES = 384 << 10
@@ -295,7 +296,9 @@ class VerifyCall:
 
     def __init__(self, parent, tokens, target_logits, draft_logits, temperature: float, uniforms, *,
                  path=None, path_len=None, bonus_token=None, residual_out=None, next_child_out=None,
-                 all_nodes: bool = False, dev_status=None, specinfer: bool = False, target_sample: bool = False):
+                 all_nodes: bool = False, dev_status=None, specinfer: bool = False, target_sample: bool = False,
+                 schedule: str = "auto", workspace=None):
+        """schedule: "auto" (node-parallel where it applies), "walk" or "nodes" (forced)."""
         n, V = target_logits.shape
         dev = target_logits.device
         if path is None:
@@ -324,7 +327,14 @@ class VerifyCall:
         p.workspace, p.workspace_bytes = None, 0
         p.dev_status = _dev(dev_status, "dev_status", torch.int32)
         p.flags = ((SEQ_VERIFY_ALL_NODES if all_nodes else 0) | (SEQ_VERIFY_SPECINFER if specinfer else 0) |
-                   (SEQ_VERIFY_TARGET_SAMPLE if target_sample else 0))
+                   (SEQ_VERIFY_TARGET_SAMPLE if target_sample else 0) |
+                   {"auto": 0, "walk": SEQ_VERIFY_SCHED_WALK, "nodes": SEQ_VERIFY_SCHED_NODES}[schedule])
+        need = load().seq_tree_verify_workspace_bytes(C.byref(p))
+        if workspace is None and need:
+            workspace = torch.empty(need, dtype=torch.uint8, device=dev)
+        if workspace is not None:
+            p.workspace, p.workspace_bytes = _dev(workspace, "workspace"), workspace.numel() * workspace.element_size()
+        self.workspace, self.workspace_bytes_needed = workspace, need
         self.params = p
         self.path, self.path_len, self.bonus_token = path, path_len, bonus_token
         self.residual_out, self.next_child_out = residual_out, next_child_out
@@ -333,6 +343,12 @@ class VerifyCall:
     def run(self, stream=None):
         _check("seq_tree_verify", load().seq_tree_verify(C.byref(self.params), _stream(stream)))
         return self.path, self.path_len, self.bonus_token
+
+    def rows_read(self):
+        """Logit rows the last call read (synchronises); None for the walk, which reads the visited nodes' rows only."""
+        if self.workspace is None or not self.workspace_bytes_needed:
+            return None
+        return int(self.workspace[:4].view(torch.int32).item())
 
 
 class VerifyBatchParams(C.Structure):

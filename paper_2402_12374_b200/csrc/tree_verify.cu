@@ -28,6 +28,7 @@
 #include <math.h>
 
 #include "common.cuh"
+#include "tree_verify_nodes.cuh"
 
 namespace cg = cooperative_groups;
 
@@ -53,18 +54,6 @@ constexpr int kVThreads = 256;
 constexpr int kVWarps = kVThreads / 32;
 constexpr uint32_t kVSpinLimit = 1u << 22;
 
-struct VerifyArgs {
-  int32_t n, V, slice_cap, flags;
-  const int32_t* parent; const int32_t* tokens;
-  const float* target; int64_t target_stride;
-  const float* draft; int64_t draft_stride;
-  float temperature;
-  const float* uniforms;
-  int32_t* path; int32_t* path_len; int32_t* bonus;
-  float* residual_out; int32_t* next_child_out; int32_t* dev_status;
-  // batched launch: request r = cluster r; elements between consecutive requests' arrays
-  int64_t tree_stride, logits_stride, unif_stride, resid_stride;
-};
 
 // Two instances of the kernel: clusters of 8 CTAs (portable size; batched launches and the all-nodes test hook, where
 // many clusters share the GPU) and of 16 (one request per launch: the vocabulary-wide sweeps are half as long, a
@@ -89,7 +78,9 @@ static int verify_validate(const seq_tree_verify_params* p) {
   if (p->n_tree < 1 || p->n_tree > SEQ_MAX_TREE || p->vocab < 1) return SEQ_ERR_INVALID_ARG;
   if (p->parent == nullptr || p->tokens == nullptr || p->target_logits == nullptr) return SEQ_ERR_INVALID_ARG;
   if (!(p->temperature >= 0.f) || isinf(p->temperature)) return SEQ_ERR_INVALID_ARG;
-  if (p->flags & ~(SEQ_VERIFY_ALL_NODES | SEQ_VERIFY_SPECINFER | SEQ_VERIFY_TARGET_SAMPLE)) return SEQ_ERR_INVALID_ARG;
+  if (p->flags & ~(SEQ_VERIFY_ALL_NODES | SEQ_VERIFY_SPECINFER | SEQ_VERIFY_TARGET_SAMPLE | SEQ_VERIFY_SCHED_WALK | SEQ_VERIFY_SCHED_NODES))
+    return SEQ_ERR_INVALID_ARG;
+  if ((p->flags & SEQ_VERIFY_SCHED_WALK) && (p->flags & SEQ_VERIFY_SCHED_NODES)) return SEQ_ERR_INVALID_ARG;
   if ((p->flags & SEQ_VERIFY_SPECINFER) && (p->flags & SEQ_VERIFY_TARGET_SAMPLE)) return SEQ_ERR_INVALID_ARG;
   const bool all_nodes = p->flags & SEQ_VERIFY_ALL_NODES;
   if (all_nodes) {
@@ -109,9 +100,16 @@ static int verify_validate(const seq_tree_verify_params* p) {
   return SEQ_OK;
 }
 
+// Which schedule a single request gets: the node-parallel one wherever it applies, unless the caller forces the walk.
+static bool wants_nodes_schedule(const seq_tree_verify_params* p) {
+  if (p->flags & SEQ_VERIFY_SCHED_WALK) return false;
+  return verify_nodes_supported(p->n_tree, p->vocab, p->flags);
+}
+
 extern "C" size_t seq_tree_verify_workspace_bytes(const seq_tree_verify_params* p) {
-  (void)p;
-  return 0;  // all scratch lives in (distributed) shared memory
+  if (verify_validate(p) != SEQ_OK) return 0;
+  // the walk keeps all its scratch in (distributed) shared memory; the node-parallel schedule needs a few words per node
+  return wants_nodes_schedule(p) ? verify_nodes_workspace_bytes(p->n_tree) : 0;
 }
 
 // One instance (cluster size) of the launch.
@@ -176,6 +174,14 @@ static int verify_launch(const seq_tree_verify_params* p, int batch, int64_t tre
     if (!fits8 && (!fits16 || batch > 0 || (p->flags & SEQ_VERIFY_ALL_NODES))) return SEQ_ERR_UNSUPPORTED;
   }
 
+  if (batch == 0 && wants_nodes_schedule(p)) {
+    const bool have_ws = p->workspace != nullptr && p->workspace_bytes >= verify_nodes_workspace_bytes(p->n_tree);
+    if (have_ws) return launch_verify_nodes(a, p->workspace, p->workspace_bytes, 0, s);
+    if (p->flags & SEQ_VERIFY_SCHED_NODES) return SEQ_ERR_WORKSPACE;
+    // no workspace given: the walk, which needs none
+  } else if (p->flags & SEQ_VERIFY_SCHED_NODES) {
+    return SEQ_ERR_UNSUPPORTED;
+  }
   if (batch > 0) return verify_launch_with<8, vcl8::VShared, 0>(vcl8::tree_verify_kernel<true>, a, p->vocab, batch, false, s);
   if (p->flags & SEQ_VERIFY_ALL_NODES)  // 18 * 8 = 144 CTAs <= 148 SMs
     return verify_launch_with<8, vcl8::VShared, 1>(vcl8::tree_verify_kernel<false>, a, p->vocab, p->n_tree < 18 ? p->n_tree : 18, false, s);

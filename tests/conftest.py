@@ -21,3 +21,22 @@ def pytest_collection_modifyitems(config, items):
     for item in items:
         if "gpu" in item.keywords:
             item.add_marker(skip)
+
+
+@pytest.fixture
+def verify_schedule(request):
+    """Runs a verification test once per schedule of seq_tree_verify (node-parallel, walk)."""
+    from tests import gpu_util as G
+
+    G.SCHEDULE = request.param
+    yield request.param
+    G.SCHEDULE = "auto"
+
+
+def pytest_generate_tests(metafunc):
+    name = metafunc.function.__name__
+    if (metafunc.module.__name__.split(".")[-1] in ("test_gpu_parity", "test_gpu_parity_full") and name.startswith("test_verify")
+            and "every_node_hook" not in name):
+        if "verify_schedule" not in metafunc.fixturenames:
+            metafunc.fixturenames.append("verify_schedule")
+        metafunc.parametrize("verify_schedule", ["nodes", "walk"], indirect=True)

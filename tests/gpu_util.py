@@ -12,6 +12,7 @@ from paper_2402_12374_b200 import workloads as W
 ATTN_TOL = {torch.float16: 2e-2, torch.bfloat16: 2e-2, torch.float32: 1e-5}  # max abs error of the output
 RESID_TOL = 1e-5   # max abs error of residual probabilities
 GAP = 1e-5         # |u - ratio| below this: the accept decision is within rounding, outcome excluded
+SCHEDULE = "auto"  # schedule of seq_tree_verify in run_verify: set per test by the `verify_schedule` fixture
 
 
 def dev():
@@ -88,11 +89,12 @@ def run_verify(vi: W.VerifyInputs, all_nodes=False, want_residual=True, specinfe
         dl = dl[:, :V]
     call = B.VerifyCall(vi.parent.to(d), vi.tokens.to(d), tl[:, :V], dl,
                         vi.temperature, vi.uniforms.to(d), residual_out=residual, next_child_out=nxt,
-                        all_nodes=all_nodes, dev_status=st, specinfer=specinfer, target_sample=target_sample)
+                        all_nodes=all_nodes, dev_status=st, specinfer=specinfer, target_sample=target_sample,
+                        schedule="auto" if all_nodes else SCHEDULE)
     call.run()
     torch.cuda.synchronize()
     plen = int(call.path_len.item())
-    return dict(path=call.path[:plen].cpu().numpy(), path_len=plen, bonus=int(call.bonus_token.item()),
+    return dict(rows_read=call.rows_read(), path=call.path[:plen].cpu().numpy(), path_len=plen, bonus=int(call.bonus_token.item()),
                 residual=None if residual is None else residual.double().cpu().numpy(),
                 next_child=nxt.cpu().numpy(), status=int(st.item()))
 
