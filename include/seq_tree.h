@@ -221,7 +221,7 @@ int seq_tree_attention_noalloc(const seq_tree_attention_params* p, void* stream)
  *                       every node is processed and gets its own decision.
  * workspace: seq_tree_verify_workspace_bytes(p) bytes, 16-byte aligned, device, contents undefined before the call
  * (the call clears what it needs); afterwards its first int32 holds the number of logit rows the call read (a
- * diagnostic: the walk's own rows are the algorithmic minimum).  May be NULL: the call then runs the walk.
+ * diagnostic: the walk's own rows are the algorithmic minimum).  Only the node-parallel schedule uses it.
  */
 enum {
   SEQ_VERIFY_ALL_NODES = 1,
@@ -240,14 +240,15 @@ enum {
   SEQ_VERIFY_TARGET_SAMPLE = 4,
   /* Schedule of a single request (results are those of Algorithm 2 either way; vocabulary-wide sums are taken in
    * another order, so a decision inside the 1e-5 band of its uniform can differ between the two):
-   *   node-parallel (the default wherever it applies: vocabulary up to 131072, not with SEQ_VERIFY_ALL_NODES) -- one
-   *     cluster per tree node, rows kept in registers, first the nodes 0 .. clusters-1, then whatever is unclaimed
-   *     at and below the deepest node known to be on the path; the path is assembled from the nodes' decisions by
-   *     atomics, nobody waits.  It reads the rows of nodes the walk never visits (speculative work) and needs
-   *     seq_tree_verify_workspace_bytes() of workspace.  Data problems are reported for visited nodes only.
-   *   walk -- one cluster follows the path from the root and reads only the visited nodes' rows; no workspace.
-   * Neither flag: node-parallel if it applies and enough workspace is given, else the walk.  SCHED_NODES without
-   * enough workspace returns SEQ_ERR_WORKSPACE, where it does not apply SEQ_ERR_UNSUPPORTED. */
+   *   walk (the default) -- one cluster of CTAs follows the path from the root and reads only the visited nodes' rows
+   *     (plus the rows of children that were tested and rejected, loaded ahead of their test); no workspace.
+   *   node-parallel -- one cluster per tree node, first the nodes 0 .. clusters-1, then whatever is unclaimed at and
+   *     below the deepest node known to be on the path; the path is assembled from the nodes' decisions by atomics,
+   *     nobody waits.  It reads the rows of nodes the walk never visits (speculative work) and needs
+   *     seq_tree_verify_workspace_bytes() of workspace; vocabulary up to 131072, not with SEQ_VERIFY_ALL_NODES.
+   *     Data problems are reported for visited nodes only.  Measured slower than the walk on all five shapes of the
+   *     paper's models; kept selectable.
+   * SCHED_NODES without enough workspace returns SEQ_ERR_WORKSPACE, where it does not apply SEQ_ERR_UNSUPPORTED. */
   SEQ_VERIFY_SCHED_WALK = 16,
   SEQ_VERIFY_SCHED_NODES = 32
 };

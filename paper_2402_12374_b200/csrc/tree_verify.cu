@@ -100,9 +100,11 @@ static int verify_validate(const seq_tree_verify_params* p) {
   return SEQ_OK;
 }
 
-// Which schedule a single request gets: the node-parallel one wherever it applies, unless the caller forces the walk.
+// Which schedule a single request gets.  Measured on the paper's five shapes (bench.py, L2-cold): the walk with its
+// rows in registers beats the node-parallel schedule on every one of them, so the walk is what a request gets unless
+// the caller asks for the other.
 static bool wants_nodes_schedule(const seq_tree_verify_params* p) {
-  if (p->flags & SEQ_VERIFY_SCHED_WALK) return false;
+  if (!(p->flags & SEQ_VERIFY_SCHED_NODES)) return false;
   return verify_nodes_supported(p->n_tree, p->vocab, p->flags);
 }
 
@@ -124,7 +126,9 @@ static int verify_launch_with(Kernel kernel, VerifyArgs a, int vocab, int n_clus
     // function attributes once per (kernel instance, device): the largest shared-memory size any vocabulary can ask for
     static int attr_done[64];  // (one array per instantiation of this template, i.e. per Slot)
     const int rc = once_per_device(attr_done, [&]() -> int {
-      SEQ_CUDA_OK(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024));
+      cudaFuncAttributes fa;
+      SEQ_CUDA_OK(cudaFuncGetAttributes(&fa, kernel));
+      SEQ_CUDA_OK(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024 - (int)fa.sharedSizeBytes));
       if (CL > 8) SEQ_CUDA_OK(cudaFuncSetAttribute(kernel, cudaFuncAttributeNonPortableClusterSizeAllowed, 1));
       return SEQ_OK;
     });
@@ -174,13 +178,9 @@ static int verify_launch(const seq_tree_verify_params* p, int batch, int64_t tre
     if (!fits8 && (!fits16 || batch > 0 || (p->flags & SEQ_VERIFY_ALL_NODES))) return SEQ_ERR_UNSUPPORTED;
   }
 
-  if (batch == 0 && wants_nodes_schedule(p)) {
-    const bool have_ws = p->workspace != nullptr && p->workspace_bytes >= verify_nodes_workspace_bytes(p->n_tree);
-    if (have_ws) return launch_verify_nodes(a, p->workspace, p->workspace_bytes, 0, s);
-    if (p->flags & SEQ_VERIFY_SCHED_NODES) return SEQ_ERR_WORKSPACE;
-    // no workspace given: the walk, which needs none
-  } else if (p->flags & SEQ_VERIFY_SCHED_NODES) {
-    return SEQ_ERR_UNSUPPORTED;
+  if (p->flags & SEQ_VERIFY_SCHED_NODES) {
+    if (batch != 0 || !wants_nodes_schedule(p)) return SEQ_ERR_UNSUPPORTED;
+    return launch_verify_nodes(a, p->workspace, p->workspace_bytes, 0, s);  // (checks the workspace)
   }
   if (batch > 0) return verify_launch_with<8, vcl8::VShared, 0>(vcl8::tree_verify_kernel<true>, a, p->vocab, batch, false, s);
   if (p->flags & SEQ_VERIFY_ALL_NODES)  // 18 * 8 = 144 CTAs <= 148 SMs
@@ -195,6 +195,8 @@ static int verify_launch(const seq_tree_verify_params* p, int batch, int64_t tre
     wide = verify_launch_with<16, vcl16::VShared, 2>(vcl16::tree_verify_kernel<false>, a, 32000, 1, true, s) == SEQ_OK ? 1 : 2;
     __atomic_store_n(&wide_ok[dev], wide, __ATOMIC_RELEASE);
   }
+  // the walk with its rows in registers, where a cluster of 16 can be placed and the mode is one it serves
+  if (wide == 1 && verify_walk_supported(p->vocab, p->flags, p->temperature)) return launch_verify_walk(a, false, s);
   if (wide == 1 && p->vocab >= 8192)
     return verify_launch_with<16, vcl16::VShared, 2>(vcl16::tree_verify_kernel<false>, a, p->vocab, 1, false, s);
   return verify_launch_with<8, vcl8::VShared, 1>(vcl8::tree_verify_kernel<false>, a, p->vocab, 1, false, s);

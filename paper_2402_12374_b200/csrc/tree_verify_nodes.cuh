@@ -26,4 +26,8 @@ size_t verify_nodes_workspace_bytes(int n_tree);
 bool verify_nodes_supported(int n_tree, int vocab, int flags);
 int launch_verify_nodes(const VerifyArgs& a, void* workspace, size_t workspace_bytes, int max_clusters, cudaStream_t stream);
 
+// The walk with rows in registers (tree_verify_walk.cu): one cluster of 16 CTAs, no workspace.
+bool verify_walk_supported(int vocab, int flags, float temperature);
+int launch_verify_walk(const VerifyArgs& a, bool check_only, cudaStream_t stream);
+
 }  // namespace seqtree

@@ -128,8 +128,9 @@ def test_host_checkable_errors_are_refused_before_launch(lib):
         assert lib.seq_tree_verify(C.byref(ver(**kw)), None) == B.SEQ_ERR_INVALID_ARG, kw
     assert lib.seq_tree_verify(C.byref(ver(vocab=400000, target_row_stride=400000, draft_row_stride=400000)), None) \
         == B.SEQ_ERR_UNSUPPORTED
-    # the node-parallel schedule (the default for a single request) keeps a few words per node in a workspace; the walk none
-    assert 0 < lib.seq_tree_verify_workspace_bytes(C.byref(ver())) <= 16384
+    # the node-parallel schedule keeps a few words per node in a workspace; the walk (the default) none
+    assert 0 < lib.seq_tree_verify_workspace_bytes(C.byref(ver(flags=B.SEQ_VERIFY_SCHED_NODES))) <= 16384
+    assert lib.seq_tree_verify_workspace_bytes(C.byref(ver())) == 0
     assert lib.seq_tree_verify_workspace_bytes(C.byref(ver(flags=B.SEQ_VERIFY_SCHED_WALK))) == 0
     assert lib.seq_tree_verify_workspace_bytes(C.byref(ver(flags=B.SEQ_VERIFY_ALL_NODES, next_child_out=fake))) == 0
     assert lib.seq_tree_verify(C.byref(ver(flags=B.SEQ_VERIFY_SCHED_WALK | B.SEQ_VERIFY_SCHED_NODES)), None) == B.SEQ_ERR_INVALID_ARG
