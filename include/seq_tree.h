@@ -60,7 +60,8 @@ enum {
   SEQ_DEV_NONFINITE = 4,   /* NaN or +inf logit on a visited row */
   SEQ_DEV_DEGENERATE = 8,  /* sum max(R-D,0) == 0 after a rejection (impossible in exact arithmetic): R kept */
   SEQ_DEV_TIMEOUT = 16,    /* a bounded on-chip wait ran out; outputs of that call are undefined */
-  SEQ_DEV_BAD_PATH = 32    /* seq_tree_kv_commit: path not a root-to-node path (see there); nothing was moved */
+  SEQ_DEV_BAD_PATH = 32,   /* seq_tree_kv_commit: path not a root-to-node path (see there); nothing was moved */
+  SEQ_DEV_BAD_LENGTH = 64  /* *prefix_len_dev outside [0, prefix_len]: clamped into that range */
 };
 
 /*
@@ -154,6 +155,14 @@ typedef struct {
   int32_t kernel; /* 0 = choose; 1 = force the CUDA-core kernel; 2 = force the tensor-core kernel; 3, 4 = the tensor-core
                      kernel with its stream / grid schedule forced (tuning and tests; results do not depend on it) */
   const int32_t* parent; /* nullable, [n_tree] int32, device: see "mask from the parent array" above */
+  /* nullable, device: the prefix length as the previous step's seq_tree_kv_commit left it.  When given, the kernels
+   * read the length from there and prefix_len is only the LARGEST value it can take (it sizes the launch, the
+   * workspace and the checks against kv_capacity); the tree's rows then sit at [*prefix_len_dev, *prefix_len_dev +
+   * n_tree).  This is what lets one CUDA graph of a whole step (attention, verification, commit) be replayed while
+   * the prefix grows (Section 4.1: the tree is fixed so that CUDA graphs can remove the launch overhead).  On the
+   * tensor-core path the rows from *prefix_len_dev + n_tree up to kv_capacity are then fetched (not used): they may
+   * hold anything, but must be readable.  A value outside [0, prefix_len] raises SEQ_DEV_BAD_LENGTH and is clamped. */
+  const int32_t* prefix_len_dev;
 } seq_tree_attention_params;
 
 size_t seq_tree_attention_workspace_bytes(const seq_tree_attention_params* p);
@@ -375,6 +384,10 @@ typedef struct {
   const int32_t* path_len;
   int32_t* new_prefix_len;
   int32_t* dev_status;
+  /* nullable, device: the prefix length is read from here and prefix_len is its upper bound (see
+   * seq_tree_attention_params).  Must not be the same word as new_prefix_len: CTAs read the one while another
+   * writes the other; copy new_prefix_len over it after the call (a 4-byte device copy, capturable). */
+  const int32_t* prefix_len_dev;
 } seq_tree_kv_commit_params;
 
 int seq_tree_kv_commit(const seq_tree_kv_commit_params* p, void* stream);

@@ -22,6 +22,7 @@ SEQ_VERIFY_SPECINFER = 2
 SEQ_VERIFY_TARGET_SAMPLE = 4
 SEQ_VERIFY_SCHED_WALK, SEQ_VERIFY_SCHED_NODES = 16, 32
 SEQ_DEV_BAD_PATH = 32
+SEQ_DEV_BAD_LENGTH = 64
 SEQ_MAX_TREE = 1024
 SEQ_NOALLOC_SCRATCH_BYTES = 384 << 10
 KERNEL_AUTO, KERNEL_CUDA_CORE, KERNEL_TENSOR_CORE = 0, 1, 2
@@ -69,7 +70,7 @@ class AttentionParams(C.Structure):
         ("out", C.c_void_p), ("o_stride_tok", C.c_int64), ("o_stride_head", C.c_int64),
         ("lse", C.c_void_p), ("workspace", C.c_void_p), ("workspace_bytes", C.c_size_t),
         ("dev_status", C.c_void_p), ("kernel", C.c_int32),
-        ("parent", C.c_void_p),
+        ("parent", C.c_void_p), ("prefix_len_dev", C.c_void_p),
     ]
 
 
@@ -192,6 +193,7 @@ class KvCommitParams(C.Structure):
         ("k_cache", C.c_void_p), ("v_cache", C.c_void_p),
         ("plane_stride_bytes", C.c_int64), ("row_stride_bytes", C.c_int64),
         ("path", C.c_void_p), ("path_len", C.c_void_p), ("new_prefix_len", C.c_void_p), ("dev_status", C.c_void_p),
+        ("prefix_len_dev", C.c_void_p),
     ]
 
 
@@ -225,7 +227,7 @@ class AttentionCall:
 
     def __init__(self, q, k_cache, v_cache, mask_bits, prefix_len: int, *, out=None, lse=None,
                  softmax_scale: float = 0.0, workspace=None, dev_status=None, kernel: int = KERNEL_AUTO,
-                 noalloc: bool = False, parent=None):
+                 noalloc: bool = False, parent=None, prefix_len_dev=None):
         """``noalloc=True`` prepares a call of ``seq_tree_attention_noalloc``: no workspace tensor is
         created or passed; the library's built-in scratch array is used (CUDA-core kernel).
         ``mask_bits=None`` with ``parent`` (int32 [n], device) lets the tensor-core kernel derive the
@@ -256,6 +258,7 @@ class AttentionCall:
                 raise ValueError("mask_bits or parent is required")
             p.mask_bits, p.mask_words_per_row = None, 0
         p.parent = _dev(parent, "parent", torch.int32)
+        p.prefix_len_dev = _dev(prefix_len_dev, "prefix_len_dev", torch.int32)  # prefix_len is then its upper bound
         p.out, p.o_stride_tok, p.o_stride_head = _dev(out, "out", q.dtype), out.stride(0), out.stride(1)
         p.lse = _dev(lse, "lse", torch.float32)
         p.dev_status = _dev(dev_status, "dev_status", torch.int32)
@@ -268,7 +271,7 @@ class AttentionCall:
         p.workspace_bytes = workspace.numel() * workspace.element_size() if workspace is not None else 0
         self.params, self.out, self.lse, self.workspace_bytes_needed = p, out, lse, need
         self.workspace = workspace
-        self._keep = (q, k_cache, v_cache, mask_bits, parent, out, lse, workspace, dev_status)
+        self._keep = (q, k_cache, v_cache, mask_bits, parent, out, lse, workspace, dev_status, prefix_len_dev)
 
     def run(self, stream=None):
         if self.noalloc:
@@ -476,7 +479,7 @@ def seq_tree_speedup_search(table, t_of_n, c: float):
 
 
 def seq_tree_kv_commit(k_cache, v_cache, prefix_len: int, n_tree: int, path, path_len, *, new_prefix_len=None,
-                       dev_status=None, stream=None):
+                       dev_status=None, stream=None, prefix_len_dev=None):
     """In place: row prefix_len+i of every plane <- row prefix_len+path[i], i < path_len (device tensors as
     seq_tree_verify wrote them).  k_cache / v_cache: [planes, rows, head_dim] (v_cache may be None), rows
     contiguous."""
@@ -492,6 +495,7 @@ def seq_tree_kv_commit(k_cache, v_cache, prefix_len: int, n_tree: int, path, pat
     p.row_stride_bytes = k_cache.stride(1) * e
     p.path, p.path_len = _dev(path, "path", torch.int32), _dev(path_len, "path_len", torch.int32)
     p.new_prefix_len = _dev(new_prefix_len, "new_prefix_len", torch.int32)
+    p.prefix_len_dev = _dev(prefix_len_dev, "prefix_len_dev", torch.int32)
     p.dev_status = _dev(dev_status, "dev_status", torch.int32)
     _check("seq_tree_kv_commit", load().seq_tree_kv_commit(C.byref(p), _stream(stream)))
 

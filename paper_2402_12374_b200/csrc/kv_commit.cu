@@ -12,7 +12,8 @@ struct CommitArgs {
   uint8_t* cache[2];
   int64_t plane_stride, row_stride;  // bytes
   int32_t planes, cols;              // cols = 16-byte columns per row
-  int32_t L, n;
+  int32_t L_host, n;
+  const int32_t* L_dev;  // nullable: the prefix length in device memory (<= L_host)
   const int32_t* path; const int32_t* path_len;
   int32_t* new_prefix_len; int32_t* dev_status;
 };
@@ -22,6 +23,12 @@ __global__ void __launch_bounds__(kCommitThreads) kv_commit_kernel(const CommitA
   // path_len and the whole path buffer (n entries, as seq_tree_verify owns it) are fetched together: one memory
   // latency instead of two.  Every CTA checks the path for itself: 0 first, strictly ascending, below n.
   const int len = *a.path_len;
+  int L = a.L_host;
+  if (a.L_dev != nullptr) {
+    const int v = *a.L_dev;
+    if ((v < 0 || v > a.L_host) && blockIdx.x == 0 && threadIdx.x == 0) dev_flag(a.dev_status, SEQ_DEV_BAD_LENGTH);
+    L = min(max(v, 0), a.L_host);
+  }
   for (int i = threadIdx.x; i < a.n; i += kCommitThreads) s_path[i] = a.path[i];
   __syncthreads();
   int bad = len < 0 || len > a.n;
@@ -33,7 +40,7 @@ __global__ void __launch_bounds__(kCommitThreads) kv_commit_kernel(const CommitA
   bad = __syncthreads_or(bad);
   if (blockIdx.x == 0 && threadIdx.x == 0) {
     if (bad) dev_flag(a.dev_status, SEQ_DEV_BAD_PATH);
-    if (a.new_prefix_len != nullptr) *a.new_prefix_len = a.L + (bad ? 0 : len);
+    if (a.new_prefix_len != nullptr) *a.new_prefix_len = L + (bad ? 0 : len);
   }
   if (bad) return;
   // rows that already sit in place (always the root, often the first levels) are skipped
@@ -48,7 +55,7 @@ __global__ void __launch_bounds__(kCommitThreads) kv_commit_kernel(const CommitA
     const int64_t r = t - which * per_cache;
     const int64_t plane = r / a.cols;
     const int col = (int)(r - plane * a.cols);
-    uint8_t* base = (which ? a.cache[1] : a.cache[0]) + plane * a.plane_stride + (int64_t)a.L * a.row_stride + (int64_t)col * 16;
+    uint8_t* base = (which ? a.cache[1] : a.cache[0]) + plane * a.plane_stride + (int64_t)L * a.row_stride + (int64_t)col * 16;
     for (int i0 = first; i0 < len; i0 += kCommitBatch) {
       uint4 v[kCommitBatch];
 #pragma unroll
@@ -68,6 +75,7 @@ using namespace seqtree;
 extern "C" int seq_tree_kv_commit(const seq_tree_kv_commit_params* p, void* stream) {
   if (p == nullptr || p->k_cache == nullptr || p->path == nullptr || p->path_len == nullptr) return SEQ_ERR_INVALID_ARG;
   if (p->num_planes < 1 || p->n_tree < 1 || p->n_tree > SEQ_MAX_TREE || p->prefix_len < 0) return SEQ_ERR_INVALID_ARG;
+  if (p->prefix_len_dev != nullptr && p->prefix_len_dev == p->new_prefix_len) return SEQ_ERR_INVALID_ARG;  // read by some CTAs while another writes
   if (p->row_bytes < 16 || p->row_bytes % 16 != 0 || p->row_stride_bytes < p->row_bytes || p->row_stride_bytes % 16 != 0 ||
       p->plane_stride_bytes % 16 != 0 ||
       p->plane_stride_bytes < ((int64_t)p->prefix_len + p->n_tree) * p->row_stride_bytes)
@@ -79,7 +87,7 @@ extern "C" int seq_tree_kv_commit(const seq_tree_kv_commit_params* p, void* stre
   a.cache[1] = static_cast<uint8_t*>(p->v_cache);
   a.plane_stride = p->plane_stride_bytes; a.row_stride = p->row_stride_bytes;
   a.planes = p->num_planes; a.cols = p->row_bytes / 16;
-  a.L = p->prefix_len; a.n = p->n_tree;
+  a.L_host = p->prefix_len; a.L_dev = p->prefix_len_dev; a.n = p->n_tree;
   a.path = p->path; a.path_len = p->path_len;
   a.new_prefix_len = p->new_prefix_len; a.dev_status = p->dev_status;
   const int64_t total = (int64_t)a.planes * a.cols * (a.cache[1] != nullptr ? 2 : 1);

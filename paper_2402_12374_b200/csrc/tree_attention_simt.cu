@@ -101,7 +101,9 @@ struct SimtArgs {
   float* lse;
   float* o_part; float2* ml;
   int64_t q_stride_tok, q_stride_head, kv_stride_tok, kv_stride_head, o_stride_tok, o_stride_head;
-  int32_t n, L, Hq, group, mask_wpr, splits;
+  int32_t n, L_host, Hq, group, mask_wpr, splits;
+  const int32_t* L_dev;  // nullable: the prefix length in device memory (<= L_host)
+  int32_t* dev_status;
   float scale_log2;  // softmax_scale * log2(e)
 };
 
@@ -110,6 +112,12 @@ __global__ void __launch_bounds__(kSimtWarps * 32)
 tree_attention_simt_kernel(const SimtArgs a) {
   const int i = blockIdx.x, h = blockIdx.y, split = blockIdx.z;
   const int g = h / a.group;
+  int L = a.L_host;
+  if (a.L_dev != nullptr) {
+    const int v = *a.L_dev;
+    if ((v < 0 || v > a.L_host) && threadIdx.x == 0) dev_flag(a.dev_status, SEQ_DEV_BAD_LENGTH);
+    L = min(max(v, 0), a.L_host);
+  }
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
   __shared__ __align__(16) float q_s[kHeadDim];
@@ -125,7 +133,7 @@ tree_attention_simt_kernel(const SimtArgs a) {
   const uint32_t* mrow = a.mask_bits + (size_t)i * a.mask_wpr;
 
   // node i can only see tree nodes <= i, so keys end at L + i + 1
-  const int n_keys = a.L + i + 1;
+  const int n_keys = L + i + 1;
   const int n_chunks = (n_keys + 31) >> 5;
   const int stride = a.splits * kSimtWarps;
 
@@ -134,9 +142,9 @@ tree_attention_simt_kernel(const SimtArgs a) {
 
   for (int c = split * kSimtWarps + warp; c < n_chunks; c += stride) {
     const int j = (c << 5) + lane;
-    bool valid = j < a.L;
+    bool valid = j < L;
     if (!valid && j < n_keys) {
-      const int t = j - a.L;
+      const int t = j - L;
       valid = (mrow[t >> 5] >> (t & 31)) & 1u;
     }
     float s = -INFINITY;
@@ -266,7 +274,7 @@ static int launch_simt_t(const seq_tree_attention_params& p, int splits, cudaStr
   a.q_stride_tok = p.q_stride_tok; a.q_stride_head = p.q_stride_head;
   a.kv_stride_tok = p.kv_stride_tok; a.kv_stride_head = p.kv_stride_head;
   a.o_stride_tok = p.o_stride_tok; a.o_stride_head = p.o_stride_head;
-  a.n = p.n_tree; a.L = p.prefix_len; a.Hq = p.num_q_heads; a.group = p.num_q_heads / p.num_kv_heads;
+  a.n = p.n_tree; a.L_host = p.prefix_len; a.L_dev = p.prefix_len_dev; a.dev_status = p.dev_status; a.Hq = p.num_q_heads; a.group = p.num_q_heads / p.num_kv_heads;
   a.mask_wpr = p.mask_words_per_row; a.splits = splits;
   const float scale = p.softmax_scale > 0.f ? p.softmax_scale : 0.08838834764831845f;
   a.scale_log2 = scale * kLog2e;

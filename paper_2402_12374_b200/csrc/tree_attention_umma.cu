@@ -126,12 +126,14 @@ struct UmmaSmem {
 static_assert(offsetof(UmmaSmem, v) == offsetof(UmmaSmem, k) + sizeof(UmmaSmem::k), "the cluster merge receives into k and v as one buffer");
 
 struct UmmaArgs {
-  int32_t n, L, Hq, Hkv, group, mask_wpr, splits, nodes_per_tile, tiles;
+  int32_t n, L_host, Hq, Hkv, group, mask_wpr, splits, nodes_per_tile, tiles;
+  const int32_t* L_dev;   // nullable: the prefix length in device memory (<= L_host)
+  int32_t zero_tail;      // the K/V maps cover the whole cache: rows past the tree are cleared in shared memory
   // Stream mode (more (tile, kv head) units than SMs): the 64-key blocks of all units, laid end to end, are
   // cut into gridDim.x equal ranges, one per CTA; a tile cut by a range boundary is completed by whichever
   // of its CTAs finishes last, from partial results in the workspace.
-  int32_t stream, blocks_per_head;
-  int64_t total_blocks;
+  int32_t stream, blocks_per_head_host;
+  int64_t total_blocks_host;
   int32_t* ws_count;   // [Hkv * tiles] arrivals per tile, zero on entry and on exit
   float2* ws_ml;       // [2 * gridDim.x][128] (m, l) of a partial result
   float4* ws_o;        // [2 * gridDim.x][2][16][128] its unnormalised accumulator, thread-major
@@ -321,8 +323,12 @@ tree_attention_umma_kernel(const __grid_constant__ CUtensorMap q_map, const __gr
   // A CTA works through segments: (kv head, tile, range of the tile's 64-key blocks).  Grid mode: the one
   // segment (blockIdx.y, blockIdx.x, this CTA's share of the cluster's key range).  Stream mode: the pieces
   // of the units that its range [range_lo, range_hi) of the flattened block space overlaps.
-  const int64_t range_lo = kStream ? (a.total_blocks * (int64_t)blockIdx.x) / (int64_t)gridDim.x : 0;
-  const int64_t range_hi = kStream ? (a.total_blocks * (int64_t)(blockIdx.x + 1)) / (int64_t)gridDim.x : 1;
+  // The prefix length: the host's, or - for a step replayed from one CUDA graph while the prefix grows - read from
+  // device memory below (the host's value is then the largest it can be, which the launch was planned for).
+  int L = a.L_host;
+  int blocks_per_head = a.blocks_per_head_host;
+  int64_t total_blocks = a.total_blocks_host;
+  int64_t range_lo = 0, range_hi = 1;
   struct Seg { int g, tile, slot_in_head, i0, i1, blk_lo, nblk, nblk_tile; int64_t next; };
   // Stream mode lays the tiles of a kv head out alternating from both ends (0, T-1, 1, T-2, ...): late tiles
   // have more masked blocks, which cost more, and this way every range gets its share of them.
@@ -334,13 +340,13 @@ tree_attention_umma_kernel(const __grid_constant__ CUtensorMap q_map, const __gr
       x.i0 = x.tile * a.nodes_per_tile;
       x.i1 = min(x.i0 + a.nodes_per_tile, a.n);
       // keys this tile can see end at L + i1 (a node sees no later node); blocks of this CTA
-      x.nblk_tile = (a.L + x.i1 + kBlockN - 1) / kBlockN;
+      x.nblk_tile = (L + x.i1 + kBlockN - 1) / kBlockN;
       x.blk_lo = (int)(((long)split * x.nblk_tile) / a.splits);
       x.nblk = (int)(((long)(split + 1) * x.nblk_tile) / a.splits) - x.blk_lo;
       x.next = 1;
     } else {
-      x.g = (int)(pos / a.blocks_per_head);
-      const int rem = (int)(pos % a.blocks_per_head);
+      x.g = (int)(pos / blocks_per_head);
+      const int rem = (int)(pos % blocks_per_head);
       int lo = 0, hi = a.tiles - 1;  // the last place in the head's layout whose first block is at or before rem
       while (lo < hi) {
         const int mid = (lo + hi + 1) >> 1;
@@ -388,6 +394,23 @@ tree_attention_umma_kernel(const __grid_constant__ CUtensorMap q_map, const __gr
   // ... and everything above ran while the previous kernel in the stream was still finishing.  Nothing before this
   // line reads or writes global memory.
   asm volatile("griddepcontrol.wait;" ::: "memory");
+  if (a.L_dev != nullptr) {
+    const int v = *a.L_dev;
+    if (v < 0 || v > a.L_host) { if (threadIdx.x == 0) dev_flag(a.dev_status, SEQ_DEV_BAD_LENGTH); }
+    L = min(max(v, 0), a.L_host);
+    if (kStream) {  // the flattened block space of this prefix length (every warp for itself)
+      int sum = 0;
+      for (int t = lane; t < a.tiles; t += 32) sum += kStreamTileCost + (L + min((t + 1) * a.nodes_per_tile, a.n) + kBlockN - 1) / kBlockN;
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, o);
+      blocks_per_head = sum;
+      total_blocks = (int64_t)sum * a.Hkv;
+    }
+  }
+  if (kStream) {
+    range_lo = (total_blocks * (int64_t)blockIdx.x) / (int64_t)gridDim.x;
+    range_hi = (total_blocks * (int64_t)(blockIdx.x + 1)) / (int64_t)gridDim.x;
+  }
   // Grid schedule: the one segment of this CTA is known from its block index, so the thread that armed the barriers
   // requests the Q tile and the first K tile of each chain right away, before the CTA-wide barrier below and the
   // hand-over to the producer warps (which skip what has been requested here).
@@ -410,7 +433,7 @@ tree_attention_umma_kernel(const __grid_constant__ CUtensorMap q_map, const __gr
 #pragma unroll
     for (int k = 0; k < kMaxStreamTiles / 32; ++k) {
       const int t = lane * per + k;
-      local[k] = (k < per && t < a.tiles) ? kStreamTileCost + (a.L + min((tile_at(t) + 1) * a.nodes_per_tile, a.n) + kBlockN - 1) / kBlockN : 0;
+      local[k] = (k < per && t < a.tiles) ? kStreamTileCost + (L + min((tile_at(t) + 1) * a.nodes_per_tile, a.n) + kBlockN - 1) / kBlockN : 0;
       sum += local[k];
     }
     int incl = sum;
@@ -528,6 +551,22 @@ tree_attention_umma_kernel(const __grid_constant__ CUtensorMap q_map, const __gr
           if (u == 0 && seg > 0 && !mbar_wait(sm, &sm->o_free, (seg - 1) & 1, a.dev_status)) break;
           if (lane == 0) UTRACE(c == 0 ? 1 : 3, 3);
           if (!mbar_wait(sm, &sm->v_full[c][b], w & 1, a.dev_status)) break;
+          if (a.zero_tail) {
+            // The tensor maps of this mode cover the whole cache, so a block that reaches past the last tree row has
+            // fetched rows that may hold anything; their probabilities are exactly 0, but 0 * NaN is not: the rows are
+            // cleared here (whole 128-byte rows of both halves: the swizzle stays inside a row), and the clearing is
+            // made visible to the tensor core's reads.
+            const int live = L + a.n - (blk_lo + 2 * u + c) * kBlockN;  // rows of this block that exist
+            if (live < kBlockN) {
+              uint4* vt = reinterpret_cast<uint4*>(sm->v[c][b]);
+              for (int i = max(live, 0) * 8 + lane; i < kBlockN * 8; i += 32) {
+                vt[i] = make_uint4(0u, 0u, 0u, 0u);
+                vt[kKvHalf / 16 + i] = make_uint4(0u, 0u, 0u, 0u);
+              }
+              fence_async_smem();
+              __syncwarp();
+            }
+          }
           tc_fence_after();
           const uint64_t vd0 = make_desc(smem_u32(sm->v[c][b]), kKvHalf, 1024);
           const uint32_t pa = tmem + 128u * c + 64u * b;
@@ -636,11 +675,11 @@ tree_attention_umma_kernel(const __grid_constant__ CUtensorMap q_map, const __gr
     tmem_ld32(tmem_s, sreg, 0);
     tmem_ld32(tmem_s + 32u, sreg, 32);
     const int kb = (blk_lo + jj) * kBlockN;
-    const bool masked = kb + kBlockN > a.L;  // the block reaches into the tree keys (or past the end)
+    const bool masked = kb + kBlockN > L;  // the block reaches into the tree keys (or past the end)
     uint32_t vis[2] = {0xFFFFFFFFu, 0xFFFFFFFFu};
     if (masked) {
-      vis[0] = mask_window(mrow, mask_wpr, a.n, kb - a.L);
-      vis[1] = mask_window(mrow, mask_wpr, a.n, kb - a.L + 32);
+      vis[0] = mask_window(mrow, mask_wpr, a.n, kb - L);
+      vis[1] = mask_window(mrow, mask_wpr, a.n, kb - L + 32);
     }
     tc_wait_ld();
     if (threadIdx.x == 128) UTRACE(2, 2);
@@ -765,9 +804,9 @@ tree_attention_umma_kernel(const __grid_constant__ CUtensorMap q_map, const __gr
     // if the piece opens the CTA's range, else 1), then counted; the CTA whose count completes the tile
     // adds the other pieces to its own and writes the output.  Nobody waits for anybody.
     // positions of the tile's blocks in the layout, and the CTAs whose ranges hold some of them
-    const int64_t t0 = (int64_t)g * a.blocks_per_head + sm->tile_prefix[sg.slot_in_head] + kStreamTileCost, t1 = t0 + sg.nblk_tile;
-    auto cta_lo = [&](int c) { return (a.total_blocks * (int64_t)c) / (int64_t)gridDim.x; };
-    int c_first = (int)((t0 * (int64_t)gridDim.x) / a.total_blocks);  // the CTA whose range holds block t0 ...
+    const int64_t t0 = (int64_t)g * blocks_per_head + sm->tile_prefix[sg.slot_in_head] + kStreamTileCost, t1 = t0 + sg.nblk_tile;
+    auto cta_lo = [&](int c) { return (total_blocks * (int64_t)c) / (int64_t)gridDim.x; };
+    int c_first = (int)((t0 * (int64_t)gridDim.x) / total_blocks);  // the CTA whose range holds block t0 ...
     while (cta_lo(c_first + 1) <= t0) ++c_first;                      // ... exactly
     while (cta_lo(c_first) > t0) --c_first;
     int c_last = c_first;
@@ -1039,8 +1078,9 @@ int launch_attention_umma(const seq_tree_attention_params& p, int splits, cudaSt
       return SEQ_ERR_CUDA;
   }
   for (int which = 0; which < 2; ++which) {
-    // only the live rows [0, prefix_len + n_tree) are mapped: anything past them reads as zero
-    cuuint64_t dims[4] = {64, (cuuint64_t)(p.prefix_len + p.n_tree), 2, (cuuint64_t)p.num_kv_heads};
+    // only the live rows [0, prefix_len + n_tree) are mapped: anything past them reads as zero.  (With the prefix
+    // length in device memory the map cannot end there: it covers the cache, and the kernel clears the tail rows.)
+    cuuint64_t dims[4] = {64, (cuuint64_t)(p.prefix_len_dev != nullptr ? p.kv_capacity : p.prefix_len + p.n_tree), 2, (cuuint64_t)p.num_kv_heads};
     cuuint64_t strides[3] = {(cuuint64_t)p.kv_stride_tok * 2, 128, (cuuint64_t)p.kv_stride_head * 2};
     cuuint32_t box[4] = {64, (cuuint32_t)kBlockN, 2, 1};
     cuuint32_t estr[4] = {1, 1, 1, 1};
@@ -1051,7 +1091,7 @@ int launch_attention_umma(const seq_tree_attention_params& p, int splits, cudaSt
   }
 
   UmmaArgs a;
-  a.n = p.n_tree; a.L = p.prefix_len; a.Hq = p.num_q_heads; a.Hkv = p.num_kv_heads; a.group = G;
+  a.n = p.n_tree; a.L_host = p.prefix_len; a.Hq = p.num_q_heads; a.Hkv = p.num_kv_heads; a.group = G;
   a.mask_wpr = p.mask_words_per_row; a.splits = splits; a.nodes_per_tile = nodes_per_tile; a.tiles = tiles;
   const float scale = p.softmax_scale > 0.f ? p.softmax_scale : 0.08838834764831845f;
   a.scale_log2 = scale * kLog2e;
@@ -1066,7 +1106,8 @@ int launch_attention_umma(const seq_tree_attention_params& p, int splits, cudaSt
   a.lse = p.lse;
   a.dev_status = p.dev_status;
   a.stream = umma_stream_mode(p, splits) ? 1 : 0;
-  a.blocks_per_head = 0; a.total_blocks = 0;
+  a.blocks_per_head_host = 0; a.total_blocks_host = 0;
+  a.L_dev = p.prefix_len_dev; a.zero_tail = p.prefix_len_dev != nullptr ? 1 : 0;
   a.ws_count = nullptr; a.ws_ml = nullptr; a.ws_o = nullptr;
   if (a.stream) {
     const size_t cnt_bytes = stream_count_bytes(p);
@@ -1074,9 +1115,9 @@ int launch_attention_umma(const seq_tree_attention_params& p, int splits, cudaSt
     if (reinterpret_cast<uintptr_t>(p.workspace) % 256 != 0) return SEQ_ERR_INVALID_ARG;
     for (int t = 0; t < tiles; ++t) {
       const int i1 = (t + 1) * nodes_per_tile < p.n_tree ? (t + 1) * nodes_per_tile : p.n_tree;
-      a.blocks_per_head += kStreamTileCost + (p.prefix_len + i1 + kBlockN - 1) / kBlockN;
+      a.blocks_per_head_host += kStreamTileCost + (p.prefix_len + i1 + kBlockN - 1) / kBlockN;
     }
-    a.total_blocks = (int64_t)a.blocks_per_head * p.num_kv_heads;
+    a.total_blocks_host = (int64_t)a.blocks_per_head_host * p.num_kv_heads;
     uint8_t* ws = static_cast<uint8_t*>(p.workspace);
     a.ws_count = reinterpret_cast<int32_t*>(ws);
     a.ws_ml = reinterpret_cast<float2*>(ws + cnt_bytes);
@@ -1089,7 +1130,7 @@ int launch_attention_umma(const seq_tree_attention_params& p, int splits, cudaSt
   // Stream schedule: one CTA per SM, but never more CTAs than positions in the layout: a range must not be empty
   // (the CTAs that share a cut tile are counted from the ranges, and each of them has to arrive).
   const int sms = device_sm_count();
-  const int stream_ctas = a.total_blocks < sms ? (int)a.total_blocks : sms;
+  const int stream_ctas = a.total_blocks_host < sms ? (int)a.total_blocks_host : sms;
   cfg.gridDim = a.stream ? dim3(stream_ctas, 1, 1) : dim3(tiles, p.num_kv_heads, splits);
   cfg.blockDim = dim3(kUmmaThreads);
   cfg.dynamicSmemBytes = smem;
