@@ -214,8 +214,9 @@ int seq_tree_attention_noalloc(const seq_tree_attention_params* p, void* stream)
  * uniforms are not read.
  *
  *   parent, tokens      [n] int32; tokens[0] is ignored.  A single root.
- *   target_logits       fp32, row v at v*target_row_stride: next-token logits after node v.
- *   draft_logits        fp32, row v at v*draft_row_stride: the logits whose softmax at T
+ *   target_logits       fp32 (bfloat16 with SEQ_VERIFY_LOGITS_BF16), row v at v*target_row_stride: next-token
+ *                       logits after node v.
+ *   draft_logits        same type, row v at v*draft_row_stride: the logits whose softmax at T
  *                       v's children were drawn from without replacement; rows of leaves
  *                       are never read.  -inf entries are legal (probability 0).
  *   temperature         >= 0, finite; one value for both models.
@@ -259,7 +260,12 @@ enum {
    *     paper's models; kept selectable.
    * SCHED_NODES without enough workspace returns SEQ_ERR_WORKSPACE, where it does not apply SEQ_ERR_UNSUPPORTED. */
   SEQ_VERIFY_SCHED_WALK = 16,
-  SEQ_VERIFY_SCHED_NODES = 32
+  SEQ_VERIFY_SCHED_NODES = 32,
+  /* target_logits and draft_logits hold bfloat16 instead of fp32 (what a 16-bit language-model head writes; half the
+   * bytes per visited node).  Every value is widened to fp32 exactly and the arithmetic is unchanged.  Row strides
+   * stay in elements (multiples of 4), rows 8-byte aligned.  One request at T > 0 in the default mode or with
+   * SEQ_VERIFY_SPECINFER, on the walk schedule; anything else returns SEQ_ERR_UNSUPPORTED. */
+  SEQ_VERIFY_LOGITS_BF16 = 8
 };
 
 typedef struct {

@@ -21,6 +21,7 @@ SEQ_VERIFY_ALL_NODES = 1
 SEQ_VERIFY_SPECINFER = 2
 SEQ_VERIFY_TARGET_SAMPLE = 4
 SEQ_VERIFY_SCHED_WALK, SEQ_VERIFY_SCHED_NODES = 16, 32
+SEQ_VERIFY_LOGITS_BF16 = 8
 SEQ_DEV_BAD_PATH = 32
 SEQ_DEV_BAD_LENGTH = 64
 SEQ_MAX_TREE = 1024
@@ -318,8 +319,11 @@ class VerifyCall:
         p = VerifyParams()
         p.n_tree, p.vocab = n, V
         p.parent, p.tokens = _dev(parent, "parent", torch.int32), _dev(tokens, "tokens", torch.int32)
-        p.target_logits, p.target_row_stride = _dev(target_logits, "target_logits", torch.float32), target_logits.stride(0)
-        p.draft_logits = _dev(draft_logits, "draft_logits", torch.float32)
+        ldt = target_logits.dtype  # fp32, or bfloat16 (then the draft's too)
+        if ldt not in (torch.float32, torch.bfloat16):
+            raise ValueError("target_logits must be float32 or bfloat16")
+        p.target_logits, p.target_row_stride = _dev(target_logits, "target_logits", ldt), target_logits.stride(0)
+        p.draft_logits = _dev(draft_logits, "draft_logits", ldt)
         p.draft_row_stride = draft_logits.stride(0) if draft_logits is not None else 0
         p.temperature = temperature
         p.uniforms = _dev(uniforms, "uniforms", torch.float32)
@@ -330,7 +334,7 @@ class VerifyCall:
         p.workspace, p.workspace_bytes = None, 0
         p.dev_status = _dev(dev_status, "dev_status", torch.int32)
         p.flags = ((SEQ_VERIFY_ALL_NODES if all_nodes else 0) | (SEQ_VERIFY_SPECINFER if specinfer else 0) |
-                   (SEQ_VERIFY_TARGET_SAMPLE if target_sample else 0) |
+                   (SEQ_VERIFY_TARGET_SAMPLE if target_sample else 0) | (SEQ_VERIFY_LOGITS_BF16 if ldt == torch.bfloat16 else 0) |
                    {"auto": 0, "walk": SEQ_VERIFY_SCHED_WALK, "nodes": SEQ_VERIFY_SCHED_NODES}[schedule])
         need = load().seq_tree_verify_workspace_bytes(C.byref(p))
         if workspace is None and need:

@@ -78,7 +78,8 @@ static int verify_validate(const seq_tree_verify_params* p) {
   if (p->n_tree < 1 || p->n_tree > SEQ_MAX_TREE || p->vocab < 1) return SEQ_ERR_INVALID_ARG;
   if (p->parent == nullptr || p->tokens == nullptr || p->target_logits == nullptr) return SEQ_ERR_INVALID_ARG;
   if (!(p->temperature >= 0.f) || isinf(p->temperature)) return SEQ_ERR_INVALID_ARG;
-  if (p->flags & ~(SEQ_VERIFY_ALL_NODES | SEQ_VERIFY_SPECINFER | SEQ_VERIFY_TARGET_SAMPLE | SEQ_VERIFY_SCHED_WALK | SEQ_VERIFY_SCHED_NODES))
+  if (p->flags & ~(SEQ_VERIFY_ALL_NODES | SEQ_VERIFY_SPECINFER | SEQ_VERIFY_TARGET_SAMPLE | SEQ_VERIFY_SCHED_WALK | SEQ_VERIFY_SCHED_NODES |
+                   SEQ_VERIFY_LOGITS_BF16))
     return SEQ_ERR_INVALID_ARG;
   if ((p->flags & SEQ_VERIFY_SCHED_WALK) && (p->flags & SEQ_VERIFY_SCHED_NODES)) return SEQ_ERR_INVALID_ARG;
   if ((p->flags & SEQ_VERIFY_SPECINFER) && (p->flags & SEQ_VERIFY_TARGET_SAMPLE)) return SEQ_ERR_INVALID_ARG;
@@ -90,12 +91,14 @@ static int verify_validate(const seq_tree_verify_params* p) {
   }
   if (p->temperature > 0.f && p->uniforms == nullptr) return SEQ_ERR_INVALID_ARG;
   if (p->temperature > 0.f && p->draft_logits == nullptr && !(p->flags & SEQ_VERIFY_TARGET_SAMPLE)) return SEQ_ERR_INVALID_ARG;
+  // rows start on 16-byte boundaries (8-byte for 16-bit logits)
+  const uintptr_t base_align = (p->flags & SEQ_VERIFY_LOGITS_BF16) ? 8 : 16;
   if (p->target_row_stride < p->vocab || p->target_row_stride % 4 != 0 ||
-      reinterpret_cast<uintptr_t>(p->target_logits) % 16 != 0)
+      reinterpret_cast<uintptr_t>(p->target_logits) % base_align != 0)
     return SEQ_ERR_INVALID_ARG;
   if (p->draft_logits != nullptr &&
       (p->draft_row_stride < p->vocab || p->draft_row_stride % 4 != 0 ||
-       reinterpret_cast<uintptr_t>(p->draft_logits) % 16 != 0))
+       reinterpret_cast<uintptr_t>(p->draft_logits) % base_align != 0))
     return SEQ_ERR_INVALID_ARG;
   return SEQ_OK;
 }
@@ -178,6 +181,11 @@ static int verify_launch(const seq_tree_verify_params* p, int batch, int64_t tre
     if (!fits8 && (!fits16 || batch > 0 || (p->flags & SEQ_VERIFY_ALL_NODES))) return SEQ_ERR_UNSUPPORTED;
   }
 
+  // 16-bit logits: served by the walk with its rows in registers only (default mode and the variant without the draft
+  // update, T > 0, one request, a device that places a cluster of 16)
+  const bool bf16 = (p->flags & SEQ_VERIFY_LOGITS_BF16) != 0;
+  if (bf16 && (batch != 0 || (p->flags & SEQ_VERIFY_SCHED_NODES) || !verify_walk_supported(p->vocab, p->flags, p->temperature)))
+    return SEQ_ERR_UNSUPPORTED;
   if (p->flags & SEQ_VERIFY_SCHED_NODES) {
     if (batch != 0 || !wants_nodes_schedule(p)) return SEQ_ERR_UNSUPPORTED;
     return launch_verify_nodes(a, p->workspace, p->workspace_bytes, 0, s);  // (checks the workspace)
@@ -197,6 +205,7 @@ static int verify_launch(const seq_tree_verify_params* p, int batch, int64_t tre
   }
   // the walk with its rows in registers, where a cluster of 16 can be placed and the mode is one it serves
   if (wide == 1 && verify_walk_supported(p->vocab, p->flags, p->temperature)) return launch_verify_walk(a, false, s);
+  if (bf16) return SEQ_ERR_UNSUPPORTED;
   if (wide == 1 && p->vocab >= 8192)
     return verify_launch_with<16, vcl16::VShared, 2>(vcl16::tree_verify_kernel<false>, a, p->vocab, 1, false, s);
   return verify_launch_with<8, vcl8::VShared, 1>(vcl8::tree_verify_kernel<false>, a, p->vocab, 1, false, s);

@@ -89,11 +89,32 @@ struct Ctx {
 // One row slice into registers: NCH independent 16-byte loads per thread, the ragged end element by element;
 // positions past the slice read as -inf (probability 0).  A warp holds 128 * NCH consecutive elements, in chunks of
 // 128; within a chunk a lane holds four consecutive ones.
-template <int NCH>
-__device__ __forceinline__ void load_row(const Ctx& c, const float* row, float* x) {
+__device__ __forceinline__ float bf16_bits_to_float(uint32_t b) { return __uint_as_float(b << 16); }  // exact
+template <bool kBf16>
+__device__ __forceinline__ float load_logit(const void* row, int64_t i) {
+  if (kBf16) return bf16_bits_to_float(__ldg(static_cast<const unsigned short*>(row) + i));
+  return __ldg(static_cast<const float*>(row) + i);
+}
+template <int NCH, bool kBf16>
+__device__ __forceinline__ void load_row(const Ctx& c, const void* row_v, float* x) {
   const int first = c.warp * (128 * NCH) + c.lane * 4;
-  const float* base = row + c.lo + first;
   const int room = c.cnt - first;
+  if (kBf16) {  // four 16-bit logits per lane and chunk: 8-byte loads
+    const unsigned short* base = static_cast<const unsigned short*>(row_v) + c.lo + first;
+#pragma unroll
+    for (int j = 0; j < NCH; ++j) {
+      if (room - 128 * j >= 4) {
+        const uint2 v = __ldcs(reinterpret_cast<const uint2*>(base + 128 * j));
+        x[4 * j] = bf16_bits_to_float(v.x & 0xFFFFu); x[4 * j + 1] = bf16_bits_to_float(v.x >> 16);
+        x[4 * j + 2] = bf16_bits_to_float(v.y & 0xFFFFu); x[4 * j + 3] = bf16_bits_to_float(v.y >> 16);
+      } else {
+#pragma unroll
+        for (int i = 0; i < 4; ++i) x[4 * j + i] = room - 128 * j > i ? bf16_bits_to_float(__ldcs(base + 128 * j + i)) : -INFINITY;
+      }
+    }
+    return;
+  }
+  const float* base = static_cast<const float*>(row_v) + c.lo + first;
 #pragma unroll
   for (int j = 0; j < NCH; ++j) {
     float4 v;
@@ -165,8 +186,11 @@ __device__ __forceinline__ void cluster_exchange(cg::cluster_group& cluster, Ctx
   exchange_pull(c, x);
 }
 
-template <int NCH>
+template <int NCH, bool kBf16>
 __global__ void __launch_bounds__(kTh, 1) tree_verify_walk_kernel(const VerifyArgs a) {
+  constexpr int kEsz = kBf16 ? 2 : 4;  // bytes per logit
+  const char* const tbase = reinterpret_cast<const char*>(a.target);
+  const char* const dbase = reinterpret_cast<const char*>(a.draft);
   constexpr int kE = 4 * NCH;        // elements per thread and row
   constexpr int kSpan = 32 * kE;     // consecutive elements of the slice that one warp holds
   cg::cluster_group cluster = cg::this_cluster();
@@ -205,8 +229,8 @@ __global__ void __launch_bounds__(kTh, 1) tree_verify_walk_kernel(const VerifyAr
     }
 #pragma unroll
     for (int k = 0; k < 5; ++k) tu[k] = c.tid + kTh * k <= a.n ? a.uniforms[c.tid + kTh * k] : 0.f;
-    load_row<NCH>(c, a.target, p);
-    if (a.n > 1) load_row<NCH>(c, a.draft, q);  // (a root without children: never read)
+    load_row<NCH, kBf16>(c, tbase, p);
+    if (a.n > 1) load_row<NCH, kBf16>(c, dbase, q);  // (a root without children: never read)
     if (c.tid < SEQ_MAX_TREE / 32) sh->has_child[c.tid] = 0u;
     if (c.tid == 0) sh->node_flags = 0;
     __syncthreads();
@@ -239,8 +263,8 @@ __global__ void __launch_bounds__(kTh, 1) tree_verify_walk_kernel(const VerifyAr
     ++plen;
     WTRACE(leader, 10);
     const int np = hop & 1;
-    const float* trow = a.target + (int64_t)cur * a.target_stride;
-    const float* drow = a.draft + (int64_t)cur * a.draft_stride;
+    const char* trow = tbase + (int64_t)cur * a.target_stride * kEsz;
+    const char* drow = dbase + (int64_t)cur * a.draft_stride * kEsz;
     // ---- exponentials relative to this thread's own maxima, with their sums; the per-warp partials go to every CTA
     const bool need_draft = cur_has_kids;
     bool bad = false;
@@ -294,7 +318,7 @@ __global__ void __launch_bounds__(kTh, 1) tree_verify_walk_kernel(const VerifyAr
           sh->kids[np][r] = ch;
           sh->kid_tok[np][r] = s;
           krank[j] = r;
-          if (s >= 0 && s < a.V) kraw[j] = make_float2(__ldg(trow + s), __ldg(drow + s));
+          if (s >= 0 && s < a.V) kraw[j] = make_float2(load_logit<kBf16>(trow, s), load_logit<kBf16>(drow, s));
         }
       }
       __syncthreads();
@@ -303,8 +327,8 @@ __global__ void __launch_bounds__(kTh, 1) tree_verify_walk_kernel(const VerifyAr
     bool nxt_has_kids = false;
     if (nxt >= 0) {
       nxt_has_kids = (sh->has_child[nxt >> 5] >> (nxt & 31)) & 1u;
-      load_row<NCH>(c, a.target + (int64_t)nxt * a.target_stride, pn);
-      if (nxt_has_kids) load_row<NCH>(c, a.draft + (int64_t)nxt * a.draft_stride, qn);
+      load_row<NCH, kBf16>(c, tbase + (int64_t)nxt * a.target_stride * kEsz, pn);
+      if (nxt_has_kids) load_row<NCH, kBf16>(c, dbase + (int64_t)nxt * a.draft_stride * kEsz, qn);
     }
     WTRACE(leader, 44);
     if (!specinfer) {  // does an earlier sibling carry the same token?
@@ -390,8 +414,8 @@ __global__ void __launch_bounds__(kTh, 1) tree_verify_walk_kernel(const VerifyAr
       if (i + 1 < n_kids) {
         nxt = sh->kids[np][i + 1];
         nxt_has_kids = (sh->has_child[nxt >> 5] >> (nxt & 31)) & 1u;
-        load_row<NCH>(c, a.target + (int64_t)nxt * a.target_stride, pn);
-        if (nxt_has_kids) load_row<NCH>(c, a.draft + (int64_t)nxt * a.draft_stride, qn);
+        load_row<NCH, kBf16>(c, tbase + (int64_t)nxt * a.target_stride * kEsz, pn);
+        if (nxt_has_kids) load_row<NCH, kBf16>(c, dbase + (int64_t)nxt * a.draft_stride * kEsz, qn);
       }
       if (!valid) continue;  // (not a token: R and D untouched)
       // R <- norm(max(R - D, 0)) with D as it stands
@@ -567,10 +591,12 @@ int launch_verify_walk(const VerifyArgs& a_in, bool check_only, cudaStream_t str
   VerifyArgs a = a_in;
   a.slice_cap = (((a.V + vwk::kCl - 1) / vwk::kCl) + 3) & ~3;
   const int nch = a.slice_cap <= vwk::kTh * 4 * 2 ? 2 : a.slice_cap <= vwk::kTh * 4 * 4 ? 4 : 8;
-  void (*kernel)(const VerifyArgs) = nch == 2 ? vwk::tree_verify_walk_kernel<2> : nch == 4 ? vwk::tree_verify_walk_kernel<4>
-                                                                                           : vwk::tree_verify_walk_kernel<8>;
-  const int slot = nch == 2 ? 0 : nch == 4 ? 1 : 2;
-  static int attr_done[3][64];
+  const bool bf16 = (a.flags & SEQ_VERIFY_LOGITS_BF16) != 0;
+  void (*kernel)(const VerifyArgs) =
+      bf16 ? (nch == 2 ? vwk::tree_verify_walk_kernel<2, true> : nch == 4 ? vwk::tree_verify_walk_kernel<4, true> : vwk::tree_verify_walk_kernel<8, true>)
+           : (nch == 2 ? vwk::tree_verify_walk_kernel<2, false> : nch == 4 ? vwk::tree_verify_walk_kernel<4, false> : vwk::tree_verify_walk_kernel<8, false>);
+  const int slot = (nch == 2 ? 0 : nch == 4 ? 1 : 2) + (bf16 ? 3 : 0);
+  static int attr_done[6][64];
   const int rc = once_per_device(attr_done[slot], [&]() -> int {
     SEQ_CUDA_OK(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sizeof(vwk::Shared)));
     SEQ_CUDA_OK(cudaFuncSetAttribute(kernel, cudaFuncAttributeNonPortableClusterSizeAllowed, 1));

@@ -72,7 +72,7 @@ def _path(parent, i):
     return out
 
 
-def run_verify(vi: W.VerifyInputs, all_nodes=False, want_residual=True, specinfer=False, target_sample=False):
+def run_verify(vi: W.VerifyInputs, all_nodes=False, want_residual=True, specinfer=False, target_sample=False, bf16_logits=False):
     d = dev()
     n, V = vi.target_logits.shape
     st = torch.zeros(1, dtype=torch.int32, device=d)
@@ -87,6 +87,12 @@ def run_verify(vi: W.VerifyInputs, all_nodes=False, want_residual=True, specinfe
         dl = torch.full((n, Vp), float("nan"), dtype=torch.float32, device=d)
         dl[:, :V] = vi.draft_logits.to(d)
         dl = dl[:, :V]
+    if bf16_logits:  # (the caller made sure the values are exact in bfloat16; the padded row stride is kept)
+        tl = tl.to(torch.bfloat16)
+        if dl is not None:
+            dl_full = torch.full((n, Vp), float("nan"), dtype=torch.bfloat16, device=d)
+            dl_full[:, :V] = dl.to(torch.bfloat16)
+            dl = dl_full[:, :V]
     call = B.VerifyCall(vi.parent.to(d), vi.tokens.to(d), tl[:, :V], dl,
                         vi.temperature, vi.uniforms.to(d), residual_out=residual, next_child_out=nxt,
                         all_nodes=all_nodes, dev_status=st, specinfer=specinfer, target_sample=target_sample,
@@ -99,10 +105,10 @@ def run_verify(vi: W.VerifyInputs, all_nodes=False, want_residual=True, specinfe
                 next_child=nxt.cpu().numpy(), status=int(st.item()))
 
 
-def check_verify(vi: W.VerifyInputs, specinfer=False):
+def check_verify(vi: W.VerifyInputs, specinfer=False, bf16_logits=False):
     """Path and bonus identical to the oracle's (outside the rounding band), residual within 1e-5.
     Returns 'ok' or 'excluded'."""
-    got = run_verify(vi, specinfer=specinfer)
+    got = run_verify(vi, specinfer=specinfer, bf16_logits=bf16_logits)
     ref = O.tree_verify(vi.parent, vi.tokens, vi.target_logits, vi.draft_logits, vi.temperature, vi.uniforms,
                         variant=O.VARIANT_SPECINFER if specinfer else O.VARIANT_SEQUOIA)
     assert got["status"] == ref["flags"] == 0

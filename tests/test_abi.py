@@ -123,7 +123,7 @@ def test_host_checkable_errors_are_refused_before_launch(lib):
     bad = [dict(parent=None), dict(n_tree=0), dict(n_tree=5000), dict(vocab=0), dict(temperature=-1.0),
            dict(temperature=float("nan")), dict(temperature=float("inf")), dict(target_row_stride=31999),
            dict(target_row_stride=32001), dict(draft_logits=None), dict(uniforms=None), dict(path=None),
-           dict(flags=8), dict(flags=6), dict(flags=1, next_child_out=None), dict(target_logits=fake + 4)]
+           dict(flags=64), dict(flags=6), dict(flags=1, next_child_out=None), dict(target_logits=fake + 4)]
     for kw in bad:
         assert lib.seq_tree_verify(C.byref(ver(**kw)), None) == B.SEQ_ERR_INVALID_ARG, kw
     assert lib.seq_tree_verify(C.byref(ver(vocab=400000, target_row_stride=400000, draft_row_stride=400000)), None) \

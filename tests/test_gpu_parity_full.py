@@ -219,3 +219,21 @@ def test_verify_bonus_draw_falls_back_to_the_last_token_with_mass():
                 t = got["bonus"]
                 lo = cdf[t - 1] if t > 0 else 0.0
                 assert lo - G.GAP <= float(last) < cdf[t] + G.GAP and ref["residual"][t] > 0
+
+
+@pytest.mark.parametrize("name,T,seeds", [("tiny", 0.6, range(4)), ("llama2-7b", 0.6, range(4)), ("llama2-7b", 1.0, range(2)),
+                                          ("llama3-70b", 0.6, range(1))])
+def test_bf16_logits_are_widened_exactly(name, T, seeds):
+    """SEQ_VERIFY_LOGITS_BF16: both logit matrices in bfloat16 (half the bytes per visited node).  The oracle is given
+    the same values as fp32 (the widening is exact), so the parity rule is the usual one; also with a ragged
+    vocabulary (rows that end inside an 8-byte load) and for the variant without the draft update."""
+    cfg = W.CONFIGS[name]
+    outcomes = []
+    for seed in seeds:
+        vi = W.make_verify_inputs(cfg, T, seed, vocab=None if seed % 2 == 0 or cfg.vocab > 100000 else 30001)
+        vi.target_logits = vi.target_logits.to(torch.bfloat16).float()
+        vi.draft_logits = vi.draft_logits.to(torch.bfloat16).float()
+        outcomes.append(G.check_verify(vi, bf16_logits=True))
+        if seed == 0:
+            outcomes.append(G.check_verify(vi, bf16_logits=True, specinfer=True))
+    assert outcomes.count("ok") >= len(outcomes) - 1, outcomes
