@@ -633,6 +633,86 @@ def spread(ms_list, per):
     return {"median": statistics.median(us), "min": us[0], "max": us[-1], "replays": len(us)}
 
 
+def verify_bf16_leg(cfg, parent, ver_sets, T, dev, stream) -> dict:
+    """Not part of the timed step: the verification with both logit matrices in bfloat16 (half the bytes per visited
+    node), L2-cold like the fp32 figure (a 160 MiB write before each launch, the same graph without launches
+    subtracted)."""
+    from paper_2402_12374_b200 import binding as B
+
+    status = torch.zeros(1, dtype=torch.int32, device=dev)
+    parent_d = torch.from_numpy(parent).to(dev)
+    calls = [B.VerifyCall(parent_d, tok, tl.to(torch.bfloat16), dl.to(torch.bfloat16), T, u, dev_status=status)
+             for tok, tl, dl, u in ver_sets[:2]]
+    flush = torch.empty(160 << 20, dtype=torch.uint8, device=dev)
+    Kc = 12
+
+    def graph_of(body):
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g, stream=stream):
+            for i in range(Kc):
+                body(i)
+        g.replay()
+        stream.synchronize()
+        return g
+
+    with torch.cuda.stream(stream):
+        calls[0].run(stream)
+        stream.synchronize()
+        g_cold = graph_of(lambda i: (flush.fill_(i & 127), calls[i % len(calls)].run(stream)))
+        g_flush = graph_of(lambda i: flush.fill_(i & 127))
+        ms = [statistics.median(timed_replays(g, stream, 7, 1, dev)) for g in (g_cold, g_flush)]
+    if int(status.item()) != 0:
+        raise RuntimeError(f"verify_bf16 dev_status = {int(status.item())}")
+    return {"us_per_launch": (ms[0] - ms[1]) * 1e3 / Kc, "l2": "cold (160 MiB written before every launch)",
+            "note": "SEQ_VERIFY_LOGITS_BF16: the same walk on bfloat16 logits; outside the timed step"}
+
+
+def robustness_leg(dev, stream, vocab=2048, requests=1500) -> dict:
+    """Not part of the timed step (--robustness): a synthetic analogue of the paper's rejection-rate figure (Section
+    3.2.2: average rejection rate against the number of speculated child tokens at T = 0.2, 0.6, 1.0, for the three
+    verification algorithms), on the library's three verifiers through seq_tree_verify_batch.  One node with k
+    children per request, target logits N(0, 3^2), draft = target + N(0, 1): Sequoia (children drawn without
+    replacement, Algorithm 2), SpecInfer (children drawn with replacement, Algorithm 2 without the draft update),
+    top-k (children = the draft's top k, verification by sampling from the target).  Rejection = no child accepted."""
+    from paper_2402_12374_b200 import binding as B
+
+    gen = torch.Generator(device=dev)
+    gen.manual_seed(W.BASE_SEED)
+    ks = [1, 2, 4, 8, 16, 32]
+    out = {"vocab": vocab, "requests_per_point": requests, "k": ks, "rejection_rate": {}}
+    status = torch.zeros(1, dtype=torch.int32, device=dev)
+    torch.cuda.synchronize()
+    with torch.cuda.stream(stream):  # inputs and launches on one stream
+        for T in (0.2, 0.6, 1.0):
+            rates = {"sequoia": [], "specinfer": [], "top_k": []}
+            for k in ks:
+                n = k + 1
+                tl = 3.0 * torch.randn((requests, 1, vocab), device=dev, generator=gen)
+                dl = tl + torch.randn((requests, 1, vocab), device=dev, generator=gen)
+                TL, DL = tl.expand(requests, n, vocab).contiguous(), dl.expand(requests, n, vocab).contiguous()
+                par = torch.zeros((requests, n), dtype=torch.int32, device=dev)
+                par[:, 0] = -1
+                u = torch.rand((requests, n + 1), device=dev, generator=gen)
+                gum = -torch.log(-torch.log(torch.rand((requests, vocab), device=dev, generator=gen).clamp_(1e-9, 1 - 1e-7)))
+                draws = {
+                    "sequoia": torch.topk(dl[:, 0] / T + gum, k, dim=1).indices,
+                    "specinfer": torch.multinomial(torch.softmax(dl[:, 0] / T, dim=1), k, replacement=True, generator=gen),
+                    "top_k": torch.topk(dl[:, 0], k, dim=1).indices,
+                }
+                for name, kids in draws.items():
+                    tok = torch.zeros((requests, n), dtype=torch.int32, device=dev)
+                    tok[:, 1:] = kids.to(torch.int32)
+                    _, plen, _ = B.seq_tree_verify_batch(par, tok, TL, None if name == "top_k" else DL, T, u, dev_status=status,
+                                                         specinfer=name == "specinfer", target_sample=name == "top_k", stream=stream)
+                    stream.synchronize()
+                    rates[name].append(float((plen == 1).float().mean().item()))
+            out["rejection_rate"][f"T={T}"] = rates
+    if int(status.item()) != 0:
+        raise RuntimeError(f"robustness dev_status = {int(status.item())}")
+    out["note"] = "synthetic logits; outside the timed step"
+    return out
+
+
 def floors_leg(dev, stream) -> dict:
     """What the device gives to a kernel that only reads (GB/s over a buffer far larger than L2) and to a launch
     that does next to nothing (one warp, one dependent load from memory that is not in L2), both through this
@@ -782,14 +862,26 @@ def run_workload(cfg, T, args, rank, local_rank, world, dev, stream, peaks, with
     has_child = np.zeros(n, dtype=bool)
     has_child[parent[1:][parent[1:] >= 0]] = True
     torch.cuda.synchronize()
-    path_bytes, visited = [], []
+    kids = W.children_lists(parent)
+    row_bytes = lambda v: 4 * cfg.vocab * (2 if has_child[v] else 1)
+    path_bytes, moved_bytes, visited = [], [], []
     for vc in ver_calls:
         plen = int(vc.path_len.item())
-        nodes = vc.path[:plen].cpu().numpy()
+        nodes = vc.path[:plen].cpu().numpy().tolist()
         visited.append(plen)
-        path_bytes.append(sum(4 * cfg.vocab * (2 if has_child[v] else 1) for v in nodes))
+        path_bytes.append(sum(row_bytes(v) for v in nodes))
+        # what the walk really loads: the root's rows, and ahead of its test the rows of every child that is tested
+        # (up to the accepted one, all of them where none is accepted)
+        m = row_bytes(0)
+        for i, v in enumerate(nodes):
+            nxt = nodes[i + 1] if i + 1 < plen else None
+            for ch in kids[v]:
+                m += row_bytes(ch)
+                if ch == nxt:
+                    break
+        moved_bytes.append(m)
     b_path = float(np.mean(path_bytes))
-    moved = ver_calls[0].bytes_moved_estimate(b_path) if hasattr(ver_calls[0], "bytes_moved_estimate") else b_path
+    moved = float(np.mean(moved_bytes))
     ver_gbs = moved / (ver_cold_us * 1e-6) / 1e9
     roofline_verify = {"bound": "hbm", "achieved": ver_gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s",
                        "frac": ver_gbs / peaks["hbm_gbs"], "frac_of_spec": ver_gbs / SPEC_HBM_GBS, "traffic": None,
@@ -798,7 +890,8 @@ def run_workload(cfg, T, args, rank, local_rank, world, dev, stream, peaks, with
                        "visited_nodes_mean": float(np.mean(visited)),
                        "timing": f"L2-cold: {Kc} launches in one graph, a 160 MiB write before each, minus the same graph "
                                  f"without the launches; L2-warm: {Kb} launches back to back over {nv} logit sets",
-                       "note": "a dependent walk: latency-bound, its HBM fraction says little"}
+                       "note": "a dependent walk on one cluster of 16 CTAs: latency-bound, its HBM fraction says little; bytes moved "
+                               "= the visited nodes' rows plus the rows of tested-and-rejected children, loaded ahead of their test"}
     res = {
         "us_per_step": step_us, "ms_per_step": step_us["median"] / 1e3,
         "attention_us": attn_us, "verify_us": ver_cold_us, "verify_us_l2_warm": ver_warm_us,
@@ -820,6 +913,7 @@ def run_workload(cfg, T, args, rank, local_rank, world, dev, stream, peaks, with
         ver_like = [_HostLike(*s) for s in ver_sets]
         legs["verify_batch"] = verify_batch_leg(cfg, parent, ver_like, T, dev, stream)
         if T > 0:
+            legs["verify_bf16_logits"] = verify_bf16_leg(cfg, parent, ver_sets, T, dev, stream)
             legs["top_p_filter"] = top_p_leg(cfg, ver_like, T, dev, stream, peaks)
             legs["draft_sample"] = draft_sample_leg(cfg, parent, ver_like, T, dev, stream, peaks)
         res["next_rows"] = legs
@@ -851,6 +945,8 @@ def main():
                     help="random: seeded random tree within the config's bounds; dp: Sequoia's dynamic program on the paper's acceptance vector")
     ap.add_argument("--tree-search", action="store_true",
                     help="also time the step on trees of growing size and run the Speedup(n, d) search on that t(n)")
+    ap.add_argument("--robustness", action="store_true",
+                    help="also sweep the three verifiers' rejection rate against the number of speculated children")
     ap.add_argument("--separate-mask", action="store_true",
                     help="build the ancestor mask with a launch of its own instead of inside the attention kernel")
     ap.add_argument("--ncu-traffic-csv", default=None,
@@ -950,6 +1046,8 @@ def main():
         line["next_rows"] = head["next_rows"]
     if not args.no_legs:
         line["floors"] = floors_leg(dev, stream)
+    if args.robustness:
+        line.setdefault("next_rows", {})["robustness"] = robustness_leg(dev, stream)
     if not args.no_cpu_baseline:
         from oracle import oracle as O
 

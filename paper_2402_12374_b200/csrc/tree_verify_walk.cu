@@ -95,38 +95,61 @@ __device__ __forceinline__ float load_logit(const void* row, int64_t i) {
   if (kBf16) return bf16_bits_to_float(__ldg(static_cast<const unsigned short*>(row) + i));
   return __ldg(static_cast<const float*>(row) + i);
 }
+// One row slice into registers, as it lies in memory: NCH independent loads per thread (16 bytes each for fp32 logits,
+// 8 for 16-bit ones), the ragged end element by element; positions past the slice read as -inf (probability 0).  A
+// warp holds 128 * NCH consecutive elements, in chunks of 128; within a chunk a lane holds four consecutive ones.
+// Nothing here touches the loaded values, so the loads stay in flight until widen() is called on them: that is what
+// lets the next node's rows travel while the current node is worked on.
 template <int NCH, bool kBf16>
-__device__ __forceinline__ void load_row(const Ctx& c, const void* row_v, float* x) {
+struct RawRow { uint32_t w[kBf16 ? 2 * NCH : 4 * NCH]; };
+template <int NCH, bool kBf16>
+__device__ __forceinline__ void load_row(const Ctx& c, const void* row_v, RawRow<NCH, kBf16>& r) {
   const int first = c.warp * (128 * NCH) + c.lane * 4;
   const int room = c.cnt - first;
-  if (kBf16) {  // four 16-bit logits per lane and chunk: 8-byte loads
+  if (kBf16) {
     const unsigned short* base = static_cast<const unsigned short*>(row_v) + c.lo + first;
 #pragma unroll
     for (int j = 0; j < NCH; ++j) {
+      uint2 v;
       if (room - 128 * j >= 4) {
-        const uint2 v = __ldcs(reinterpret_cast<const uint2*>(base + 128 * j));
-        x[4 * j] = bf16_bits_to_float(v.x & 0xFFFFu); x[4 * j + 1] = bf16_bits_to_float(v.x >> 16);
-        x[4 * j + 2] = bf16_bits_to_float(v.y & 0xFFFFu); x[4 * j + 3] = bf16_bits_to_float(v.y >> 16);
+        v = __ldcs(reinterpret_cast<const uint2*>(base + 128 * j));
       } else {
-#pragma unroll
-        for (int i = 0; i < 4; ++i) x[4 * j + i] = room - 128 * j > i ? bf16_bits_to_float(__ldcs(base + 128 * j + i)) : -INFINITY;
+        const uint32_t h0 = room - 128 * j > 0 ? __ldcs(base + 128 * j) : 0xFF80u, h1 = room - 128 * j > 1 ? __ldcs(base + 128 * j + 1) : 0xFF80u;
+        const uint32_t h2 = room - 128 * j > 2 ? __ldcs(base + 128 * j + 2) : 0xFF80u;  // (0xFF80: -inf)
+        v = make_uint2(h0 | (h1 << 16), h2 | (0xFF80u << 16));
       }
+      r.w[2 * j] = v.x; r.w[2 * j + 1] = v.y;
     }
-    return;
+  } else {
+    const float* base = static_cast<const float*>(row_v) + c.lo + first;
+#pragma unroll
+    for (int j = 0; j < NCH; ++j) {
+      float4 v;
+      if (room - 128 * j >= 4) {
+        v = __ldcs(reinterpret_cast<const float4*>(base + 128 * j));
+      } else {
+        v.x = room - 128 * j > 0 ? __ldcs(base + 128 * j) : -INFINITY;
+        v.y = room - 128 * j > 1 ? __ldcs(base + 128 * j + 1) : -INFINITY;
+        v.z = room - 128 * j > 2 ? __ldcs(base + 128 * j + 2) : -INFINITY;
+        v.w = -INFINITY;
+      }
+      r.w[4 * j] = __float_as_uint(v.x); r.w[4 * j + 1] = __float_as_uint(v.y);
+      r.w[4 * j + 2] = __float_as_uint(v.z); r.w[4 * j + 3] = __float_as_uint(v.w);
+    }
   }
-  const float* base = static_cast<const float*>(row_v) + c.lo + first;
+}
+// ... and widened to fp32 (exact)
+template <int NCH, bool kBf16>
+__device__ __forceinline__ void widen(const RawRow<NCH, kBf16>& r, float* x) {
 #pragma unroll
   for (int j = 0; j < NCH; ++j) {
-    float4 v;
-    if (room - 128 * j >= 4) {
-      v = __ldcs(reinterpret_cast<const float4*>(base + 128 * j));
+    if (kBf16) {
+      x[4 * j] = __uint_as_float(r.w[2 * j] << 16); x[4 * j + 1] = __uint_as_float(r.w[2 * j] & 0xFFFF0000u);
+      x[4 * j + 2] = __uint_as_float(r.w[2 * j + 1] << 16); x[4 * j + 3] = __uint_as_float(r.w[2 * j + 1] & 0xFFFF0000u);
     } else {
-      v.x = room - 128 * j > 0 ? __ldcs(base + 128 * j) : -INFINITY;
-      v.y = room - 128 * j > 1 ? __ldcs(base + 128 * j + 1) : -INFINITY;
-      v.z = room - 128 * j > 2 ? __ldcs(base + 128 * j + 2) : -INFINITY;
-      v.w = -INFINITY;
+#pragma unroll
+      for (int i = 0; i < 4; ++i) x[4 * j + i] = __uint_as_float(r.w[4 * j + i]);
     }
-    x[4 * j] = v.x; x[4 * j + 1] = v.y; x[4 * j + 2] = v.z; x[4 * j + 3] = v.w;
   }
 }
 
@@ -215,8 +238,8 @@ __global__ void __launch_bounds__(kTh, 1) tree_verify_walk_kernel(const VerifyAr
   asm volatile("griddepcontrol.wait;" ::: "memory");
   WTRACE(leader, 1);
 
-  float p[kE], q[kE];      // the current node's rows
-  float pn[kE], qn[kE];    // the rows of the child under test, on their way
+  float p[kE], q[kE];                // the current node's rows
+  RawRow<NCH, kBf16> pn, qn;         // the rows of the child under test, on their way (as they lie in memory)
   {
     // The tree first - a few words per thread, and everything waits for them - then the root's rows.
     int tp[4], tt[4];
@@ -229,8 +252,8 @@ __global__ void __launch_bounds__(kTh, 1) tree_verify_walk_kernel(const VerifyAr
     }
 #pragma unroll
     for (int k = 0; k < 5; ++k) tu[k] = c.tid + kTh * k <= a.n ? a.uniforms[c.tid + kTh * k] : 0.f;
-    load_row<NCH, kBf16>(c, tbase, p);
-    if (a.n > 1) load_row<NCH, kBf16>(c, dbase, q);  // (a root without children: never read)
+    load_row<NCH, kBf16>(c, tbase, pn);
+    if (a.n > 1) load_row<NCH, kBf16>(c, dbase, qn);  // (a root without children: never read)
     if (c.tid < SEQ_MAX_TREE / 32) sh->has_child[c.tid] = 0u;
     if (c.tid == 0) sh->node_flags = 0;
     __syncthreads();
@@ -253,6 +276,8 @@ __global__ void __launch_bounds__(kTh, 1) tree_verify_walk_kernel(const VerifyAr
       for (int i = c.tid; i < a.n; i += kTh) a.next_child_out[i] = -2;  // nodes the walk does not visit
   }
   cluster.sync();  // the tree is in place; every CTA of the cluster is resident before any remote write
+  widen<NCH, kBf16>(pn, p);
+  widen<NCH, kBf16>(qn, q);  // (a tree of one node: never loaded, never read)
   WTRACE(leader, 2);
 
   int cur = 0, plen = 0, bonus_found = -1;
@@ -464,8 +489,8 @@ __global__ void __launch_bounds__(kTh, 1) tree_verify_walk_kernel(const VerifyAr
     if (leader && a.next_child_out != nullptr) a.next_child_out[cur] = accepted;
     if (accepted >= 0) {
       // ---- on to the accepted child: its rows are in the second set of registers (or about to land there)
-#pragma unroll
-      for (int e = 0; e < kE; ++e) { p[e] = pn[e]; q[e] = qn[e]; }
+      widen<NCH, kBf16>(pn, p);
+      widen<NCH, kBf16>(qn, q);
       cur = accepted;
       cur_has_kids = nxt_has_kids;
       continue;
