@@ -1,5 +1,7 @@
-// seq_tree_verify: Algorithm 2 of the Sequoia paper walked from the root, on one thread-block
-// cluster, plus the final draw x ~ R.
+// seq_tree_verify: entry points, argument checks and the choice of kernel; and the walk of Algorithm 2 from the root
+// with its rows in SHARED memory (greedy decoding, sampling from the target, the every-node hook, batches of requests,
+// and devices that cannot place a cluster of 16 CTAs).  The default walk keeps its rows in registers
+// (tree_verify_walk.cu); the node-parallel schedule is tree_verify_nodes.cu.
 //
 // Schedule.  One cluster of CTAs follows the walk (16 CTAs for a single request where the device can place such a
 // cluster, 8 per request in a batched launch).  At each visited node the two logit rows

@@ -384,7 +384,7 @@ __device__ int process_node(cg::cluster_group& cluster, Ctx& c, const VerifyArgs
     const int ch = c.sh->kids[i];
     const int s = c.sh->tokens[ch];
     if (s < 0 || s >= a.V) { dev_flag(a.dev_status, SEQ_DEV_BAD_TOKEN); continue; }
-    // an earlier (hence rejected) sibling carried the same token: it is in S.  (Without lines 10-16 there is no
+    // an earlier (hence rejected) sibling carried the same token: it is in S.  (Without the draft update there is no
     // S: a repeated token is tested like any other, and its R is 0 by then.)
     const bool in_S = !specinfer && c.sh->dup[i] != 0;
     float pn = 0.f, qn = 0.f;
@@ -393,7 +393,7 @@ __device__ int process_node(cg::cluster_group& cluster, Ctx& c, const VerifyArgs
       pn = pq.x * (rel_exp(pq.z, st.Mp, c2) * st.invSp);
       qn = pq.y * (rel_exp(pq.w, st.Mq, c2) * st.invSq);
     }
-    // line 6: accept iff u < R[s]/D[s], with R[s] = rs/Z and D[s] = qn/ZD (or 1/(V-|S|)); cross-multiplied,
+    // the acceptance test: accept iff u < R[s]/D[s], with R[s] = rs/Z and D[s] = qn/ZD (or 1/(V-|S|)); cross-multiplied,
     // which also covers D[s] = 0 (accept iff R[s] > 0)
     const double rs = in_S ? 0.0 : (double)resid(pn, qn, (float)st.C, (float)st.U);
     const double u = (double)c.sh->uniforms[ch];
@@ -401,11 +401,11 @@ __device__ int process_node(cg::cluster_group& cluster, Ctx& c, const VerifyArgs
     TRACE(8);
     if (accept) return ch;
 
-    // line 9: R <- norm(max(R - D, 0)) with D as it stands
+    // the residual update: R <- norm(max(R - D, 0)) with D as it stands
     double Cn = st.C, Un = st.U;
     if (st.mode == 0) Cn += st.Z / st.ZD;
     else if (a.V - st.nS > 0) Un += st.Z / (double)(a.V - st.nS);
-    // lines 10-11: D[s] <- 0, S.add(s); done by the warp that owns s
+    // the draft update: D[s] <- 0, s joins S; done by the warp that owns s
     if (!in_S && !specinfer) {
       const int sl = s - c.lo;
       if (sl >= c.s_lo && sl < c.s_hi && c.lane == 0) { c.ps[sl] = 0.f; c.qs[sl] = 0.f; }
@@ -448,7 +448,7 @@ __device__ int process_node(cg::cluster_group& cluster, Ctx& c, const VerifyArgs
     }
     if (!specinfer) {
       st.ZD = ZDn;
-      if (st.mode == 0 && !(ZDn > 0.0)) st.mode = 1;  // lines 12-15: uniform over the non-rejected set
+      if (st.mode == 0 && !(ZDn > 0.0)) st.mode = 1;  // no mass left in D: uniform over the non-rejected set
     }
   }
   return -1;
@@ -522,7 +522,7 @@ __device__ int draw_token(Ctx& c, const NodeState& st, float u, float Cf, float 
 }
 
 
-// Line 18, x ~ R with uniforms[n]; optionally writes R.  (Greedy, and verification by sampling from the target:
+// Algorithm 2's final draw, x ~ R with uniforms[n]; optionally writes R.  (Greedy, and verification by sampling from the target:
 // the token was fixed at the last node, R is the distribution it came from.)
 __device__ void draw_bonus(Ctx& c, const VerifyArgs& a, const NodeState& st) {
   if (a.temperature == 0.f) {

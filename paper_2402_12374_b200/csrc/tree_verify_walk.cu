@@ -435,14 +435,20 @@ __global__ void __launch_bounds__(kTh, 1) tree_verify_walk_kernel(const VerifyAr
       }
       WTRACE(leader, 16);
       if (accept) { accepted = ch; break; }
-      // ---- rejected: the next child's rows start their way, then the residual update
-      if (i + 1 < n_kids) {
+      // ---- rejected: the next child's rows must start their way, and the residual is updated.  The loads are issued
+      // behind the exchange's barrier arrival (its release fence would otherwise wait for them to land).
+      const bool more = i + 1 < n_kids;
+      if (more) {
         nxt = sh->kids[np][i + 1];
         nxt_has_kids = (sh->has_child[nxt >> 5] >> (nxt & 31)) & 1u;
-        load_row<NCH, kBf16>(c, tbase + (int64_t)nxt * a.target_stride * kEsz, pn);
-        if (nxt_has_kids) load_row<NCH, kBf16>(c, dbase + (int64_t)nxt * a.draft_stride * kEsz, qn);
       }
-      if (!valid) continue;  // (not a token: R and D untouched)
+      if (!valid) {  // (not a token: R and D untouched)
+        if (more) {
+          load_row<NCH, kBf16>(c, tbase + (int64_t)nxt * a.target_stride * kEsz, pn);
+          if (nxt_has_kids) load_row<NCH, kBf16>(c, dbase + (int64_t)nxt * a.draft_stride * kEsz, qn);
+        }
+        continue;
+      }
       // R <- norm(max(R - D, 0)) with D as it stands
       float Cn = C, Un = U;
       if (mode == 0) Cn += Z * __frcp_rn(ZD);
@@ -468,7 +474,12 @@ __global__ void __launch_bounds__(kTh, 1) tree_verify_walk_kernel(const VerifyAr
       for (int e = 0; e < kE; e += 2) { z0 += resid(p[e], q[e], Cnf, Unf); z1 += resid(p[e + 1], q[e + 1], Cnf, Unf); }
       const float zr = warp_sum(z0 + z1), zd = warp_sum(zd_mine);
       WTRACE(leader, 17);
-      cluster_exchange(cluster, c, make_float4(zr, zd, 0.f, 0.f), x);
+      exchange_push(cluster, c, make_float4(zr, zd, 0.f, 0.f));
+      if (more) {
+        load_row<NCH, kBf16>(c, tbase + (int64_t)nxt * a.target_stride * kEsz, pn);
+        if (nxt_has_kids) load_row<NCH, kBf16>(c, dbase + (int64_t)nxt * a.draft_stride * kEsz, qn);
+      }
+      exchange_pull(c, x);
       WTRACE(leader, 18);
       float zsum = 0.f, zdsum = 0.f;
 #pragma unroll
