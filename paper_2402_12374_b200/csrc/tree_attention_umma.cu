@@ -61,6 +61,9 @@ namespace cg = cooperative_groups;
 
 namespace seqtree {
 
+#ifndef SEQ_TRACE_ROW
+#define SEQ_TRACE_ROW 128  // the row thread whose steps a trace build records
+#endif
 #ifdef SEQ_TRACE
 // Debug builds only: per role (0 TMA, 1 MMA chain A, 2 rows, 3 MMA chain B) a list of (tag, clock) events of
 // CTA (0, 0, 0), one 8-byte store each.  SEQ_TRACE_ROLES (bit per role) limits which roles record.
@@ -70,6 +73,7 @@ namespace seqtree {
 #ifndef SEQ_TRACE_CTA
 #define SEQ_TRACE_CTA 0
 #endif
+
 __device__ unsigned long long g_utrace[4][2048];
 __device__ unsigned long long g_cta_times[1024][2];
 __device__ __forceinline__ unsigned long long gtimer() { unsigned long long t; asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t)); return t; }
@@ -111,6 +115,7 @@ struct UmmaSmem {
   uint64_t q_full;
   uint64_t k_full[2][2], k_empty[2][2], v_full[2][2], v_empty[2][2], s_full[2][2], p_full[2][2];  // [chain][stage]
   uint64_t pv_done[2];                       // [chain]: one phase per block of the chain
+  uint64_t turn[2][4];                       // [chain][lane quarter]: the other chain's warp of the same quarter has finished its exponentials
   uint64_t all_done[2];                      // [chain]: every MMA of the chain in this segment has completed (one phase per segment)
   uint64_t o_free;                           // the row threads have read both accumulators (one phase per segment)
   uint32_t tmem_base;
@@ -265,6 +270,11 @@ __device__ __forceinline__ void tmem_st16(uint32_t taddr, const uint32_t* r) {
         "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15]), "r"(taddr) : "memory");
 }
 
+__device__ __forceinline__ float max3(float a, float b, float c) {
+  float d;
+  asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
+  return d;
+}
 __device__ __forceinline__ float ex2(float x) {
   float y;
   asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
@@ -314,7 +324,7 @@ tree_attention_umma_kernel(const __grid_constant__ CUtensorMap q_map, const __gr
   int utrace_i = 0;
 #endif
   const int split = blockIdx.z;  // the cluster spans blockIdx.z
-  if (threadIdx.x == 128) UTRACE(2, 10);
+  if (threadIdx.x == SEQ_TRACE_ROW) UTRACE(2, 10);
 #ifdef SEQ_TRACE
   const unsigned cta_lin = (blockIdx.z * gridDim.y + blockIdx.y) * gridDim.x + blockIdx.x;
   if (threadIdx.x == 128 && cta_lin < 1024) g_cta_times[cta_lin][0] = gtimer();
@@ -379,6 +389,7 @@ tree_attention_umma_kernel(const __grid_constant__ CUtensorMap q_map, const __gr
         mbar_init(&sm->s_full[c][b], 1); mbar_init(&sm->p_full[c][b], 4);
       }
       mbar_init(&sm->pv_done[c], 1);
+      for (int q = 0; q < 4; ++q) mbar_init(&sm->turn[c][q], 1);
     }
     mbar_init(&sm->all_done[0], 1); mbar_init(&sm->all_done[1], 1);  // each has one arriver: its chain's MMA warp
     mbar_init(&sm->o_free, 8);    // one arrival per warp of row threads
@@ -451,7 +462,7 @@ tree_attention_umma_kernel(const __grid_constant__ CUtensorMap q_map, const __gr
     }
     if (lane == 31) sm->tile_prefix[a.tiles] = incl;
   }
-  if (threadIdx.x == 128) UTRACE(2, 11);
+  if (threadIdx.x == SEQ_TRACE_ROW) UTRACE(2, 11);
   if (warp == 1) {  // all 512 tensor-memory columns: per chain two S buffers of 64 (P over them), then O_A, O_B
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], 512;" ::"r"(smem_u32(&sm->tmem_base)) : "memory");
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
@@ -460,7 +471,7 @@ tree_attention_umma_kernel(const __grid_constant__ CUtensorMap q_map, const __gr
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem = sm->tmem_base;
-  if (threadIdx.x == 128) UTRACE(2, 0);
+  if (threadIdx.x == SEQ_TRACE_ROW) UTRACE(2, 0);
 
   if (warp < 4) {
     // ============================ warp group 0: data movement and MMA issue, few registers =========
@@ -621,6 +632,7 @@ tree_attention_umma_kernel(const __grid_constant__ CUtensorMap q_map, const __gr
   const uint32_t lane_sel = (uint32_t)(quad * 32) << 16;
   const uint32_t tmem_o = tmem + 256u + 128u * chain + lane_sel;
   int seg_n = 0, base_n = 0;  // segments done; blocks this chain has processed in them
+  int turn_waits = 0;         // waits this warp has taken on its turn barrier (its phase runs on across segments)
   for (int64_t pos = range_lo; pos < range_hi;) {
   const Seg sg = seg_at(pos);
   if (kStream && sg.nblk == 0) { pos = sg.next; continue; }
@@ -664,7 +676,7 @@ tree_attention_umma_kernel(const __grid_constant__ CUtensorMap q_map, const __gr
     const int jj = 2 * u + chain, b = (base + u) & 1, w = (base + u) >> 1;
     const uint32_t tmem_s = tmem + 128u * chain + 64u * b + lane_sel;
     if (!mbar_wait(sm, &sm->s_full[chain][b], w & 1, a.dev_status)) { ok = false; break; }
-    if (threadIdx.x == 128) UTRACE(2, 1);
+    if (threadIdx.x == SEQ_TRACE_ROW) UTRACE(2, 1);
     if (!warp_live) {  // 32 padding rows: nothing to compute, only keep in step with the barriers
       __syncwarp();
       if (lane == 0) mbar_arrive(&sm->p_full[chain][b]);
@@ -682,7 +694,7 @@ tree_attention_umma_kernel(const __grid_constant__ CUtensorMap q_map, const __gr
       vis[1] = mask_window(mrow, mask_wpr, a.n, kb - L + 32);
     }
     tc_wait_ld();
-    if (threadIdx.x == 128) UTRACE(2, 2);
+    if (threadIdx.x == SEQ_TRACE_ROW) UTRACE(2, 2);
     if (masked) {  // masked scores become -inf: probability exactly 0, and they cannot raise the maximum
 #pragma unroll
       for (int e = 0; e < 64; ++e)
@@ -695,7 +707,8 @@ tree_attention_umma_kernel(const __grid_constant__ CUtensorMap q_map, const __gr
     {
       float mx[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
 #pragma unroll
-      for (int e = 0; e < 64; ++e) mx[e & 3] = fmaxf(mx[e & 3], __uint_as_float(sreg[e]));
+      for (int e = 0; e < 64; e += 2)  // three-input maximum: two scores per instruction
+        mx[(e >> 1) & 3] = max3(mx[(e >> 1) & 3], __uint_as_float(sreg[e]), __uint_as_float(sreg[e + 1]));
       const float m_blk = fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3])) * sc;  // scale > 0
       const bool move = m_blk > m_used + kRescaleThreshold || (m_used == -INFINITY && m_blk != -INFINITY);
       if (__any_sync(0xffffffffu, move)) {  // rare after the first blocks
@@ -719,6 +732,14 @@ tree_attention_umma_kernel(const __grid_constant__ CUtensorMap q_map, const __gr
         }
       }
     }
+    // The two warps of one lane quarter (one per chain) sit on the same scheduler and share its special-function
+    // unit.  Left alone they run in step: both take exponentials at once, at half rate each, and both then idle the
+    // unit while they read S and hand P over.  So the exponentials are taken in turns, in the order of the blocks:
+    // block jj waits here until block jj-1 (the other chain's) has taken its own, and meanwhile reads and scans.
+    if (jj > 0) {
+      if (!mbar_wait(sm, &sm->turn[chain][quad], turn_waits & 1, a.dev_status)) { ok = false; break; }
+      ++turn_waits;
+    }
     // P = 2^(scale*s - m) written over S as packed 16-bit values (32 columns, two stores of 16).
     // (A row without a reference sees nothing in this block: its scores are all -inf and its P are 0.)
     float sum;
@@ -740,13 +761,16 @@ tree_attention_umma_kernel(const __grid_constant__ CUtensorMap q_map, const __gr
       }
       sum = (sm4[0] + sm4[1]) + (sm4[2] + sm4[3]);
     }
-    if (threadIdx.x == 128) UTRACE(2, 3);
+    if (jj + 1 < nblk && lane == 0) mbar_arrive(&sm->turn[chain ^ 1][quad]);  // the exponentials are issued: the next block's turn
+    if (threadIdx.x == SEQ_TRACE_ROW) UTRACE(2, 3);
     l = l * alpha + sum;
-    if (threadIdx.x == 128) UTRACE(2, 4);
+    if (threadIdx.x == SEQ_TRACE_ROW) UTRACE(2, 4);
     tc_wait_st();
+    if (threadIdx.x == SEQ_TRACE_ROW) UTRACE(2, 12);
     tc_fence_before();
     __syncwarp();
     if (lane == 0) mbar_arrive(&sm->p_full[chain][b]);  // one arrival per warp
+    if (threadIdx.x == SEQ_TRACE_ROW) UTRACE(2, 5);
   }
   // Both chains must be done with the tensor pipe before O is read and the K stages are reused.  (A
   // parity wait on pv_done could be fooled here: the other chain may be several phases behind.)
@@ -757,7 +781,7 @@ tree_attention_umma_kernel(const __grid_constant__ CUtensorMap q_map, const __gr
   // Step 1, inside the CTA: both accumulators live in this CTA's tensor memory and a warp may read
   // any column of its 32 lanes, so the thread of chain c and row r merges columns [64c, 64c+64) of
   // O_A and O_B itself; only (m, l) goes through shared memory.
-  if (threadIdx.x == 128) UTRACE(2, 6);
+  if (threadIdx.x == SEQ_TRACE_ROW) UTRACE(2, 6);
   sm->ml_chain[seg & 1][chain][r] = (ok && n_mine > 0) ? make_float2(m_used, l) : make_float2(-INFINITY, 0.f);
   // Whether to stop after this segment is decided once for all row threads: a flag raised between two threads' own
   // reads would send some to the closing barrier and the rest into the next segment's bar.sync, which has no bound.
@@ -905,7 +929,7 @@ tree_attention_umma_kernel(const __grid_constant__ CUtensorMap q_map, const __gr
     const int cs = a.splits, slots = (16 + cs - 1) / cs;  // (any cs from 2 to 8; the last slots of some CTAs may be empty)
     tc_fence_before();
     cluster.sync();  // every CTA of the cluster is done with its K and V stages before anyone writes into them
-    if (threadIdx.x == 128) UTRACE(2, 7);
+    if (threadIdx.x == SEQ_TRACE_ROW) UTRACE(2, 7);
     // (rows past the tile's last node are padding: nothing of theirs is pushed, reduced or stored)
     if (chain == 0 && row_valid)
       for (int q = 0; q < cs; ++q) *cluster.map_shared_rank(&sm->ml_cta[split][r], q) = make_float2(M, Lc);
@@ -921,7 +945,7 @@ tree_attention_umma_kernel(const __grid_constant__ CUtensorMap q_map, const __gr
                                __float_as_uint(merged[8 * j + 6]), __float_as_uint(merged[8 * j + 7]));
     }
     cluster.sync();
-    if (threadIdx.x == 128) UTRACE(2, 8);
+    if (threadIdx.x == SEQ_TRACE_ROW) UTRACE(2, 8);
     float Mg = -INFINITY;
     for (int q = 0; q < cs; ++q) Mg = fmaxf(Mg, sm->ml_cta[q][r].x);
     float Ls = 0.f;
@@ -954,7 +978,7 @@ tree_attention_umma_kernel(const __grid_constant__ CUtensorMap q_map, const __gr
     }
     if (split == 0 && chain == 0 && row_valid && a.lse != nullptr) a.lse[(size_t)h * a.n + i] = (Mg + log2f(Ls)) * kLn2;
   }
-  if (threadIdx.x == 128) UTRACE(2, 9);
+  if (threadIdx.x == SEQ_TRACE_ROW) UTRACE(2, 9);
   pos = sg.next;
   ++seg_n; base_n += n_mine;
   if (stop_here) break;
