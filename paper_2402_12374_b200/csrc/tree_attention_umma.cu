@@ -103,6 +103,7 @@ constexpr uint32_t kHalfBytes = kTileBytes / 2;  // one 128-row x 64-element sub
 constexpr uint32_t kKvBytes = kBlockN * 128 * 2; // a K or V tile: 64 keys x 128 elements
 constexpr uint32_t kKvHalf = kKvBytes / 2;       // one 64-row x 64-element sub-tile of K or V
 constexpr float kRescaleThreshold = 8.f;         // log2 units
+constexpr float kRescaleLimit = 256.f;           // 2^kRescaleThreshold: no term of a row sum at or below it came from a score above the threshold
 constexpr uint32_t kSpinLimit = 1u << 22;
 
 struct UmmaSmem {
@@ -115,7 +116,6 @@ struct UmmaSmem {
   uint64_t q_full;
   uint64_t k_full[2][2], k_empty[2][2], v_full[2][2], v_empty[2][2], s_full[2][2], p_full[2][2];  // [chain][stage]
   uint64_t pv_done[2];                       // [chain]: one phase per block of the chain
-  uint64_t turn[2][4];                       // [chain][lane quarter]: the other chain's warp of the same quarter has finished its exponentials
   uint64_t all_done[2];                      // [chain]: every MMA of the chain in this segment has completed (one phase per segment)
   uint64_t o_free;                           // the row threads have read both accumulators (one phase per segment)
   uint32_t tmem_base;
@@ -275,6 +275,23 @@ __device__ __forceinline__ float max3(float a, float b, float c) {
   asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
   return d;
 }
+// Two single-precision values in one 64-bit register, for the packed fused multiply-add and add: half the issue slots.
+__device__ __forceinline__ uint64_t pair_of(float lo, float hi) {
+  uint64_t d;
+  asm("mov.b64 %0, {%1, %2};" : "=l"(d) : "f"(lo), "f"(hi));
+  return d;
+}
+__device__ __forceinline__ void unpair(uint64_t v, float& lo, float& hi) { asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v)); }
+__device__ __forceinline__ uint64_t fma2(uint64_t a, uint64_t b, uint64_t c) {
+  uint64_t d;
+  asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
+  return d;
+}
+__device__ __forceinline__ uint64_t add2(uint64_t a, uint64_t b) {
+  uint64_t d;
+  asm("add.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+  return d;
+}
 __device__ __forceinline__ float ex2(float x) {
   float y;
   asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
@@ -389,7 +406,6 @@ tree_attention_umma_kernel(const __grid_constant__ CUtensorMap q_map, const __gr
         mbar_init(&sm->s_full[c][b], 1); mbar_init(&sm->p_full[c][b], 4);
       }
       mbar_init(&sm->pv_done[c], 1);
-      for (int q = 0; q < 4; ++q) mbar_init(&sm->turn[c][q], 1);
     }
     mbar_init(&sm->all_done[0], 1); mbar_init(&sm->all_done[1], 1);  // each has one arriver: its chain's MMA warp
     mbar_init(&sm->o_free, 8);    // one arrival per warp of row threads
@@ -632,7 +648,6 @@ tree_attention_umma_kernel(const __grid_constant__ CUtensorMap q_map, const __gr
   const uint32_t lane_sel = (uint32_t)(quad * 32) << 16;
   const uint32_t tmem_o = tmem + 256u + 128u * chain + lane_sel;
   int seg_n = 0, base_n = 0;  // segments done; blocks this chain has processed in them
-  int turn_waits = 0;         // waits this warp has taken on its turn barrier (its phase runs on across segments)
   for (int64_t pos = range_lo; pos < range_hi;) {
   const Seg sg = seg_at(pos);
   if (kStream && sg.nblk == 0) { pos = sg.next; continue; }
@@ -700,18 +715,49 @@ tree_attention_umma_kernel(const __grid_constant__ CUtensorMap q_map, const __gr
       for (int e = 0; e < 64; ++e)
         if (!(vis[e >> 5] & (1u << (e & 31)))) sreg[e] = __float_as_uint(-INFINITY);
     }
-    // Block maximum first (a pass of comparisons only, on another pipe than the exponentials), so that
-    // the reference maximum is settled before any exponential is taken.  It only moves when the block
-    // maximum exceeds it by more than the threshold, or when the row has no reference yet.
-    float alpha = 1.f;
-    {
+    // P = 2^(scale*s - m) written over S as packed 16-bit values (32 columns, two stores of 16); returns the row sum.
+    // (A row without a reference sees nothing in this block: its scores are all -inf and its P are 0.)
+    auto exponentials = [&]() -> float {
+      const float neg_m = m_used == -INFINITY ? 0.f : -m_used;
+      const uint64_t sc2 = pair_of(sc, sc), neg_m2 = pair_of(neg_m, neg_m);
+      uint64_t sm2[2] = {pair_of(0.f, 0.f), pair_of(0.f, 0.f)};
+#pragma unroll
+      for (int c = 0; c < 2; ++c) {
+        uint32_t packed[16];
+#pragma unroll
+        for (int e = 0; e < 16; ++e) {  // two scores at a time: one packed multiply-add, two exponentials, one packed add
+          float x0, x1;
+          unpair(fma2(pair_of(__uint_as_float(sreg[32 * c + 2 * e]), __uint_as_float(sreg[32 * c + 2 * e + 1])), sc2, neg_m2), x0, x1);
+          const float p0 = ex2(x0), p1 = ex2(x1);
+          sm2[e & 1] = add2(sm2[e & 1], pair_of(p0, p1));
+          packed[e] = pack2<kBf16>(p0, p1);
+        }
+        tmem_st16(tmem_s + 16u * c, packed);
+      }
+      float s0, s1, s2, s3;
+      unpair(sm2[0], s0, s1);
+      unpair(sm2[1], s2, s3);
+      return (s0 + s1) + (s2 + s3);
+    };
+    // The reference maximum only moves when the block maximum exceeds it by more than the threshold, or when the row
+    // has no reference yet: rare after the first blocks.  So the exponentials are taken against the reference as it
+    // stands, and their sum tells whether that was right: a score more than the threshold above the reference gives a
+    // term, hence a sum, above 2^threshold.  Only then (or without a reference) is the block maximum taken, the
+    // reference moved, O rescaled, and the pass repeated (the scores are still in registers).
+    float alpha = 1.f, sum = 0.f;
+    bool settle = __any_sync(0xffffffffu, m_used == -INFINITY);
+    if (!settle) {
+      sum = exponentials();
+      settle = __any_sync(0xffffffffu, !(sum <= kRescaleLimit));
+    }
+    if (settle) {
       float mx[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
 #pragma unroll
       for (int e = 0; e < 64; e += 2)  // three-input maximum: two scores per instruction
         mx[(e >> 1) & 3] = max3(mx[(e >> 1) & 3], __uint_as_float(sreg[e]), __uint_as_float(sreg[e + 1]));
       const float m_blk = fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3])) * sc;  // scale > 0
       const bool move = m_blk > m_used + kRescaleThreshold || (m_used == -INFINITY && m_blk != -INFINITY);
-      if (__any_sync(0xffffffffu, move)) {  // rare after the first blocks
+      if (__any_sync(0xffffffffu, move)) {
         if (move) {
           alpha = m_used == -INFINITY ? 0.f : ex2(m_used - m_blk);
           m_used = m_blk;
@@ -731,37 +777,8 @@ tree_attention_umma_kernel(const __grid_constant__ CUtensorMap q_map, const __gr
           }
         }
       }
+      sum = exponentials();
     }
-    // The two warps of one lane quarter (one per chain) sit on the same scheduler and share its special-function
-    // unit.  Left alone they run in step: both take exponentials at once, at half rate each, and both then idle the
-    // unit while they read S and hand P over.  So the exponentials are taken in turns, in the order of the blocks:
-    // block jj waits here until block jj-1 (the other chain's) has taken its own, and meanwhile reads and scans.
-    if (jj > 0) {
-      if (!mbar_wait(sm, &sm->turn[chain][quad], turn_waits & 1, a.dev_status)) { ok = false; break; }
-      ++turn_waits;
-    }
-    // P = 2^(scale*s - m) written over S as packed 16-bit values (32 columns, two stores of 16).
-    // (A row without a reference sees nothing in this block: its scores are all -inf and its P are 0.)
-    float sum;
-    {
-      const float neg_m = m_used == -INFINITY ? 0.f : -m_used;
-      float sm4[4] = {0.f, 0.f, 0.f, 0.f};
-#pragma unroll
-      for (int c = 0; c < 2; ++c) {
-        uint32_t packed[16];
-#pragma unroll
-        for (int e = 0; e < 16; ++e) {
-          const float p0 = ex2(fmaf(__uint_as_float(sreg[32 * c + 2 * e]), sc, neg_m));
-          const float p1 = ex2(fmaf(__uint_as_float(sreg[32 * c + 2 * e + 1]), sc, neg_m));
-          sm4[e & 1] += p0;
-          sm4[2 + (e & 1)] += p1;
-          packed[e] = pack2<kBf16>(p0, p1);
-        }
-        tmem_st16(tmem_s + 16u * c, packed);
-      }
-      sum = (sm4[0] + sm4[1]) + (sm4[2] + sm4[3]);
-    }
-    if (jj + 1 < nblk && lane == 0) mbar_arrive(&sm->turn[chain ^ 1][quad]);  // the exponentials are issued: the next block's turn
     if (threadIdx.x == SEQ_TRACE_ROW) UTRACE(2, 3);
     l = l * alpha + sum;
     if (threadIdx.x == SEQ_TRACE_ROW) UTRACE(2, 4);
