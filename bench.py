@@ -89,8 +89,10 @@ def measured_peaks():
     path = os.path.join(ROOT, "MEASURED_PEAKS.json")
     if os.path.exists(path):
         d = json.load(open(path))
-        return dict(hbm_gbs=d["hbm_gbs"], bf16_tflops=d["bf16_tflops"], source="measured")  # burst figure: kernels are timed alone
-    return dict(hbm_gbs=6650.0, bf16_tflops=1590.0, source="fallback")
+        # the burst figure for a kernel timed alone in bursts of a few ms, the sustained one for a long loop of it
+        return dict(hbm_gbs=d["hbm_gbs"], bf16_tflops=d["bf16_tflops"],
+                    bf16_tflops_sustained=d.get("bf16_tflops_sustained", d["bf16_tflops"]), source="measured")
+    return dict(hbm_gbs=6650.0, bf16_tflops=1590.0, bf16_tflops_sustained=1400.0, source="fallback")
 
 
 class ClockSampler:
@@ -797,7 +799,11 @@ def run_workload(cfg, T, args, rank, local_rank, world, dev, stream, peaks, with
         ver_calls[i % nv].run(s)
 
     flush = torch.empty(160 << 20, dtype=torch.uint8, device=dev)
-    Kb = max(K, 4 * na)   # launches per graph of the per-kernel timings: every attention set a few times
+    # Launches per graph of the per-kernel timings: every attention set four times, whatever K is.  On the 768-node
+    # workload that is a burst of about 5 ms per replay, as the burst peak it is set against was measured (single GEMMs,
+    # best of ten); a hundred such launches in a row run into the 1 kW power cap, and that figure is reported beside
+    # it, against the sustained peak.
+    Kb = 4 * na
 
     def graph_of(body, count):
         g = torch.cuda.CUDAGraph()
@@ -828,6 +834,16 @@ def run_workload(cfg, T, args, rank, local_rank, world, dev, stream, peaks, with
                 g_step.replay()
                 stream.synchronize()
         ms_attn = timed_replays(g_attn, stream, 9, world, dev)
+        # the same graph 30 times without a pause (a tensor-bound workload: > 100 ms of dense work under the power cap)
+        sustained_reps = 30
+        ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        stream.synchronize()
+        ev0.record(stream)
+        for _ in range(sustained_reps):
+            g_attn.replay()
+        ev1.record(stream)
+        stream.synchronize()
+        attn_sustained_us = ev0.elapsed_time(ev1) * 1e3 / (sustained_reps * Kb)
         ms_ver_warm = timed_replays(g_ver_warm, stream, 9, world, dev)
         ms_cold = timed_replays(g_ver_cold, stream, 9, world, dev)
         ms_flush = timed_replays(g_flush, stream, 9, world, dev)
@@ -850,6 +866,10 @@ def run_workload(cfg, T, args, rank, local_rank, world, dev, stream, peaks, with
         roofline = {"bound": "tensor", "achieved": achieved, "peak": peaks["bf16_tflops"], "unit": "TFLOP/s",
                     "frac": achieved / peaks["bf16_tflops"], "frac_of_spec": achieved / SPEC_BF16_TFLOPS,
                     "spec_peak": SPEC_BF16_TFLOPS}
+        ach_s = flops / (attn_sustained_us * 1e-6) / 1e12
+        roofline["sustained"] = {"us_per_launch": attn_sustained_us, "achieved": ach_s, "peak": peaks["bf16_tflops_sustained"],
+                                 "frac": ach_s / peaks["bf16_tflops_sustained"], "launches": sustained_reps * Kb,
+                                 "note": "the same launches in one unbroken run, against the sustained peak"}
     roofline.update({
         "traffic": ncu_traffic_bytes(cfg.name), "kernel": "seq_tree_attention", "us_per_launch": attn_us,
         "algorithmic_bytes": attn_bytes, "algorithmic_flops": flops, "peak_source": f"of {peaks['source']}",

@@ -493,6 +493,7 @@ tree_attention_umma_kernel(const __grid_constant__ CUtensorMap q_map, const __gr
     // ============================ warp group 0: data movement and MMA issue, few registers =========
     asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(kRegsLight));
     int seg_n = 0, base_an = 0, base_bn = 0;  // segments done; blocks chains A, B have processed in them
+    uint32_t issued = 0, issued_parity = 0;   // producers: stages (bit 2*chain + stage; bit 4: Q) this warp has requested a tile for, and the phase of the last request
     for (int64_t pos = range_lo; pos < range_hi;) {
     const Seg sg = seg_at(pos);
     if (kStream && sg.nblk == 0) { pos = sg.next; continue; }
@@ -515,6 +516,7 @@ tree_attention_umma_kernel(const __grid_constant__ CUtensorMap q_map, const __gr
           tma_load_5d(sm->q, &q_map, &sm->q_full, 0, 0, i0, 0, g);  // both 64-element halves by one copy
         }
         __syncwarp();
+        if (kStream && !is_v) { issued |= 16u; issued_parity = (issued_parity & ~16u) | ((uint32_t)(seg & 1) << 4); }
         const CUtensorMap* map = is_v ? &v_map : &k_map;
         for (int jj = (!kStream && !is_v) ? min(2, nblk) : 0; jj < nblk; ++jj) {
           const int c = jj & 1, u = (c ? base_b : base_a) + (jj >> 1);  // chain, the chain's running block count
@@ -529,6 +531,8 @@ tree_attention_umma_kernel(const __grid_constant__ CUtensorMap q_map, const __gr
             tma_load_4d(dst, map, full, 0, row, 0, g);  // both 64-element halves by one copy
           }
           __syncwarp();
+          issued |= 1u << (2 * c + b);
+          issued_parity = (issued_parity & ~(1u << (2 * c + b))) | ((uint32_t)(w & 1) << (2 * c + b));
           if (lane == 0 && !is_v) UTRACE(0, 1);
         }
       }
@@ -631,6 +635,18 @@ tree_attention_umma_kernel(const __grid_constant__ CUtensorMap q_map, const __gr
     ++seg_n; base_an += (nblk + 1) >> 1; base_bn += nblk >> 1;
     if (kStream && sm->abort_flag) break;
     }  // segments
+    // A CTA that gives up must not leave while a tile it has requested is still on its way into its shared memory
+    // (the next CTA on this SM could get that memory): the producers wait, with a bound of their own, for the last
+    // tile requested into each stage.  (Whether its consumer has taken that phase or not, the parity test answers
+    // when the bytes have landed.  Tiles requested earlier into the same stage landed before the stage was reused.)
+    if (sm->abort_flag && (warp == 0 || warp == 3)) {
+      for (int st = 0; st < 5; ++st) {
+        if (!((issued >> st) & 1u)) continue;
+        uint64_t* full = st == 4 ? &sm->q_full : (warp == 3 ? &sm->v_full[st >> 1][st & 1] : &sm->k_full[st >> 1][st & 1]);
+        for (uint32_t it = 0; it < (1u << 16); ++it)
+          if (mbar_try_wait(full, (issued_parity >> st) & 1u)) break;
+      }
+    }
     tc_fence_before();
     __syncthreads();
     if (warp == 1) {
