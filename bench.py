@@ -1026,17 +1026,31 @@ def main():
                       v0.tokens, v0.target_logits, v0.draft_logits, T, v0.uniforms, device=dev,
                       fused_mask=head_state["fused_mask"], kernel=args.kernel)
     Ke = max(3, min(args.steps, 10))
-    with torch.cuda.stream(stream):
-        for _ in range(3):
-            host.run(stream)
-            stream.synchronize()
-        torch.cuda.synchronize()
-        t0 = time.perf_counter()
-        for _ in range(Ke):
-            host.run(stream)
-            stream.synchronize()
-        e2e_us = 1e6 * (time.perf_counter() - t0) / Ke
-    e2e_us = max_over_ranks(e2e_us, dev) / world
+
+    def time_host_step(hs):
+        with torch.cuda.stream(stream):
+            for _ in range(3):
+                hs.run(stream)
+                stream.synchronize()
+            torch.cuda.synchronize()
+            t0 = time.perf_counter()
+            for _ in range(Ke):
+                hs.run(stream)
+                stream.synchronize()
+            return 1e6 * (time.perf_counter() - t0) / Ke
+
+    e2e_us = max_over_ranks(time_host_step(host), dev) / world
+    # the same step with the verification's inputs on a second stream, and with the prefix of the cache resident
+    e2e_variants = {}
+    if not args.no_legs:
+        for label, kw in (("two_streams", dict(two_streams=True)), ("resident_cache", dict(resident_cache=True)),
+                          ("resident_cache_two_streams", dict(resident_cache=True, two_streams=True))):
+            hs = B.HostStep(a0.q, a0.k_cache, a0.v_cache, torch.from_numpy(head_state["parent"]), cfg.prefix_len,
+                            v0.tokens, v0.target_logits, v0.draft_logits, T, v0.uniforms, device=dev,
+                            fused_mask=head_state["fused_mask"], kernel=args.kernel, **kw)
+            e2e_variants[label] = {"value": max_over_ranks(time_host_step(hs), dev) / world, "unit": UNIT,
+                                   "h2d_bytes_per_step": hs.h2d_bytes, "d2h_bytes_per_step": hs.d2h_bytes}
+            del hs
 
     if rank != 0:
         if world > 1:
@@ -1053,7 +1067,7 @@ def main():
         "us_per_step_spread": head["us_per_step"],
         "clocks": head["clocks"],
         "e2e": {"value": e2e_us, "unit": UNIT, "h2d_bytes_per_step": host.h2d_bytes, "d2h_bytes_per_step": host.d2h_bytes,
-                "steps": Ke},
+                "steps": Ke, "variants": e2e_variants},
         "gpu_launches": sum(p["gpu_launches"] for p in per.values()),
         "roofline": head["roofline"],
         "roofline_verify": head["roofline_verify"],

@@ -508,10 +508,17 @@ class HostStep:
     """One whole verify step fed from pinned HOST buffers: per call it copies the step's inputs to
     the device, builds the ancestor mask (inside the attention kernel with ``fused_mask``, else by a
     launch of its own), runs attention and verification, and copies the results (attention output,
-    path, bonus token) back.  Device staging buffers are allocated once here."""
+    path, bonus token) back.  Device staging buffers are allocated once here.
+
+    ``resident_cache``: the prefix rows of the key/value cache are copied once, here, and a step copies only what a
+    step changes: the tree's rows ``[prefix_len, prefix_len + n)`` of every head, the queries, the tree, the logits
+    and the uniforms.  ``two_streams``: the logits, tokens and uniforms travel on a second stream while the first
+    copies q/k/v and runs the attention; the verification waits for them, and the attention output returns on the
+    second stream while the verification runs."""
 
     def __init__(self, q, k_cache, v_cache, parent, prefix_len, tokens, target_logits, draft_logits, temperature,
-                 uniforms, device="cuda", fused_mask: bool = False, kernel: int = KERNEL_AUTO):
+                 uniforms, device="cuda", fused_mask: bool = False, kernel: int = KERNEL_AUTO,
+                 resident_cache: bool = False, two_streams: bool = False):
         self.host_in = [t if t.is_pinned() else t.pin_memory()
                         for t in (q, k_cache, v_cache, parent, tokens, target_logits, draft_logits, uniforms)]
         self.dev_in = [torch.empty_like(t, device=device) for t in self.host_in]
@@ -528,19 +535,59 @@ class HostStep:
                          torch.empty(n, dtype=torch.int32).pin_memory(),
                          torch.empty(1, dtype=torch.int32).pin_memory(),
                          torch.empty(1, dtype=torch.int32).pin_memory()]
-        self.h2d_bytes = sum(t.numel() * t.element_size() for t in self.host_in)
+        # (host, device) pairs per group: what the attention needs, what only the verification needs
+        hq, hk, hv, hparent, htok, htl, hdl, hu = self.host_in
+        if resident_cache:
+            dk.copy_(hk)
+            dv.copy_(hv)
+            rows = slice(prefix_len, prefix_len + n)
+            kv_pairs = [(hk[:, rows], dk[:, rows]), (hv[:, rows], dv[:, rows])]
+        else:
+            kv_pairs = [(hk, dk), (hv, dv)]
+        self.copies_attention = [(hq, dq)] + kv_pairs + [(hparent, dparent)]
+        self.copies_verify = [(htok, dtok), (htl, dtl), (hdl, ddl), (hu, du)]
+        self.h2d_bytes = sum(h.numel() * h.element_size() for h, _ in self.copies_attention + self.copies_verify)
         self.d2h_bytes = sum(t.numel() * t.element_size() for t in self.host_out)
+        self.side = torch.cuda.Stream(device=device) if two_streams else None
+        self.ev_inputs = torch.cuda.Event() if two_streams else None
+        self.ev_attention = torch.cuda.Event() if two_streams else None
+        self.ev_side_done = torch.cuda.Event() if two_streams else None
+        self.ev_start = torch.cuda.Event() if two_streams else None
 
     def run(self, stream=None):
-        for h, d in zip(self.host_in, self.dev_in):
-            d.copy_(h, non_blocking=True)
-        if not self.fused_mask:
-            seq_tree_mask_from_parents(self.dev_in[3], mask_bits=self.mask, depth=self.depth, dev_status=self.status,
-                                       stream=stream)
-        self.attn.run(stream)
-        self.verify.run(stream)
-        for h, d in zip(self.host_out, (self.attn.out, self.verify.path, self.verify.path_len, self.verify.bonus_token)):
-            h.copy_(d, non_blocking=True)
+        main = stream if stream is not None else torch.cuda.current_stream()
+        with torch.cuda.stream(main):
+            if self.side is not None:
+                self.ev_start.record(main)
+                with torch.cuda.stream(self.side):
+                    self.side.wait_event(self.ev_start)  # not before the previous step has finished with the buffers
+                    for h, d in self.copies_verify:
+                        d.copy_(h, non_blocking=True)
+                    self.ev_inputs.record(self.side)
+            for h, d in self.copies_attention:
+                d.copy_(h, non_blocking=True)
+            if self.side is None:
+                for h, d in self.copies_verify:
+                    d.copy_(h, non_blocking=True)
+            if not self.fused_mask:
+                seq_tree_mask_from_parents(self.dev_in[3], mask_bits=self.mask, depth=self.depth, dev_status=self.status,
+                                           stream=main)
+            self.attn.run(main)
+            if self.side is not None:
+                self.ev_attention.record(main)
+                main.wait_event(self.ev_inputs)
+            self.verify.run(main)
+            if self.side is not None:
+                with torch.cuda.stream(self.side):
+                    self.side.wait_event(self.ev_attention)
+                    self.host_out[0].copy_(self.attn.out, non_blocking=True)
+                    self.ev_side_done.record(self.side)
+            else:
+                self.host_out[0].copy_(self.attn.out, non_blocking=True)
+            for h, d in zip(self.host_out[1:], (self.verify.path, self.verify.path_len, self.verify.bonus_token)):
+                h.copy_(d, non_blocking=True)
+            if self.side is not None:
+                main.wait_event(self.ev_side_done)  # a caller that waits for `stream` has everything
         return self.host_out
 
 
