@@ -11,10 +11,12 @@
  *   - All data pointers are DEVICE pointers owned by the caller, valid on the
  *     device that is current when the call is made.  The library allocates
  *     no device memory and never synchronises the host.  Between calls it keeps
- *     only per-device facts that it looks up once (a driver entry point, whether
- *     a 16-CTA cluster can be placed, function attributes already set, the
- *     address of the built-in scratch array); those lookups are guarded, so
- *     calls may come from several host threads.
+ *     only per-device facts that it looks up once (a driver entry point, the
+ *     SM count, whether a 16-CTA cluster can be placed, function attributes
+ *     already set, the address of the built-in scratch array) and the last 16
+ *     tensor maps it has encoded, keyed by the arguments of the encode (pointer,
+ *     extents, strides), so that a repeated launch makes no driver call; those
+ *     lookups are guarded, so calls may come from several host threads.
  *   - `stream` is a cudaStream_t passed as void* (NULL = the legacy default
  *     stream).  Work is enqueued on it and the call returns at once.
  *   - Problems the host can see (null pointers, sizes out of range, bad

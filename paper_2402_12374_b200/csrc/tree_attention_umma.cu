@@ -54,39 +54,14 @@
 #include <cstddef>
 #include <cuda.h>
 #include <stdlib.h>
+#include <string.h>
 
 #include "common.cuh"
+#include "trace_attention.cuh"
 
 namespace cg = cooperative_groups;
 
 namespace seqtree {
-
-#ifndef SEQ_TRACE_ROW
-#define SEQ_TRACE_ROW 128  // the row thread whose steps a trace build records
-#endif
-#ifdef SEQ_TRACE
-// Debug builds only: per role (0 TMA, 1 MMA chain A, 2 rows, 3 MMA chain B) a list of (tag, clock) events of
-// CTA (0, 0, 0), one 8-byte store each.  SEQ_TRACE_ROLES (bit per role) limits which roles record.
-#ifndef SEQ_TRACE_ROLES
-#define SEQ_TRACE_ROLES 15
-#endif
-#ifndef SEQ_TRACE_CTA
-#define SEQ_TRACE_CTA 0
-#endif
-
-__device__ unsigned long long g_utrace[4][2048];
-__device__ unsigned long long g_cta_times[1024][2];
-__device__ __forceinline__ unsigned long long gtimer() { unsigned long long t; asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t)); return t; }
-#define UTRACE(role, tag)                                                       \
-  do {                                                                          \
-    if (((SEQ_TRACE_ROLES) >> (role)) & 1) {                                    \
-      if (blockIdx.x == (SEQ_TRACE_CTA) && blockIdx.y == 0 && blockIdx.z == 0 && utrace_i < 2047) \
-        g_utrace[role][++utrace_i] = ((unsigned long long)(tag) << 56) | ((unsigned long long)clock64() & 0xFFFFFFFFFFFFFFull); \
-    }                                                                           \
-  } while (0)
-#else
-#define UTRACE(role, tag) do { } while (0)
-#endif
 
 constexpr int kTileM = 128;         // query rows per CTA
 constexpr int kBlockN = 64;         // keys per block
@@ -1042,6 +1017,49 @@ static EncodeTiledFn encode_fn() {
   return reinterpret_cast<EncodeTiledFn>(p);
 }
 
+// Encoded tensor maps are kept: a caller that launches directly (no CUDA graph) passes the same pointers and shapes
+// step after step, and an encode is a driver call of a microsecond or two.  A map depends on nothing but the
+// arguments of the encode (the swizzle, interleave, promotion and fill are the same for every map of this file), so
+// the key is those arguments, compared byte for byte; 16 entries, replaced in turn; one lock around the table.
+namespace {
+struct MapKey {
+  const void* base;
+  cuuint64_t dims[5], strides[4];
+  cuuint32_t box[5];
+  int32_t rank, dtype;
+};
+struct MapEntry { MapKey key; CUtensorMap map; bool used; };
+MapEntry g_maps[16];
+unsigned g_maps_next = 0;
+int g_maps_lock = 0;
+
+CUresult encode_cached(EncodeTiledFn encode, CUtensorMap* out, CUtensorMapDataType dt, cuuint32_t rank, const void* base,
+                       const cuuint64_t* dims, const cuuint64_t* strides, const cuuint32_t* box) {
+  MapKey key;
+  memset(&key, 0, sizeof(key));
+  key.base = base; key.rank = (int32_t)rank; key.dtype = (int32_t)dt;
+  for (cuuint32_t i = 0; i < rank; ++i) { key.dims[i] = dims[i]; key.box[i] = box[i]; }
+  for (cuuint32_t i = 0; i + 1 < rank; ++i) key.strides[i] = strides[i];
+  while (__atomic_exchange_n(&g_maps_lock, 1, __ATOMIC_ACQUIRE) != 0) { }
+  for (MapEntry& e : g_maps)
+    if (e.used && memcmp(&e.key, &key, sizeof(key)) == 0) {
+      *out = e.map;
+      __atomic_store_n(&g_maps_lock, 0, __ATOMIC_RELEASE);
+      return CUDA_SUCCESS;
+    }
+  __atomic_store_n(&g_maps_lock, 0, __ATOMIC_RELEASE);
+  const cuuint32_t estr[5] = {1, 1, 1, 1, 1};
+  const CUresult r = encode(out, dt, rank, const_cast<void*>(base), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                            CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  if (r != CUDA_SUCCESS) return r;
+  while (__atomic_exchange_n(&g_maps_lock, 1, __ATOMIC_ACQUIRE) != 0) { }
+  MapEntry& e = g_maps[g_maps_next++ % 16];
+  e.key = key; e.map = *out; e.used = true;
+  __atomic_store_n(&g_maps_lock, 0, __ATOMIC_RELEASE);
+  return CUDA_SUCCESS;
+}
+}  // namespace
+
 bool umma_supported(const seq_tree_attention_params& p) {
   if (p.dtype != SEQ_F16 && p.dtype != SEQ_BF16) return false;
   const int G = p.num_q_heads / p.num_kv_heads;
@@ -1128,11 +1146,7 @@ int launch_attention_umma(const seq_tree_attention_params& p, int splits, cudaSt
     cuuint64_t strides[4] = {(cuuint64_t)p.q_stride_head * 2, (cuuint64_t)p.q_stride_tok * 2, 128,
                              (cuuint64_t)p.q_stride_head * 2 * G};
     cuuint32_t box[5] = {64, (cuuint32_t)G, (cuuint32_t)nodes_per_tile, 2, 1};
-    cuuint32_t estr[5] = {1, 1, 1, 1, 1};
-    if (encode(&q_map, dt, 5, const_cast<void*>(p.q), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
-               CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
-      return SEQ_ERR_CUDA;
+    if (encode_cached(encode, &q_map, dt, 5, p.q, dims, strides, box) != CUDA_SUCCESS) return SEQ_ERR_CUDA;
   }
   for (int which = 0; which < 2; ++which) {
     // only the live rows [0, prefix_len + n_tree) are mapped: anything past them reads as zero.  (With the prefix
@@ -1140,10 +1154,7 @@ int launch_attention_umma(const seq_tree_attention_params& p, int splits, cudaSt
     cuuint64_t dims[4] = {64, (cuuint64_t)(p.prefix_len_dev != nullptr ? p.kv_capacity : p.prefix_len + p.n_tree), 2, (cuuint64_t)p.num_kv_heads};
     cuuint64_t strides[3] = {(cuuint64_t)p.kv_stride_tok * 2, 128, (cuuint64_t)p.kv_stride_head * 2};
     cuuint32_t box[4] = {64, (cuuint32_t)kBlockN, 2, 1};
-    cuuint32_t estr[4] = {1, 1, 1, 1};
-    if (encode(which == 0 ? &k_map : &v_map, dt, 4, const_cast<void*>(which == 0 ? p.k_cache : p.v_cache), dims,
-               strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
-               CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+    if (encode_cached(encode, which == 0 ? &k_map : &v_map, dt, 4, which == 0 ? p.k_cache : p.v_cache, dims, strides, box) != CUDA_SUCCESS)
       return SEQ_ERR_CUDA;
   }
 
@@ -1217,18 +1228,3 @@ int launch_attention_umma(const seq_tree_attention_params& p, int splits, cudaSt
 }
 
 }  // namespace seqtree
-
-#ifdef SEQ_TRACE
-extern "C" int seq_debug_cta_times(unsigned long long* host_out) {
-  cudaDeviceSynchronize();
-  cudaMemcpyFromSymbol(host_out, seqtree::g_cta_times, sizeof(unsigned long long) * 2048);
-  return 0;
-}
-extern "C" int seq_debug_utrace_dump(unsigned long long* host_out) {
-  cudaDeviceSynchronize();
-  cudaMemcpyFromSymbol(host_out, seqtree::g_utrace, sizeof(unsigned long long) * 4 * 2048);
-  static unsigned long long zeros[4 * 2048];
-  cudaMemcpyToSymbol(seqtree::g_utrace, zeros, sizeof(zeros));
-  return 0;
-}
-#endif
