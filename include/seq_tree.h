@@ -165,6 +165,12 @@ typedef struct {
    * tensor-core path the rows from *prefix_len_dev + n_tree up to kv_capacity are then fetched (not used): they may
    * hold anything, but must be readable.  A value outside [0, prefix_len] raises SEQ_DEV_BAD_LENGTH and is clamped. */
   const int32_t* prefix_len_dev;
+  /* 0 or 1: *prefix_len_dev is the length of every head's prefix.  R > 1: a batch of R requests stacked as heads
+   * (request r owns kv heads [r * num_kv_heads / R, (r + 1) * num_kv_heads / R) and their query heads; the tree is
+   * common, Section 4.1: it is fixed in advance) with one prefix length each, prefix_len_dev[r]; request r's tree
+   * rows sit at [prefix_len_dev[r], prefix_len_dev[r] + n_tree) of ITS heads' caches.  R must divide num_kv_heads
+   * and prefix_len_dev must be given; the tensor-core kernel then runs its grid schedule (kernel = 3 is refused). */
+  int32_t prefix_len_dev_count;
 } seq_tree_attention_params;
 
 size_t seq_tree_attention_workspace_bytes(const seq_tree_attention_params* p);

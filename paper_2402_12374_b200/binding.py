@@ -71,7 +71,7 @@ class AttentionParams(C.Structure):
         ("out", C.c_void_p), ("o_stride_tok", C.c_int64), ("o_stride_head", C.c_int64),
         ("lse", C.c_void_p), ("workspace", C.c_void_p), ("workspace_bytes", C.c_size_t),
         ("dev_status", C.c_void_p), ("kernel", C.c_int32),
-        ("parent", C.c_void_p), ("prefix_len_dev", C.c_void_p),
+        ("parent", C.c_void_p), ("prefix_len_dev", C.c_void_p), ("prefix_len_dev_count", C.c_int32),
     ]
 
 
@@ -260,6 +260,8 @@ class AttentionCall:
             p.mask_bits, p.mask_words_per_row = None, 0
         p.parent = _dev(parent, "parent", torch.int32)
         p.prefix_len_dev = _dev(prefix_len_dev, "prefix_len_dev", torch.int32)  # prefix_len is then its upper bound
+        # more than one element: one length per request of a batch stacked as heads
+        p.prefix_len_dev_count = 0 if prefix_len_dev is None else prefix_len_dev.numel()
         p.out, p.o_stride_tok, p.o_stride_head = _dev(out, "out", q.dtype), out.stride(0), out.stride(1)
         p.lse = _dev(lse, "lse", torch.float32)
         p.dev_status = _dev(dev_status, "dev_status", torch.int32)

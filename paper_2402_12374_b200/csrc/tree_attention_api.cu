@@ -53,6 +53,10 @@ int validate_attention_params(const seq_tree_attention_params* p) {
   for (const void* q : ptrs)
     if (reinterpret_cast<uintptr_t>(q) % 16 != 0) return SEQ_ERR_INVALID_ARG;
   if (p->kernel < 0 || p->kernel > 4) return SEQ_ERR_INVALID_ARG;
+  if (p->prefix_len_dev_count < 0) return SEQ_ERR_INVALID_ARG;
+  if (p->prefix_len_dev_count > 1 &&
+      (p->prefix_len_dev == nullptr || p->num_kv_heads % p->prefix_len_dev_count != 0 || p->kernel == 3))
+    return SEQ_ERR_INVALID_ARG;
   return SEQ_OK;
 }
 

@@ -102,6 +102,7 @@ struct SimtArgs {
   float* o_part; float2* ml;
   int64_t q_stride_tok, q_stride_head, kv_stride_tok, kv_stride_head, o_stride_tok, o_stride_head;
   int32_t n, L_host, Hq, group, mask_wpr, splits;
+  int32_t L_count;       // > 1: one prefix length per request, requests stacked as heads
   const int32_t* L_dev;  // nullable: the prefix length in device memory (<= L_host)
   int32_t* dev_status;
   float scale_log2;  // softmax_scale * log2(e)
@@ -114,7 +115,7 @@ tree_attention_simt_kernel(const SimtArgs a) {
   const int g = h / a.group;
   int L = a.L_host;
   if (a.L_dev != nullptr) {
-    const int v = *a.L_dev;
+    const int v = a.L_dev[a.L_count > 1 ? (g * a.L_count) / (a.Hq / a.group) : 0];
     if ((v < 0 || v > a.L_host) && threadIdx.x == 0) dev_flag(a.dev_status, SEQ_DEV_BAD_LENGTH);
     L = min(max(v, 0), a.L_host);
   }
@@ -274,7 +275,7 @@ static int launch_simt_t(const seq_tree_attention_params& p, int splits, cudaStr
   a.q_stride_tok = p.q_stride_tok; a.q_stride_head = p.q_stride_head;
   a.kv_stride_tok = p.kv_stride_tok; a.kv_stride_head = p.kv_stride_head;
   a.o_stride_tok = p.o_stride_tok; a.o_stride_head = p.o_stride_head;
-  a.n = p.n_tree; a.L_host = p.prefix_len; a.L_dev = p.prefix_len_dev; a.dev_status = p.dev_status; a.Hq = p.num_q_heads; a.group = p.num_q_heads / p.num_kv_heads;
+  a.n = p.n_tree; a.L_host = p.prefix_len; a.L_dev = p.prefix_len_dev; a.L_count = p.prefix_len_dev_count; a.dev_status = p.dev_status; a.Hq = p.num_q_heads; a.group = p.num_q_heads / p.num_kv_heads;
   a.mask_wpr = p.mask_words_per_row; a.splits = splits;
   const float scale = p.softmax_scale > 0.f ? p.softmax_scale : 0.08838834764831845f;
   a.scale_log2 = scale * kLog2e;

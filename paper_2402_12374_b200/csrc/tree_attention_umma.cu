@@ -108,6 +108,7 @@ static_assert(offsetof(UmmaSmem, v) == offsetof(UmmaSmem, k) + sizeof(UmmaSmem::
 struct UmmaArgs {
   int32_t n, L_host, Hq, Hkv, group, mask_wpr, splits, nodes_per_tile, tiles;
   const int32_t* L_dev;   // nullable: the prefix length in device memory (<= L_host)
+  int32_t L_count;        // > 1: one length per request, requests stacked as heads (grid schedule only: a CTA has one kv head)
   int32_t zero_tail;      // the K/V maps cover the whole cache: rows past the tree are cleared in shared memory
   // Stream mode (more (tile, kv head) units than SMs): the 64-key blocks of all units, laid end to end, are
   // cut into gridDim.x equal ranges, one per CTA; a tile cut by a range boundary is completed by whichever
@@ -397,7 +398,7 @@ tree_attention_umma_kernel(const __grid_constant__ CUtensorMap q_map, const __gr
   // line reads or writes global memory.
   asm volatile("griddepcontrol.wait;" ::: "memory");
   if (a.L_dev != nullptr) {
-    const int v = *a.L_dev;
+    const int v = a.L_dev[(!kStream && a.L_count > 1) ? ((int)blockIdx.y * a.L_count) / a.Hkv : 0];
     if (v < 0 || v > a.L_host) { if (threadIdx.x == 0) dev_flag(a.dev_status, SEQ_DEV_BAD_LENGTH); }
     L = min(max(v, 0), a.L_host);
     if (kStream) {  // the flattened block space of this prefix length (every warp for itself)
@@ -1077,7 +1078,7 @@ static UmmaPlan umma_plan(const seq_tree_attention_params& p) {
   const int tiles = (p.n_tree + nodes_per_tile - 1) / nodes_per_tile;
   const long units = (long)tiles * p.num_kv_heads;
   const int nblk = (p.prefix_len + p.n_tree + kBlockN - 1) / kBlockN;
-  const bool can_stream = tiles <= kMaxStreamTiles;
+  const bool can_stream = tiles <= kMaxStreamTiles && p.prefix_len_dev_count <= 1;  // (a range of the stream schedule crosses kv heads: one length)
   const int kNumSMs = device_sm_count();
 #ifdef SEQ_TRACE
   if (const char* e = getenv("SEQ_DEBUG_SPLITS")) return {atoi(e), false};  // debug builds only
@@ -1175,7 +1176,7 @@ int launch_attention_umma(const seq_tree_attention_params& p, int splits, cudaSt
   a.dev_status = p.dev_status;
   a.stream = umma_stream_mode(p, splits) ? 1 : 0;
   a.blocks_per_head_host = 0; a.total_blocks_host = 0;
-  a.L_dev = p.prefix_len_dev; a.zero_tail = p.prefix_len_dev != nullptr ? 1 : 0;
+  a.L_dev = p.prefix_len_dev; a.L_count = p.prefix_len_dev_count; a.zero_tail = p.prefix_len_dev != nullptr ? 1 : 0;
   a.ws_count = nullptr; a.ws_ml = nullptr; a.ws_o = nullptr;
   if (a.stream) {
     const size_t cnt_bytes = stream_count_bytes(p);

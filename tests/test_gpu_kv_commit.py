@@ -250,3 +250,54 @@ def test_attention_reads_the_prefix_length_from_device_memory_on_every_kernel_pa
         B.seq_tree_attention(q, kc, vc, mask, cap - n, kernel=kernel, dev_status=st, prefix_len_dev=L_dev)
         torch.cuda.synchronize()
         assert int(st.item()) == B.SEQ_DEV_BAD_LENGTH
+
+
+@pytest.mark.parametrize("kernel,given_mask,heads_kv,group,n,lengths", [
+    (B.KERNEL_AUTO, False, 2, 4, 40, (50, 300, 171)),       # the tensor-core kernel, mask from the parent array
+    (B.KERNEL_AUTO, True, 2, 4, 40, (0, 64, 65)),           # ... with the mask given; an empty prefix among them
+    (B.KERNEL_CUDA_CORE, True, 2, 4, 40, (50, 300, 171)),   # the CUDA-core kernel
+    (B.KERNEL_AUTO, False, 40, 1, 130, (100, 37, 222, 160)),  # 320 (tile, kv head) units: more than SMs, still the grid schedule
+])
+def test_batch_of_requests_with_a_prefix_length_each(kernel, given_mask, heads_kv, group, n, lengths):
+    """Requests stacked as heads, each with its own prefix length in device memory (the tree is common: Section 4.1 fixes
+    it in advance): every request's rows against the oracle run on that request alone."""
+    import dataclasses
+
+    from paper_2402_12374_b200 import workloads as W
+
+    d = G.dev()
+    R, cap = len(lengths), max(lengths) + n + 24
+    cfg = dataclasses.replace(W.CONFIGS["tiny"], num_q_heads=heads_kv * group, num_kv_heads=heads_kv, prefix_len=max(lengths),
+                              n_tree=n, max_depth=9, max_fanout=5)
+    parent = torch.from_numpy(W.make_tree(cfg, 7))
+    rng = np.random.default_rng(17)
+    q = torch.from_numpy(rng.standard_normal((n, R * heads_kv * group, 128)).astype(np.float32)).to(torch.bfloat16)
+    k = torch.from_numpy(rng.standard_normal((R * heads_kv, cap, 128)).astype(np.float32)).to(torch.bfloat16)
+    v = torch.from_numpy(rng.standard_normal((R * heads_kv, cap, 128)).astype(np.float32)).to(torch.bfloat16)
+    st = torch.zeros(1, dtype=torch.int32, device=d)
+    L_dev = torch.tensor(lengths, dtype=torch.int32, device=d)
+    mask = G.gpu_mask(parent.numpy())[0] if given_mask else None
+    call = B.AttentionCall(q.to(d), k.to(d), v.to(d), mask, max(lengths), parent=parent.to(d), dev_status=st,
+                           prefix_len_dev=L_dev, kernel=kernel)
+    call.run()
+    torch.cuda.synchronize()
+    assert int(st.item()) == 0
+    got = call.out.double().cpu().numpy()
+    hq = heads_kv * group
+    for r, L in enumerate(lengths):
+        ref, _, _ = O.tree_attention(q[:, r * hq:(r + 1) * hq], k[r * heads_kv:(r + 1) * heads_kv, :L + n],
+                                     v[r * heads_kv:(r + 1) * heads_kv, :L + n], parent, L)
+        assert np.abs(got[:, r * hq:(r + 1) * hq] - ref).max() < 2e-2, f"request {r} (prefix {L})"
+
+
+def test_per_request_lengths_are_refused_where_they_cannot_work():
+    d = G.dev()
+    q = torch.zeros((8, 6, 128), dtype=torch.bfloat16, device=d)
+    kv = torch.zeros((6, 64, 128), dtype=torch.bfloat16, device=d)
+    parent = torch.tensor([-1, 0, 0, 1, 1, 2, 2, 3], dtype=torch.int32, device=d)
+    four = torch.zeros(4, dtype=torch.int32, device=d)   # 4 does not divide 6 kv heads
+    with pytest.raises(Exception):
+        B.AttentionCall(q, kv, kv.clone(), None, 16, parent=parent, prefix_len_dev=four).run()
+    three = torch.zeros(3, dtype=torch.int32, device=d)
+    with pytest.raises(Exception):  # the stream schedule works on ranges that cross kv heads
+        B.AttentionCall(q, kv, kv.clone(), None, 16, parent=parent, prefix_len_dev=three, kernel=B.KERNEL_TENSOR_CORE_STREAM).run()
