@@ -98,7 +98,11 @@ def test_host_checkable_errors_are_refused_before_launch(lib):
 
     bad = [dict(q=None), dict(n_tree=0), dict(n_tree=1025), dict(num_kv_heads=5), dict(kv_capacity=100),
            dict(dtype=7), dict(q_stride_head=100), dict(kv_stride_tok=129), dict(k_cache=fake + 2),
-           dict(mask_words_per_row=0), dict(softmax_scale=float("nan")), dict(kernel=9), dict(prefix_len=-1)]
+           dict(mask_words_per_row=0), dict(softmax_scale=float("nan")), dict(kernel=9), dict(prefix_len=-1),
+           # one prefix length per request: a negative count, no lengths given, a count that does not divide the kv heads,
+           # the stream schedule forced
+           dict(prefix_len_dev_count=-1), dict(prefix_len_dev_count=4), dict(prefix_len_dev_count=5, prefix_len_dev=fake),
+           dict(prefix_len_dev_count=4, prefix_len_dev=fake, kernel=3)]
     for kw in bad:
         assert lib.seq_tree_attention(C.byref(attn(**kw)), None) == B.SEQ_ERR_INVALID_ARG, kw
         assert lib.seq_tree_attention_workspace_bytes(C.byref(attn(**kw))) == 0
