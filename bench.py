@@ -669,6 +669,42 @@ def verify_bf16_leg(cfg, parent, ver_sets, T, dev, stream) -> dict:
             "note": "SEQ_VERIFY_LOGITS_BF16: the same walk on bfloat16 logits; outside the timed step"}
 
 
+def verify_greedy_leg(cfg, parent, ver_sets, dev, stream) -> dict:
+    """Not part of the timed step: the verification at T = 0 (greedy decoding, the setting of the paper's first result
+    tables), L2-cold like the sampling figure.  The walk is as long as the synthetic draft happens to agree with the
+    target's arg-max; its length is reported beside the time."""
+    from paper_2402_12374_b200 import binding as B
+
+    status = torch.zeros(1, dtype=torch.int32, device=dev)
+    parent_d = torch.from_numpy(parent).to(dev)
+    calls = [B.VerifyCall(parent_d, tok, tl, dl, 0.0, u, dev_status=status) for tok, tl, dl, u in ver_sets[:2]]
+    flush = torch.empty(160 << 20, dtype=torch.uint8, device=dev)
+    Kc = 12
+
+    def graph_of(body):
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g, stream=stream):
+            for i in range(Kc):
+                body(i)
+        g.replay()
+        stream.synchronize()
+        return g
+
+    with torch.cuda.stream(stream):
+        for c in calls:
+            c.run(stream)
+        stream.synchronize()
+        visited = sum(int(c.path_len.item()) for c in calls) / len(calls)
+        g_cold = graph_of(lambda i: (flush.fill_(i & 127), calls[i % len(calls)].run(stream)))
+        g_flush = graph_of(lambda i: flush.fill_(i & 127))
+        ms = [statistics.median(timed_replays(g, stream, 7, 1, dev)) for g in (g_cold, g_flush)]
+    if int(status.item()) != 0:
+        raise RuntimeError(f"verify_greedy dev_status = {int(status.item())}")
+    return {"us_per_launch": (ms[0] - ms[1]) * 1e3 / Kc, "visited_nodes_mean": visited,
+            "l2": "cold (160 MiB written before every launch)",
+            "note": "T = 0: arg-max matching, one exchange per visited node; outside the timed step"}
+
+
 def robustness_leg(dev, stream, vocab=2048, requests=1500) -> dict:
     """Not part of the timed step (--robustness): a synthetic analogue of the paper's rejection-rate figure (Section
     3.2.2: average rejection rate against the number of speculated child tokens at T = 0.2, 0.6, 1.0, for the three
@@ -937,6 +973,7 @@ def run_workload(cfg, T, args, rank, local_rank, world, dev, stream, peaks, with
         legs["verify_batch"] = verify_batch_leg(cfg, parent, ver_like, T, dev, stream)
         if T > 0:
             legs["verify_bf16_logits"] = verify_bf16_leg(cfg, parent, ver_sets, T, dev, stream)
+            legs["verify_greedy"] = verify_greedy_leg(cfg, parent, ver_sets, dev, stream)
             legs["top_p_filter"] = top_p_leg(cfg, ver_like, T, dev, stream, peaks)
             legs["draft_sample"] = draft_sample_leg(cfg, parent, ver_like, T, dev, stream, peaks)
         res["next_rows"] = legs

@@ -1,6 +1,6 @@
 // seq_tree_verify: entry points, argument checks and the choice of kernel; and the walk of Algorithm 2 from the root
-// with its rows in SHARED memory (greedy decoding, sampling from the target, the every-node hook, batches of requests,
-// and devices that cannot place a cluster of 16 CTAs).  The default walk keeps its rows in registers
+// with its rows in SHARED memory (sampling from the target at T > 0, the every-node hook, batches of requests, and
+// devices that cannot place a cluster of 16 CTAs).  The default walk keeps its rows in registers
 // (tree_verify_walk.cu); the node-parallel schedule is tree_verify_nodes.cu.
 //
 // Schedule.  One cluster of CTAs follows the walk (16 CTAs for a single request where the device can place such a

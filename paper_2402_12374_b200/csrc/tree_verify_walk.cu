@@ -20,10 +20,12 @@
 // marks all the same.  The per-warp partial sums of the last pass are the coarse level of the final inverse CDF,
 // which the one warp that holds the crossing finishes on its own.
 //
-// Serves the default mode and the variant without the draft update at T > 0; greedy decoding, sampling from the
-// target, the every-node hook and batches run on the kernels of tree_verify.cu.
+// Serves the default mode and the variant without the draft update at T > 0, and - with a kernel of its own at the
+// end of this file - greedy decoding (T = 0, every mode); sampling from the target at T > 0, the every-node hook and
+// batches run on the kernels of tree_verify.cu.
 #include <cooperative_groups.h>
 #include <float.h>
+#include <limits.h>
 #include <math.h>
 
 #include "common.cuh"
@@ -56,6 +58,7 @@ struct Shared {
   int32_t chunk_cnt[32];              // children among nodes [32 j, 32 j + 32)
   float4 xbuf[2][kParts];             // cluster exchange: one entry per (rank, warp), double-buffered
   int32_t node_flags;
+  int32_t pick[2][4];                 // greedy walk, by hop parity: the matching child, the first child with a bad token, the first child
 };
 
 __device__ __forceinline__ float fast_ex2(float x) {
@@ -614,11 +617,151 @@ __global__ void __launch_bounds__(kTh, 1) tree_verify_walk_kernel(const VerifyAr
   // so nothing can still address a CTA that has left.
 }
 
+
+// ---------------------------------------------------------------- greedy decoding (T = 0) -----------------------
+// R is the one-hot at the target arg-max (lowest index on ties), a child is accepted iff its token is that arg-max;
+// draft logits and uniforms play no part.  Per visited node: the target row in registers, one arg-max over the
+// cluster (one exchange), one look at the children.  While the exchange gathers, the row of the node's first child -
+// the draft's most probable token, the likeliest match - is requested; any other match is fetched when it is known.
+__device__ __forceinline__ int ordered_key(float x) {  // an integer that orders like the (non-NaN) float
+  int b = __float_as_int(x);
+  return b ^ ((b >> 31) & 0x7fffffff);
+}
+// (key, index) of the larger key, then the lower index; index 0x7fffffff = nothing
+__device__ __forceinline__ void warp_argmax(int& key, int& idx) {
+  const int k = idx == 0x7fffffff ? INT_MIN : key;
+  const int m = __reduce_max_sync(0xffffffffu, k);
+  idx = __reduce_min_sync(0xffffffffu, (k == m) ? idx : 0x7fffffff);
+  key = m;
+}
+
+template <int NCH, bool kBf16>
+__global__ void __launch_bounds__(kTh, 1) tree_verify_greedy_kernel(const VerifyArgs a) {
+  constexpr int kEsz = kBf16 ? 2 : 4;
+  constexpr int kE = 4 * NCH, kSpan = 32 * kE;
+  const char* const tbase = reinterpret_cast<const char*>(a.target);
+  cg::cluster_group cluster = cg::this_cluster();
+  extern __shared__ __align__(16) uint8_t dyn_smem[];
+  Shared* sh = reinterpret_cast<Shared*>(dyn_smem);
+  Ctx c;
+  c.sh = sh;
+  c.rank = (int)cluster.block_rank();
+  c.lo = min(c.rank * a.slice_cap, a.V);
+  c.cnt = min(a.V - c.lo, a.slice_cap);
+  c.tid = threadIdx.x; c.warp = threadIdx.x >> 5; c.lane = threadIdx.x & 31;
+  c.xpar = 0;
+  const bool leader = c.rank == 0 && c.tid == 0;
+  if (c.tid == 0) asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+  asm volatile("griddepcontrol.wait;" ::: "memory");
+
+  RawRow<NCH, kBf16> pn;
+  {
+    int tp[4], tt[4];
+#pragma unroll
+    for (int k = 0; k < 4; ++k) {
+      const int i = c.tid + kTh * k;
+      tp[k] = i < a.n ? a.parent[i] : -1;
+      tt[k] = i < a.n ? a.tokens[i] : 0;
+    }
+    load_row<NCH, kBf16>(c, tbase, pn);
+#pragma unroll
+    for (int k = 0; k < 4; ++k) {
+      const int i = c.tid + kTh * k;
+      if (i < a.n) {
+        int pp = tp[k];
+        if (i == 0) pp = -1;
+        else if (pp < -1 || pp >= i) { if (c.rank == 0) dev_flag(a.dev_status, SEQ_DEV_BAD_PARENT); pp = -1; }
+        sh->parent[i] = pp;
+        sh->tokens[i] = tt[k];
+      }
+    }
+    if (c.rank == 0 && a.next_child_out != nullptr)
+      for (int i = c.tid; i < a.n; i += kTh) a.next_child_out[i] = -2;  // nodes the walk does not visit
+  }
+  cluster.sync();  // the tree is in place; every CTA of the cluster is resident before any remote write
+
+  int cur = 0, plen = 0, g = 0;
+  bool bad = false;
+#pragma unroll 1
+  for (int hop = 0; hop < a.n; ++hop) {  // a walk visits at most n nodes
+    if (leader) a.path[plen] = cur;
+    ++plen;
+    int32_t* pick = sh->pick[hop & 1];
+    if (c.tid < 3) pick[c.tid] = 0x7fffffff;  // (the other set is the one the previous hop may still be reading)
+    float x[kE];
+    widen<NCH, kBf16>(pn, x);
+    // this thread's arg-max: its elements in ascending index order, the first of equal values stays
+    int key = INT_MIN, idx = 0x7fffffff;
+#pragma unroll
+    for (int e = 0; e < kE; ++e) {
+      const int local = c.warp * kSpan + (e >> 2) * 128 + c.lane * 4 + (e & 3);
+      if (local < c.cnt) {
+        bad |= !(x[e] < INFINITY);
+        const int k = ordered_key(clean_logit(x[e]));
+        if (idx == 0x7fffffff || k > key) { key = k; idx = c.lo + local; }
+      }
+    }
+    warp_argmax(key, idx);
+    exchange_push(cluster, c, make_float4(__int_as_float(key), __int_as_float(idx), 0.f, 0.f));
+    // ---- while the barrier gathers: the node's first child, and its row on the way
+    __syncthreads();  // pick[] is reset
+#pragma unroll
+    for (int k = 0; k < 4; ++k) {
+      const int i = c.tid + kTh * k;
+      if (i < a.n && sh->parent[i] == cur) atomicMin(&pick[2], i);
+    }
+    __syncthreads();
+    const int first_kid = pick[2];
+    if (first_kid != 0x7fffffff) load_row<NCH, kBf16>(c, tbase + (int64_t)first_kid * a.target_stride * kEsz, pn);
+    Exch t;
+    exchange_pull(c, t);
+    key = INT_MIN; idx = 0x7fffffff;
+#pragma unroll
+    for (int m = 0; m < kPPL; ++m) {  // entries in vocabulary order: the first of equal keys stays
+      const int k = __float_as_int(t.e[m].x), i = __float_as_int(t.e[m].y);
+      if (i != 0x7fffffff && (idx == 0x7fffffff || k > key)) { key = k; idx = i; }
+    }
+    warp_argmax(key, idx);
+    g = idx == 0x7fffffff ? 0 : idx;
+    // ---- the child that carries the arg-max (the first, should several); a child with a token outside the vocabulary
+    // is reported if the loop over the children would have met it before the match
+#pragma unroll
+    for (int k = 0; k < 4; ++k) {
+      const int i = c.tid + kTh * k;
+      if (i < a.n && sh->parent[i] == cur) {
+        const int s = sh->tokens[i];
+        if (s < 0 || s >= a.V) atomicMin(&pick[1], i);
+        else if (s == g) atomicMin(&pick[0], i);
+      }
+    }
+    __syncthreads();
+    const int match = pick[0];
+    if (leader) {
+      if (pick[1] < match) dev_flag(a.dev_status, SEQ_DEV_BAD_TOKEN);
+      if (a.next_child_out != nullptr) a.next_child_out[cur] = match == 0x7fffffff ? -1 : match;
+    }
+    if (match == 0x7fffffff) break;
+    if (match != first_kid) load_row<NCH, kBf16>(c, tbase + (int64_t)match * a.target_stride * kEsz, pn);
+    cur = match;
+  }
+  if (bad) dev_flag(a.dev_status, SEQ_DEV_NONFINITE);
+  if (a.residual_out != nullptr) {
+#pragma unroll
+    for (int e = 0; e < kE; ++e) {
+      const int local = c.warp * kSpan + (e >> 2) * 128 + c.lane * 4 + (e & 3);
+      if (local < c.cnt) a.residual_out[c.lo + local] = (c.lo + local == g) ? 1.f : 0.f;
+    }
+  }
+  if (leader) { *a.path_len = plen; *a.bonus = g; }
+}
+
 }  // namespace vwk
 
 // Elements a cluster of this kernel holds per row: 16 CTAs x 256 threads x 4 NCH.
 bool verify_walk_supported(int vocab, int flags, float temperature) {
-  if (flags & (SEQ_VERIFY_ALL_NODES | SEQ_VERIFY_TARGET_SAMPLE)) return false;
+  if (flags & SEQ_VERIFY_ALL_NODES) return false;
+  if (temperature == 0.f) return vocab >= 1 && (size_t)vocab <= (size_t)vwk::kCl * vwk::kTh * 4 * 8;  // greedy: its own kernel, whatever the mode flags say
+  if (flags & SEQ_VERIFY_TARGET_SAMPLE) return false;
   if (!(temperature > 0.f)) return false;
   return vocab >= 1 && (size_t)vocab <= (size_t)vwk::kCl * vwk::kTh * 4 * 8;
 }
@@ -628,11 +771,14 @@ int launch_verify_walk(const VerifyArgs& a_in, bool check_only, cudaStream_t str
   a.slice_cap = (((a.V + vwk::kCl - 1) / vwk::kCl) + 3) & ~3;
   const int nch = a.slice_cap <= vwk::kTh * 4 * 2 ? 2 : a.slice_cap <= vwk::kTh * 4 * 4 ? 4 : 8;
   const bool bf16 = (a.flags & SEQ_VERIFY_LOGITS_BF16) != 0;
+  const bool greedy = a.temperature == 0.f;
   void (*kernel)(const VerifyArgs) =
-      bf16 ? (nch == 2 ? vwk::tree_verify_walk_kernel<2, true> : nch == 4 ? vwk::tree_verify_walk_kernel<4, true> : vwk::tree_verify_walk_kernel<8, true>)
-           : (nch == 2 ? vwk::tree_verify_walk_kernel<2, false> : nch == 4 ? vwk::tree_verify_walk_kernel<4, false> : vwk::tree_verify_walk_kernel<8, false>);
-  const int slot = (nch == 2 ? 0 : nch == 4 ? 1 : 2) + (bf16 ? 3 : 0);
-  static int attr_done[6][64];
+      greedy ? (bf16 ? (nch == 2 ? vwk::tree_verify_greedy_kernel<2, true> : nch == 4 ? vwk::tree_verify_greedy_kernel<4, true> : vwk::tree_verify_greedy_kernel<8, true>)
+                     : (nch == 2 ? vwk::tree_verify_greedy_kernel<2, false> : nch == 4 ? vwk::tree_verify_greedy_kernel<4, false> : vwk::tree_verify_greedy_kernel<8, false>))
+      : bf16 ? (nch == 2 ? vwk::tree_verify_walk_kernel<2, true> : nch == 4 ? vwk::tree_verify_walk_kernel<4, true> : vwk::tree_verify_walk_kernel<8, true>)
+             : (nch == 2 ? vwk::tree_verify_walk_kernel<2, false> : nch == 4 ? vwk::tree_verify_walk_kernel<4, false> : vwk::tree_verify_walk_kernel<8, false>);
+  const int slot = (nch == 2 ? 0 : nch == 4 ? 1 : 2) + (bf16 ? 3 : 0) + (greedy ? 6 : 0);
+  static int attr_done[12][64];
   const int rc = once_per_device(attr_done[slot], [&]() -> int {
     SEQ_CUDA_OK(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sizeof(vwk::Shared)));
     SEQ_CUDA_OK(cudaFuncSetAttribute(kernel, cudaFuncAttributeNonPortableClusterSizeAllowed, 1));

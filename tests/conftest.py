@@ -35,7 +35,8 @@ def verify_schedule(request):
 
 def pytest_generate_tests(metafunc):
     name = metafunc.function.__name__
-    if (metafunc.module.__name__.split(".")[-1] in ("test_gpu_parity", "test_gpu_parity_full") and name.startswith("test_verify")
+    if ((metafunc.module.__name__.split(".")[-1] in ("test_gpu_parity", "test_gpu_parity_full") and name.startswith("test_verify")
+         or metafunc.module.__name__.split(".")[-1] == "test_gpu_greedy" and "verify_schedule" in metafunc.fixturenames)
             and "every_node_hook" not in name):
         if "verify_schedule" not in metafunc.fixturenames:
             metafunc.fixturenames.append("verify_schedule")
