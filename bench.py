@@ -528,7 +528,7 @@ def verify_batch_leg(cfg, parent, ver_h, T, dev, stream) -> dict:
         raise RuntimeError(f"verify_batch: dev_status {int(status.item())}, {same} of {R} bonus tokens equal to single launches")
     return {"requests": R, "us_per_launch": us_b, "us_per_request": us_b / R, "us_per_request_single_launches": us_s / R,
             "gpu_launches_per_call": 1, "bonus_tokens_equal_to_single_launches": f"{same}/{R}",
-            "note": "one cluster of 8 CTAs per request (a single request runs on a cluster of 16); outside the timed step"}
+            "note": "one cluster per request: of 16 CTAs (rows in registers) while the batch fits the GPU side by side, else of 8; outside the timed step"}
 
 
 def attention_batch_leg(cfg, parent, attn_h, dev, stream, peaks) -> dict:

@@ -300,8 +300,10 @@ typedef struct {
 size_t seq_tree_verify_workspace_bytes(const seq_tree_verify_params* p);
 int seq_tree_verify(const seq_tree_verify_params* p, void* stream);
 
-/* seq_tree_verify_batch -- `batch` independent requests in one launch, one cluster of 8 CTAs per request (18
- * clusters run at a time on 148 SMs).  Every request is verified as seq_tree_verify would verify it (the same
+/* seq_tree_verify_batch -- `batch` independent requests in one launch, one cluster of CTAs per request: clusters of 16
+ * with the request's rows in registers while the batch fits the device side by side (9 requests on 148 SMs; the
+ * modes that seq_tree_verify serves that way), else clusters of 8 with the rows in shared memory (18 clusters run at a
+ * time).  Every request is verified as seq_tree_verify would verify it (the same
  * algorithm; seq_tree_verify may spread one request over a larger cluster, so vocabulary-wide sums can round
  * differently and a decision inside the 1e-5 band can differ): same sizes, temperature and flags for all
  * (SEQ_VERIFY_ALL_NODES is not allowed), each with its own tree, tokens, logits and uniforms.  request0 describes request 0; request r's arrays start r strides further:

@@ -186,25 +186,34 @@ static int verify_launch(const seq_tree_verify_params* p, int batch, int64_t tre
   // 16-bit logits: served by the walk with its rows in registers only (default mode and the variant without the draft
   // update, T > 0, one request, a device that places a cluster of 16)
   const bool bf16 = (p->flags & SEQ_VERIFY_LOGITS_BF16) != 0;
-  if (bf16 && (batch != 0 || (p->flags & SEQ_VERIFY_SCHED_NODES) || !verify_walk_supported(p->vocab, p->flags, p->temperature)))
+  if (bf16 && ((p->flags & SEQ_VERIFY_SCHED_NODES) || !verify_walk_supported(p->vocab, p->flags, p->temperature)))
     return SEQ_ERR_UNSUPPORTED;
   if (p->flags & SEQ_VERIFY_SCHED_NODES) {
     if (batch != 0 || !wants_nodes_schedule(p)) return SEQ_ERR_UNSUPPORTED;
     return launch_verify_nodes(a, p->workspace, p->workspace_bytes, 0, s);  // (checks the workspace)
   }
-  if (batch > 0) return verify_launch_with<8, vcl8::VShared, 0>(vcl8::tree_verify_kernel<true>, a, p->vocab, batch, false, s);
-  if (p->flags & SEQ_VERIFY_ALL_NODES)  // 18 * 8 = 144 CTAs <= 148 SMs
-    return verify_launch_with<8, vcl8::VShared, 1>(vcl8::tree_verify_kernel<false>, a, p->vocab, p->n_tree < 18 ? p->n_tree : 18, false, s);
-  // One request: the cluster of 16 where the device can place one (asked once per device), else the cluster of 8.
-  // Vocabularies below 8192 tokens gain nothing from more CTAs.
+  // The cluster of 16 where the device can place one (asked once per device), else the cluster of 8.
   static int wide_ok[64];  // per device: 0 = not asked yet, 1 = yes, 2 = no
   int dev = 0;
   SEQ_CUDA_OK(cudaGetDevice(&dev));
   int wide = (dev >= 0 && dev < 64) ? __atomic_load_n(&wide_ok[dev], __ATOMIC_ACQUIRE) : 2;
   if (wide == 0) {  // (two threads asking at once get the same answer)
-    wide = verify_launch_with<16, vcl16::VShared, 2>(vcl16::tree_verify_kernel<false>, a, 32000, 1, true, s) == SEQ_OK ? 1 : 2;
+    VerifyArgs one = a;
+    wide = verify_launch_with<16, vcl16::VShared, 2>(vcl16::tree_verify_kernel<false>, one, 32000, 1, true, s) == SEQ_OK ? 1 : 2;
     __atomic_store_n(&wide_ok[dev], wide, __ATOMIC_RELEASE);
   }
+  if (batch > 0) {
+    // A batch that fits the GPU as clusters of 16 side by side runs the walk with its rows in registers, one cluster
+    // per request (one request then costs what it costs alone); a larger one the shared-memory walk on clusters of 8,
+    // eighteen requests at a time.
+    if (wide == 1 && batch * 16 <= device_sm_count() && verify_walk_supported(p->vocab, p->flags, p->temperature))
+      return launch_verify_walk(a, false, s, batch);
+    if (bf16) return SEQ_ERR_UNSUPPORTED;
+    return verify_launch_with<8, vcl8::VShared, 0>(vcl8::tree_verify_kernel<true>, a, p->vocab, batch, false, s);
+  }
+  if (p->flags & SEQ_VERIFY_ALL_NODES)  // 18 * 8 = 144 CTAs <= 148 SMs
+    return verify_launch_with<8, vcl8::VShared, 1>(vcl8::tree_verify_kernel<false>, a, p->vocab, p->n_tree < 18 ? p->n_tree : 18, false, s);
+  // One request.  Vocabularies below 8192 tokens gain nothing from more CTAs.
   // the walk with its rows in registers, where a cluster of 16 can be placed and the mode is one it serves
   if (wide == 1 && verify_walk_supported(p->vocab, p->flags, p->temperature)) return launch_verify_walk(a, false, s);
   if (bf16) return SEQ_ERR_UNSUPPORTED;

@@ -28,6 +28,7 @@ int launch_verify_nodes(const VerifyArgs& a, void* workspace, size_t workspace_b
 
 // The walk with rows in registers (tree_verify_walk.cu): one cluster of 16 CTAs, no workspace.
 bool verify_walk_supported(int vocab, int flags, float temperature);
-int launch_verify_walk(const VerifyArgs& a, bool check_only, cudaStream_t stream);
+// `requests` > 1: a batched launch, one cluster per request (the strides of VerifyArgs lead from one request to the next).
+int launch_verify_walk(const VerifyArgs& a, bool check_only, cudaStream_t stream, int requests = 1);
 
 }  // namespace seqtree

@@ -212,8 +212,25 @@ __device__ __forceinline__ void cluster_exchange(cg::cluster_group& cluster, Ctx
   exchange_pull(c, x);
 }
 
+// A batched launch runs one request per cluster: the same code on that request's arrays.
+__device__ __forceinline__ VerifyArgs request_args(const VerifyArgs& in) {
+  VerifyArgs a = in;
+  const int64_t r = blockIdx.x / kCl;
+  if (r > 0) {
+    a.parent += r * in.tree_stride; a.tokens += r * in.tree_stride;
+    a.target = reinterpret_cast<const float*>(reinterpret_cast<const char*>(in.target) + r * in.logits_stride * ((in.flags & SEQ_VERIFY_LOGITS_BF16) ? 2 : 4));
+    a.draft = reinterpret_cast<const float*>(reinterpret_cast<const char*>(in.draft) + r * in.logits_stride * ((in.flags & SEQ_VERIFY_LOGITS_BF16) ? 2 : 4));
+    a.uniforms += r * in.unif_stride;
+    a.path += r * in.tree_stride; a.path_len += r; a.bonus += r;
+    if (in.residual_out != nullptr) a.residual_out += r * in.resid_stride;
+    if (in.next_child_out != nullptr) a.next_child_out += r * in.tree_stride;
+  }
+  return a;
+}
+
 template <int NCH, bool kBf16>
-__global__ void __launch_bounds__(kTh, 1) tree_verify_walk_kernel(const VerifyArgs a) {
+__global__ void __launch_bounds__(kTh, 1) tree_verify_walk_kernel(const VerifyArgs a_in) {
+  const VerifyArgs a = request_args(a_in);
   constexpr int kEsz = kBf16 ? 2 : 4;  // bytes per logit
   const char* const tbase = reinterpret_cast<const char*>(a.target);
   const char* const dbase = reinterpret_cast<const char*>(a.draft);
@@ -636,7 +653,8 @@ __device__ __forceinline__ void warp_argmax(int& key, int& idx) {
 }
 
 template <int NCH, bool kBf16>
-__global__ void __launch_bounds__(kTh, 1) tree_verify_greedy_kernel(const VerifyArgs a) {
+__global__ void __launch_bounds__(kTh, 1) tree_verify_greedy_kernel(const VerifyArgs a_in) {
+  const VerifyArgs a = request_args(a_in);
   constexpr int kEsz = kBf16 ? 2 : 4;
   constexpr int kE = 4 * NCH, kSpan = 32 * kE;
   const char* const tbase = reinterpret_cast<const char*>(a.target);
@@ -766,7 +784,7 @@ bool verify_walk_supported(int vocab, int flags, float temperature) {
   return vocab >= 1 && (size_t)vocab <= (size_t)vwk::kCl * vwk::kTh * 4 * 8;
 }
 
-int launch_verify_walk(const VerifyArgs& a_in, bool check_only, cudaStream_t stream) {
+int launch_verify_walk(const VerifyArgs& a_in, bool check_only, cudaStream_t stream, int requests) {
   VerifyArgs a = a_in;
   a.slice_cap = (((a.V + vwk::kCl - 1) / vwk::kCl) + 3) & ~3;
   const int nch = a.slice_cap <= vwk::kTh * 4 * 2 ? 2 : a.slice_cap <= vwk::kTh * 4 * 4 ? 4 : 8;
@@ -786,7 +804,7 @@ int launch_verify_walk(const VerifyArgs& a_in, bool check_only, cudaStream_t str
   });
   if (rc != SEQ_OK) return rc;
   cudaLaunchConfig_t cfg = {};
-  cfg.gridDim = dim3(vwk::kCl);
+  cfg.gridDim = dim3(vwk::kCl * (requests > 0 ? requests : 1));
   cfg.blockDim = dim3(vwk::kTh);
   cfg.dynamicSmemBytes = sizeof(vwk::Shared);
   cfg.stream = stream;

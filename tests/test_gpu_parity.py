@@ -485,7 +485,8 @@ def test_verify_on_dp_shaped_trees(name, T):
 
 # ---------------------------------------------------------------- batched verification --------------
 @pytest.mark.parametrize("name,T,R,mode", [("tiny", 0.6, 5, "sequoia"), ("llama2-7b", 0.6, 20, "sequoia"), ("llama2-7b", 1.0, 7, "specinfer"),
-                                           ("llama2-7b", 0.6, 6, "target"), ("llama2-7b", 0.0, 4, "sequoia")])
+                                           ("llama2-7b", 0.6, 6, "target"), ("llama2-7b", 0.0, 4, "sequoia"),
+                                           ("llama3-70b", 0.6, 3, "sequoia")])  # (up to 9 requests: one cluster of 16 each, rows in registers)
 def test_verify_batch_equals_one_request_at_a_time(name, T, R, mode):
     """R requests (own tree, tokens, logits, uniforms) in one launch: every request's path, bonus and residual are
     the oracle's, and equal (to rounding) to what a launch of its own returns."""
