@@ -132,7 +132,7 @@ def test_verify_tiny_config():
 
 @pytest.mark.parametrize("T", [0.0, 0.6, 1.0])
 def test_verify_llama2_7b_config(T):
-    _verify_cases("llama2-7b", T, range(4))
+    _verify_cases("llama2-7b", T, range(8) if T == 0.6 else range(4))
 
 
 def test_verify_llama2_13b_config():
