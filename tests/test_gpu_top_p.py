@@ -169,3 +169,18 @@ def test_filter_then_verify_matches_the_oracle_chain(tp):
         vi2 = W.VerifyInputs(vi.parent, vi.tokens, filt.cpu(), vi.draft_logits, vi.uniforms, vi.temperature)
         checked += G.check_verify(vi2) == "ok"
     assert checked >= 1
+
+
+def test_top_p_cut_with_a_clear_margin_is_the_oracles_on_every_row():
+    """Rows whose probabilities fall off geometrically (each token 0.6 of the one before, in a shuffled order): the
+    cumulative mass passes top_p with a margin of percents, far outside the rounding band, so every row's kept set must
+    be exactly the oracle's — an off-by-one at the cut could not hide here."""
+    rng = np.random.default_rng(5)
+    rows, V, T = 48, 5000, 0.7
+    logits = np.full((rows, V), -60.0, np.float32)
+    for r in range(rows):
+        perm = rng.permutation(V)[:40]
+        logits[r, perm] = (T * np.log(0.6) * np.arange(40)).astype(np.float32) + np.float32(rng.normal())
+    for tp in (0.5, 0.8, 0.95, 0.999):
+        same, st = _check(logits, T, tp)
+        assert st == 0 and same == rows, (tp, same)
